@@ -1,0 +1,110 @@
+"""ctypes front end of the CPU oracle (``attn_ref.c``).
+
+TEST INFRASTRUCTURE ONLY: imported by the test-suite, the smoke check and the
+benchmark's cpu-baseline / reference legs.  The CUDA library and its Python
+binding never import this module, and this module never imports them.
+
+Every function takes and returns numpy float64 arrays shaped ``[B,H,S,D]``
+(``[B,H,S]`` for LSE).  Inputs in f32 or bf16 convert to f64 exactly, so the
+caller just passes ``x.double().numpy()``.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "attn_ref.c")
+_LIB = os.path.join(_HERE, "libmgn_oracle.so")
+_lib = None
+
+_dp = ctypes.POINTER(ctypes.c_double)
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (-O2, OpenMP, no fast-math). Returns the .so path."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + f".tmp{os.getpid()}"
+        subprocess.check_call(
+            ["gcc", "-O2", "-std=c11", "-fopenmp", "-fPIC", "-shared", "-o", tmp, _SRC, "-lm"]
+        )
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(build())
+        i, d = ctypes.c_int, ctypes.c_double
+        lib.ref_attn_fwd.argtypes = [_dp] * 5 + [i, i, i, i, i, d, i]
+        lib.ref_attn_fwd.restype = None
+        lib.ref_attn_bwd.argtypes = [_dp] * 9 + [i, i, i, i, i, d, i]
+        lib.ref_attn_bwd.restype = None
+        lib.ref_attn_head_matrices.argtypes = [_dp] * 7 + [i, i, i, d]
+        lib.ref_attn_head_matrices.restype = None
+        lib.ref_grads_from_ds.argtypes = [_dp] * 5 + [i, i, d]
+        lib.ref_grads_from_ds.restype = None
+        lib.ref_max_threads.argtypes = []
+        lib.ref_max_threads.restype = i
+        _lib = lib
+    return _lib
+
+
+def _c(a: np.ndarray) -> np.ndarray:
+    return np.ascontiguousarray(a, dtype=np.float64)
+
+
+def _p(a: np.ndarray):
+    return a.ctypes.data_as(_dp)
+
+
+def max_threads() -> int:
+    return int(_load().ref_max_threads())
+
+
+def attn_fwd(q, k, v, causal: bool, scale: float, nthreads: int = 0):
+    """Returns (O, LSE) in float64."""
+    q, k, v = _c(q), _c(k), _c(v)
+    B, H, S, D = q.shape
+    assert k.shape == q.shape and v.shape == q.shape
+    o = np.empty_like(q)
+    lse = np.empty((B, H, S), dtype=np.float64)
+    _load().ref_attn_fwd(_p(q), _p(k), _p(v), _p(o), _p(lse), B, H, S, D,
+                         int(bool(causal)), float(scale), int(nthreads))
+    return o, lse
+
+
+def attn_bwd(q, k, v, d_o, causal: bool, scale: float, nthreads: int = 0):
+    """Returns (O, LSE, dQ, dK, dV) in float64; O and LSE are recomputed here."""
+    q, k, v, d_o = _c(q), _c(k), _c(v), _c(d_o)
+    B, H, S, D = q.shape
+    assert k.shape == q.shape and v.shape == q.shape and d_o.shape == q.shape
+    o = np.empty_like(q)
+    lse = np.empty((B, H, S), dtype=np.float64)
+    dq, dk, dv = np.empty_like(q), np.empty_like(q), np.empty_like(q)
+    _load().ref_attn_bwd(_p(q), _p(k), _p(v), _p(d_o), _p(o), _p(lse), _p(dq), _p(dk), _p(dv),
+                         B, H, S, D, int(bool(causal)), float(scale), int(nthreads))
+    return o, lse, dq, dk, dv
+
+
+def head_matrices(q, k, v, d_o, causal: bool, scale: float):
+    """One head ([S,D] inputs): dense P, dP, dS as [S,S] float64 (masked entries 0)."""
+    q, k, v, d_o = _c(q), _c(k), _c(v), _c(d_o)
+    S, D = q.shape
+    P = np.empty((S, S)); dP = np.empty((S, S)); dS = np.empty((S, S))
+    _load().ref_attn_head_matrices(_p(q), _p(k), _p(v), _p(d_o), _p(P), _p(dP), _p(dS),
+                                   S, D, int(bool(causal)), float(scale))
+    return P, dP, dS
+
+
+def grads_from_ds(dS, q, k, scale: float):
+    """One head: (dQ, dK) = (scale dS K, scale dS^T Q)."""
+    dS, q, k = _c(dS), _c(q), _c(k)
+    S, D = q.shape
+    dq = np.empty_like(q); dk = np.empty_like(q)
+    _load().ref_grads_from_ds(_p(dS), _p(q), _p(k), _p(dq), _p(dk), S, D, float(scale))
+    return dq, dk
