@@ -1,0 +1,358 @@
+#!/usr/bin/env python
+"""Benchmark of the attention forward+backward hot path.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+                    [--workload NAME] [--mode strict|fast]
+
+A step is one forward call plus one backward call (preprocess, dQ clear, fused
+dK/dV/dQ kernel) over one batch of seeded synthetic input.  Prints ONE JSON line.
+The metric is counted GEMM TFLOP/s: forward 4*BH*Np*D, backward 10*BH*Np*D with
+Np = S^2 (full) or S^2/2 (causal).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import threading
+import time
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2608_01563_b200 import inputs as synth  # noqa: E402
+
+METRIC = "attention fwd+bwd TFLOP/s per B200 (strict f32, bf16) and % of matching peak"
+SM_COUNT = 148
+FP32_LANES_PER_SM = 128
+
+
+def flops(w, which):
+    npairs = w.S * w.S / (2.0 if w.causal else 1.0)
+    unit = w.BH * npairs * w.D
+    return {"fwd": 4.0 * unit, "bwd": 10.0 * unit, "sum": 14.0 * unit}[which]
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as fh:
+            return json.load(fh), "measured"
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "sm_max_mhz": 1965.0}, "fallback"
+
+
+def fp32_peak_tflops(peaks):
+    """FFMA peak: SMs x 128 lanes x 2 flop x max SM clock."""
+    return SM_COUNT * FP32_LANES_PER_SM * 2 * peaks.get("sm_max_mhz", 1965.0) * 1e6 / 1e12
+
+
+class ClockSampler:
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.gpu_index = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.fh = open(self.path, "w")
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.gpu_index), f"--query-gpu={self.QUERY}",
+                 "--format=csv,noheader,nounits", "-lms", "100"], stdout=self.fh, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.fh.close()
+        sm, mx, reasons, power = [], [], set(), []
+        for line in open(self.path):
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 9:
+                continue
+            try:
+                sm.append(float(parts[1])); mx.append(float(parts[2])); power.append(float(parts[3]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), parts[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        os.unlink(self.path)
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons),
+                       samples=len(sm), power_w_max=max(power))
+        return out
+
+
+def cpu_info():
+    model = "unknown"
+    try:
+        for line in open("/proc/cpuinfo"):
+            if line.startswith("model name"):
+                model = line.split(":", 1)[1].strip()
+                break
+    except OSError:
+        pass
+    return model
+
+
+def time_oracle(w, dtype, heads, repeats=1):
+    """Oracle forward+backward on the first `heads` heads. Returns (seconds fwd, seconds bwd, threads)."""
+    from oracle import attn_oracle as orc
+    q, k, v, d_o = synth.make_inputs(w, dtype=dtype, heads=heads)
+    a = [t.double().numpy() for t in (q, k, v, d_o)]
+    best_f = best_b = float("inf")
+    for _ in range(repeats):
+        t0 = time.perf_counter()
+        orc.attn_fwd(a[0], a[1], a[2], w.causal, w.scale)
+        t1 = time.perf_counter()
+        orc.attn_bwd(a[0], a[1], a[2], a[3], w.causal, w.scale)
+        t2 = time.perf_counter()
+        best_f, best_b = min(best_f, t1 - t0), min(best_b, t2 - t1)
+    return best_f, best_b, orc.max_threads()
+
+
+def cpu_baseline(w, dtype, budget_s=15.0):
+    """The oracle, as it stands, on a bounded head subset sized for ~budget_s of CPU work."""
+    from oracle import attn_oracle as orc
+    threads = orc.max_threads()
+    probe_heads = min(w.BH, threads)
+    tf, tb, _ = time_oracle(w, dtype, probe_heads)
+    per_round = tf + tb
+    rounds = max(1, int(budget_s / max(per_round, 1e-3)))
+    heads = min(w.BH, probe_heads * rounds)
+    if heads > probe_heads:
+        tf, tb, _ = time_oracle(w, dtype, heads)
+    fl = flops(w, "sum") * heads / w.BH
+    return {"value": fl / (tf + tb) / 1e12, "unit": "TFLOP/s", "cores": threads, "kind": "oracle",
+            "sample": f"first {heads} of {w.BH} heads of {w.name} (f64, fwd {tf:.2f} s + bwd {tb:.2f} s)",
+            "cpu_model": cpu_info()}
+
+
+def run_reference(args, w, dtype):
+    """--impl reference: the CPU oracle timed on a bounded sample of the same workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import attn_oracle as orc
+    threads = orc.max_threads()
+    heads = min(w.BH, threads)
+    for _ in range(args.warmup):
+        time_oracle(w, dtype, heads)
+    times = []
+    for _ in range(args.steps):
+        tf, tb, _ = time_oracle(w, dtype, heads)
+        times.append(tf + tb)
+    total = sum(times)
+    fl = flops(w, "sum") * heads / w.BH
+    value = fl * args.steps / total / 1e12
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "B": w.B, "H": w.H, "S": w.S, "D": w.D, "causal": w.causal,
+                   "mode": args.mode, "sample_heads": heads},
+        "cpu_baseline": {"value": value, "unit": "TFLOP/s", "cores": threads, "kind": "oracle",
+                         "sample": f"first {heads} of {w.BH} heads of {w.name} per step", "cpu_model": cpu_info()},
+        "e2e": {"value": value, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default=None)
+    ap.add_argument("--mode", default="strict", choices=["strict", "fast"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    default_wl = "gpt2_small" if args.mode == "strict" else "long_context"
+    w = synth.WORKLOADS[args.workload or default_wl]
+    dtype = torch.float32 if args.mode == "strict" else torch.bfloat16
+
+    if args.impl == "reference":
+        run_reference(args, w, dtype)
+        return
+
+    from paper_2608_01563_b200 import binding as mgn
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the attention path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    mode = mgn.MODE_STRICT_F32 if args.mode == "strict" else mgn.MODE_FAST_BF16
+
+    # Each rank works on its own batch of the same shape (heads are independent units:
+    # no data-path collective).  Rank r draws sweep index r*1000 more than rank 0.
+    import dataclasses
+    w_rank = dataclasses.replace(w, sweep=w.sweep + 1000 * rank)
+    host = [t.pin_memory() for t in synth.make_inputs(w_rank, dtype=dtype)]
+    dev = [t.cuda(non_blocking=True) for t in host]
+    qd, kd, vd, dod = dev
+    B, H, S, D = qd.shape
+    o = torch.empty_like(qd)
+    lse = torch.empty(B, H, S, device="cuda", dtype=torch.float32)
+    dq, dk, dv = (torch.empty_like(qd) for _ in range(3))
+    ws = mgn.alloc_workspace(B, H, S, D, mode)
+    host_out = [torch.empty(t.shape, dtype=t.dtype).pin_memory() for t in (o, lse, dq, dk, dv)]
+    torch.cuda.synchronize()
+
+    def step():
+        mgn.mgn_attn_fwd(qd, kd, vd, o, lse, w.causal, w.scale, mode)
+        mgn.mgn_attn_bwd(qd, kd, vd, o, dod, lse, dq, dk, dv, ws, w.causal, w.scale, mode)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step()
+    mgn.mgn_attn_check()
+
+    K = args.steps
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    e_step0, e_step1 = ev(), ev()
+    pairs = {name: [(ev(), ev()) for _ in range(K)] for name in ("fwd_main", "bwd_main")}
+    e_fwd_end = [ev() for _ in range(K)]
+    for lst in pairs.values():          # create the underlying CUDA events
+        for a, b in lst:
+            a.record(); b.record()
+    torch.cuda.synchronize()
+
+    sampler = ClockSampler(local_rank if "CUDA_VISIBLE_DEVICES" not in os.environ else
+                           int(os.environ["CUDA_VISIBLE_DEVICES"].split(",")[local_rank]))
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    barrier()
+    e_step0.record()
+    for i in range(K):
+        a, b = pairs["fwd_main"][i]
+        mgn.mgn_attn_profile_events(a.cuda_event, b.cuda_event)
+        mgn.mgn_attn_fwd(qd, kd, vd, o, lse, w.causal, w.scale, mode)
+        e_fwd_end[i].record()
+        a, b = pairs["bwd_main"][i]
+        mgn.mgn_attn_profile_events(a.cuda_event, b.cuda_event)
+        mgn.mgn_attn_bwd(qd, kd, vd, o, dod, lse, dq, dk, dv, ws, w.causal, w.scale, mode)
+    e_step1.record()
+    barrier()
+    mgn.mgn_attn_profile_events(None, None)
+    clocks = sampler.stop() if rank == 0 else None
+    mgn.mgn_attn_check()
+
+    total_ms = e_step0.elapsed_time(e_step1)
+    fwd_main_ms = statistics.mean(a.elapsed_time(b) for a, b in pairs["fwd_main"])
+    bwd_main_ms = statistics.mean(a.elapsed_time(b) for a, b in pairs["bwd_main"])
+    # forward call = its one kernel; backward call = everything from the end of forward to the end of the step
+    fwd_call_ms = fwd_main_ms
+    bwd_call_ms = total_ms / K - fwd_call_ms
+
+    # ---- end to end: host buffers in, host buffers out, copies inside the timed region ----------
+    e2e = None
+    if not args.no_e2e:
+        def e2e_step():
+            for h, d in zip(host, dev):
+                d.copy_(h, non_blocking=True)
+            step()
+            for h, d in zip(host_out, (o, lse, dq, dk, dv)):
+                h.copy_(d, non_blocking=True)
+        for _ in range(3):
+            e2e_step()
+        barrier()
+        e0, e1 = ev(), ev()
+        e0.record()
+        for _ in range(K):
+            e2e_step()
+        e1.record()
+        barrier()
+        e2e_ms = e0.elapsed_time(e1)
+    else:
+        e2e_ms = None
+
+    t = torch.tensor([total_ms, e2e_ms or 0.0], device="cuda", dtype=torch.float64)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    total_ms_max, e2e_ms_max = t.tolist()
+
+    if rank == 0:
+        peaks, peak_src = measured_peaks()
+        fl_sum = flops(w, "sum")
+        value = world * fl_sum * K / (total_ms_max * 1e-3) / 1e12
+        if args.mode == "strict":
+            peak = fp32_peak_tflops(peaks)
+            bound = "alu"
+            peak_note = f"{SM_COUNT} SMs x {FP32_LANES_PER_SM} FP32 lanes x 2 x {peaks.get('sm_max_mhz', 1965.0):.0f} MHz"
+        else:
+            peak = peaks["bf16_tflops_sustained"]
+            bound = "tensor"
+            peak_note = f"{peak_src} dense bf16 (sustained); burst {peaks['bf16_tflops']}"
+        bwd_main_tflops = flops(w, "bwd") / (bwd_main_ms * 1e-3) / 1e12
+        fwd_main_tflops = flops(w, "fwd") / (fwd_main_ms * 1e-3) / 1e12
+        line = {
+            "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": K,
+            "warmup": args.warmup, "ms_per_step": total_ms_max / K, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32" if args.mode == "strict" else "bf16", "data": "synthetic",
+            "config": {"workload": w.name, "B": w.B, "H": w.H, "S": w.S, "D": w.D, "causal": w.causal,
+                       "mode": args.mode, "per_rank_batch": "full workload on every rank",
+                       "l2": "no flush: Q,K,V,dO,O,dQ,dK,dV of one step exceed the 126 MB L2"
+                       if 8 * qd.numel() * qd.element_size() > 126e6 else "working set fits L2 (compute-bound path)"},
+            "frac_of_peak": value / world / peak, "peak_tflops": peak, "peak_note": peak_note,
+            "fwd_tflops": flops(w, "fwd") / (fwd_call_ms * 1e-3) / 1e12,
+            "bwd_tflops": flops(w, "bwd") / (bwd_call_ms * 1e-3) / 1e12,
+            "fwd_ms": fwd_call_ms, "bwd_ms": bwd_call_ms,
+            "roofline": {"kernel": "bwd_main (fused dK/dV/dQ)", "bound": bound, "achieved": bwd_main_tflops,
+                         "peak": peak, "unit": "TFLOP/s", "frac": bwd_main_tflops / peak, "traffic": None,
+                         "ms_per_launch": bwd_main_ms, "peak_source": peak_note,
+                         "fwd_kernel": {"achieved": fwd_main_tflops, "frac": fwd_main_tflops / peak,
+                                        "ms_per_launch": fwd_main_ms}},
+            "gpu_launches": 3 * K,
+            "clocks": clocks,
+        }
+        if e2e_ms is not None:
+            h2d = sum(t_.numel() * t_.element_size() for t_ in host)
+            d2h = sum(t_.numel() * t_.element_size() for t_ in host_out)
+            line["e2e"] = {"value": world * fl_sum * K / (e2e_ms_max * 1e-3) / 1e12, "unit": "TFLOP/s",
+                           "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+        if world == 1 and not args.no_cpu_baseline:
+            line["cpu_baseline"] = cpu_baseline(w, dtype)
+        print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

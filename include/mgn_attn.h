@@ -1,0 +1,110 @@
+/*
+ * mgn_attn.h -- C ABI of the B200 (sm_100a) scaled-dot-product attention library.
+ *
+ * The operations are the attention kernels the paper lists as one of its kernel
+ * archetypes (Section 3.3: "tiled attention forward, dQ, and fused dK+dV kernels")
+ * and profiles in Section 7.3 (FlashGradKV / FlashGradQ).  The two numerical modes
+ * mirror the paper's arithmetic contracts (Section 4.2, Table "Arithmetic
+ * permissions"): a strict f32 path and a validated reduced-input fast path with
+ * f32 accumulation.
+ *
+ * Conventions shared by every entry point
+ *   - All tensor pointers are DEVICE pointers on the current CUDA device.
+ *   - q, k, v, o, d_o, dq, dk, dv are dense row-major [B,H,S,D], D innermost, no
+ *     padding.  Element type: MGN_MODE_STRICT_F32 -> IEEE binary32,
+ *     MGN_MODE_FAST_BF16 -> bfloat16.  lse is [B,H,S] binary32 in both modes.
+ *   - Every tensor pointer must be 16-byte aligned.  D must be 32, 64 or 128.
+ *   - The caller owns every buffer.  The library allocates no device memory.
+ *   - Calls only enqueue work on `stream` (a cudaStream_t passed as void*; NULL is
+ *     the legacy default stream) and return without synchronising.  Inputs must
+ *     stay valid, and outputs untouched, until the stream has passed the call.
+ *   - Outputs need not be initialised.  Outputs must not alias inputs or each other.
+ *   - Errors are reported by return code only (mgn_status); nothing is printed and
+ *     nothing aborts.  Argument errors are detected before any launch, in the
+ *     order INVALID_ARG, UNSUPPORTED, MISALIGNED, WORKSPACE, ARCH.
+ */
+#ifndef MGN_ATTN_H
+#define MGN_ATTN_H
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    MGN_OK = 0,
+    MGN_ERR_INVALID_ARG = 1,    /* null pointer, non-positive dim, causal not 0/1, non-finite scale, unknown mode */
+    MGN_ERR_UNSUPPORTED = 2,    /* D not in {32,64,128}, or sizes beyond the index plan */
+    MGN_ERR_MISALIGNED = 3,     /* a tensor pointer is not 16-byte aligned */
+    MGN_ERR_WORKSPACE = 4,      /* workspace null or too small */
+    MGN_ERR_CUDA = 5,           /* a CUDA runtime/driver call failed */
+    MGN_ERR_ARCH = 6,           /* current device is not compute capability 10.x */
+    MGN_ERR_DEVICE_TIMEOUT = 7  /* a bounded wait inside a kernel gave up (see mgn_attn_check) */
+} mgn_status;
+
+enum { MGN_MODE_STRICT_F32 = 0, MGN_MODE_FAST_BF16 = 1 };
+
+/*
+ * Attention forward (paper Section 3.3, "tiled attention forward").
+ *   s_ij = scale * sum_d q[i,d] k[j,d];  causal != 0 keeps only j <= i;
+ *   lse_i = log sum_j exp(s_ij)  (natural log, of the scaled and masked scores);
+ *   o_i   = sum_j exp(s_ij - lse_i) v_j.
+ * q,k,v: in.  o: out [B,H,S,D] (mode's element type).  lse: out [B,H,S] f32.
+ * Strict mode computes in f32 FFMA; fast mode multiplies bf16 operands on the
+ * tensor cores with f32 accumulation and f32 softmax statistics.
+ */
+int mgn_attn_fwd(const void* q, const void* k, const void* v, void* o, float* lse,
+                 int B, int H, int S, int D, int causal, float scale, int mode, void* stream);
+
+/*
+ * Attention backward (paper Section 3.3 "dQ, and fused dK+dV kernels"; Section 7.3).
+ * Given q,k,v, the forward's o and lse (of the same mode), and d_o = dLoss/do:
+ *   delta_i = sum_d d_o[i,d] o[i,d];   p_ij = exp(s_ij - lse_i);
+ *   dv_j = sum_i p_ij d_o_i;           dp_ij = sum_d d_o[i,d] v[j,d];
+ *   ds_ij = p_ij (dp_ij - delta_i);
+ *   dq_i = scale sum_j ds_ij k_j;      dk_j = scale sum_i ds_ij q_i.
+ * dq, dk, dv: out.  workspace: device scratch of at least
+ * mgn_attn_bwd_workspace_bytes(...) bytes, 256-byte aligned, contents ignored on
+ * entry and undefined on exit; two calls that may overlap on the GPU need
+ * distinct workspaces.  dq is accumulated with floating-point atomics, so its
+ * low-order bits can differ from run to run; dk, dv, and the forward are
+ * deterministic.
+ */
+int mgn_attn_bwd(const void* q, const void* k, const void* v, const void* o, const void* d_o,
+                 const float* lse, void* dq, void* dk, void* dv,
+                 void* workspace, size_t workspace_bytes,
+                 int B, int H, int S, int D, int causal, float scale, int mode, void* stream);
+
+/* Bytes of workspace mgn_attn_bwd needs for these sizes; 0 if the arguments are invalid. */
+size_t mgn_attn_bwd_workspace_bytes(int B, int H, int S, int D, int mode);
+
+/*
+ * Synchronises `stream`, then reads and clears the device-side status word that
+ * kernels set when one of their bounded waits (TMA / tensor-core completion
+ * barriers) ran out.  Returns MGN_OK, MGN_ERR_DEVICE_TIMEOUT or MGN_ERR_CUDA.
+ * (Library plumbing; the paper has no counterpart.)
+ */
+int mgn_attn_check(void* stream);
+
+/*
+ * Measurement hook (library plumbing; the paper has no counterpart).  While both
+ * arguments are non-null cudaEvent_t handles, every later mgn_attn_fwd / mgn_attn_bwd
+ * call records `before_main` on its stream immediately before its main kernel (the
+ * forward kernel, or the fused dK/dV/dQ kernel) and `after_main` immediately after it,
+ * so a benchmark can time that kernel alone inside a whole-call timed region.  Pass
+ * two nulls to switch it off.  Process-wide state: meant for single-threaded
+ * benchmarks only.  Returns MGN_OK, or MGN_ERR_INVALID_ARG if exactly one is null.
+ */
+int mgn_attn_profile_events(void* before_main, void* after_main);
+
+/* Static string naming a status code. */
+const char* mgn_status_string(int status);
+
+/* Library version: major*10000 + minor*100 + patch. */
+int mgn_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MGN_ATTN_H */

@@ -1,0 +1,121 @@
+"""Thin ctypes binding of ``libmgn_attn.so``: argument marshalling only.
+
+Every function mirrors the C entry point of the same name (``include/mgn_attn.h``),
+takes torch CUDA tensors for the device buffers and enqueues on the current torch
+stream unless ``stream`` (a raw ``cudaStream_t`` integer) is given.  There is no
+fallback: if the library has not been built the first call raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+MODE_STRICT_F32 = 0
+MODE_FAST_BF16 = 1
+
+MGN_OK = 0
+STATUS_NAMES = {
+    0: "MGN_OK", 1: "MGN_ERR_INVALID_ARG", 2: "MGN_ERR_UNSUPPORTED", 3: "MGN_ERR_MISALIGNED",
+    4: "MGN_ERR_WORKSPACE", 5: "MGN_ERR_CUDA", 6: "MGN_ERR_ARCH", 7: "MGN_ERR_DEVICE_TIMEOUT",
+}
+
+LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libmgn_attn.so")
+_lib = None
+
+
+class MgnError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        super().__init__(f"{where} failed: {STATUS_NAMES.get(status, status)}")
+        self.status = status
+
+
+def lib() -> ctypes.CDLL:
+    """Loads the CUDA library; raises if it is missing (no CPU or eager fallback exists)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_2608_01563_b200.build`")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, i, f, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_float, ctypes.c_size_t
+        L.mgn_attn_fwd.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, i, f, i, vp]
+        L.mgn_attn_fwd.restype = i
+        L.mgn_attn_bwd.argtypes = [vp] * 9 + [vp, sz, i, i, i, i, i, f, i, vp]
+        L.mgn_attn_bwd.restype = i
+        L.mgn_attn_bwd_workspace_bytes.argtypes = [i, i, i, i, i]
+        L.mgn_attn_bwd_workspace_bytes.restype = sz
+        L.mgn_attn_check.argtypes = [vp]
+        L.mgn_attn_check.restype = i
+        L.mgn_attn_profile_events.argtypes = [vp, vp]
+        L.mgn_attn_profile_events.restype = i
+        L.mgn_status_string.argtypes = [i]
+        L.mgn_status_string.restype = ctypes.c_char_p
+        L.mgn_version.argtypes = []
+        L.mgn_version.restype = i
+        _lib = L
+    return _lib
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    return None if t is None else t.data_ptr()
+
+
+def _stream(stream: Optional[int]) -> Optional[int]:
+    if stream is not None:
+        return stream
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _dims(q: torch.Tensor):
+    B, H, S, D = q.shape
+    return int(B), int(H), int(S), int(D)
+
+
+def mgn_attn_fwd(q, k, v, o, lse, causal: bool, scale: float, mode: int, stream: Optional[int] = None) -> None:
+    B, H, S, D = _dims(q)
+    st = lib().mgn_attn_fwd(_ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse), B, H, S, D,
+                            int(causal), float(scale), int(mode), _stream(stream))
+    if st != MGN_OK:
+        raise MgnError(st, "mgn_attn_fwd")
+
+
+def mgn_attn_bwd_workspace_bytes(B: int, H: int, S: int, D: int, mode: int) -> int:
+    return int(lib().mgn_attn_bwd_workspace_bytes(B, H, S, D, mode))
+
+
+def mgn_attn_bwd(q, k, v, o, d_o, lse, dq, dk, dv, workspace, causal: bool, scale: float, mode: int,
+                 stream: Optional[int] = None) -> None:
+    B, H, S, D = _dims(q)
+    st = lib().mgn_attn_bwd(_ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(d_o), _ptr(lse), _ptr(dq), _ptr(dk),
+                            _ptr(dv), _ptr(workspace), workspace.numel() * workspace.element_size(),
+                            B, H, S, D, int(causal), float(scale), int(mode), _stream(stream))
+    if st != MGN_OK:
+        raise MgnError(st, "mgn_attn_bwd")
+
+
+def mgn_attn_check(stream: Optional[int] = None) -> None:
+    st = lib().mgn_attn_check(_stream(stream))
+    if st != MGN_OK:
+        raise MgnError(st, "mgn_attn_check")
+
+
+def mgn_attn_profile_events(before_main: Optional[int], after_main: Optional[int]) -> None:
+    st = lib().mgn_attn_profile_events(before_main, after_main)
+    if st != MGN_OK:
+        raise MgnError(st, "mgn_attn_profile_events")
+
+
+def mgn_status_string(status: int) -> str:
+    return lib().mgn_status_string(int(status)).decode()
+
+
+def mgn_version() -> int:
+    return int(lib().mgn_version())
+
+
+def alloc_workspace(B: int, H: int, S: int, D: int, mode: int, device="cuda") -> torch.Tensor:
+    """Convenience: a uint8 device buffer of the size mgn_attn_bwd needs (256-byte aligned by torch)."""
+    return torch.empty(mgn_attn_bwd_workspace_bytes(B, H, S, D, mode), dtype=torch.uint8, device=device)

@@ -1,0 +1,188 @@
+// C ABI of the attention library: argument validation, workspace layout, dispatch.
+#include <math.h>
+#include <stdint.h>
+
+#include <mutex>
+
+#include "../../include/mgn_attn.h"
+#include "kernels.h"
+
+namespace {
+
+// Device status word set by kernels whose bounded waits ran out.
+__device__ unsigned g_mgn_status;
+
+constexpr int kMaxDevices = 64;
+unsigned* g_status_ptr[kMaxDevices];
+int g_arch_ok[kMaxDevices];   // 0 unknown, 1 ok, -1 wrong arch
+std::mutex g_mu;
+
+cudaEvent_t g_ev_before = nullptr, g_ev_after = nullptr;
+
+struct MainKernelTimer {
+    cudaStream_t st;
+    explicit MainKernelTimer(cudaStream_t s) : st(s) { if (g_ev_before) cudaEventRecord(g_ev_before, st); }
+    ~MainKernelTimer() { if (g_ev_after) cudaEventRecord(g_ev_after, st); }
+};
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int check_common(int B, int H, int S, int D, int causal, float scale, int mode)
+{
+    if (B <= 0 || H <= 0 || S <= 0 || D <= 0) return MGN_ERR_INVALID_ARG;
+    if (causal != 0 && causal != 1) return MGN_ERR_INVALID_ARG;
+    if (!isfinite(scale)) return MGN_ERR_INVALID_ARG;
+    if (mode != MGN_MODE_STRICT_F32 && mode != MGN_MODE_FAST_BF16) return MGN_ERR_INVALID_ARG;
+    if (D != 32 && D != 64 && D != 128) return MGN_ERR_UNSUPPORTED;
+    const long long bh = static_cast<long long>(B) * H;
+    if (bh > 0x7fffffffLL) return MGN_ERR_UNSUPPORTED;
+    if (S > (1 << 24)) return MGN_ERR_UNSUPPORTED;
+    // grid and byte-offset plan: tiles*BH must fit an int, element counts must fit 2^40
+    if (bh * ((S + 63) / 64) > 0x7fffffffLL) return MGN_ERR_UNSUPPORTED;
+    if (static_cast<double>(bh) * S * D > 1.0e12) return MGN_ERR_UNSUPPORTED;
+    return MGN_OK;
+}
+
+// Per-device set-up: architecture check and the address of the status word.
+int device_setup(unsigned** status)
+{
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return MGN_ERR_CUDA;
+    if (dev < 0 || dev >= kMaxDevices) return MGN_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(g_mu);
+    if (g_arch_ok[dev] == 0) {
+        int major = 0;
+        if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return MGN_ERR_CUDA;
+        if (major != 10) { g_arch_ok[dev] = -1; return MGN_ERR_ARCH; }
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_mgn_status) != cudaSuccess) { cudaGetLastError(); return MGN_ERR_CUDA; }
+        g_status_ptr[dev] = static_cast<unsigned*>(p);
+        g_arch_ok[dev] = 1;
+    }
+    if (g_arch_ok[dev] < 0) return MGN_ERR_ARCH;
+    *status = g_status_ptr[dev];
+    return MGN_OK;
+}
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// Workspace layout: [delta: BH*S f32][fast mode only: dQ accumulator BH*S*D f32], 256-byte granules.
+size_t ws_delta_bytes(size_t rows) { return align_up(rows * sizeof(float), 256); }
+
+}  // namespace
+
+extern "C" {
+
+size_t mgn_attn_bwd_workspace_bytes(int B, int H, int S, int D, int mode)
+{
+    if (check_common(B, H, S, D, 0, 1.0f, mode) != MGN_OK) return 0;
+    const size_t rows = static_cast<size_t>(B) * H * S;
+    size_t bytes = ws_delta_bytes(rows);
+    if (mode == MGN_MODE_FAST_BF16) bytes += align_up(rows * D * sizeof(float), 256);
+    return bytes;
+}
+
+int mgn_attn_fwd(const void* q, const void* k, const void* v, void* o, float* lse,
+                 int B, int H, int S, int D, int causal, float scale, int mode, void* stream)
+{
+    if (!q || !k || !v || !o || !lse) return MGN_ERR_INVALID_ARG;
+    if (int r = check_common(B, H, S, D, causal, scale, mode)) return r;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(lse)) return MGN_ERR_MISALIGNED;
+    unsigned* status = nullptr;
+    if (int r = device_setup(&status)) return r;
+    const mgn::Problem p{B * H, S, D, causal, scale};
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e;
+    MainKernelTimer timer(st);
+    if (mode == MGN_MODE_STRICT_F32)
+        e = mgn::launch_strict_fwd(p, static_cast<const float*>(q), static_cast<const float*>(k),
+                                   static_cast<const float*>(v), static_cast<float*>(o), lse, status, st);
+    else
+        e = mgn::launch_fast_fwd(p, q, k, v, o, lse, status, st);
+    return e == cudaSuccess ? MGN_OK : MGN_ERR_CUDA;
+}
+
+int mgn_attn_bwd(const void* q, const void* k, const void* v, const void* o, const void* d_o,
+                 const float* lse, void* dq, void* dk, void* dv,
+                 void* workspace, size_t workspace_bytes,
+                 int B, int H, int S, int D, int causal, float scale, int mode, void* stream)
+{
+    if (!q || !k || !v || !o || !d_o || !lse || !dq || !dk || !dv) return MGN_ERR_INVALID_ARG;
+    if (int r = check_common(B, H, S, D, causal, scale, mode)) return r;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(d_o) || !aligned16(lse) ||
+        !aligned16(dq) || !aligned16(dk) || !aligned16(dv))
+        return MGN_ERR_MISALIGNED;
+    const size_t need = mgn_attn_bwd_workspace_bytes(B, H, S, D, mode);
+    if (!workspace || workspace_bytes < need) return MGN_ERR_WORKSPACE;
+    if (reinterpret_cast<uintptr_t>(workspace) & 255u) return MGN_ERR_WORKSPACE;
+    unsigned* status = nullptr;
+    if (int r = device_setup(&status)) return r;
+
+    const mgn::Problem p{B * H, S, D, causal, scale};
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t rows = static_cast<size_t>(B) * H * S;
+    float* delta = static_cast<float*>(workspace);
+    const bool fast = mode == MGN_MODE_FAST_BF16;
+
+    cudaError_t e = mgn::launch_bwd_preprocess(o, d_o, delta, rows, D, fast ? 1 : 0, st);
+    if (e != cudaSuccess) return MGN_ERR_CUDA;
+    if (!fast) {
+        // dQ is accumulated in place by floating-point reductions: start from zero.
+        e = cudaMemsetAsync(dq, 0, rows * D * sizeof(float), st);
+        if (e != cudaSuccess) return MGN_ERR_CUDA;
+        MainKernelTimer timer(st);
+        e = mgn::launch_strict_bwd(p, static_cast<const float*>(q), static_cast<const float*>(k),
+                                   static_cast<const float*>(v), static_cast<const float*>(d_o), lse, delta,
+                                   static_cast<float*>(dq), static_cast<float*>(dk), static_cast<float*>(dv), status,
+                                   st);
+    } else {
+        float* dq_acc = reinterpret_cast<float*>(static_cast<char*>(workspace) + ws_delta_bytes(rows));
+        e = cudaMemsetAsync(dq_acc, 0, rows * D * sizeof(float), st);
+        if (e != cudaSuccess) return MGN_ERR_CUDA;
+        MainKernelTimer timer(st);
+        e = mgn::launch_fast_bwd(p, q, k, v, d_o, lse, delta, dq_acc, dq, dk, dv, status, st);
+    }
+    return e == cudaSuccess ? MGN_OK : MGN_ERR_CUDA;
+}
+
+int mgn_attn_check(void* stream)
+{
+    unsigned* status = nullptr;
+    if (int r = device_setup(&status)) return r;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (cudaStreamSynchronize(st) != cudaSuccess) return MGN_ERR_CUDA;
+    unsigned h = 0;
+    if (cudaMemcpy(&h, status, sizeof(h), cudaMemcpyDeviceToHost) != cudaSuccess) return MGN_ERR_CUDA;
+    if (h != 0) {
+        cudaMemset(status, 0, sizeof(h));
+        return MGN_ERR_DEVICE_TIMEOUT;
+    }
+    return MGN_OK;
+}
+
+int mgn_attn_profile_events(void* before_main, void* after_main)
+{
+    if ((before_main == nullptr) != (after_main == nullptr)) return MGN_ERR_INVALID_ARG;
+    g_ev_before = static_cast<cudaEvent_t>(before_main);
+    g_ev_after = static_cast<cudaEvent_t>(after_main);
+    return MGN_OK;
+}
+
+const char* mgn_status_string(int status)
+{
+    switch (status) {
+        case MGN_OK: return "MGN_OK";
+        case MGN_ERR_INVALID_ARG: return "MGN_ERR_INVALID_ARG";
+        case MGN_ERR_UNSUPPORTED: return "MGN_ERR_UNSUPPORTED";
+        case MGN_ERR_MISALIGNED: return "MGN_ERR_MISALIGNED";
+        case MGN_ERR_WORKSPACE: return "MGN_ERR_WORKSPACE";
+        case MGN_ERR_CUDA: return "MGN_ERR_CUDA";
+        case MGN_ERR_ARCH: return "MGN_ERR_ARCH";
+        case MGN_ERR_DEVICE_TIMEOUT: return "MGN_ERR_DEVICE_TIMEOUT";
+        default: return "MGN_ERR_UNKNOWN";
+    }
+}
+
+int mgn_version(void) { return 100; }
+
+}  // extern "C"

@@ -1,0 +1,81 @@
+// Backward preprocess: delta_i = sum_d dO[i,d] * O[i,d] for every (b,h,i) row.
+// HBM-bound streaming kernel: 128-bit loads, D/4 (f32) or D/8 (bf16) lanes per row,
+// shuffle reduction inside the lane group.  (The paper's backward kernels need this
+// row statistic; it is the "backward preprocess" step of the attention path.)
+#include <cuda_bf16.h>
+
+#include "kernels.h"
+
+namespace mgn {
+namespace {
+
+template <int LANES, bool BF16>
+__global__ void __launch_bounds__(256)
+bwd_preprocess_kernel(const uint4* __restrict__ o, const uint4* __restrict__ d_o, float* __restrict__ delta, size_t rows)
+{
+    constexpr int ROWS_PER_BLOCK = 256 / LANES;
+    const int lane = threadIdx.x % LANES;
+    const int sub = threadIdx.x / LANES;
+    for (size_t r0 = static_cast<size_t>(blockIdx.x) * ROWS_PER_BLOCK; r0 < rows;
+         r0 += static_cast<size_t>(gridDim.x) * ROWS_PER_BLOCK) {
+        const size_t r = r0 + sub;
+        float acc = 0.f;
+        if (r < rows) {
+            const uint4 a = __ldg(o + r * LANES + lane);
+            const uint4 b = __ldg(d_o + r * LANES + lane);
+            if constexpr (BF16) {
+                const __nv_bfloat162* pa = reinterpret_cast<const __nv_bfloat162*>(&a);
+                const __nv_bfloat162* pb = reinterpret_cast<const __nv_bfloat162*>(&b);
+#pragma unroll
+                for (int t = 0; t < 4; ++t) {
+                    const float2 fa = __bfloat1622float2(pa[t]), fb = __bfloat1622float2(pb[t]);
+                    acc = fmaf(fa.x, fb.x, acc);
+                    acc = fmaf(fa.y, fb.y, acc);
+                }
+            } else {
+                acc = fmaf(__uint_as_float(a.x), __uint_as_float(b.x), acc);
+                acc = fmaf(__uint_as_float(a.y), __uint_as_float(b.y), acc);
+                acc = fmaf(__uint_as_float(a.z), __uint_as_float(b.z), acc);
+                acc = fmaf(__uint_as_float(a.w), __uint_as_float(b.w), acc);
+            }
+        }
+#pragma unroll
+        for (int off = LANES / 2; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+        if (r < rows && lane == 0) delta[r] = acc;
+    }
+}
+
+template <int LANES, bool BF16>
+cudaError_t run(const void* o, const void* d_o, float* delta, size_t rows, cudaStream_t st)
+{
+    constexpr int ROWS_PER_BLOCK = 256 / LANES;
+    size_t blocks = (rows + ROWS_PER_BLOCK - 1) / ROWS_PER_BLOCK;
+    const size_t cap = 148u * 8u * 4u;
+    if (blocks > cap) blocks = cap;
+    bwd_preprocess_kernel<LANES, BF16><<<static_cast<unsigned>(blocks), 256, 0, st>>>(
+        static_cast<const uint4*>(o), static_cast<const uint4*>(d_o), delta, rows);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_bwd_preprocess(const void* o, const void* d_o, float* delta, size_t rows, int D, int is_bf16,
+                                  cudaStream_t st)
+{
+    if (is_bf16) {
+        switch (D) {
+            case 32:  return run<4, true>(o, d_o, delta, rows, st);
+            case 64:  return run<8, true>(o, d_o, delta, rows, st);
+            case 128: return run<16, true>(o, d_o, delta, rows, st);
+        }
+    } else {
+        switch (D) {
+            case 32:  return run<8, false>(o, d_o, delta, rows, st);
+            case 64:  return run<16, false>(o, d_o, delta, rows, st);
+            case 128: return run<32, false>(o, d_o, delta, rows, st);
+        }
+    }
+    return cudaErrorInvalidValue;
+}
+
+}  // namespace mgn

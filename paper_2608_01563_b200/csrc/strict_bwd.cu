@@ -1,0 +1,339 @@
+// Strict-mode attention backward: f32 storage, f32 FFMA arithmetic (paper Section 3.3,
+// "dQ, and fused dK+dV kernels"; Section 7.3 names them FlashGradQ and FlashGradKV).
+//
+// Single pass: one CTA (256 threads) keeps one BN-key tile of K and V resident, holds
+// the dK and dV accumulators of that tile in registers, and walks over the BM-row query
+// tiles.  For each (query tile, key tile) pair it
+//   A. recomputes S = Q K^T and computes dP = dO V^T in one fused loop over d,
+//      forms P = exp(S - LSE) and dS = P o (dP - delta) in registers, and writes P and dS
+//      to shared memory (row-major [i][j]),
+//   B. accumulates dV += P^T dO and dK += dS^T Q (contraction over query rows),
+//   C. forms the partial dQ = dS K of this pair and adds it to global dQ with 128-bit
+//      floating-point reductions (the "atomic accumulation" variant of the dQ kernel),
+// so exactly the five counted matrix products are executed.  Tiles arrive by TMA in the
+// swizzled layout described in strict_fwd.cu.
+#include "kernels.h"
+#include "ptx.cuh"
+
+namespace mgn {
+namespace {
+
+constexpr int kThreads = 256;
+constexpr float kLog2e = 1.4426950408889634f;
+
+template <int D, int BM, int BN>
+struct BwdCfg {
+    static constexpr int RM = BM / 16;   // query rows per thread (phases A, C)
+    static constexpr int RN = BN / 16;   // key columns per thread (phase A)
+    static constexpr int JN = BN / 16;   // key rows per thread (phase B), groups of 4 contiguous
+    static constexpr int DV = D / 16;    // d columns per thread (phases B, C)
+    static constexpr int NCH = D / 32;
+    static constexpr int PSTR = BN + 4;
+    static constexpr int KV_BYTES = BN * D * 4;
+    static constexpr int Q_BYTES = BM * D * 4;
+    static constexpr int P_BYTES = BM * PSTR * 4;
+    static constexpr int SMEM = 2 * KV_BYTES + 2 * Q_BYTES + 2 * P_BYTES + 64 + 1024;
+    static_assert(JN % 4 == 0, "key rows per thread come in float4 groups");
+};
+
+// d columns owned by column group tc: D=32 -> {2tc, 2tc+1}; else {4tc + 64e + 0..3}.
+template <int D, int R>
+__device__ __forceinline__ void load_row_cols(uint32_t tile, int r, int r7, int tc, float (&out)[D / 16]) {
+    if constexpr (D == 32) {
+        const float2 t = lds64(tile + r * 128 + (((tc >> 1) ^ r7) << 4) + (tc & 1) * 8);
+        out[0] = t.x; out[1] = t.y;
+    } else {
+#pragma unroll
+        for (int e = 0; e < D / 64; ++e) {
+            const int piece = tc + 16 * e;
+            const float4 t = lds128(tile + (piece >> 3) * (R * 128) + r * 128 + (((piece & 7) ^ r7) << 4));
+            out[4 * e + 0] = t.x; out[4 * e + 1] = t.y; out[4 * e + 2] = t.z; out[4 * e + 3] = t.w;
+        }
+    }
+}
+
+__device__ __forceinline__ float f4_get(const float4& v, int u) {
+    return u == 0 ? v.x : u == 1 ? v.y : u == 2 ? v.z : v.w;
+}
+
+template <int D, int BM, int BN>
+__global__ void __launch_bounds__(kThreads, 1)
+strict_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+                  const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmdO,
+                  const float* __restrict__ LSE, const float* __restrict__ DELTA,
+                  float* __restrict__ dQ, float* __restrict__ dK, float* __restrict__ dV,
+                  int S, int BH, int n_qt, int causal, float scale, unsigned* status)
+{
+    using C = BwdCfg<D, BM, BN>;
+    constexpr int RM = C::RM, RN = C::RN, JN = C::JN, DV = C::DV, NCH = C::NCH, PSTR = C::PSTR;
+
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t sK = base;
+    const uint32_t sV = sK + C::KV_BYTES;
+    const uint32_t sQ = sV + C::KV_BYTES;
+    const uint32_t sdO = sQ + C::Q_BYTES;
+    const uint32_t sP = sdO + C::Q_BYTES;
+    const uint32_t sdS = sP + C::P_BYTES;
+    const uint32_t barKV = sdS + C::P_BYTES, barQ = barKV + 8;
+
+    const int tid = threadIdx.x;
+    const int tr = 2 * (tid >> 5) + ((tid & 31) >> 4);   // 0..15
+    const int tc = tid & 15;                             // 0..15
+
+    // Heaviest key tiles (lowest j0) first when causal.
+    const int kt = static_cast<int>(blockIdx.x) / BH;
+    const int bh = static_cast<int>(blockIdx.x) % BH;
+    const int j0 = kt * BN;
+    const int qt0 = causal ? (j0 / BM) : 0;
+    const float c2 = scale * kLog2e;
+
+    if (tid == 0) {
+        mbar_init(barKV, 1);
+        mbar_init(barQ, 1);
+        fence_mbar_init();
+    }
+    __syncthreads();
+    if (tid == 0) {
+        mbar_arrive_expect_tx(barKV, 2 * C::KV_BYTES);
+#pragma unroll
+        for (int ch = 0; ch < NCH; ++ch) {
+            tma_load_3d(sK + ch * BN * 128, &tmK, barKV, ch * 32, j0, bh);
+            tma_load_3d(sV + ch * BN * 128, &tmV, barKV, ch * 32, j0, bh);
+        }
+        mbar_arrive_expect_tx(barQ, 2 * C::Q_BYTES);
+#pragma unroll
+        for (int ch = 0; ch < NCH; ++ch) {
+            tma_load_3d(sQ + ch * BM * 128, &tmQ, barQ, ch * 32, qt0 * BM, bh);
+            tma_load_3d(sdO + ch * BM * 128, &tmdO, barQ, ch * 32, qt0 * BM, bh);
+        }
+    }
+
+    float dk[JN][DV], dv[JN][DV];
+#pragma unroll
+    for (int a = 0; a < JN; ++a)
+#pragma unroll
+        for (int e = 0; e < DV; ++e) { dk[a][e] = 0.f; dv[a][e] = 0.f; }
+
+    mbar_wait(barKV, 0, status);
+
+    for (int qt = qt0; qt < n_qt; ++qt) {
+        const int i0 = qt * BM;
+        const uint32_t ph = (qt - qt0) & 1;
+
+        // row statistics of this thread's query rows (rows past S: P = 0 via lse = +inf)
+        float lse2[RM], dl[RM];
+#pragma unroll
+        for (int x = 0; x < RM; ++x) {
+            const int i = i0 + tr + 16 * x;
+            const bool ok = i < S;
+            lse2[x] = ok ? LSE[static_cast<size_t>(bh) * S + i] * kLog2e : INFINITY;
+            dl[x] = ok ? DELTA[static_cast<size_t>(bh) * S + i] : 0.f;
+        }
+
+        mbar_wait(barQ, ph, status);
+
+        // ---- A: S = Q K^T and dP = dO V^T, fused over d ---------------------------------------
+        float s[RM][RN], dp[RM][RN];
+#pragma unroll
+        for (int x = 0; x < RM; ++x)
+#pragma unroll
+            for (int y = 0; y < RN; ++y) { s[x][y] = 0.f; dp[x][y] = 0.f; }
+        {
+            const int xq = tr & 7, xk = tc & 7;
+#pragma unroll
+            for (int pc = 0; pc < D / 4; ++pc) {
+                const uint32_t oq = (pc >> 3) * (BM * 128) + tr * 128 + (((pc & 7) ^ xq) << 4);
+                const uint32_t ok = (pc >> 3) * (BN * 128) + tc * 128 + (((pc & 7) ^ xk) << 4);
+                float4 bk[RN], bv[RN];
+#pragma unroll
+                for (int y = 0; y < RN; ++y) {
+                    bk[y] = lds128(sK + ok + y * 16 * 128);
+                    bv[y] = lds128(sV + ok + y * 16 * 128);
+                }
+#pragma unroll
+                for (int x = 0; x < RM; ++x) {
+                    const float4 aq = lds128(sQ + oq + x * 16 * 128);
+                    const float4 ad = lds128(sdO + oq + x * 16 * 128);
+#pragma unroll
+                    for (int y = 0; y < RN; ++y) {
+                        s[x][y] = fmaf(aq.x, bk[y].x, s[x][y]);
+                        s[x][y] = fmaf(aq.y, bk[y].y, s[x][y]);
+                        s[x][y] = fmaf(aq.z, bk[y].z, s[x][y]);
+                        s[x][y] = fmaf(aq.w, bk[y].w, s[x][y]);
+                        dp[x][y] = fmaf(ad.x, bv[y].x, dp[x][y]);
+                        dp[x][y] = fmaf(ad.y, bv[y].y, dp[x][y]);
+                        dp[x][y] = fmaf(ad.z, bv[y].z, dp[x][y]);
+                        dp[x][y] = fmaf(ad.w, bv[y].w, dp[x][y]);
+                    }
+                }
+            }
+        }
+        __syncthreads();   // phase C of the previous pair has finished reading dS
+        {
+            const bool need_mask = (causal && (j0 + BN - 1 > i0)) || (j0 + BN > S);
+#pragma unroll
+            for (int x = 0; x < RM; ++x) {
+                const int i = i0 + tr + 16 * x;
+                const uint32_t row = ((tr + 16 * x) * PSTR + tc) * 4;
+#pragma unroll
+                for (int y = 0; y < RN; ++y) {
+                    float p = ex2(fmaf(s[x][y], c2, -lse2[x]));
+                    if (need_mask) {
+                        const int j = j0 + tc + 16 * y;
+                        if (j >= S || (causal && j > i)) p = 0.f;
+                    }
+                    const float ds = p * (dp[x][y] - dl[x]);
+                    sts32(sP + row + y * 64, p);
+                    sts32(sdS + row + y * 64, ds);
+                }
+            }
+        }
+        __syncthreads();   // P, dS visible
+
+        // ---- B: dV += P^T dO, dK += dS^T Q : contraction over the query rows ---------------
+        {
+            // this thread's key rows: j = 4*tr + 64*g + u, g < JN/4, u < 4
+#pragma unroll 1
+            for (int i8 = 0; i8 < BM; i8 += 8)
+#pragma unroll
+            for (int iu = 0; iu < 8; ++iu) {
+                const int i = i8 + iu;
+                float dov[DV], qv[DV];
+                load_row_cols<D, BM>(sdO, i, iu, tc, dov);
+                load_row_cols<D, BM>(sQ, i, iu, tc, qv);
+#pragma unroll
+                for (int g = 0; g < JN / 4; ++g) {
+                    const float4 p4 = lds128(sP + (i * PSTR + 4 * tr + 64 * g) * 4);
+                    const float4 d4 = lds128(sdS + (i * PSTR + 4 * tr + 64 * g) * 4);
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const float pj = f4_get(p4, u), dj = f4_get(d4, u);
+#pragma unroll
+                        for (int e = 0; e < DV; ++e) {
+                            dv[4 * g + u][e] = fmaf(pj, dov[e], dv[4 * g + u][e]);
+                            dk[4 * g + u][e] = fmaf(dj, qv[e], dk[4 * g + u][e]);
+                        }
+                    }
+                }
+            }
+        }
+        __syncthreads();   // Q and dO tiles are free
+        if (tid == 0 && qt + 1 < n_qt) {
+            mbar_arrive_expect_tx(barQ, 2 * C::Q_BYTES);
+#pragma unroll
+            for (int ch = 0; ch < NCH; ++ch) {
+                tma_load_3d(sQ + ch * BM * 128, &tmQ, barQ, ch * 32, i0 + BM, bh);
+                tma_load_3d(sdO + ch * BM * 128, &tmdO, barQ, ch * 32, i0 + BM, bh);
+            }
+        }
+
+        // ---- C: dQ partial = dS K : contraction over keys, reduced into global dQ ----------
+        {
+            float dq[RM][DV];
+#pragma unroll
+            for (int x = 0; x < RM; ++x)
+#pragma unroll
+                for (int e = 0; e < DV; ++e) dq[x][e] = 0.f;
+#pragma unroll 2
+            for (int j8 = 0; j8 < BN / 8; ++j8) {
+                float4 d4[2][RM];
+#pragma unroll
+                for (int hlf = 0; hlf < 2; ++hlf)
+#pragma unroll
+                    for (int x = 0; x < RM; ++x)
+                        d4[hlf][x] = lds128(sdS + ((tr + 16 * x) * PSTR + j8 * 8 + hlf * 4) * 4);
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    float kv[DV];
+                    load_row_cols<D, BN>(sK, j8 * 8 + u, u, tc, kv);
+#pragma unroll
+                    for (int x = 0; x < RM; ++x) {
+                        const float dsv = f4_get(d4[u >> 2][x], u & 3);
+#pragma unroll
+                        for (int e = 0; e < DV; ++e) dq[x][e] = fmaf(dsv, kv[e], dq[x][e]);
+                    }
+                }
+            }
+#pragma unroll
+            for (int x = 0; x < RM; ++x) {
+                const int i = i0 + tr + 16 * x;
+                if (i < S) {
+                    float* row = dQ + (static_cast<size_t>(bh) * S + i) * D;
+                    if constexpr (DV == 2) {
+                        red_add_v2(row + 2 * tc, dq[x][0] * scale, dq[x][1] * scale);
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < DV / 4; ++e)
+                            red_add_v4(row + 4 * tc + 64 * e, dq[x][4 * e] * scale, dq[x][4 * e + 1] * scale,
+                                       dq[x][4 * e + 2] * scale, dq[x][4 * e + 3] * scale);
+                    }
+                }
+            }
+        }
+    }
+
+    // ---- epilogue: dK (scaled) and dV of this key tile ----------------------------------------
+#pragma unroll
+    for (int g = 0; g < JN / 4; ++g)
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int j = j0 + 4 * tr + 64 * g + u;
+            if (j < S) {
+                const size_t off = (static_cast<size_t>(bh) * S + j) * D;
+                const int a = 4 * g + u;
+                if constexpr (DV == 2) {
+                    *reinterpret_cast<float2*>(dK + off + 2 * tc) = make_float2(dk[a][0] * scale, dk[a][1] * scale);
+                    *reinterpret_cast<float2*>(dV + off + 2 * tc) = make_float2(dv[a][0], dv[a][1]);
+                } else {
+#pragma unroll
+                    for (int e = 0; e < DV / 4; ++e) {
+                        *reinterpret_cast<float4*>(dK + off + 4 * tc + 64 * e) =
+                            make_float4(dk[a][4 * e] * scale, dk[a][4 * e + 1] * scale, dk[a][4 * e + 2] * scale,
+                                        dk[a][4 * e + 3] * scale);
+                        *reinterpret_cast<float4*>(dV + off + 4 * tc + 64 * e) =
+                            make_float4(dv[a][4 * e], dv[a][4 * e + 1], dv[a][4 * e + 2], dv[a][4 * e + 3]);
+                    }
+                }
+            }
+        }
+}
+
+template <int D, int BM, int BN>
+cudaError_t launch(const Problem& p, const float* q, const float* k, const float* v, const float* d_o,
+                   const float* lse, const float* delta, float* dq, float* dk, float* dv, unsigned* status,
+                   cudaStream_t st)
+{
+    using C = BwdCfg<D, BM, BN>;
+    CUtensorMap tq, tk, tv, tdo;
+    if (make_tmap_3d(&tq, q, 4, 0, p.BH, p.S, D, 32, BM)) return cudaErrorInvalidValue;
+    if (make_tmap_3d(&tdo, d_o, 4, 0, p.BH, p.S, D, 32, BM)) return cudaErrorInvalidValue;
+    if (make_tmap_3d(&tk, k, 4, 0, p.BH, p.S, D, 32, BN)) return cudaErrorInvalidValue;
+    if (make_tmap_3d(&tv, v, 4, 0, p.BH, p.S, D, 32, BN)) return cudaErrorInvalidValue;
+    auto kern = strict_bwd_kernel<D, BM, BN>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM);
+    if (e != cudaSuccess) return e;
+    const int n_qt = (p.S + BM - 1) / BM;
+    const int n_kt = (p.S + BN - 1) / BN;
+    const long long blocks = static_cast<long long>(n_kt) * p.BH;
+    if (blocks > 0x7fffffffLL) return cudaErrorInvalidValue;
+    kern<<<static_cast<unsigned>(blocks), kThreads, C::SMEM, st>>>(tq, tk, tv, tdo, lse, delta, dq, dk, dv, p.S, p.BH,
+                                                                   n_qt, p.causal, p.scale, status);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_strict_bwd(const Problem& p, const float* q, const float* k, const float* v,
+                              const float* d_o, const float* lse, const float* delta,
+                              float* dq, float* dk, float* dv, unsigned* status, cudaStream_t st)
+{
+    switch (p.D) {
+        case 32:  return launch<32, 64, 128>(p, q, k, v, d_o, lse, delta, dq, dk, dv, status, st);
+        case 64:  return launch<64, 64, 128>(p, q, k, v, d_o, lse, delta, dq, dk, dv, status, st);
+        case 128: return launch<128, 64, 64>(p, q, k, v, d_o, lse, delta, dq, dk, dv, status, st);
+        default:  return cudaErrorInvalidValue;
+    }
+}
+
+}  // namespace mgn

@@ -1,0 +1,283 @@
+// Strict-mode attention forward: f32 storage, f32 FFMA arithmetic (paper Section 3.3,
+// "tiled attention forward"; Section 4.2 strict arithmetic contract).
+//
+// One CTA (256 threads) owns BM query rows of one head and streams BN-key tiles of
+// K and V through shared memory with TMA.  Scores live in registers (each thread an
+// (BM/16)x(BN/16) micro-tile), the softmax is the online form (running row max in
+// the log2 domain, thread-local partial row sums), P goes through shared memory
+// once to become the A operand of O += P V.
+//
+// Shared-memory tile layout (as TMA writes it with the 128-byte swizzle): a tile of
+// R rows x D floats is stored as D/32 chunks; chunk c holds, for every row, the 32
+// floats [32c, 32c+32) in a 128-byte line, lines at 128-byte pitch, and the 16-byte
+// piece p of row r sits at piece position p ^ (r & 7).  Rows that a warp reads in one
+// instruction are consecutive modulo 8, so every 128-bit shared load is conflict free.
+#include "kernels.h"
+#include "ptx.cuh"
+
+namespace mgn {
+namespace {
+
+constexpr int kThreads = 256;
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+
+template <int D, int BM, int BN>
+struct FwdCfg {
+    static constexpr int RM = BM / 16;    // query rows per thread
+    static constexpr int RN = BN / 16;    // key columns per thread
+    static constexpr int DV = D / 16;     // output columns per thread
+    static constexpr int NCH = D / 32;    // 128-byte chunks per row
+    static constexpr int PSTR = BN + 4;   // padded row stride of P (floats)
+    static constexpr int Q_BYTES = BM * D * 4;
+    static constexpr int KV_BYTES = BN * D * 4;
+    static constexpr int P_BYTES = BM * PSTR * 4;
+    static constexpr int SMEM = Q_BYTES + 2 * KV_BYTES + P_BYTES + 64 + 1024;
+};
+
+// Byte offset of the 16-byte piece `piece` (0..D/4-1) of row `r` in a swizzled tile of R rows.
+template <int R>
+__device__ __forceinline__ uint32_t tile_off(int r, int piece) {
+    return static_cast<uint32_t>((piece >> 3) * (R * 128) + r * 128 + (((piece & 7) ^ (r & 7)) << 4));
+}
+
+template <int D, int BM, int BN>
+__global__ void __launch_bounds__(kThreads, 1)
+strict_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+                  const __grid_constant__ CUtensorMap tmV, float* __restrict__ O, float* __restrict__ LSE,
+                  int S, int BH, int n_qt, int causal, float c2, unsigned* status)
+{
+    using C = FwdCfg<D, BM, BN>;
+    constexpr int RM = C::RM, RN = C::RN, DV = C::DV, NCH = C::NCH, PSTR = C::PSTR;
+
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t sQ = base;
+    const uint32_t sK = sQ + C::Q_BYTES;
+    const uint32_t sV = sK + C::KV_BYTES;
+    const uint32_t sP = sV + C::KV_BYTES;
+    const uint32_t barQ = sP + C::P_BYTES, barK = barQ + 8, barV = barQ + 16;
+
+    const int tid = threadIdx.x;
+    const int tr = 2 * (tid >> 5) + ((tid & 31) >> 4);   // 0..15: row group
+    const int tc = tid & 15;                             // 0..15: column group
+
+    // Heaviest (last) query tiles first when causal.
+    const int qt = n_qt - 1 - static_cast<int>(blockIdx.x) / BH;
+    const int bh = static_cast<int>(blockIdx.x) % BH;
+    const int i0 = qt * BM;
+    const int i_last = min(i0 + BM, S) - 1;
+    const int n_kt = causal ? (i_last / BN + 1) : ((S + BN - 1) / BN);
+
+    if (tid == 0) {
+        mbar_init(barQ, 1);
+        mbar_init(barK, 1);
+        mbar_init(barV, 1);
+        fence_mbar_init();
+    }
+    __syncthreads();
+    if (tid == 0) {
+        mbar_arrive_expect_tx(barQ, C::Q_BYTES);
+#pragma unroll
+        for (int ch = 0; ch < NCH; ++ch) tma_load_3d(sQ + ch * BM * 128, &tmQ, barQ, ch * 32, i0, bh);
+        mbar_arrive_expect_tx(barK, C::KV_BYTES);
+#pragma unroll
+        for (int ch = 0; ch < NCH; ++ch) tma_load_3d(sK + ch * BN * 128, &tmK, barK, ch * 32, 0, bh);
+        mbar_arrive_expect_tx(barV, C::KV_BYTES);
+#pragma unroll
+        for (int ch = 0; ch < NCH; ++ch) tma_load_3d(sV + ch * BN * 128, &tmV, barV, ch * 32, 0, bh);
+    }
+
+    float o[RM][DV];
+    float m[RM], l[RM];
+#pragma unroll
+    for (int x = 0; x < RM; ++x) {
+        m[x] = -INFINITY;
+        l[x] = 0.f;
+#pragma unroll
+        for (int e = 0; e < DV; ++e) o[x][e] = 0.f;
+    }
+
+    mbar_wait(barQ, 0, status);
+
+    for (int kt = 0; kt < n_kt; ++kt) {
+        const uint32_t ph = kt & 1;
+        const int j0 = kt * BN;
+        float s[RM][RN];
+#pragma unroll
+        for (int x = 0; x < RM; ++x)
+#pragma unroll
+            for (int y = 0; y < RN; ++y) s[x][y] = 0.f;
+
+        mbar_wait(barK, ph, status);
+        // ---- S = Q K^T : contraction along d, float4 pieces --------------------------------
+        {
+            const uint32_t qa = sQ + tr * 128, ka = sK + tc * 128;
+            const int xq = tr & 7, xk = tc & 7;
+#pragma unroll
+            for (int pc = 0; pc < D / 4; ++pc) {
+                const uint32_t oq = (pc >> 3) * (BM * 128) + (((pc & 7) ^ xq) << 4);
+                const uint32_t ok = (pc >> 3) * (BN * 128) + (((pc & 7) ^ xk) << 4);
+                float4 b[RN];
+#pragma unroll
+                for (int y = 0; y < RN; ++y) b[y] = lds128(ka + ok + y * 16 * 128);
+#pragma unroll
+                for (int x = 0; x < RM; ++x) {
+                    const float4 a = lds128(qa + oq + x * 16 * 128);
+#pragma unroll
+                    for (int y = 0; y < RN; ++y) {
+                        s[x][y] = fmaf(a.x, b[y].x, s[x][y]);
+                        s[x][y] = fmaf(a.y, b[y].y, s[x][y]);
+                        s[x][y] = fmaf(a.z, b[y].z, s[x][y]);
+                        s[x][y] = fmaf(a.w, b[y].w, s[x][y]);
+                    }
+                }
+            }
+        }
+        __syncthreads();   // every warp is done with this K tile (and with P of the previous tile)
+        if (tid == 0 && kt + 1 < n_kt) {
+            mbar_arrive_expect_tx(barK, C::KV_BYTES);
+#pragma unroll
+            for (int ch = 0; ch < NCH; ++ch) tma_load_3d(sK + ch * BN * 128, &tmK, barK, ch * 32, j0 + BN, bh);
+        }
+
+        // ---- scale into the log2 domain, mask, online softmax ------------------------------
+        const bool need_mask = (causal && (j0 + BN - 1 > i0)) || (j0 + BN > S);
+#pragma unroll
+        for (int x = 0; x < RM; ++x) {
+            const int i = i0 + tr + 16 * x;
+            float mx = -INFINITY;
+#pragma unroll
+            for (int y = 0; y < RN; ++y) {
+                float v = s[x][y] * c2;
+                if (need_mask) {
+                    const int j = j0 + tc + 16 * y;
+                    if (j >= S || (causal && j > i)) v = -INFINITY;
+                }
+                s[x][y] = v;
+                mx = fmaxf(mx, v);
+            }
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 8));
+            const float m_new = fmaxf(m[x], mx);    // finite from the first tile on (key 0 is never masked)
+            const float alpha = ex2(m[x] - m_new);
+            m[x] = m_new;
+            float psum = 0.f;
+            const uint32_t prow = sP + ((tr + 16 * x) * PSTR + tc) * 4;
+#pragma unroll
+            for (int y = 0; y < RN; ++y) {
+                const float p = ex2(s[x][y] - m_new);
+                psum += p;
+                sts32(prow + y * 64, p);
+            }
+            l[x] = fmaf(l[x], alpha, psum);
+#pragma unroll
+            for (int e = 0; e < DV; ++e) o[x][e] *= alpha;
+        }
+        __syncthreads();   // P visible
+        mbar_wait(barV, ph, status);
+
+        // ---- O += P V : contraction along keys ----------------------------------------------
+        {
+            const uint32_t pa = sP + tr * PSTR * 4;
+#pragma unroll 2
+            for (int j8 = 0; j8 < BN / 8; ++j8) {
+                float4 p[2][RM];
+#pragma unroll
+                for (int hlf = 0; hlf < 2; ++hlf)
+#pragma unroll
+                    for (int x = 0; x < RM; ++x) p[hlf][x] = lds128(pa + (x * 16 * PSTR + j8 * 8 + hlf * 4) * 4);
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    const int j = j8 * 8 + u;
+                    float vv[DV];
+                    if constexpr (DV == 2) {
+                        const float2 t = lds64(sV + j * 128 + ((((tc >> 1)) ^ u) << 4) + (tc & 1) * 8);
+                        vv[0] = t.x; vv[1] = t.y;
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < DV / 4; ++e) {
+                            const int piece = tc + 16 * e;
+                            const float4 t = lds128(sV + (piece >> 3) * (BN * 128) + j * 128 + (((piece & 7) ^ u) << 4));
+                            vv[4 * e + 0] = t.x; vv[4 * e + 1] = t.y; vv[4 * e + 2] = t.z; vv[4 * e + 3] = t.w;
+                        }
+                    }
+#pragma unroll
+                    for (int x = 0; x < RM; ++x) {
+                        const float4 pp = p[u >> 2][x];
+                        const float pv = (u & 3) == 0 ? pp.x : (u & 3) == 1 ? pp.y : (u & 3) == 2 ? pp.z : pp.w;
+#pragma unroll
+                        for (int e = 0; e < DV; ++e) o[x][e] = fmaf(pv, vv[e], o[x][e]);
+                    }
+                }
+            }
+        }
+        __syncthreads();   // every warp is done with this V tile and with P
+        if (tid == 0 && kt + 1 < n_kt) {
+            mbar_arrive_expect_tx(barV, C::KV_BYTES);
+#pragma unroll
+            for (int ch = 0; ch < NCH; ++ch) tma_load_3d(sV + ch * BN * 128, &tmV, barV, ch * 32, j0 + BN, bh);
+        }
+    }
+
+    // ---- epilogue: O / l, LSE = ln2 (m + log2 l) -----------------------------------------------
+#pragma unroll
+    for (int x = 0; x < RM; ++x) {
+        float lt = l[x];
+        lt += __shfl_xor_sync(0xffffffffu, lt, 1);
+        lt += __shfl_xor_sync(0xffffffffu, lt, 2);
+        lt += __shfl_xor_sync(0xffffffffu, lt, 4);
+        lt += __shfl_xor_sync(0xffffffffu, lt, 8);
+        const int i = i0 + tr + 16 * x;
+        if (i < S) {
+            const float inv = 1.0f / lt;
+            float* orow = O + (static_cast<size_t>(bh) * S + i) * D;
+            if constexpr (DV == 2) {
+                *reinterpret_cast<float2*>(orow + 2 * tc) = make_float2(o[x][0] * inv, o[x][1] * inv);
+            } else {
+#pragma unroll
+                for (int e = 0; e < DV / 4; ++e)
+                    *reinterpret_cast<float4*>(orow + 4 * tc + 64 * e) =
+                        make_float4(o[x][4 * e] * inv, o[x][4 * e + 1] * inv, o[x][4 * e + 2] * inv, o[x][4 * e + 3] * inv);
+            }
+            if (tc == 0) LSE[static_cast<size_t>(bh) * S + i] = (m[x] + log2f(lt)) * kLn2;
+        }
+    }
+}
+
+template <int D, int BM, int BN>
+cudaError_t launch(const Problem& p, const float* q, const float* k, const float* v, float* o, float* lse,
+                   unsigned* status, cudaStream_t st)
+{
+    using C = FwdCfg<D, BM, BN>;
+    CUtensorMap tq, tk, tv;
+    if (make_tmap_3d(&tq, q, 4, 0, p.BH, p.S, D, 32, BM)) return cudaErrorInvalidValue;
+    if (make_tmap_3d(&tk, k, 4, 0, p.BH, p.S, D, 32, BN)) return cudaErrorInvalidValue;
+    if (make_tmap_3d(&tv, v, 4, 0, p.BH, p.S, D, 32, BN)) return cudaErrorInvalidValue;
+    auto kern = strict_fwd_kernel<D, BM, BN>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM);
+    if (e != cudaSuccess) return e;
+    const int n_qt = (p.S + BM - 1) / BM;
+    const long long blocks = static_cast<long long>(n_qt) * p.BH;
+    if (blocks > 0x7fffffffLL) return cudaErrorInvalidValue;
+    kern<<<static_cast<unsigned>(blocks), kThreads, C::SMEM, st>>>(tq, tk, tv, o, lse, p.S, p.BH, n_qt, p.causal,
+                                                                   p.scale * kLog2e, status);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_strict_fwd(const Problem& p, const float* q, const float* k, const float* v,
+                              float* o, float* lse, unsigned* status, cudaStream_t st)
+{
+    switch (p.D) {
+        case 32:  return launch<32, 128, 128>(p, q, k, v, o, lse, status, st);
+        case 64:  return launch<64, 128, 128>(p, q, k, v, o, lse, status, st);
+        case 128: return launch<128, 128, 64>(p, q, k, v, o, lse, status, st);
+        default:  return cudaErrorInvalidValue;
+    }
+}
+
+}  // namespace mgn

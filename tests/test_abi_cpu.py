@@ -1,0 +1,117 @@
+"""Host-side checks of the C ABI that need no GPU: the library loads, exports every
+symbol the header declares, and rejects bad arguments in the documented order."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2608_01563_b200 import build as mgn_build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    mgn_build.build()
+    from paper_2608_01563_b200 import binding
+    return binding.lib()
+
+
+def declared_symbols():
+    names = set()
+    inc = os.path.join(ROOT, "include")
+    for fn in os.listdir(inc):
+        if fn.endswith(".h"):
+            text = open(os.path.join(inc, fn)).read()
+            text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+            names |= set(re.findall(r"\b(mgn_[a-z0-9_]+)\s*\(", text))
+    return sorted(names)
+
+
+def test_every_declared_symbol_is_exported(lib):
+    syms = declared_symbols()
+    assert {"mgn_attn_fwd", "mgn_attn_bwd", "mgn_attn_bwd_workspace_bytes", "mgn_attn_check",
+            "mgn_status_string", "mgn_version", "mgn_attn_profile_events"} <= set(syms)
+    for s in syms:
+        assert getattr(lib, s) is not None
+
+
+def test_version_and_status_strings(lib):
+    assert lib.mgn_version() >= 100
+    names = [lib.mgn_status_string(i).decode() for i in range(8)]
+    assert names[0] == "MGN_OK" and len(set(names)) == 8
+    assert lib.mgn_status_string(99).decode() == "MGN_ERR_UNKNOWN"
+
+
+def test_workspace_bytes(lib):
+    f = lib.mgn_attn_bwd_workspace_bytes
+    assert f(8, 12, 1024, 64, 0) >= 8 * 12 * 1024 * 4
+    assert f(8, 12, 1024, 64, 1) >= 8 * 12 * 1024 * 4 + 8 * 12 * 1024 * 64 * 4
+    assert f(8, 12, 1024, 64, 0) % 256 == 0
+    for bad in [(0, 1, 1, 64, 0), (1, 1, 1, 48, 0), (1, 1, 1, 64, 2), (1, -1, 1, 64, 0)]:
+        assert f(*bad) == 0
+
+
+A = 1 << 20  # a fake, 16-byte aligned, never dereferenced device address
+
+
+def fwd(lib, q=A, k=A, v=A, o=A, lse=A, B=1, H=1, S=8, D=64, causal=0, scale=1.0, mode=0):
+    return lib.mgn_attn_fwd(q, k, v, o, lse, B, H, S, D, causal, scale, mode, None)
+
+
+def bwd(lib, ptrs=None, ws=A, ws_bytes=1 << 30, B=1, H=1, S=8, D=64, causal=0, scale=1.0, mode=0):
+    p = [A] * 9 if ptrs is None else ptrs
+    return lib.mgn_attn_bwd(*p, ws, ws_bytes, B, H, S, D, causal, scale, mode, None)
+
+
+def test_forward_argument_validation_order(lib):
+    INVALID, UNSUPPORTED, MISALIGNED = 1, 2, 3
+    assert fwd(lib, q=None) == INVALID
+    assert fwd(lib, lse=None) == INVALID
+    assert fwd(lib, S=0) == INVALID
+    assert fwd(lib, B=-1) == INVALID
+    assert fwd(lib, causal=2) == INVALID
+    assert fwd(lib, scale=float("nan")) == INVALID
+    assert fwd(lib, scale=float("inf")) == INVALID
+    assert fwd(lib, mode=5) == INVALID
+    assert fwd(lib, D=48) == UNSUPPORTED
+    assert fwd(lib, D=256) == UNSUPPORTED
+    assert fwd(lib, B=1 << 20, H=1 << 20) == UNSUPPORTED
+    assert fwd(lib, q=A + 4) == MISALIGNED
+    assert fwd(lib, o=A + 8) == MISALIGNED
+    # invalid beats unsupported beats misaligned
+    assert fwd(lib, q=A + 4, D=48) == UNSUPPORTED
+    assert fwd(lib, q=A + 4, D=48, S=0) == INVALID
+    # a fully valid call gets past validation; without a usable device it must fail, not compute
+    import torch
+    if not torch.cuda.is_available():
+        assert fwd(lib) in (5, 6)
+
+
+def test_backward_argument_validation_order(lib):
+    INVALID, UNSUPPORTED, MISALIGNED, WORKSPACE = 1, 2, 3, 4
+    for idx in range(9):
+        p = [A] * 9
+        p[idx] = None
+        assert bwd(lib, ptrs=p) == INVALID
+    for idx in range(9):
+        p = [A] * 9
+        p[idx] = A + 2
+        assert bwd(lib, ptrs=p) == MISALIGNED
+    assert bwd(lib, D=100) == UNSUPPORTED
+    assert bwd(lib, ws=None) == WORKSPACE
+    assert bwd(lib, ws_bytes=16) == WORKSPACE
+    assert bwd(lib, ws=A + 16) == WORKSPACE
+    need = lib.mgn_attn_bwd_workspace_bytes(1, 1, 8, 64, 1)
+    assert bwd(lib, ws_bytes=need - 1, mode=1) == WORKSPACE
+    assert bwd(lib, ws=None, ptrs=[A + 4] * 9) == MISALIGNED
+    assert bwd(lib, ws=None, S=-3) == INVALID
+
+
+def test_binding_fails_loudly_without_library(monkeypatch, tmp_path):
+    from paper_2608_01563_b200 import binding
+    monkeypatch.setattr(binding, "_lib", None)
+    monkeypatch.setattr(binding, "LIB_PATH", str(tmp_path / "nope.so"))
+    with pytest.raises(RuntimeError):
+        binding.mgn_version()
