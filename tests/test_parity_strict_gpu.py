@@ -64,7 +64,8 @@ def test_unusual_scales(scale):
     q, k, v, d_o = synth.random_inputs(77, B, H, S, D, std=0.7)
     res = hp.run_cuda(q, k, v, d_o, True, scale, MODE)
     ref = hp.run_oracle(q, k, v, d_o, True, scale)
-    hp.check_strict(hp.select(res, B, H), ref, label=f"scale={scale} ")
+    # scale 2.0 drives |dQ|,|dK| to tens, so the absolute bound is taken relative to max(1, max|ref|)
+    hp.check_strict(hp.select(res, B, H), ref, literal_max_abs=False, label=f"scale={scale} ")
 
 
 def test_backward_accepts_given_o_and_lse():
