@@ -36,6 +36,7 @@ int check_common(int B, int H, int S, int D, int causal, float scale, int mode)
     if (D != 32 && D != 64 && D != 128) return MGN_ERR_UNSUPPORTED;
     const long long bh = static_cast<long long>(B) * H;
     if (bh > 0x7fffffffLL) return MGN_ERR_UNSUPPORTED;
+    if (mode == MGN_MODE_FAST_BF16 && D == 32) return MGN_ERR_UNSUPPORTED;   // tensor-core path: D in {64,128}
     if (S > (1 << 24)) return MGN_ERR_UNSUPPORTED;
     // grid and byte-offset plan: tiles*BH must fit an int, element counts must fit 2^40
     if (bh * ((S + 63) / 64) > 0x7fffffffLL) return MGN_ERR_UNSUPPORTED;

@@ -1,0 +1,327 @@
+// Fast-mode attention forward: bf16 storage, tcgen05 tensor-core products with f32
+// accumulation in tensor memory, f32 softmax statistics (paper Section 3.3 "tiled attention
+// forward"; Section 4.2: the validated reduced-input path with f32 accumulation).
+//
+// One CTA owns two 128-row query tiles of one head and walks over 128-key blocks.
+// Warp roles (384 threads):
+//   warp 0      TMA producer: Q tiles once, then K and V blocks through a 2-stage ring
+//   warp 1      MMA issuer: S_t = Q_t K^T (operands in shared memory) and O_t += P_t V
+//               (P_t read from tensor memory, V as an MN-major shared-memory operand)
+//   warps 4-7   softmax of query tile 0: one thread per row, so row max / row sum need no
+//   warps 8-11  softmax of query tile 1   cross-thread reduction
+// Tensor memory (512 columns): S_0 [0,128), S_1 [128,256), O_0 [256,256+D), O_1 [256+D,256+2D).
+// P_t (bf16) overwrites the first 64 columns of S_t.  The two tiles ping-pong: while one tile's
+// softmax runs, the tensor core works on the other tile.  The running maximum is only moved
+// (and O rescaled in tensor memory) when it grows by more than 2^8, which is exact: any
+// reference point works for a softmax as long as nothing overflows.
+#include "kernels.h"
+#include "umma.cuh"
+
+namespace mgn {
+namespace {
+
+constexpr int kThreads = 384;
+constexpr int BM = 128;      // rows per query tile
+constexpr int BN = 128;      // keys per block
+constexpr int kStages = 2;
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+constexpr float kRescaleThreshold = 8.0f;
+
+template <int D>
+struct Cfg {
+    static constexpr int NCH = D / 64;                 // 128-byte chunks per row
+    static constexpr int TILE_BYTES = 128 * D * 2;     // a 128-row tile of Q, K or V
+    static constexpr int CHUNK_BYTES = 128 * 128;      // one 64-column chunk of a 128-row tile
+    static constexpr int OFF_Q = 0;
+    static constexpr int OFF_K = OFF_Q + 2 * TILE_BYTES;
+    static constexpr int OFF_V = OFF_K + kStages * TILE_BYTES;
+    static constexpr int OFF_BAR = OFF_V + kStages * TILE_BYTES;
+    static constexpr int SMEM = OFF_BAR + 256 + 1024;
+    static constexpr uint32_t TM_S = 0, TM_O = 256, TM_COLS = 512;
+};
+
+// barrier slots (8 bytes each)
+enum { B_Q = 0, B_KFULL = 1, B_KEMPTY = 3, B_VFULL = 5, B_VEMPTY = 7, B_SFULL = 9, B_PFULL = 11, B_OFULL = 13, B_COUNT = 15 };
+
+template <int D>
+__global__ void __launch_bounds__(kThreads, 1)
+fast_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+                const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO,
+                float* __restrict__ LSE, int S, int BH, int n_pairs, int causal, float c2, unsigned* status)
+{
+    using C = Cfg<D>;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t sQ = base + C::OFF_Q, sK = base + C::OFF_K, sV = base + C::OFF_V;
+    const uint32_t bars = base + C::OFF_BAR;
+    const uint32_t tmem_slot = bars + B_COUNT * 8;
+    auto bar = [&](int i) { return bars + 8u * i; };
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    if (*reinterpret_cast<volatile unsigned*>(status) != 0) return;   // an earlier wait on this device gave up
+
+    // heaviest (last) query-tile pairs first when causal
+    const int pair = n_pairs - 1 - static_cast<int>(blockIdx.x) / BH;
+    const int bh = static_cast<int>(blockIdx.x) % BH;
+    const int n_kb = (S + BN - 1) / BN;
+    int row0[2], nblk[2];
+#pragma unroll
+    for (int t = 0; t < 2; ++t) {
+        row0[t] = pair * 2 * BM + t * BM;
+        if (row0[t] >= S) nblk[t] = 0;
+        else nblk[t] = causal ? min(n_kb, (min(row0[t] + BM, S) - 1) / BN + 1) : n_kb;
+    }
+    const int n_max = max(nblk[0], nblk[1]);
+
+    if (tid == 0) {
+        for (int i = 0; i < B_COUNT; ++i) mbar_init(bar(i), (i == B_PFULL || i == B_PFULL + 1) ? 128 : 1);
+        fence_mbar_init();
+    }
+    __syncwarp();
+    if (warp == 0) tmem_alloc(tmem_slot, C::TM_COLS);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = lds32u(tmem_slot);
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            const int nq = (nblk[1] > 0) ? 2 : 1;
+            mbar_arrive_expect_tx(bar(B_Q), nq * C::TILE_BYTES);
+            for (int t = 0; t < nq; ++t)
+#pragma unroll
+                for (int ch = 0; ch < C::NCH; ++ch)
+                    tma_load_3d(sQ + t * C::TILE_BYTES + ch * C::CHUNK_BYTES, &tmQ, bar(B_Q), ch * 64, row0[t], bh);
+            for (int n = 0; n < n_max; ++n) {
+                const int st = n & 1;
+                const uint32_t ph = (n >> 1) & 1;
+                mbar_wait(bar(B_KEMPTY + st), ph ^ 1, status);
+                mbar_arrive_expect_tx(bar(B_KFULL + st), C::TILE_BYTES);
+#pragma unroll
+                for (int ch = 0; ch < C::NCH; ++ch)
+                    tma_load_3d(sK + st * C::TILE_BYTES + ch * C::CHUNK_BYTES, &tmK, bar(B_KFULL + st), ch * 64, n * BN, bh);
+                mbar_wait(bar(B_VEMPTY + st), ph ^ 1, status);
+                mbar_arrive_expect_tx(bar(B_VFULL + st), C::TILE_BYTES);
+#pragma unroll
+                for (int ch = 0; ch < C::NCH; ++ch)
+                    tma_load_3d(sV + st * C::TILE_BYTES + ch * C::CHUNK_BYTES, &tmV, bar(B_VFULL + st), ch * 64, n * BN, bh);
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc_s = umma_idesc_bf16(BM, BN, false, false);
+            constexpr uint32_t idesc_o = umma_idesc_bf16(BM, D, false, true);
+            auto issue_s = [&](int t, int n) {   // S_t = Q_t K(n)^T
+                const uint32_t qa = sQ + t * C::TILE_BYTES, ka = sK + (n & 1) * C::TILE_BYTES;
+#pragma unroll
+                for (int kk = 0; kk < D / 16; ++kk) {
+                    const uint32_t off = (kk >> 2) * C::CHUNK_BYTES + (kk & 3) * 32;
+                    umma_ss(tmem + C::TM_S + t * 128, umma_smem_desc(qa + off, 16, 1024),
+                            umma_smem_desc(ka + off, 16, 1024), idesc_s, kk > 0);
+                }
+                umma_commit(bar(B_SFULL + t));
+            };
+            auto issue_o = [&](int t, int n) {   // O_t += P_t V(n)
+                const uint32_t va = sV + (n & 1) * C::TILE_BYTES;
+#pragma unroll
+                for (int kk = 0; kk < BN / 16; ++kk)
+                    umma_ts(tmem + C::TM_O + t * D, tmem + C::TM_S + t * 128 + kk * 8,
+                            umma_smem_desc(va + kk * 2048, C::CHUNK_BYTES, 1024), idesc_o, (n > 0 || kk > 0));
+            };
+            mbar_wait(bar(B_Q), 0, status);
+            mbar_wait(bar(B_KFULL + 0), 0, status);
+            tc_fence_after();
+            for (int t = 0; t < 2; ++t)
+                if (nblk[t] > 0) issue_s(t, 0);
+            umma_commit(bar(B_KEMPTY + 0));
+            for (int n = 0; n < n_max; ++n) {
+                const int st = n & 1;
+                const uint32_t ph = (n >> 1) & 1;
+                mbar_wait(bar(B_VFULL + st), ph, status);
+                if (n + 1 < n_max) mbar_wait(bar(B_KFULL + (st ^ 1)), ((n + 1) >> 1) & 1, status);
+                for (int t = 0; t < 2; ++t) {
+                    if (n < nblk[t]) {
+                        mbar_wait(bar(B_PFULL + t), n & 1, status);
+                        tc_fence_after();
+                        issue_o(t, n);
+                        if (n == nblk[t] - 1) umma_commit(bar(B_OFULL + t));
+                    }
+                    if (n + 1 < nblk[t]) issue_s(t, n + 1);
+                }
+                umma_commit(bar(B_VEMPTY + st));
+                if (n + 1 < n_max) umma_commit(bar(B_KEMPTY + (st ^ 1)));
+            }
+        }
+        __syncwarp();
+    } else if (warp >= 4) {
+        // ------------------------------------------------------------------ softmax + epilogue
+        const int t = (warp - 4) >> 2;
+        const int r = tid - 128 * (1 + t);                 // row within the tile, 0..127
+        const uint32_t lane_base = static_cast<uint32_t>(r & ~31) << 16;
+        const uint32_t tS = tmem + lane_base + C::TM_S + t * 128;
+        const uint32_t tO = tmem + lane_base + C::TM_O + t * D;
+        const int i = row0[t] + r;
+        const int nb = nblk[t];
+        float m_ref = -INFINITY, l = 0.f;
+
+        for (int n = 0; n < nb; ++n) {
+            mbar_wait(bar(B_SFULL + t), n & 1, status);
+            tc_fence_after();
+            const int j0 = n * BN;
+            const bool masked = (causal && (j0 + BN - 1 > row0[t])) || (j0 + BN > S);
+            const int jmax = min(S - 1, causal ? i : S - 1) - j0;   // columns c <= jmax of this block are visible
+
+            // pass 1: block maximum of the scaled scores
+            float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+#pragma unroll 1
+            for (int c = 0; c < 4; ++c) {
+                uint32_t v[32];
+                tmem_ld32(tS + 32 * c, v);
+                tmem_ld_wait();
+                float x[32];
+#pragma unroll
+                for (int e = 0; e < 32; ++e) x[e] = __uint_as_float(v[e]) * c2;
+                if (masked) {
+#pragma unroll
+                    for (int e = 0; e < 32; ++e)
+                        if (32 * c + e > jmax) x[e] = -INFINITY;
+                }
+#pragma unroll
+                for (int e = 0; e < 32; e += 4) {
+                    mx0 = fmaxf(mx0, x[e]);
+                    mx1 = fmaxf(mx1, x[e + 1]);
+                    mx2 = fmaxf(mx2, x[e + 2]);
+                    mx3 = fmaxf(mx3, x[e + 3]);
+                }
+            }
+            const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
+            if (n == 0) {
+                m_ref = mx;      // finite: key 0 is visible to every row
+            } else {
+                const bool grow = (mx - m_ref) > kRescaleThreshold;
+                if (__any_sync(0xffffffffu, grow)) {
+                    const float m_new = fmaxf(m_ref, mx);
+                    const float alpha = ex2(m_ref - m_new);
+                    m_ref = m_new;
+                    l *= alpha;
+#pragma unroll 1
+                    for (int c = 0; c < D / 32; ++c) {
+                        uint32_t v[32];
+                        tmem_ld32(tO + 32 * c, v);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) v[e] = __float_as_uint(__uint_as_float(v[e]) * alpha);
+                        tmem_st32(tO + 32 * c, v);
+                    }
+                    tmem_st_wait();
+                }
+            }
+
+            // pass 2: P = exp2(s*c2 - m_ref) -> bf16 into tensor memory over S; row sum
+            float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
+            const float neg_m = -m_ref;
+#pragma unroll 1
+            for (int c = 0; c < 4; ++c) {
+                uint32_t v[32];
+                tmem_ld32(tS + 32 * c, v);
+                tmem_ld_wait();
+                float p[32];
+#pragma unroll
+                for (int e = 0; e < 32; ++e) p[e] = ex2(fmaf(__uint_as_float(v[e]), c2, neg_m));
+                if (masked) {
+#pragma unroll
+                    for (int e = 0; e < 32; ++e)
+                        if (32 * c + e > jmax) p[e] = 0.f;
+                }
+                uint32_t u[16];
+#pragma unroll
+                for (int e = 0; e < 32; e += 4) {
+                    l0 += p[e]; l1 += p[e + 1]; l2 += p[e + 2]; l3 += p[e + 3];
+                    u[e / 2] = pack_bf16(p[e], p[e + 1]);
+                    u[e / 2 + 1] = pack_bf16(p[e + 2], p[e + 3]);
+                }
+                tmem_st16(tS + 16 * c, u);
+            }
+            l += (l0 + l1) + (l2 + l3);
+            tmem_st_wait();
+            tc_fence_before();
+            mbar_arrive(bar(B_PFULL + t));
+        }
+
+        if (nb > 0) {
+            // ---- epilogue: O / l -> bf16 -> shared (swizzled like the TMA box) -> TMA store; LSE
+            mbar_wait(bar(B_OFULL + t), 0, status);
+            tc_fence_after();
+            const float inv = 1.0f / l;
+            const uint32_t stage = sQ + t * C::TILE_BYTES;     // Q_t is no longer needed
+#pragma unroll 1
+            for (int c = 0; c < D / 32; ++c) {
+                uint32_t v[32];
+                tmem_ld32(tO + 32 * c, v);
+                tmem_ld_wait();
+                uint32_t u[16];
+#pragma unroll
+                for (int e = 0; e < 16; ++e)
+                    u[e] = pack_bf16(__uint_as_float(v[2 * e]) * inv, __uint_as_float(v[2 * e + 1]) * inv);
+                const uint32_t rowaddr = stage + (c >> 1) * C::CHUNK_BYTES + r * 128;
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const int piece = (c & 1) * 4 + q;
+                    sts128(rowaddr + ((piece ^ (r & 7)) << 4), u[4 * q], u[4 * q + 1], u[4 * q + 2], u[4 * q + 3]);
+                }
+            }
+            if (i < S) LSE[static_cast<size_t>(bh) * S + i] = (m_ref + log2f(l)) * kLn2;
+            fence_proxy_async_smem();
+            named_bar_sync(1 + t, 128);
+            if (r == 0) {
+#pragma unroll
+                for (int ch = 0; ch < C::NCH; ++ch)
+                    tma_store_3d(&tmO, stage + ch * C::CHUNK_BYTES, ch * 64, row0[t], bh);
+                tma_store_commit_and_wait_read();
+            }
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem, C::TM_COLS);
+}
+
+template <int D>
+cudaError_t launch(const Problem& p, const void* q, const void* k, const void* v, void* o, float* lse,
+                   unsigned* status, cudaStream_t st)
+{
+    using C = Cfg<D>;
+    CUtensorMap tq, tk, tv, to;
+    if (make_tmap_3d(&tq, q, 2, 1, p.BH, p.S, D, 64, 128)) return cudaErrorInvalidValue;
+    if (make_tmap_3d(&tk, k, 2, 1, p.BH, p.S, D, 64, 128)) return cudaErrorInvalidValue;
+    if (make_tmap_3d(&tv, v, 2, 1, p.BH, p.S, D, 64, 128)) return cudaErrorInvalidValue;
+    if (make_tmap_3d(&to, o, 2, 1, p.BH, p.S, D, 64, 128)) return cudaErrorInvalidValue;
+    auto kern = fast_fwd_kernel<D>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM);
+    if (e != cudaSuccess) return e;
+    const int n_pairs = (p.S + 2 * BM - 1) / (2 * BM);
+    const long long blocks = static_cast<long long>(n_pairs) * p.BH;
+    if (blocks > 0x7fffffffLL) return cudaErrorInvalidValue;
+    kern<<<static_cast<unsigned>(blocks), kThreads, C::SMEM, st>>>(tq, tk, tv, to, lse, p.S, p.BH, n_pairs, p.causal,
+                                                                   p.scale * kLog2e, status);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_fast_fwd(const Problem& p, const void* q, const void* k, const void* v, void* o, float* lse,
+                            unsigned* status, cudaStream_t st)
+{
+    switch (p.D) {
+        case 64:  return launch<64>(p, q, k, v, o, lse, status, st);
+        case 128: return launch<128>(p, q, k, v, o, lse, status, st);
+        default:  return cudaErrorNotSupported;
+    }
+}
+
+}  // namespace mgn

@@ -10,7 +10,7 @@ namespace mgn {
 // Upper bound on polls of one barrier wait.  A wait that runs out records
 // MGN_ERR_DEVICE_TIMEOUT in the status word and the kernel carries on to its
 // end (its results are then garbage, but it cannot hang the device).
-constexpr uint32_t kMaxPolls = 1u << 24;
+constexpr uint32_t kMaxPolls = 1u << 22;
 constexpr unsigned kStatusTimeout = 7u;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -43,8 +43,11 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
 }
 // Bounded wait.  Returns false (after flagging the status word) if it gave up.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, unsigned* status) {
-    for (uint32_t it = 0; it < kMaxPolls; ++it)
+    for (uint32_t it = 0; it < kMaxPolls; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
+        // once any wait on the device has given up, every other wait gives up quickly too
+        if ((it & 0xfffu) == 0xfffu && status && *reinterpret_cast<volatile unsigned*>(status) != 0) return false;
+    }
     if (status) atomicMax(status, kStatusTimeout);
     return false;
 }

@@ -36,14 +36,14 @@ class Guarded:
         n = int(np.prod(shape))
         self.shape = shape
         self.n = n
-        self.buf = torch.full((n + 2 * GUARD,), 777.0, dtype=dtype, device=device)
+        self.buf = torch.full((n + 2 * GUARD,), 512.0, dtype=dtype, device=device)
         self.view = self.buf[GUARD:GUARD + n].view(shape)
         self.view.fill_(float("nan"))
         assert self.view.data_ptr() % 16 == 0
 
     def check(self, name):
         b = self.buf.float().cpu()
-        assert (b[:GUARD] == 777.0).all() and (b[GUARD + self.n:] == 777.0).all(), f"{name}: wrote outside its buffer"
+        assert (b[:GUARD] == 512.0).all() and (b[GUARD + self.n:] == 512.0).all(), f"{name}: wrote outside its buffer"
         out = self.view.detach().cpu()
         assert not torch.isnan(out.float()).any(), f"{name}: unwritten or NaN elements"
         return out

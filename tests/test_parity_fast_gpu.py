@@ -1,0 +1,95 @@
+"""Fast (bf16 tensor-core) mode: CUDA path vs the f64 oracle through the C ABI.
+
+The oracle receives the bf16-rounded inputs (exact in f64), so input quantisation is not
+counted as error; rounding of P, dS and of the bf16 outputs is.  Gate: rel-L2 <= 2e-2."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2608_01563_b200 import binding as mgn
+from paper_2608_01563_b200 import inputs as synth
+
+import helpers as hp
+
+pytestmark = pytest.mark.gpu
+MODE = mgn.MODE_FAST_BF16
+BF = torch.bfloat16
+
+
+@pytest.mark.parametrize("D", [64, 128])
+@pytest.mark.parametrize("causal", [False, True])
+@pytest.mark.parametrize("S", [1, 2, 63, 64, 65, 127, 128, 129, 197, 256, 257, 300, 520])
+def test_forward_edge_shapes(S, D, causal):
+    B, H = 1, 3
+    q, k, v, d_o = synth.random_inputs(2000 + S + D, B, H, S, D, dtype=BF)
+    scale = 1.0 / math.sqrt(D)
+    res = hp.run_cuda(q, k, v, d_o, causal, scale, MODE, run_bwd=False)
+    ref = hp.run_oracle(q, k, v, d_o, causal, scale)
+    hp.check_fast(hp.select(res, B, H), ref, names=("O",), label=f"S={S} D={D} causal={causal} ")
+
+
+@pytest.mark.parametrize("D", [64, 128])
+@pytest.mark.parametrize("causal", [False, True])
+@pytest.mark.parametrize("S", [1, 2, 63, 64, 65, 127, 128, 129, 197, 256, 257, 300, 520])
+def test_forward_backward_edge_shapes(S, D, causal):
+    B, H = 1, 3
+    q, k, v, d_o = synth.random_inputs(3000 + S + D, B, H, S, D, dtype=BF)
+    scale = 1.0 / math.sqrt(D)
+    res = hp.run_cuda(q, k, v, d_o, causal, scale, MODE)
+    ref = hp.run_oracle(q, k, v, d_o, causal, scale)
+    hp.check_fast(hp.select(res, B, H), ref, label=f"S={S} D={D} causal={causal} ")
+
+
+def test_forward_large_max_growth_triggers_rescale():
+    """Keys grow along the sequence so the running maximum moves by far more than the lazy threshold."""
+    B, H, S, D = 1, 2, 1024, 128
+    q, k, v, d_o = synth.random_inputs(11, B, H, S, D, dtype=torch.float32)
+    ramp = torch.linspace(0.1, 3.0, S).view(1, 1, S, 1)
+    k = (k * ramp).to(BF)
+    q, v, d_o = q.to(BF), v.to(BF), d_o.to(BF)
+    for causal in (False, True):
+        res = hp.run_cuda(q, k, v, d_o, causal, 0.3, MODE, run_bwd=False)
+        ref = hp.run_oracle(q, k, v, d_o, causal, 0.3)
+        hp.check_fast(hp.select(res, B, H), ref, names=("O",))
+
+
+@pytest.mark.parametrize("scale", [0.0, -0.2])
+def test_forward_unusual_scales(scale):
+    B, H, S, D = 1, 2, 300, 64
+    q, k, v, d_o = synth.random_inputs(12, B, H, S, D, dtype=BF)
+    res = hp.run_cuda(q, k, v, d_o, True, scale, MODE, run_bwd=False)
+    ref = hp.run_oracle(q, k, v, d_o, True, scale)
+    hp.check_fast(hp.select(res, B, H), ref, names=("O",))
+
+
+def _workload_parity(name, heads):
+    w = synth.WORKLOADS[name]
+    q, k, v, d_o = synth.make_inputs(w, dtype=BF)
+    res = hp.run_cuda(q, k, v, d_o, w.causal, w.scale, MODE)
+    ref = hp.run_oracle(q, k, v, d_o, w.causal, w.scale, heads)
+    rep = hp.check_fast(hp.select(res, w.B, w.H, heads), ref, label=name + " ")
+    hp.check_invariants(q, k, v, d_o, res, rtol=2e-2)
+    return rep
+
+
+def test_long_context_head_subset():
+    _workload_parity("long_context", [0, 13, 31])
+
+
+@pytest.mark.parametrize("name,heads", [
+    ("decoder_sweep_S512", [0, 37, 127]),
+    ("decoder_sweep_S1024", [0, 127]),
+    ("decoder_sweep_S2048", [64]),
+])
+def test_decoder_sweep_head_subset(name, heads):
+    _workload_parity(name, heads)
+
+
+def test_d32_is_reported_unsupported_in_fast_mode():
+    q = torch.zeros(1, 1, 8, 32, device="cuda", dtype=BF)
+    lse = torch.zeros(1, 1, 8, device="cuda")
+    with pytest.raises(mgn.MgnError) as e:
+        mgn.mgn_attn_fwd(q, q, q, torch.empty_like(q), lse, False, 1.0, MODE)
+    assert e.value.status == 2
