@@ -1,0 +1,378 @@
+// Fast-mode attention backward: bf16 storage, tcgen05 tensor-core products with f32
+// accumulation in tensor memory (paper Section 3.3 "dQ, and fused dK+dV kernels"; Section 7.3
+// FlashGradKV / FlashGradQ; Section 4.2 for the reduced-input arithmetic contract).
+//
+// Single pass.  One CTA keeps one 128-key block (K, V tiles) resident in shared memory, holds the
+// dK and dV accumulators of that block in tensor memory, and walks over the 128-row query blocks
+// (from the diagonal down when causal).  All score-shaped tiles are computed TRANSPOSED
+// (lanes = keys, columns = queries) so that P^T can feed dV = P^T dO straight from tensor
+// memory.  Per (key block, query block) pair:
+//   MMA1  S^T  = K Q^T            -> X            MMA2  dP^T = V dO^T -> Y
+//   compute (256 threads, one key lane x 64 query columns each):
+//         P^T = exp2(S^T c - LSE) -> bf16 into X;  dS^T = P^T (dP^T - delta) -> bf16 into shared
+//         memory, one buffer whose bytes are at once the K-major operand dS^T (rows = keys) and
+//         the MN-major operand dS (rows = queries)
+//   MMA4  dV  += P^T dO   (A from tensor memory)
+//   MMA5  dK  += dS^T Q   (A from shared memory)
+//   MMA6  dQp  = dS K  -> Y, then read out and added to the f32 dQ accumulator in global memory
+//         with 128-bit reductions (a later kernel scales and converts it to bf16).
+// Tensor memory: X [0,128)  Y [128,256)  dK [256,256+D)  dV [256+D,256+2D).
+// Warp roles (384 threads): warp 0 TMA producer, warp 1 MMA issuer, warps 4-11 compute.
+#include <cuda_bf16.h>
+
+#include "kernels.h"
+#include "umma.cuh"
+
+namespace mgn {
+namespace {
+
+constexpr int kThreads = 384;
+constexpr int BLK = 128;     // keys per CTA block and query rows per step
+constexpr float kLog2e = 1.4426950408889634f;
+
+template <int D>
+struct Cfg {
+    static constexpr int NCH = D / 64;
+    static constexpr int TILE_BYTES = BLK * D * 2;
+    static constexpr int CHUNK_BYTES = BLK * 128;
+    static constexpr int DS_BYTES = BLK * BLK * 2;
+    static constexpr int OFF_K = 0;
+    static constexpr int OFF_V = OFF_K + TILE_BYTES;
+    static constexpr int OFF_Q = OFF_V + TILE_BYTES;           // two stages
+    static constexpr int OFF_DO = OFF_Q + 2 * TILE_BYTES;
+    static constexpr int OFF_DS = OFF_DO + TILE_BYTES;
+    static constexpr int OFF_STAT = OFF_DS + DS_BYTES;         // [2 stages][lse2 | delta][128] f32
+    static constexpr int OFF_BAR = OFF_STAT + 2 * 2 * BLK * 4;
+    static constexpr int SMEM = OFF_BAR + 256 + 1024;
+    static constexpr uint32_t TM_X = 0, TM_Y = 128, TM_DK = 256, TM_DV = 256 + D, TM_COLS = 512;
+};
+
+enum { B_KV = 0, B_QFULL = 1, B_QEMPTY = 3, B_DOFULL = 5, B_DOEMPTY = 6, B_SFULL = 7, B_DPFULL = 8,
+       B_PDSFULL = 9, B_DQFULL = 10, B_DQEMPTY = 11, B_DKVFULL = 12, B_COUNT = 13 };
+
+template <int D>
+__global__ void __launch_bounds__(kThreads, 1)
+fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+                const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmdO,
+                const __grid_constant__ CUtensorMap tmdK, const __grid_constant__ CUtensorMap tmdV,
+                const float* __restrict__ LSE, const float* __restrict__ DELTA, float* __restrict__ dQacc,
+                int S, int BH, int causal, float scale, unsigned* status)
+{
+    using C = Cfg<D>;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t sK = base + C::OFF_K, sV = base + C::OFF_V, sQ = base + C::OFF_Q, sdO = base + C::OFF_DO;
+    const uint32_t sdS = base + C::OFF_DS, sStat = base + C::OFF_STAT, bars = base + C::OFF_BAR;
+    const uint32_t tmem_slot = bars + B_COUNT * 8;
+    auto bar = [&](int i) { return bars + 8u * i; };
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    if (*reinterpret_cast<volatile unsigned*>(status) != 0) return;   // an earlier wait on this device gave up
+
+    // heaviest key blocks (lowest j0) first when causal
+    const int kb = static_cast<int>(blockIdx.x) / BH;
+    const int bh = static_cast<int>(blockIdx.x) % BH;
+    const int j0 = kb * BLK;
+    const int n_qb = (S + BLK - 1) / BLK;
+    const int qb0 = causal ? kb : 0;
+    const int N = n_qb - qb0;                 // query blocks this CTA visits (>= 1)
+    const float c2 = scale * kLog2e;
+
+    if (tid == 0) {
+        for (int i = 0; i < B_COUNT; ++i) mbar_init(bar(i), (i == B_PDSFULL || i == B_DQEMPTY) ? 256 : 1);
+        fence_mbar_init();
+    }
+    __syncwarp();
+    if (warp == 0) tmem_alloc(tmem_slot, C::TM_COLS);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = lds32u(tmem_slot);
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            mbar_arrive_expect_tx(bar(B_KV), 2 * C::TILE_BYTES);
+#pragma unroll
+            for (int ch = 0; ch < C::NCH; ++ch) {
+                tma_load_3d(sK + ch * C::CHUNK_BYTES, &tmK, bar(B_KV), ch * 64, j0, bh);
+                tma_load_3d(sV + ch * C::CHUNK_BYTES, &tmV, bar(B_KV), ch * 64, j0, bh);
+            }
+            for (int n = 0; n < N; ++n) {
+                const int st = n & 1;
+                const int i0 = (qb0 + n) * BLK;
+                mbar_wait(bar(B_QEMPTY + st), ((n >> 1) & 1) ^ 1, status);
+                mbar_arrive_expect_tx(bar(B_QFULL + st), C::TILE_BYTES);
+#pragma unroll
+                for (int ch = 0; ch < C::NCH; ++ch)
+                    tma_load_3d(sQ + st * C::TILE_BYTES + ch * C::CHUNK_BYTES, &tmQ, bar(B_QFULL + st), ch * 64, i0, bh);
+                mbar_wait(bar(B_DOEMPTY), (n & 1) ^ 1, status);
+                mbar_arrive_expect_tx(bar(B_DOFULL), C::TILE_BYTES);
+#pragma unroll
+                for (int ch = 0; ch < C::NCH; ++ch)
+                    tma_load_3d(sdO + ch * C::CHUNK_BYTES, &tmdO, bar(B_DOFULL), ch * 64, i0, bh);
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc_st = umma_idesc_bf16(BLK, BLK, false, false);   // S^T, dP^T
+            constexpr uint32_t idesc_dv = umma_idesc_bf16(BLK, D, false, true);      // A tmem / K-major, B MN-major
+            constexpr uint32_t idesc_dq = umma_idesc_bf16(BLK, D, true, true);       // A MN-major, B MN-major
+            auto kmajor_off = [](int kk) { return static_cast<uint32_t>((kk >> 2) * C::CHUNK_BYTES + (kk & 3) * 32); };
+            auto mma1 = [&](int n) {   // S^T = K Q(n)^T -> X
+                const uint32_t qa = sQ + (n & 1) * C::TILE_BYTES;
+#pragma unroll
+                for (int kk = 0; kk < D / 16; ++kk)
+                    umma_ss(tmem + C::TM_X, umma_smem_desc(sK + kmajor_off(kk), 16, 1024),
+                            umma_smem_desc(qa + kmajor_off(kk), 16, 1024), idesc_st, kk > 0);
+                umma_commit(bar(B_SFULL));
+            };
+            auto mma2 = [&]() {        // dP^T = V dO^T -> Y
+#pragma unroll
+                for (int kk = 0; kk < D / 16; ++kk)
+                    umma_ss(tmem + C::TM_Y, umma_smem_desc(sV + kmajor_off(kk), 16, 1024),
+                            umma_smem_desc(sdO + kmajor_off(kk), 16, 1024), idesc_st, kk > 0);
+                umma_commit(bar(B_DPFULL));
+            };
+            mbar_wait(bar(B_KV), 0, status);
+            mbar_wait(bar(B_QFULL + 0), 0, status);
+            tc_fence_after();
+            mma1(0);
+            mbar_wait(bar(B_DOFULL), 0, status);
+            tc_fence_after();
+            mma2();
+            for (int n = 0; n < N; ++n) {
+                const uint32_t qa = sQ + (n & 1) * C::TILE_BYTES;
+                mbar_wait(bar(B_PDSFULL), n & 1, status);
+                tc_fence_after();
+                // MMA4: dV += P^T dO(n).  P^T: queries 0-63 at X[0,32), queries 64-127 at X[64,96)
+#pragma unroll
+                for (int kk = 0; kk < BLK / 16; ++kk)
+                    umma_ts(tmem + C::TM_DV, tmem + C::TM_X + (kk >> 2) * 64 + (kk & 3) * 8,
+                            umma_smem_desc(sdO + kk * 2048, C::CHUNK_BYTES, 1024), idesc_dv, (n > 0 || kk > 0));
+                umma_commit(bar(B_DOEMPTY));
+                // MMA5: dK += dS^T Q(n)
+#pragma unroll
+                for (int kk = 0; kk < BLK / 16; ++kk)
+                    umma_ss(tmem + C::TM_DK, umma_smem_desc(sdS + kmajor_off(kk), 16, 1024),
+                            umma_smem_desc(qa + kk * 2048, C::CHUNK_BYTES, 1024), idesc_dv, (n > 0 || kk > 0));
+                umma_commit(bar(B_QEMPTY + (n & 1)));
+                // MMA6: dQ partial = dS K -> Y
+#pragma unroll
+                for (int kk = 0; kk < BLK / 16; ++kk)
+                    umma_ss(tmem + C::TM_Y, umma_smem_desc(sdS + kk * 2048, C::CHUNK_BYTES, 1024),
+                            umma_smem_desc(sK + kk * 2048, C::CHUNK_BYTES, 1024), idesc_dq, kk > 0);
+                umma_commit(bar(B_DQFULL));
+                if (n + 1 < N) {
+                    mbar_wait(bar(B_QFULL + ((n + 1) & 1)), ((n + 1) >> 1) & 1, status);
+                    tc_fence_after();
+                    mma1(n + 1);
+                    mbar_wait(bar(B_DQEMPTY), n & 1, status);
+                    mbar_wait(bar(B_DOFULL), (n + 1) & 1, status);
+                    tc_fence_after();
+                    mma2();
+                }
+            }
+            umma_commit(bar(B_DKVFULL));
+        }
+        __syncwarp();
+    } else if (warp >= 4) {
+        // ------------------------------------------------------------------ compute warps
+        const int half = (warp - 4) >> 2;                  // which 64 query columns
+        const int r = (tid - 128) & 127;                   // key lane 0..127
+        const uint32_t lane_base = static_cast<uint32_t>(r & ~31) << 16;
+        const uint32_t tX = tmem + lane_base + C::TM_X, tY = tmem + lane_base + C::TM_Y;
+        const int ctid = tid - 128;                        // 0..255
+
+        for (int n = 0; n < N; ++n) {
+            const int i0 = (qb0 + n) * BLK;
+            const uint32_t statL = sStat + (n & 1) * (2 * BLK * 4), statD = statL + BLK * 4;
+            {   // stage LSE (log2 domain) and delta of this query block
+                const int i = i0 + r;
+                if (half == 0) sts32(statL + r * 4, i < S ? LSE[static_cast<size_t>(bh) * S + i] * kLog2e : INFINITY);
+                else           sts32(statD + r * 4, i < S ? DELTA[static_cast<size_t>(bh) * S + i] : 0.f);
+            }
+            named_bar_sync(1, 256);
+            const bool diag = causal && (i0 == j0);
+
+            // P^T = exp2(S^T c - lse)
+            mbar_wait(bar(B_SFULL), n & 1, status);
+            tc_fence_after();
+            float p[64];
+#pragma unroll
+            for (int c = 0; c < 2; ++c) {
+                uint32_t v[32];
+                tmem_ld32(tX + half * 64 + 32 * c, v);
+                tmem_ld_wait();
+#pragma unroll
+                for (int e4 = 0; e4 < 8; ++e4) {
+                    const float4 l4 = lds128(statL + (half * 64 + 32 * c + 4 * e4) * 4);
+                    p[32 * c + 4 * e4 + 0] = ex2(fmaf(__uint_as_float(v[4 * e4 + 0]), c2, -l4.x));
+                    p[32 * c + 4 * e4 + 1] = ex2(fmaf(__uint_as_float(v[4 * e4 + 1]), c2, -l4.y));
+                    p[32 * c + 4 * e4 + 2] = ex2(fmaf(__uint_as_float(v[4 * e4 + 2]), c2, -l4.z));
+                    p[32 * c + 4 * e4 + 3] = ex2(fmaf(__uint_as_float(v[4 * e4 + 3]), c2, -l4.w));
+                }
+                if (diag) {   // keep key j <= query i, i.e. lane r <= column
+#pragma unroll
+                    for (int e = 0; e < 32; ++e)
+                        if (r > half * 64 + 32 * c + e) p[32 * c + e] = 0.f;
+                }
+                uint32_t u[16];
+#pragma unroll
+                for (int e = 0; e < 16; ++e) u[e] = pack_bf16(p[32 * c + 2 * e], p[32 * c + 2 * e + 1]);
+                tmem_st16(tX + half * 64 + 16 * c, u);
+            }
+
+            // dS^T = P^T (dP^T - delta) -> bf16 -> shared memory [key][query]
+            mbar_wait(bar(B_DPFULL), n & 1, status);
+            tc_fence_after();
+#pragma unroll
+            for (int c = 0; c < 2; ++c) {
+                uint32_t v[32];
+                tmem_ld32(tY + half * 64 + 32 * c, v);
+                tmem_ld_wait();
+                uint32_t u[16];
+#pragma unroll
+                for (int e4 = 0; e4 < 8; ++e4) {
+                    const float4 d4 = lds128(statD + (half * 64 + 32 * c + 4 * e4) * 4);
+                    const float a0 = p[32 * c + 4 * e4 + 0] * (__uint_as_float(v[4 * e4 + 0]) - d4.x);
+                    const float a1 = p[32 * c + 4 * e4 + 1] * (__uint_as_float(v[4 * e4 + 1]) - d4.y);
+                    const float a2 = p[32 * c + 4 * e4 + 2] * (__uint_as_float(v[4 * e4 + 2]) - d4.z);
+                    const float a3 = p[32 * c + 4 * e4 + 3] * (__uint_as_float(v[4 * e4 + 3]) - d4.w);
+                    u[2 * e4] = pack_bf16(a0, a1);
+                    u[2 * e4 + 1] = pack_bf16(a2, a3);
+                }
+                const uint32_t rowaddr = sdS + half * C::CHUNK_BYTES + r * 128;
+#pragma unroll
+                for (int q = 0; q < 4; ++q)
+                    sts128(rowaddr + (((4 * c + q) ^ (r & 7)) << 4), u[4 * q], u[4 * q + 1], u[4 * q + 2], u[4 * q + 3]);
+            }
+            tmem_st_wait();
+            fence_proxy_async_smem();
+            tc_fence_before();
+            mbar_arrive(bar(B_PDSFULL));
+
+            // dQ partial of this pair: lanes = queries, columns = d
+            mbar_wait(bar(B_DQFULL), n & 1, status);
+            tc_fence_after();
+            {
+                const int i = i0 + r;
+                float* row = dQacc + (static_cast<size_t>(bh) * S + i) * D;
+#pragma unroll
+                for (int c = 0; c < D / 64; ++c) {
+                    uint32_t v[32];
+                    const int col = half * (D / 2) + 32 * c;
+                    tmem_ld32(tY + col, v);
+                    tmem_ld_wait();
+                    if (i < S) {
+#pragma unroll
+                        for (int e = 0; e < 32; e += 4)
+                            red_add_v4(row + col + e, __uint_as_float(v[e]), __uint_as_float(v[e + 1]),
+                                       __uint_as_float(v[e + 2]), __uint_as_float(v[e + 3]));
+                    }
+                }
+            }
+            tc_fence_before();
+            mbar_arrive(bar(B_DQEMPTY));
+        }
+
+        // ---- epilogue: dK (scaled) by half 0, dV by half 1 -> bf16 -> shared -> TMA store
+        mbar_wait(bar(B_DKVFULL), 0, status);
+        tc_fence_after();
+        {
+            const uint32_t tAcc = tmem + lane_base + (half == 0 ? C::TM_DK : C::TM_DV);
+            const float mul = half == 0 ? scale : 1.0f;
+            const uint32_t stage = sQ + half * C::TILE_BYTES;
+#pragma unroll 1
+            for (int c = 0; c < D / 32; ++c) {
+                uint32_t v[32];
+                tmem_ld32(tAcc + 32 * c, v);
+                tmem_ld_wait();
+                uint32_t u[16];
+#pragma unroll
+                for (int e = 0; e < 16; ++e)
+                    u[e] = pack_bf16(__uint_as_float(v[2 * e]) * mul, __uint_as_float(v[2 * e + 1]) * mul);
+                const uint32_t rowaddr = stage + (c >> 1) * C::CHUNK_BYTES + r * 128;
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const int piece = (c & 1) * 4 + q;
+                    sts128(rowaddr + ((piece ^ (r & 7)) << 4), u[4 * q], u[4 * q + 1], u[4 * q + 2], u[4 * q + 3]);
+                }
+            }
+            fence_proxy_async_smem();
+            named_bar_sync(2 + half, 128);
+            if (r == 0) {
+#pragma unroll
+                for (int ch = 0; ch < C::NCH; ++ch)
+                    tma_store_3d(half == 0 ? &tmdK : &tmdV, stage + ch * C::CHUNK_BYTES, ch * 64, j0, bh);
+                tma_store_commit_and_wait_read();
+            }
+        }
+        (void)ctid;
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem, C::TM_COLS);
+}
+
+// dq = bf16(scale * dq_acc)
+__global__ void __launch_bounds__(256)
+dq_convert_kernel(const float4* __restrict__ acc, uint2* __restrict__ out, size_t n4, float scale)
+{
+    for (size_t i = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x; i < n4;
+         i += static_cast<size_t>(gridDim.x) * blockDim.x) {
+        const float4 a = acc[i];
+        uint2 o;
+        o.x = pack_bf16(a.x * scale, a.y * scale);
+        o.y = pack_bf16(a.z * scale, a.w * scale);
+        out[i] = o;
+    }
+}
+
+template <int D>
+cudaError_t launch(const Problem& p, const void* q, const void* k, const void* v, const void* d_o,
+                   const float* lse, const float* delta, float* dq_acc, void* dq, void* dk, void* dv,
+                   unsigned* status, cudaStream_t st)
+{
+    using C = Cfg<D>;
+    CUtensorMap tq, tk, tv, tdo, tdk, tdv;
+    if (make_tmap_3d(&tq, q, 2, 1, p.BH, p.S, D, 64, BLK)) return cudaErrorInvalidValue;
+    if (make_tmap_3d(&tk, k, 2, 1, p.BH, p.S, D, 64, BLK)) return cudaErrorInvalidValue;
+    if (make_tmap_3d(&tv, v, 2, 1, p.BH, p.S, D, 64, BLK)) return cudaErrorInvalidValue;
+    if (make_tmap_3d(&tdo, d_o, 2, 1, p.BH, p.S, D, 64, BLK)) return cudaErrorInvalidValue;
+    if (make_tmap_3d(&tdk, dk, 2, 1, p.BH, p.S, D, 64, BLK)) return cudaErrorInvalidValue;
+    if (make_tmap_3d(&tdv, dv, 2, 1, p.BH, p.S, D, 64, BLK)) return cudaErrorInvalidValue;
+    auto kern = fast_bwd_kernel<D>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM);
+    if (e != cudaSuccess) return e;
+    const int n_kb = (p.S + BLK - 1) / BLK;
+    const long long blocks = static_cast<long long>(n_kb) * p.BH;
+    if (blocks > 0x7fffffffLL) return cudaErrorInvalidValue;
+    kern<<<static_cast<unsigned>(blocks), kThreads, C::SMEM, st>>>(tq, tk, tv, tdo, tdk, tdv, lse, delta, dq_acc, p.S,
+                                                                   p.BH, p.causal, p.scale, status);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    const size_t n4 = static_cast<size_t>(p.BH) * p.S * D / 4;
+    const unsigned cblocks = static_cast<unsigned>(n4 / 256 + 1 < 148u * 16u ? n4 / 256 + 1 : 148u * 16u);
+    dq_convert_kernel<<<cblocks, 256, 0, st>>>(reinterpret_cast<const float4*>(dq_acc), reinterpret_cast<uint2*>(dq), n4,
+                                               p.scale);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_fast_bwd(const Problem& p, const void* q, const void* k, const void* v, const void* d_o,
+                            const float* lse, const float* delta, float* dq_acc, void* dq, void* dk, void* dv,
+                            unsigned* status, cudaStream_t st)
+{
+    switch (p.D) {
+        case 64:  return launch<64>(p, q, k, v, d_o, lse, delta, dq_acc, dq, dk, dv, status, st);
+        case 128: return launch<128>(p, q, k, v, d_o, lse, delta, dq_acc, dq, dk, dv, status, st);
+        default:  return cudaErrorNotSupported;
+    }
+}
+
+}  // namespace mgn
