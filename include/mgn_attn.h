@@ -99,6 +99,39 @@ int mgn_attn_check(void* stream);
  */
 int mgn_attn_profile_events(void* before_main, void* after_main);
 
+/*
+ * Backward for callers that cannot allocate device memory.  (The paper has no counterpart:
+ * this is a convenience of this library.)
+ *
+ * Who needs it: code that is handed tensors but may not call cudaMalloc -- a plug-in inside a
+ * framework whose memory pool owns the whole GPU, a serving loop where an allocation would
+ * synchronise the device, a caller that has only the pointers it was given.  mgn_attn_bwd asks
+ * such a caller for a workspace it cannot produce; this entry point takes none.  The workspace
+ * is a fixed MGN_NOALLOC_MAX_WORKSPACE_BYTES array inside the library image, so every GPU that
+ * loads the library gives up that much memory until the process exits.
+ *
+ * Arguments, layouts, results and error codes are those of mgn_attn_bwd without `workspace`
+ * and `workspace_bytes`.  Differences:
+ *   - Sizes for which mgn_attn_bwd_workspace_bytes(B,H,S,D,mode) exceeds
+ *     MGN_NOALLOC_MAX_WORKSPACE_BYTES are refused with MGN_ERR_WORKSPACE before anything is
+ *     enqueued (strict mode needs 4 bytes per (b,h,s) row; fast mode 4*(D+1) bytes per row).
+ *   - It calls no cudaMalloc, cudaFree or other allocating routine.
+ *   - The first call on each device looks up the array's device address (a one-time, per-device
+ *     set-up done with that device current); make that first call outside any stream capture.
+ *   - All calls on a device share the one array and it keeps whatever the last call left in it.
+ *     Each call clears or overwrites everything it reads, so calls issued one after another on a
+ *     stream are independent; calls that can overlap on the GPU (different streams, no ordering)
+ *     race on the array and corrupt each other -- serialise them, or use mgn_attn_bwd with
+ *     separate workspaces.
+ */
+#define MGN_NOALLOC_MAX_WORKSPACE_BYTES (8u << 20)
+int mgn_attn_bwd_noalloc(const void* q, const void* k, const void* v, const void* o, const void* d_o,
+                         const float* lse, void* dq, void* dk, void* dv,
+                         int B, int H, int S, int D, int causal, float scale, int mode, void* stream);
+
+/* The constant above, for callers that bind the library without the header. */
+size_t mgn_attn_bwd_noalloc_max_workspace_bytes(void);
+
 /* Static string naming a status code. */
 const char* mgn_status_string(int status);
 

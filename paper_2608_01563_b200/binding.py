@@ -49,6 +49,10 @@ def lib() -> ctypes.CDLL:
         L.mgn_attn_bwd_workspace_bytes.restype = sz
         L.mgn_attn_check.argtypes = [vp]
         L.mgn_attn_check.restype = i
+        L.mgn_attn_bwd_noalloc.argtypes = [vp] * 9 + [i, i, i, i, i, f, i, vp]
+        L.mgn_attn_bwd_noalloc.restype = i
+        L.mgn_attn_bwd_noalloc_max_workspace_bytes.argtypes = []
+        L.mgn_attn_bwd_noalloc_max_workspace_bytes.restype = sz
         L.mgn_attn_profile_events.argtypes = [vp, vp]
         L.mgn_attn_profile_events.restype = i
         L.mgn_status_string.argtypes = [i]
@@ -94,6 +98,21 @@ def mgn_attn_bwd(q, k, v, o, d_o, lse, dq, dk, dv, workspace, causal: bool, scal
                             B, H, S, D, int(causal), float(scale), int(mode), _stream(stream))
     if st != MGN_OK:
         raise MgnError(st, "mgn_attn_bwd")
+
+
+def mgn_attn_bwd_noalloc(q, k, v, o, d_o, lse, dq, dk, dv, causal: bool, scale: float, mode: int,
+                         stream: Optional[int] = None) -> None:
+    """Backward without a caller workspace: for callers that may not allocate device memory.
+    Uses the library's built-in scratch array; sizes beyond it raise MgnError(MGN_ERR_WORKSPACE)."""
+    B, H, S, D = _dims(q)
+    st = lib().mgn_attn_bwd_noalloc(_ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(d_o), _ptr(lse), _ptr(dq), _ptr(dk),
+                                    _ptr(dv), B, H, S, D, int(causal), float(scale), int(mode), _stream(stream))
+    if st != MGN_OK:
+        raise MgnError(st, "mgn_attn_bwd_noalloc")
+
+
+def mgn_attn_bwd_noalloc_max_workspace_bytes() -> int:
+    return int(lib().mgn_attn_bwd_noalloc_max_workspace_bytes())
 
 
 def mgn_attn_check(stream: Optional[int] = None) -> None:
