@@ -52,6 +52,26 @@ def fp32_peak_tflops(peaks):
     return SM_COUNT * FP32_LANES_PER_SM * 2 * peaks.get("sm_max_mhz", 1965.0) * 1e6 / 1e12
 
 
+def rank_workload(w, rank):
+    """Rank r works on its own batch of the same shape (heads are independent units, so there is
+    no data-path collective): same workload, sweep index offset by 1000*r in the seed."""
+    import dataclasses
+    return dataclasses.replace(w, sweep=w.sweep + 1000 * rank)
+
+
+def max_over_ranks(values, dist, device):
+    """Element-wise MAX over ranks of a list of floats (identity without a process group)."""
+    t = torch.tensor(list(values), device=device, dtype=torch.float64)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.tolist()
+
+
+def whole_job_tflops(w, world, steps, total_ms):
+    """Weak scaling: every rank runs the full workload; value = all ranks' counted FLOPs / max time."""
+    return world * flops(w, "sum") * steps / (total_ms * 1e-3) / 1e12
+
+
 class ClockSampler:
     QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
@@ -114,11 +134,17 @@ def cpu_info():
     return model
 
 
+_oracle_inputs = {}
+
+
 def time_oracle(w, dtype, heads, repeats=1):
     """Oracle forward+backward on the first `heads` heads. Returns (seconds fwd, seconds bwd, threads)."""
     from oracle import attn_oracle as orc
-    q, k, v, d_o = synth.make_inputs(w, dtype=dtype, heads=heads)
-    a = [t.double().numpy() for t in (q, k, v, d_o)]
+    key = (w.name, w.sweep, dtype, heads)
+    if key not in _oracle_inputs:
+        _oracle_inputs.clear()
+        _oracle_inputs[key] = [t.double().numpy() for t in synth.make_inputs(w, dtype=dtype, heads=heads)]
+    a = _oracle_inputs[key]
     best_f = best_b = float("inf")
     for _ in range(repeats):
         t0 = time.perf_counter()
@@ -216,8 +242,7 @@ def main():
 
     # Each rank works on its own batch of the same shape (heads are independent units:
     # no data-path collective).  Rank r draws sweep index r*1000 more than rank 0.
-    import dataclasses
-    w_rank = dataclasses.replace(w, sweep=w.sweep + 1000 * rank)
+    w_rank = rank_workload(w, rank)
     host = [t.pin_memory() for t in synth.make_inputs(w_rank, dtype=dtype)]
     dev = [t.cuda(non_blocking=True) for t in host]
     qd, kd, vd, dod = dev
@@ -302,23 +327,21 @@ def main():
     else:
         e2e_ms = None
 
-    t = torch.tensor([total_ms, e2e_ms or 0.0], device="cuda", dtype=torch.float64)
-    if dist is not None:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    total_ms_max, e2e_ms_max = t.tolist()
+    total_ms_max, e2e_ms_max = max_over_ranks([total_ms, e2e_ms or 0.0], dist, "cuda")
 
     if rank == 0:
         peaks, peak_src = measured_peaks()
         fl_sum = flops(w, "sum")
-        value = world * fl_sum * K / (total_ms_max * 1e-3) / 1e12
+        value = whole_job_tflops(w, world, K, total_ms_max)
         if args.mode == "strict":
             peak = fp32_peak_tflops(peaks)
             bound = "alu"
             peak_note = f"{SM_COUNT} SMs x {FP32_LANES_PER_SM} FP32 lanes x 2 x {peaks.get('sm_max_mhz', 1965.0):.0f} MHz"
         else:
-            peak = peaks["bf16_tflops_sustained"]
+            peak = peaks["bf16_tflops"]
             bound = "tensor"
-            peak_note = f"{peak_src} dense bf16 (sustained); burst {peaks['bf16_tflops']}"
+            peak_note = (f"{peak_src} dense bf16, burst figure (steps are ~1 ms bursts); "
+                         f"sustained {peaks['bf16_tflops_sustained']}")
         bwd_main_tflops = flops(w, "bwd") / (bwd_main_ms * 1e-3) / 1e12
         fwd_main_tflops = flops(w, "fwd") / (fwd_main_ms * 1e-3) / 1e12
         line = {
@@ -339,13 +362,13 @@ def main():
                          "ms_per_launch": bwd_main_ms, "peak_source": peak_note,
                          "fwd_kernel": {"achieved": fwd_main_tflops, "frac": fwd_main_tflops / peak,
                                         "ms_per_launch": fwd_main_ms}},
-            "gpu_launches": 3 * K,
+            "gpu_launches": (3 if args.mode == "strict" else 4) * K,
             "clocks": clocks,
         }
         if e2e_ms is not None:
             h2d = sum(t_.numel() * t_.element_size() for t_ in host)
             d2h = sum(t_.numel() * t_.element_size() for t_ in host_out)
-            line["e2e"] = {"value": world * fl_sum * K / (e2e_ms_max * 1e-3) / 1e12, "unit": "TFLOP/s",
+            line["e2e"] = {"value": whole_job_tflops(w, world, K, e2e_ms_max), "unit": "TFLOP/s",
                            "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
         if world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline(w, dtype)
