@@ -14,8 +14,9 @@
 //         the MN-major operand dS (rows = queries)
 //   MMA4  dV  += P^T dO   (A from tensor memory)
 //   MMA5  dK  += dS^T Q   (A from shared memory)
-//   MMA6  dQp  = dS K  -> Y, then read out and added to the f32 dQ accumulator in global memory
-//         with 128-bit reductions (a later kernel scales and converts it to bf16).
+//   MMA6  dQp  = dS K  -> Y, then read out, staged in shared memory (the dS buffer, free by then)
+//         and added to the f32 dQ accumulator in global memory by TMA reduce-add (a later kernel
+//         scales and converts it to bf16).
 // Tensor memory: X [0,128)  Y [128,256)  dK [256,256+D)  dV [256+D,256+2D).
 // Warp roles (384 threads): warp 0 TMA producer, warp 1 MMA issuer, warps 4-11 compute.
 #include <cuda_bf16.h>
@@ -55,7 +56,8 @@ __global__ void __launch_bounds__(kThreads, 1)
 fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                 const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmdO,
                 const __grid_constant__ CUtensorMap tmdK, const __grid_constant__ CUtensorMap tmdV,
-                const float* __restrict__ LSE, const float* __restrict__ DELTA, float* __restrict__ dQacc,
+                const __grid_constant__ CUtensorMap tmdQ,
+                const float* __restrict__ LSE, const float* __restrict__ DELTA,
                 int S, int BH, int causal, float scale, unsigned* status)
 {
     using C = Cfg<D>;
@@ -184,17 +186,23 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         const int r = (tid - 128) & 127;                   // key lane 0..127
         const uint32_t lane_base = static_cast<uint32_t>(r & ~31) << 16;
         const uint32_t tX = tmem + lane_base + C::TM_X, tY = tmem + lane_base + C::TM_Y;
-        const int ctid = tid - 128;                        // 0..255
+
+        // row statistic of query (qb0*BLK + r), prefetched one block ahead: LSE (log2 domain) in
+        // half 0, delta in half 1
+        auto load_stat = [&](int n) -> float {
+            const int i = (qb0 + n) * BLK + r;
+            if (n >= N || i >= S) return half == 0 ? INFINITY : 0.f;
+            return half == 0 ? LSE[static_cast<size_t>(bh) * S + i] * kLog2e : DELTA[static_cast<size_t>(bh) * S + i];
+        };
+        float stat_next = load_stat(0);
+        const uint32_t dq_stage = sdS + half * C::CHUNK_BYTES;     // this warpgroup's 16 KB of the dS buffer
 
         for (int n = 0; n < N; ++n) {
             const int i0 = (qb0 + n) * BLK;
             const uint32_t statL = sStat + (n & 1) * (2 * BLK * 4), statD = statL + BLK * 4;
-            {   // stage LSE (log2 domain) and delta of this query block
-                const int i = i0 + r;
-                if (half == 0) sts32(statL + r * 4, i < S ? LSE[static_cast<size_t>(bh) * S + i] * kLog2e : INFINITY);
-                else           sts32(statD + r * 4, i < S ? DELTA[static_cast<size_t>(bh) * S + i] : 0.f);
-            }
+            sts32((half == 0 ? statL : statD) + r * 4, stat_next);
             named_bar_sync(1, 256);
+            stat_next = load_stat(n + 1);
             const bool diag = causal && (i0 == j0);
 
             // P^T = exp2(S^T c - lse)
@@ -228,6 +236,9 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             // dS^T = P^T (dP^T - delta) -> bf16 -> shared memory [key][query]
             mbar_wait(bar(B_DPFULL), n & 1, status);
             tc_fence_after();
+            // the dQ reduction of the previous pair read its staging from this buffer: let it finish
+            if (r == 0) bulk_wait_group_read0();
+            named_bar_sync(2 + half, 128);
 #pragma unroll
             for (int c = 0; c < 2; ++c) {
                 uint32_t v[32];
@@ -254,29 +265,37 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             tc_fence_before();
             mbar_arrive(bar(B_PDSFULL));
 
-            // dQ partial of this pair: lanes = queries, columns = d
+            // dQ partial of this pair (lanes = queries, columns = d): tensor memory -> registers ->
+            // shared memory (f32, swizzled 32-column boxes, in the dS buffer that MMA5/MMA6 have
+            // finished with) -> TMA reduce-add into the f32 accumulator in global memory.
             mbar_wait(bar(B_DQFULL), n & 1, status);
             tc_fence_after();
-            {
-                const int i = i0 + r;
-                float* row = dQacc + (static_cast<size_t>(bh) * S + i) * D;
 #pragma unroll
-                for (int c = 0; c < D / 64; ++c) {
-                    uint32_t v[32];
-                    const int col = half * (D / 2) + 32 * c;
-                    tmem_ld32(tY + col, v);
-                    tmem_ld_wait();
-                    if (i < S) {
+            for (int c = 0; c < D / 64; ++c) {
+                uint32_t v[32];
+                const int col = half * (D / 2) + 32 * c;
+                tmem_ld32(tY + col, v);
+                tmem_ld_wait();
+                if (c == D / 64 - 1) {          // tensor memory Y is free again
+                    tc_fence_before();
+                    mbar_arrive(bar(B_DQEMPTY));
+                }
+                if (c > 0) {                    // staging is still being read by the previous box
+                    if (r == 0) bulk_wait_group_read0();
+                    named_bar_sync(2 + half, 128);
+                }
 #pragma unroll
-                        for (int e = 0; e < 32; e += 4)
-                            red_add_v4(row + col + e, __uint_as_float(v[e]), __uint_as_float(v[e + 1]),
-                                       __uint_as_float(v[e + 2]), __uint_as_float(v[e + 3]));
-                    }
+                for (int q = 0; q < 8; ++q)
+                    sts128(dq_stage + r * 128 + ((q ^ (r & 7)) << 4), v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+                fence_proxy_async_smem();
+                named_bar_sync(2 + half, 128);
+                if (r == 0) {
+                    tma_reduce_add_3d(&tmdQ, dq_stage, col, i0, bh);
+                    bulk_commit_group();
                 }
             }
-            tc_fence_before();
-            mbar_arrive(bar(B_DQEMPTY));
         }
+        if (r == 0) bulk_wait_group_read0();
 
         // ---- epilogue: dK (scaled) by half 0, dV by half 1 -> bf16 -> shared -> TMA store
         mbar_wait(bar(B_DKVFULL), 0, status);
@@ -310,7 +329,6 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                 tma_store_commit_and_wait_read();
             }
         }
-        (void)ctid;
     }
 
     tc_fence_before();
@@ -338,7 +356,8 @@ cudaError_t launch(const Problem& p, const void* q, const void* k, const void* v
                    unsigned* status, cudaStream_t st)
 {
     using C = Cfg<D>;
-    CUtensorMap tq, tk, tv, tdo, tdk, tdv;
+    CUtensorMap tq, tk, tv, tdo, tdk, tdv, tdq;
+    if (make_tmap_3d(&tdq, dq_acc, 4, 0, p.BH, p.S, D, 32, BLK)) return cudaErrorInvalidValue;
     if (make_tmap_3d(&tq, q, 2, 1, p.BH, p.S, D, 64, BLK)) return cudaErrorInvalidValue;
     if (make_tmap_3d(&tk, k, 2, 1, p.BH, p.S, D, 64, BLK)) return cudaErrorInvalidValue;
     if (make_tmap_3d(&tv, v, 2, 1, p.BH, p.S, D, 64, BLK)) return cudaErrorInvalidValue;
@@ -351,7 +370,7 @@ cudaError_t launch(const Problem& p, const void* q, const void* k, const void* v
     const int n_kb = (p.S + BLK - 1) / BLK;
     const long long blocks = static_cast<long long>(n_kb) * p.BH;
     if (blocks > 0x7fffffffLL) return cudaErrorInvalidValue;
-    kern<<<static_cast<unsigned>(blocks), kThreads, C::SMEM, st>>>(tq, tk, tv, tdo, tdk, tdv, lse, delta, dq_acc, p.S,
+    kern<<<static_cast<unsigned>(blocks), kThreads, C::SMEM, st>>>(tq, tk, tv, tdo, tdk, tdv, tdq, lse, delta, p.S,
                                                                    p.BH, p.causal, p.scale, status);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
