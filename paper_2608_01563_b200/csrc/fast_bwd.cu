@@ -42,9 +42,12 @@ struct Cfg {
     static constexpr int OFF_Q = OFF_V + TILE_BYTES;           // two stages
     static constexpr int OFF_DO = OFF_Q + 2 * TILE_BYTES;
     static constexpr int OFF_DS = OFF_DO + TILE_BYTES;
-    static constexpr int OFF_STAT = OFF_DS + DS_BYTES;         // [2 stages][lse2 | delta][128] f32
-    static constexpr int OFF_BAR = OFF_STAT + 2 * 2 * BLK * 4;
-    static constexpr int SMEM = OFF_BAR + 256 + 1024;
+    static constexpr int OFF_DQ1 = OFF_DS + DS_BYTES;          // second dQ staging box (D = 128 only)
+    static constexpr int DQ1_BYTES = (D == 128) ? 2 * CHUNK_BYTES : 0;
+    static constexpr int OFF_STAT = OFF_DQ1 + DQ1_BYTES;       // [lse2 | delta][128] f32
+    static constexpr int OFF_BAR = OFF_STAT + 2 * BLK * 4;
+    static constexpr int SMEM = OFF_BAR + 128 + 1024;
+    static_assert(SMEM <= 232448, "shared memory budget");
     static constexpr uint32_t TM_X = 0, TM_Y = 128, TM_DK = 256, TM_DV = 256 + D, TM_COLS = 512;
 };
 
@@ -155,6 +158,13 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                     umma_ts(tmem + C::TM_DV, tmem + C::TM_X + (kk >> 2) * 64 + (kk & 3) * 8,
                             umma_smem_desc(sdO + kk * 2048, C::CHUNK_BYTES, 1024), idesc_dv, (n > 0 || kk > 0));
                 umma_commit(bar(B_DOEMPTY));
+                // MMA1 of the next pair right behind it: X is free once MMA4 has read P^T, and the
+                // compute warps can then exponentiate the next scores while MMA5/MMA6 run
+                if (n + 1 < N) {
+                    mbar_wait(bar(B_QFULL + ((n + 1) & 1)), ((n + 1) >> 1) & 1, status);
+                    tc_fence_after();
+                    mma1(n + 1);
+                }
                 // MMA5: dK += dS^T Q(n)
 #pragma unroll
                 for (int kk = 0; kk < BLK / 16; ++kk)
@@ -168,9 +178,6 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                             umma_smem_desc(sK + kk * 2048, C::CHUNK_BYTES, 1024), idesc_dq, kk > 0);
                 umma_commit(bar(B_DQFULL));
                 if (n + 1 < N) {
-                    mbar_wait(bar(B_QFULL + ((n + 1) & 1)), ((n + 1) >> 1) & 1, status);
-                    tc_fence_after();
-                    mma1(n + 1);
                     mbar_wait(bar(B_DQEMPTY), n & 1, status);
                     mbar_wait(bar(B_DOFULL), (n + 1) & 1, status);
                     tc_fence_after();
@@ -194,49 +201,58 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             if (n >= N || i >= S) return half == 0 ? INFINITY : 0.f;
             return half == 0 ? LSE[static_cast<size_t>(bh) * S + i] * kLog2e : DELTA[static_cast<size_t>(bh) * S + i];
         };
-        float stat_next = load_stat(0);
-        const uint32_t dq_stage = sdS + half * C::CHUNK_BYTES;     // this warpgroup's 16 KB of the dS buffer
+        const uint32_t statL = sStat, statD = sStat + BLK * 4;
+        const uint32_t dq_stage0 = sdS + half * C::CHUNK_BYTES;              // this warpgroup's 16 KB of the dS buffer
+        const uint32_t dq_stage1 = base + C::OFF_DQ1 + half * C::CHUNK_BYTES;
+        uint32_t pk[32];                                                     // P^T of the current pair, packed bf16
 
-        for (int n = 0; n < N; ++n) {
-            const int i0 = (qb0 + n) * BLK;
-            const uint32_t statL = sStat + (n & 1) * (2 * BLK * 4), statD = statL + BLK * 4;
-            sts32((half == 0 ? statL : statD) + r * 4, stat_next);
-            named_bar_sync(1, 256);
-            stat_next = load_stat(n + 1);
-            const bool diag = causal && (i0 == j0);
-
-            // P^T = exp2(S^T c - lse)
+        // P^T = exp2(S^T c - lse) of pair n: bf16 into X (A operand of dV) and into pk (for dS)
+        auto exp_phase = [&](int n) {
+            const bool diag = causal && ((qb0 + n) * BLK == j0);
             mbar_wait(bar(B_SFULL), n & 1, status);
             tc_fence_after();
-            float p[64];
 #pragma unroll
             for (int c = 0; c < 2; ++c) {
                 uint32_t v[32];
                 tmem_ld32(tX + half * 64 + 32 * c, v);
                 tmem_ld_wait();
+                float p[32];
 #pragma unroll
                 for (int e4 = 0; e4 < 8; ++e4) {
                     const float4 l4 = lds128(statL + (half * 64 + 32 * c + 4 * e4) * 4);
-                    p[32 * c + 4 * e4 + 0] = ex2(fmaf(__uint_as_float(v[4 * e4 + 0]), c2, -l4.x));
-                    p[32 * c + 4 * e4 + 1] = ex2(fmaf(__uint_as_float(v[4 * e4 + 1]), c2, -l4.y));
-                    p[32 * c + 4 * e4 + 2] = ex2(fmaf(__uint_as_float(v[4 * e4 + 2]), c2, -l4.z));
-                    p[32 * c + 4 * e4 + 3] = ex2(fmaf(__uint_as_float(v[4 * e4 + 3]), c2, -l4.w));
+                    p[4 * e4 + 0] = ex2(fmaf(__uint_as_float(v[4 * e4 + 0]), c2, -l4.x));
+                    p[4 * e4 + 1] = ex2(fmaf(__uint_as_float(v[4 * e4 + 1]), c2, -l4.y));
+                    p[4 * e4 + 2] = ex2(fmaf(__uint_as_float(v[4 * e4 + 2]), c2, -l4.z));
+                    p[4 * e4 + 3] = ex2(fmaf(__uint_as_float(v[4 * e4 + 3]), c2, -l4.w));
                 }
                 if (diag) {   // keep key j <= query i, i.e. lane r <= column
 #pragma unroll
                     for (int e = 0; e < 32; ++e)
-                        if (r > half * 64 + 32 * c + e) p[32 * c + e] = 0.f;
+                        if (r > half * 64 + 32 * c + e) p[e] = 0.f;
                 }
                 uint32_t u[16];
 #pragma unroll
-                for (int e = 0; e < 16; ++e) u[e] = pack_bf16(p[32 * c + 2 * e], p[32 * c + 2 * e + 1]);
+                for (int e = 0; e < 16; ++e) {
+                    u[e] = pack_bf16(p[2 * e], p[2 * e + 1]);
+                    pk[16 * c + e] = u[e];
+                }
                 tmem_st16(tX + half * 64 + 16 * c, u);
             }
+        };
+
+        float stat_next = load_stat(0);
+        sts32((half == 0 ? statL : statD) + r * 4, stat_next);
+        named_bar_sync(1, 256);
+        stat_next = load_stat(1);
+        exp_phase(0);
+
+        for (int n = 0; n < N; ++n) {
+            const int i0 = (qb0 + n) * BLK;
 
             // dS^T = P^T (dP^T - delta) -> bf16 -> shared memory [key][query]
             mbar_wait(bar(B_DPFULL), n & 1, status);
             tc_fence_after();
-            // the dQ reduction of the previous pair read its staging from this buffer: let it finish
+            // earlier dQ reductions read their staging from this buffer: let them finish
             if (r == 0) bulk_wait_group_read0();
             named_bar_sync(2 + half, 128);
 #pragma unroll
@@ -248,10 +264,11 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
 #pragma unroll
                 for (int e4 = 0; e4 < 8; ++e4) {
                     const float4 d4 = lds128(statD + (half * 64 + 32 * c + 4 * e4) * 4);
-                    const float a0 = p[32 * c + 4 * e4 + 0] * (__uint_as_float(v[4 * e4 + 0]) - d4.x);
-                    const float a1 = p[32 * c + 4 * e4 + 1] * (__uint_as_float(v[4 * e4 + 1]) - d4.y);
-                    const float a2 = p[32 * c + 4 * e4 + 2] * (__uint_as_float(v[4 * e4 + 2]) - d4.z);
-                    const float a3 = p[32 * c + 4 * e4 + 3] * (__uint_as_float(v[4 * e4 + 3]) - d4.w);
+                    const uint32_t k0 = pk[16 * c + 2 * e4], k1 = pk[16 * c + 2 * e4 + 1];
+                    const float a0 = __uint_as_float(k0 << 16) * (__uint_as_float(v[4 * e4 + 0]) - d4.x);
+                    const float a1 = __uint_as_float(k0 & 0xffff0000u) * (__uint_as_float(v[4 * e4 + 1]) - d4.y);
+                    const float a2 = __uint_as_float(k1 << 16) * (__uint_as_float(v[4 * e4 + 2]) - d4.z);
+                    const float a3 = __uint_as_float(k1 & 0xffff0000u) * (__uint_as_float(v[4 * e4 + 3]) - d4.w);
                     u[2 * e4] = pack_bf16(a0, a1);
                     u[2 * e4 + 1] = pack_bf16(a2, a3);
                 }
@@ -265,32 +282,41 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             tc_fence_before();
             mbar_arrive(bar(B_PDSFULL));
 
+            // next pair's statistics and exponentials while MMA5/MMA6 of this pair run
+            if (n + 1 < N) {
+                named_bar_sync(1, 256);        // everyone is done reading this pair's statistics
+                sts32((half == 0 ? statL : statD) + r * 4, stat_next);
+                named_bar_sync(1, 256);
+                stat_next = load_stat(n + 2);
+                exp_phase(n + 1);
+            }
+
             // dQ partial of this pair (lanes = queries, columns = d): tensor memory -> registers ->
-            // shared memory (f32, swizzled 32-column boxes, in the dS buffer that MMA5/MMA6 have
-            // finished with) -> TMA reduce-add into the f32 accumulator in global memory.
+            // shared memory (f32, swizzled 32-column boxes; the first box in the dS buffer that
+            // MMA5/MMA6 have finished with) -> TMA reduce-add into the f32 accumulator in global memory.
             mbar_wait(bar(B_DQFULL), n & 1, status);
             tc_fence_after();
-#pragma unroll
-            for (int c = 0; c < D / 64; ++c) {
-                uint32_t v[32];
-                const int col = half * (D / 2) + 32 * c;
-                tmem_ld32(tY + col, v);
+            {
+                uint32_t v0[32], v1[32];
+                const int col = half * (D / 2);
+                tmem_ld32(tY + col, v0);
+                if constexpr (D == 128) tmem_ld32(tY + col + 32, v1);
                 tmem_ld_wait();
-                if (c == D / 64 - 1) {          // tensor memory Y is free again
-                    tc_fence_before();
-                    mbar_arrive(bar(B_DQEMPTY));
-                }
-                if (c > 0) {                    // staging is still being read by the previous box
-                    if (r == 0) bulk_wait_group_read0();
-                    named_bar_sync(2 + half, 128);
-                }
+                tc_fence_before();
+                mbar_arrive(bar(B_DQEMPTY));     // tensor memory Y is free again
 #pragma unroll
                 for (int q = 0; q < 8; ++q)
-                    sts128(dq_stage + r * 128 + ((q ^ (r & 7)) << 4), v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+                    sts128(dq_stage0 + r * 128 + ((q ^ (r & 7)) << 4), v0[4 * q], v0[4 * q + 1], v0[4 * q + 2], v0[4 * q + 3]);
+                if constexpr (D == 128) {
+#pragma unroll
+                    for (int q = 0; q < 8; ++q)
+                        sts128(dq_stage1 + r * 128 + ((q ^ (r & 7)) << 4), v1[4 * q], v1[4 * q + 1], v1[4 * q + 2], v1[4 * q + 3]);
+                }
                 fence_proxy_async_smem();
                 named_bar_sync(2 + half, 128);
                 if (r == 0) {
-                    tma_reduce_add_3d(&tmdQ, dq_stage, col, i0, bh);
+                    tma_reduce_add_3d(&tmdQ, dq_stage0, col, i0, bh);
+                    if constexpr (D == 128) tma_reduce_add_3d(&tmdQ, dq_stage1, col + 32, i0, bh);
                     bulk_commit_group();
                 }
             }
