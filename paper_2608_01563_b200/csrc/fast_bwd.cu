@@ -14,11 +14,17 @@
 //         the MN-major operand dS (rows = queries)
 //   MMA4  dV  += P^T dO   (A from tensor memory)
 //   MMA5  dK  += dS^T Q   (A from shared memory)
-//   MMA6  dQp  = dS K  -> Y, then read out, staged in shared memory (the dS buffer, free by then)
-//         and added to the f32 dQ accumulator in global memory by TMA reduce-add (a later kernel
-//         scales and converts it to bf16).
+//   MMA6  dQp  = dS K  -> Y, then drained by a dedicated warpgroup: tensor memory -> registers ->
+//         a 32 KB shared-memory staging area (f32, swizzled 32-column boxes) -> TMA reduce-add into
+//         the f32 dQ accumulator in global memory (a later kernel scales and converts it to bf16).
+//         Global f32 reduce-add runs at about 20 bytes per clock per SM on this part (3300 clocks
+//         for one 64 KB partial), and issued from the load/store unit it stalls every shared-memory
+//         access of the SM; so it goes through TMA and is waited for only by the drain warps.
+// Issue order per pair: MMA4(n), MMA1(n+1), MMA6(n), MMA5(n), MMA2(n+1): the next scores are ready
+// while dQ/dK are still being multiplied, and dP^T(n+1) follows as soon as Y has been drained.
 // Tensor memory: X [0,128)  Y [128,256)  dK [256,256+D)  dV [256+D,256+2D).
-// Warp roles (384 threads): warp 0 TMA producer, warp 1 MMA issuer, warps 4-11 compute.
+// Warp roles (512 threads): warp 0 TMA producer, warp 1 MMA issuer, warps 4-11 compute,
+// warps 12-15 dQ drain; register budgets are rebalanced with setmaxnreg (88 / 136 / 136 / 144).
 #include <cuda_bf16.h>
 
 #include "kernels.h"
@@ -27,7 +33,7 @@
 namespace mgn {
 namespace {
 
-constexpr int kThreads = 384;
+constexpr int kThreads = 512;
 constexpr int BLK = 128;     // keys per CTA block and query rows per step
 constexpr float kLog2e = 1.4426950408889634f;
 
@@ -42,9 +48,8 @@ struct Cfg {
     static constexpr int OFF_Q = OFF_V + TILE_BYTES;           // two stages
     static constexpr int OFF_DO = OFF_Q + 2 * TILE_BYTES;
     static constexpr int OFF_DS = OFF_DO + TILE_BYTES;
-    static constexpr int OFF_DQ1 = OFF_DS + DS_BYTES;          // second dQ staging box (D = 128 only)
-    static constexpr int DQ1_BYTES = (D == 128) ? 2 * CHUNK_BYTES : 0;
-    static constexpr int OFF_STAT = OFF_DQ1 + DQ1_BYTES;       // [lse2 | delta][128] f32
+    static constexpr int OFF_DQ = OFF_DS + DS_BYTES;           // dQ staging: 2 boxes of 128 rows x 32 f32
+    static constexpr int OFF_STAT = OFF_DQ + 2 * CHUNK_BYTES;  // [lse2 | delta][128] f32
     static constexpr int OFF_BAR = OFF_STAT + 2 * BLK * 4;
     static constexpr int SMEM = OFF_BAR + 128 + 1024;
     static_assert(SMEM <= 232448, "shared memory budget");
@@ -84,7 +89,7 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     const float c2 = scale * kLog2e;
 
     if (tid == 0) {
-        for (int i = 0; i < B_COUNT; ++i) mbar_init(bar(i), (i == B_PDSFULL || i == B_DQEMPTY) ? 256 : 1);
+        for (int i = 0; i < B_COUNT; ++i) mbar_init(bar(i), i == B_PDSFULL ? 256 : (i == B_DQEMPTY ? 128 : 1));
         fence_mbar_init();
     }
     __syncwarp();
@@ -94,9 +99,11 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     tc_fence_after();
     const uint32_t tmem = lds32u(tmem_slot);
 
-    if (warp == 0) {
+    if (warp < 4) {
+        reg_dealloc<88>();
+        if (warp == 0 && lane == 0) {
         // ------------------------------------------------------------------ TMA producer
-        if (lane == 0) {
+        {
             mbar_arrive_expect_tx(bar(B_KV), 2 * C::TILE_BYTES);
 #pragma unroll
             for (int ch = 0; ch < C::NCH; ++ch) {
@@ -118,10 +125,9 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                     tma_load_3d(sdO + ch * C::CHUNK_BYTES, &tmdO, bar(B_DOFULL), ch * 64, i0, bh);
             }
         }
-        __syncwarp();
-    } else if (warp == 1) {
+        } else if (warp == 1 && lane == 0) {
         // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
+        {
             constexpr uint32_t idesc_st = umma_idesc_bf16(BLK, BLK, false, false);   // S^T, dP^T
             constexpr uint32_t idesc_dv = umma_idesc_bf16(BLK, D, false, true);      // A tmem / K-major, B MN-major
             constexpr uint32_t idesc_dq = umma_idesc_bf16(BLK, D, true, true);       // A MN-major, B MN-major
@@ -165,18 +171,18 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                     tc_fence_after();
                     mma1(n + 1);
                 }
+                // MMA6: dQ partial = dS K -> Y (first, so that the drain can start early)
+#pragma unroll
+                for (int kk = 0; kk < BLK / 16; ++kk)
+                    umma_ss(tmem + C::TM_Y, umma_smem_desc(sdS + kk * 2048, C::CHUNK_BYTES, 1024),
+                            umma_smem_desc(sK + kk * 2048, C::CHUNK_BYTES, 1024), idesc_dq, kk > 0);
+                umma_commit(bar(B_DQFULL));
                 // MMA5: dK += dS^T Q(n)
 #pragma unroll
                 for (int kk = 0; kk < BLK / 16; ++kk)
                     umma_ss(tmem + C::TM_DK, umma_smem_desc(sdS + kmajor_off(kk), 16, 1024),
                             umma_smem_desc(qa + kk * 2048, C::CHUNK_BYTES, 1024), idesc_dv, (n > 0 || kk > 0));
                 umma_commit(bar(B_QEMPTY + (n & 1)));
-                // MMA6: dQ partial = dS K -> Y
-#pragma unroll
-                for (int kk = 0; kk < BLK / 16; ++kk)
-                    umma_ss(tmem + C::TM_Y, umma_smem_desc(sdS + kk * 2048, C::CHUNK_BYTES, 1024),
-                            umma_smem_desc(sK + kk * 2048, C::CHUNK_BYTES, 1024), idesc_dq, kk > 0);
-                umma_commit(bar(B_DQFULL));
                 if (n + 1 < N) {
                     mbar_wait(bar(B_DQEMPTY), n & 1, status);
                     mbar_wait(bar(B_DOFULL), (n + 1) & 1, status);
@@ -186,24 +192,63 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             }
             umma_commit(bar(B_DKVFULL));
         }
+        }
         __syncwarp();
-    } else if (warp >= 4) {
+    } else if (warp >= 12) {
+        // ------------------------------------------------------------------ dQ drain warps
+        reg_alloc<144>();
+        const int r = tid - 384;                           // query row of the block = tensor-memory lane
+        const uint32_t tY = tmem + (static_cast<uint32_t>(r & ~31) << 16) + C::TM_Y;
+        const uint32_t stage = base + C::OFF_DQ;
+        for (int n = 0; n < N; ++n) {
+            const int i0 = (qb0 + n) * BLK;
+            mbar_wait(bar(B_DQFULL), n & 1, status);
+            tc_fence_after();
+            uint32_t v[D / 32][32];
+#pragma unroll
+            for (int c = 0; c < D / 32; ++c) tmem_ld32(tY + 32 * c, v[c]);
+            tmem_ld_wait();
+            tc_fence_before();
+            mbar_arrive(bar(B_DQEMPTY));                   // Y may be overwritten by dP^T of the next pair
+#pragma unroll
+            for (int round = 0; round < D / 64; ++round) {
+                // the previous reduction must have finished reading the staging area
+                if (r == 0) bulk_wait_group_read0();
+                named_bar_sync(4, 128);
+#pragma unroll
+                for (int b = 0; b < 2; ++b)
+#pragma unroll
+                    for (int q = 0; q < 8; ++q)
+                        sts128(stage + b * C::CHUNK_BYTES + r * 128 + ((q ^ (r & 7)) << 4), v[2 * round + b][4 * q],
+                               v[2 * round + b][4 * q + 1], v[2 * round + b][4 * q + 2], v[2 * round + b][4 * q + 3]);
+                fence_proxy_async_smem();
+                named_bar_sync(4, 128);
+                if (r == 0) {
+                    tma_reduce_add_3d(&tmdQ, stage, 64 * round, i0, bh);
+                    tma_reduce_add_3d(&tmdQ, stage + C::CHUNK_BYTES, 64 * round + 32, i0, bh);
+                    bulk_commit_group();
+                }
+            }
+        }
+        if (r == 0) bulk_wait_group_read0();
+    } else {
         // ------------------------------------------------------------------ compute warps
+        reg_alloc<136>();
         const int half = (warp - 4) >> 2;                  // which 64 query columns
         const int r = (tid - 128) & 127;                   // key lane 0..127
         const uint32_t lane_base = static_cast<uint32_t>(r & ~31) << 16;
         const uint32_t tX = tmem + lane_base + C::TM_X, tY = tmem + lane_base + C::TM_Y;
 
-        // row statistic of query (qb0*BLK + r), prefetched one block ahead: LSE (log2 domain) in
-        // half 0, delta in half 1
-        auto load_stat = [&](int n) -> float {
-            const int i = (qb0 + n) * BLK + r;
-            if (n >= N || i >= S) return half == 0 ? INFINITY : 0.f;
-            return half == 0 ? LSE[static_cast<size_t>(bh) * S + i] * kLog2e : DELTA[static_cast<size_t>(bh) * S + i];
-        };
+        // Row statistics of the 64 query columns this warpgroup works on, prefetched one block
+        // ahead: threads 0-63 of the warpgroup fetch LSE (log2 domain), threads 64-127 fetch delta.
+        // Each warpgroup writes only the entries it reads, so the buffer needs no cross-warpgroup sync.
         const uint32_t statL = sStat, statD = sStat + BLK * 4;
-        const uint32_t dq_stage0 = sdS + half * C::CHUNK_BYTES;              // this warpgroup's 16 KB of the dS buffer
-        const uint32_t dq_stage1 = base + C::OFF_DQ1 + half * C::CHUNK_BYTES;
+        const uint32_t my_stat = (r < 64 ? statL : statD) + (half * 64 + (r & 63)) * 4;
+        auto load_stat = [&](int n) -> float {
+            const int i = (qb0 + n) * BLK + half * 64 + (r & 63);
+            if (n >= N || i >= S) return r < 64 ? INFINITY : 0.f;
+            return r < 64 ? LSE[static_cast<size_t>(bh) * S + i] * kLog2e : DELTA[static_cast<size_t>(bh) * S + i];
+        };
         uint32_t pk[32];                                                     // P^T of the current pair, packed bf16
 
         // P^T = exp2(S^T c - lse) of pair n: bf16 into X (A operand of dV) and into pk (for dS)
@@ -241,20 +286,15 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         };
 
         float stat_next = load_stat(0);
-        sts32((half == 0 ? statL : statD) + r * 4, stat_next);
-        named_bar_sync(1, 256);
+        sts32(my_stat, stat_next);
+        named_bar_sync(2 + half, 128);
         stat_next = load_stat(1);
         exp_phase(0);
 
         for (int n = 0; n < N; ++n) {
-            const int i0 = (qb0 + n) * BLK;
-
             // dS^T = P^T (dP^T - delta) -> bf16 -> shared memory [key][query]
             mbar_wait(bar(B_DPFULL), n & 1, status);
             tc_fence_after();
-            // earlier dQ reductions read their staging from this buffer: let them finish
-            if (r == 0) bulk_wait_group_read0();
-            named_bar_sync(2 + half, 128);
 #pragma unroll
             for (int c = 0; c < 2; ++c) {
                 uint32_t v[32];
@@ -282,46 +322,15 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             tc_fence_before();
             mbar_arrive(bar(B_PDSFULL));
 
-            // next pair's statistics and exponentials while MMA5/MMA6 of this pair run
+            // next pair's statistics and exponentials while the dQ/dK products of this pair run
             if (n + 1 < N) {
-                named_bar_sync(1, 256);        // everyone is done reading this pair's statistics
-                sts32((half == 0 ? statL : statD) + r * 4, stat_next);
-                named_bar_sync(1, 256);
+                named_bar_sync(2 + half, 128);     // this warpgroup is done reading the old statistics
+                sts32(my_stat, stat_next);
+                named_bar_sync(2 + half, 128);
                 stat_next = load_stat(n + 2);
                 exp_phase(n + 1);
             }
-
-            // dQ partial of this pair (lanes = queries, columns = d): tensor memory -> registers ->
-            // shared memory (f32, swizzled 32-column boxes; the first box in the dS buffer that
-            // MMA5/MMA6 have finished with) -> TMA reduce-add into the f32 accumulator in global memory.
-            mbar_wait(bar(B_DQFULL), n & 1, status);
-            tc_fence_after();
-            {
-                uint32_t v0[32], v1[32];
-                const int col = half * (D / 2);
-                tmem_ld32(tY + col, v0);
-                if constexpr (D == 128) tmem_ld32(tY + col + 32, v1);
-                tmem_ld_wait();
-                tc_fence_before();
-                mbar_arrive(bar(B_DQEMPTY));     // tensor memory Y is free again
-#pragma unroll
-                for (int q = 0; q < 8; ++q)
-                    sts128(dq_stage0 + r * 128 + ((q ^ (r & 7)) << 4), v0[4 * q], v0[4 * q + 1], v0[4 * q + 2], v0[4 * q + 3]);
-                if constexpr (D == 128) {
-#pragma unroll
-                    for (int q = 0; q < 8; ++q)
-                        sts128(dq_stage1 + r * 128 + ((q ^ (r & 7)) << 4), v1[4 * q], v1[4 * q + 1], v1[4 * q + 2], v1[4 * q + 3]);
-                }
-                fence_proxy_async_smem();
-                named_bar_sync(2 + half, 128);
-                if (r == 0) {
-                    tma_reduce_add_3d(&tmdQ, dq_stage0, col, i0, bh);
-                    if constexpr (D == 128) tma_reduce_add_3d(&tmdQ, dq_stage1, col + 32, i0, bh);
-                    bulk_commit_group();
-                }
-            }
         }
-        if (r == 0) bulk_wait_group_read0();
 
         // ---- epilogue: dK (scaled) by half 0, dV by half 1 -> bf16 -> shared -> TMA store
         mbar_wait(bar(B_DKVFULL), 0, status);
