@@ -85,9 +85,11 @@ fast_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     tc_fence_after();
     const uint32_t tmem = lds32u(tmem_slot);
 
-    if (warp == 0) {
+    if (warp < 4) {
+        reg_dealloc<72>();
+        if (warp == 0 && lane == 0) {
         // ------------------------------------------------------------------ TMA producer
-        if (lane == 0) {
+        {
             const int nq = (nblk[1] > 0) ? 2 : 1;
             mbar_arrive_expect_tx(bar(B_Q), nq * C::TILE_BYTES);
             for (int t = 0; t < nq; ++t)
@@ -109,10 +111,9 @@ fast_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                     tma_load_3d(sV + st * C::TILE_BYTES + ch * C::CHUNK_BYTES, &tmV, bar(B_VFULL + st), ch * 64, n * BN, bh);
             }
         }
-        __syncwarp();
-    } else if (warp == 1) {
+        } else if (warp == 1 && lane == 0) {
         // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
+        {
             constexpr uint32_t idesc_s = umma_idesc_bf16(BM, BN, false, false);
             constexpr uint32_t idesc_o = umma_idesc_bf16(BM, D, false, true);
             auto issue_s = [&](int t, int n) {   // S_t = Q_t K(n)^T
@@ -156,9 +157,11 @@ fast_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                 if (n + 1 < n_max) umma_commit(bar(B_KEMPTY + (st ^ 1)));
             }
         }
+        }
         __syncwarp();
-    } else if (warp >= 4) {
+    } else {
         // ------------------------------------------------------------------ softmax + epilogue
+        reg_alloc<216>();
         const int t = (warp - 4) >> 2;
         const int r = tid - 128 * (1 + t);                 // row within the tile, 0..127
         const uint32_t lane_base = static_cast<uint32_t>(r & ~31) << 16;
@@ -175,78 +178,92 @@ fast_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             const bool masked = (causal && (j0 + BN - 1 > row0[t])) || (j0 + BN > S);
             const int jmax = min(S - 1, causal ? i : S - 1) - j0;   // columns c <= jmax of this block are visible
 
-            // pass 1: block maximum of the scaled scores
-            float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
-#pragma unroll 1
-            for (int c = 0; c < 4; ++c) {
-                uint32_t v[32];
-                tmem_ld32(tS + 32 * c, v);
-                tmem_ld_wait();
-                float x[32];
-#pragma unroll
-                for (int e = 0; e < 32; ++e) x[e] = __uint_as_float(v[e]) * c2;
-                if (masked) {
-#pragma unroll
-                    for (int e = 0; e < 32; ++e)
-                        if (32 * c + e > jmax) x[e] = -INFINITY;
-                }
-#pragma unroll
-                for (int e = 0; e < 32; e += 4) {
-                    mx0 = fmaxf(mx0, x[e]);
-                    mx1 = fmaxf(mx1, x[e + 1]);
-                    mx2 = fmaxf(mx2, x[e + 2]);
-                    mx3 = fmaxf(mx3, x[e + 3]);
-                }
-            }
-            const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
             if (n == 0) {
-                m_ref = mx;      // finite: key 0 is visible to every row
-            } else {
-                const bool grow = (mx - m_ref) > kRescaleThreshold;
-                if (__any_sync(0xffffffffu, grow)) {
-                    const float m_new = fmaxf(m_ref, mx);
-                    const float alpha = ex2(m_ref - m_new);
-                    m_ref = m_new;
-                    l *= alpha;
+                // first block: the reference point is the block maximum of the scaled scores
+                float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
 #pragma unroll 1
-                    for (int c = 0; c < D / 32; ++c) {
-                        uint32_t v[32];
-                        tmem_ld32(tO + 32 * c, v);
-                        tmem_ld_wait();
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t v[32];
+                    tmem_ld32(tS + 32 * c, v);
+                    tmem_ld_wait();
+                    float x[32];
 #pragma unroll
-                        for (int e = 0; e < 32; ++e) v[e] = __float_as_uint(__uint_as_float(v[e]) * alpha);
-                        tmem_st32(tO + 32 * c, v);
+                    for (int e = 0; e < 32; ++e) x[e] = __uint_as_float(v[e]) * c2;
+                    if (masked) {
+#pragma unroll
+                        for (int e = 0; e < 32; ++e)
+                            if (32 * c + e > jmax) x[e] = -INFINITY;
                     }
-                    tmem_st_wait();
+#pragma unroll
+                    for (int e = 0; e < 32; e += 4) {
+                        mx0 = fmaxf(mx0, x[e]);
+                        mx1 = fmaxf(mx1, x[e + 1]);
+                        mx2 = fmaxf(mx2, x[e + 2]);
+                        mx3 = fmaxf(mx3, x[e + 3]);
+                    }
                 }
+                m_ref = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));      // finite: key 0 is visible to every row
             }
 
-            // pass 2: P = exp2(s*c2 - m_ref) -> bf16 into tensor memory over S; row sum
-            float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
-            const float neg_m = -m_ref;
-#pragma unroll 1
-            for (int c = 0; c < 4; ++c) {
-                uint32_t v[32];
-                tmem_ld32(tS + 32 * c, v);
-                tmem_ld_wait();
-                float p[32];
+            // One pass: y = s*c2 - m_ref, p = exp2(y), row sum, bf16 pack (kept in registers), and the
+            // largest y.  If some row of the warp outgrew the reference point by more than the
+            // threshold, move the reference, rescale O and l, and redo the pass (S is still intact:
+            // P is written over it only afterwards).
+            uint32_t pk[64];
+            float lsum = 0.f;
+            for (int attempt = 0; attempt < 2; ++attempt) {
+                float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
+                float y0 = -INFINITY, y1 = -INFINITY, y2 = -INFINITY, y3 = -INFINITY;
+                const float neg_m = -m_ref;
 #pragma unroll
-                for (int e = 0; e < 32; ++e) p[e] = ex2(fmaf(__uint_as_float(v[e]), c2, neg_m));
-                if (masked) {
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t v[32];
+                    tmem_ld32(tS + 32 * c, v);
+                    tmem_ld_wait();
+                    float y[32];
 #pragma unroll
-                    for (int e = 0; e < 32; ++e)
-                        if (32 * c + e > jmax) p[e] = 0.f;
+                    for (int e = 0; e < 32; ++e) y[e] = fmaf(__uint_as_float(v[e]), c2, neg_m);
+                    if (masked) {
+#pragma unroll
+                        for (int e = 0; e < 32; ++e)
+                            if (32 * c + e > jmax) y[e] = -INFINITY;
+                    }
+#pragma unroll
+                    for (int e = 0; e < 32; e += 4) {
+                        y0 = fmaxf(y0, y[e]); y1 = fmaxf(y1, y[e + 1]); y2 = fmaxf(y2, y[e + 2]); y3 = fmaxf(y3, y[e + 3]);
+                        const float p0 = ex2(y[e]), p1 = ex2(y[e + 1]), p2 = ex2(y[e + 2]), p3 = ex2(y[e + 3]);
+                        l0 += p0; l1 += p1; l2 += p2; l3 += p3;
+                        pk[16 * c + e / 2] = pack_bf16(p0, p1);
+                        pk[16 * c + e / 2 + 1] = pack_bf16(p2, p3);
+                    }
                 }
+                lsum = (l0 + l1) + (l2 + l3);
+                const float ymax = fmaxf(fmaxf(y0, y1), fmaxf(y2, y3));
+                const bool grow = ymax > kRescaleThreshold;
+                if (attempt == 1 || !__any_sync(0xffffffffu, grow)) break;
+                // move the reference point of every row of this warp
+                const float m_new = fmaxf(m_ref, m_ref + ymax);
+                const float alpha = ex2(m_ref - m_new);
+                m_ref = m_new;
+                l *= alpha;
+#pragma unroll 1
+                for (int c = 0; c < D / 32; ++c) {
+                    uint32_t v[32];
+                    tmem_ld32(tO + 32 * c, v);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) v[e] = __float_as_uint(__uint_as_float(v[e]) * alpha);
+                    tmem_st32(tO + 32 * c, v);
+                }
+            }
+            l += lsum;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
                 uint32_t u[16];
 #pragma unroll
-                for (int e = 0; e < 32; e += 4) {
-                    l0 += p[e]; l1 += p[e + 1]; l2 += p[e + 2]; l3 += p[e + 3];
-                    u[e / 2] = pack_bf16(p[e], p[e + 1]);
-                    u[e / 2 + 1] = pack_bf16(p[e + 2], p[e + 3]);
-                }
+                for (int e = 0; e < 16; ++e) u[e] = pk[16 * c + e];
                 tmem_st16(tS + 16 * c, u);
             }
-            l += (l0 + l1) + (l2 + l3);
             tmem_st_wait();
             tc_fence_before();
             mbar_arrive(bar(B_PFULL + t));
