@@ -24,7 +24,7 @@
 // while dQ/dK are still being multiplied, and dP^T(n+1) follows as soon as Y has been drained.
 // Tensor memory: X [0,128)  Y [128,256)  dK [256,256+D)  dV [256+D,256+2D).
 // Warp roles (512 threads): warp 0 TMA producer, warp 1 MMA issuer, warps 4-11 compute,
-// warps 12-15 dQ drain; register budgets are rebalanced with setmaxnreg (88 / 136 / 136 / 144).
+// warps 12-15 dQ drain; register budgets are rebalanced with setmaxnreg (104 / 128 / 128 / 144).
 #include <cuda_bf16.h>
 
 #include "kernels.h"
@@ -100,7 +100,7 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     const uint32_t tmem = lds32u(tmem_slot);
 
     if (warp < 4) {
-        reg_dealloc<88>();
+        reg_dealloc<104>();
         if (warp == 0 && lane == 0) {
         // ------------------------------------------------------------------ TMA producer
         {
@@ -131,20 +131,27 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             constexpr uint32_t idesc_st = umma_idesc_bf16(BLK, BLK, false, false);   // S^T, dP^T
             constexpr uint32_t idesc_dv = umma_idesc_bf16(BLK, D, false, true);      // A tmem / K-major, B MN-major
             constexpr uint32_t idesc_dq = umma_idesc_bf16(BLK, D, true, true);       // A MN-major, B MN-major
-            auto kmajor_off = [](int kk) { return static_cast<uint32_t>((kk >> 2) * C::CHUNK_BYTES + (kk & 3) * 32); };
+            // Descriptors are built once; inside the loops only the start-address field moves (it
+            // holds address >> 4 and cannot carry out of its 14 bits within shared memory).  The
+            // issuing thread is a single lane: every instruction it saves shortens the gap between
+            // two tensor-core instructions.
+            auto kmajor_off = [](int kk) { return static_cast<uint64_t>(((kk >> 2) * C::CHUNK_BYTES + (kk & 3) * 32) >> 4); };
+            auto mn_off = [](int kk) { return static_cast<uint64_t>((kk * 2048) >> 4); };
+            const uint64_t kK = umma_smem_desc(sK, 16, 1024), kV = umma_smem_desc(sV, 16, 1024);
+            const uint64_t kQ = umma_smem_desc(sQ, 16, 1024), kdO = umma_smem_desc(sdO, 16, 1024);
+            const uint64_t kdS = umma_smem_desc(sdS, 16, 1024);
+            const uint64_t mK = umma_smem_desc(sK, C::CHUNK_BYTES, 1024), mQ = umma_smem_desc(sQ, C::CHUNK_BYTES, 1024);
+            const uint64_t mdO = umma_smem_desc(sdO, C::CHUNK_BYTES, 1024), mdS = umma_smem_desc(sdS, C::CHUNK_BYTES, 1024);
+            const uint32_t tXa = tmem + C::TM_X, tYa = tmem + C::TM_Y, tDK = tmem + C::TM_DK, tDV = tmem + C::TM_DV;
             auto mma1 = [&](int n) {   // S^T = K Q(n)^T -> X
-                const uint32_t qa = sQ + (n & 1) * C::TILE_BYTES;
+                const uint64_t qd = kQ + static_cast<uint64_t>(((n & 1) * C::TILE_BYTES) >> 4);
 #pragma unroll
-                for (int kk = 0; kk < D / 16; ++kk)
-                    umma_ss(tmem + C::TM_X, umma_smem_desc(sK + kmajor_off(kk), 16, 1024),
-                            umma_smem_desc(qa + kmajor_off(kk), 16, 1024), idesc_st, kk > 0);
+                for (int kk = 0; kk < D / 16; ++kk) umma_ss(tXa, kK + kmajor_off(kk), qd + kmajor_off(kk), idesc_st, kk > 0);
                 umma_commit(bar(B_SFULL));
             };
             auto mma2 = [&]() {        // dP^T = V dO^T -> Y
 #pragma unroll
-                for (int kk = 0; kk < D / 16; ++kk)
-                    umma_ss(tmem + C::TM_Y, umma_smem_desc(sV + kmajor_off(kk), 16, 1024),
-                            umma_smem_desc(sdO + kmajor_off(kk), 16, 1024), idesc_st, kk > 0);
+                for (int kk = 0; kk < D / 16; ++kk) umma_ss(tYa, kV + kmajor_off(kk), kdO + kmajor_off(kk), idesc_st, kk > 0);
                 umma_commit(bar(B_DPFULL));
             };
             mbar_wait(bar(B_KV), 0, status);
@@ -155,14 +162,14 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             tc_fence_after();
             mma2();
             for (int n = 0; n < N; ++n) {
-                const uint32_t qa = sQ + (n & 1) * C::TILE_BYTES;
+                const uint64_t qm = mQ + static_cast<uint64_t>(((n & 1) * C::TILE_BYTES) >> 4);
+                const uint32_t acc0 = n > 0;
                 mbar_wait(bar(B_PDSFULL), n & 1, status);
                 tc_fence_after();
                 // MMA4: dV += P^T dO(n).  P^T: queries 0-63 at X[0,32), queries 64-127 at X[64,96)
 #pragma unroll
                 for (int kk = 0; kk < BLK / 16; ++kk)
-                    umma_ts(tmem + C::TM_DV, tmem + C::TM_X + (kk >> 2) * 64 + (kk & 3) * 8,
-                            umma_smem_desc(sdO + kk * 2048, C::CHUNK_BYTES, 1024), idesc_dv, (n > 0 || kk > 0));
+                    umma_ts(tDV, tXa + (kk >> 2) * 64 + (kk & 3) * 8, mdO + mn_off(kk), idesc_dv, kk > 0 ? 1u : acc0);
                 umma_commit(bar(B_DOEMPTY));
                 // MMA1 of the next pair right behind it: X is free once MMA4 has read P^T, and the
                 // compute warps can then exponentiate the next scores while MMA5/MMA6 run
@@ -173,15 +180,12 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                 }
                 // MMA6: dQ partial = dS K -> Y (first, so that the drain can start early)
 #pragma unroll
-                for (int kk = 0; kk < BLK / 16; ++kk)
-                    umma_ss(tmem + C::TM_Y, umma_smem_desc(sdS + kk * 2048, C::CHUNK_BYTES, 1024),
-                            umma_smem_desc(sK + kk * 2048, C::CHUNK_BYTES, 1024), idesc_dq, kk > 0);
+                for (int kk = 0; kk < BLK / 16; ++kk) umma_ss(tYa, mdS + mn_off(kk), mK + mn_off(kk), idesc_dq, kk > 0);
                 umma_commit(bar(B_DQFULL));
                 // MMA5: dK += dS^T Q(n)
 #pragma unroll
                 for (int kk = 0; kk < BLK / 16; ++kk)
-                    umma_ss(tmem + C::TM_DK, umma_smem_desc(sdS + kmajor_off(kk), 16, 1024),
-                            umma_smem_desc(qa + kk * 2048, C::CHUNK_BYTES, 1024), idesc_dv, (n > 0 || kk > 0));
+                    umma_ss(tDK, kdS + kmajor_off(kk), qm + mn_off(kk), idesc_dv, kk > 0 ? 1u : acc0);
                 umma_commit(bar(B_QEMPTY + (n & 1)));
                 if (n + 1 < N) {
                     mbar_wait(bar(B_DQEMPTY), n & 1, status);
@@ -233,7 +237,7 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         if (r == 0) bulk_wait_group_read0();
     } else {
         // ------------------------------------------------------------------ compute warps
-        reg_alloc<136>();
+        reg_alloc<128>();
         const int half = (warp - 4) >> 2;                  // which 64 query columns
         const int r = (tid - 128) & 127;                   // key lane 0..127
         const uint32_t lane_base = static_cast<uint32_t>(r & ~31) << 16;

@@ -7,13 +7,16 @@
 //   warp 0      TMA producer: Q tiles once, then K and V blocks through a 2-stage ring
 //   warp 1      MMA issuer: S_t = Q_t K^T (operands in shared memory) and O_t += P_t V
 //               (P_t read from tensor memory, V as an MN-major shared-memory operand)
-//   warps 4-7   softmax of query tile 0: one thread per row, so row max / row sum need no
-//   warps 8-11  softmax of query tile 1   cross-thread reduction
+//   warps 4-11  softmax: all 256 threads work on ONE query tile at a time, two threads per row
+//               (64 key columns each), alternating between the two tiles.  A lone warp per
+//               scheduler cannot keep the exp2 unit busy; two can, so a tile's softmax takes half
+//               as long and the tensor core's S/PV products of the other tile hide it.
 // Tensor memory (512 columns): S_0 [0,128), S_1 [128,256), O_0 [256,256+D), O_1 [256+D,256+2D).
-// P_t (bf16) overwrites the first 64 columns of S_t.  The two tiles ping-pong: while one tile's
-// softmax runs, the tensor core works on the other tile.  The running maximum is only moved
-// (and O rescaled in tensor memory) when it grows by more than 2^8, which is exact: any
-// reference point works for a softmax as long as nothing overflows.
+// P_t (bf16) overwrites S_t: keys 0-63 at S_t[0,32), keys 64-127 at S_t[64,96) (each half in the
+// columns its own threads have already read).  The softmax reference point of a row only moves
+// (and O is rescaled in tensor memory) when a score outgrows it by more than 2^8, which is exact:
+// any reference point works for a softmax as long as nothing overflows.  The two threads of a
+// row agree on that through a barrier with an OR-reduction per block.
 #include "kernels.h"
 #include "umma.cuh"
 
@@ -36,7 +39,8 @@ struct Cfg {
     static constexpr int OFF_Q = 0;
     static constexpr int OFF_K = OFF_Q + 2 * TILE_BYTES;
     static constexpr int OFF_V = OFF_K + kStages * TILE_BYTES;
-    static constexpr int OFF_BAR = OFF_V + kStages * TILE_BYTES;
+    static constexpr int OFF_XCHG = OFF_V + kStages * TILE_BYTES;   // [2 halves][128 rows] f32 exchange
+    static constexpr int OFF_BAR = OFF_XCHG + 2 * 128 * 4;
     static constexpr int SMEM = OFF_BAR + 256 + 1024;
     static constexpr uint32_t TM_S = 0, TM_O = 256, TM_COLS = 512;
 };
@@ -75,7 +79,7 @@ fast_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     const int n_max = max(nblk[0], nblk[1]);
 
     if (tid == 0) {
-        for (int i = 0; i < B_COUNT; ++i) mbar_init(bar(i), (i == B_PFULL || i == B_PFULL + 1) ? 128 : 1);
+        for (int i = 0; i < B_COUNT; ++i) mbar_init(bar(i), (i == B_PFULL || i == B_PFULL + 1) ? 256 : 1);
         fence_mbar_init();
     }
     __syncwarp();
@@ -86,7 +90,7 @@ fast_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     const uint32_t tmem = lds32u(tmem_slot);
 
     if (warp < 4) {
-        reg_dealloc<72>();
+        reg_dealloc<96>();
         if (warp == 0 && lane == 0) {
         // ------------------------------------------------------------------ TMA producer
         {
@@ -116,22 +120,31 @@ fast_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         {
             constexpr uint32_t idesc_s = umma_idesc_bf16(BM, BN, false, false);
             constexpr uint32_t idesc_o = umma_idesc_bf16(BM, D, false, true);
+            // Descriptors are built once; inside the loops only the start-address field moves (the
+            // field holds address >> 4 and cannot carry out of its 14 bits within shared memory).
+            // The issuing thread is a single lane: every instruction it saves shortens the time
+            // between two tensor-core instructions.
+            const uint64_t dQ0 = umma_smem_desc(sQ, 16, 1024), dK0 = umma_smem_desc(sK, 16, 1024);
+            const uint64_t dV0 = umma_smem_desc(sV, C::CHUNK_BYTES, 1024);
             auto issue_s = [&](int t, int n) {   // S_t = Q_t K(n)^T
-                const uint32_t qa = sQ + t * C::TILE_BYTES, ka = sK + (n & 1) * C::TILE_BYTES;
+                const uint64_t qd = dQ0 + static_cast<uint64_t>((t * C::TILE_BYTES) >> 4);
+                const uint64_t kd = dK0 + static_cast<uint64_t>(((n & 1) * C::TILE_BYTES) >> 4);
+                const uint32_t dst = tmem + C::TM_S + t * 128;
 #pragma unroll
                 for (int kk = 0; kk < D / 16; ++kk) {
-                    const uint32_t off = (kk >> 2) * C::CHUNK_BYTES + (kk & 3) * 32;
-                    umma_ss(tmem + C::TM_S + t * 128, umma_smem_desc(qa + off, 16, 1024),
-                            umma_smem_desc(ka + off, 16, 1024), idesc_s, kk > 0);
+                    const uint64_t off = static_cast<uint64_t>(((kk >> 2) * C::CHUNK_BYTES + (kk & 3) * 32) >> 4);
+                    umma_ss(dst, qd + off, kd + off, idesc_s, kk > 0);
                 }
                 umma_commit(bar(B_SFULL + t));
             };
             auto issue_o = [&](int t, int n) {   // O_t += P_t V(n)
-                const uint32_t va = sV + (n & 1) * C::TILE_BYTES;
+                const uint64_t vd = dV0 + static_cast<uint64_t>(((n & 1) * C::TILE_BYTES) >> 4);
+                const uint32_t dst = tmem + C::TM_O + t * D, src = tmem + C::TM_S + t * 128;
+                const uint32_t acc0 = n > 0;
 #pragma unroll
                 for (int kk = 0; kk < BN / 16; ++kk)
-                    umma_ts(tmem + C::TM_O + t * D, tmem + C::TM_S + t * 128 + kk * 8,
-                            umma_smem_desc(va + kk * 2048, C::CHUNK_BYTES, 1024), idesc_o, (n > 0 || kk > 0));
+                    umma_ts(dst, src + (kk >> 2) * 64 + (kk & 3) * 8, vd + static_cast<uint64_t>((kk * 2048) >> 4), idesc_o,
+                            kk > 0 ? 1u : acc0);
             };
             mbar_wait(bar(B_Q), 0, status);
             mbar_wait(bar(B_KFULL + 0), 0, status);
@@ -161,122 +174,151 @@ fast_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         __syncwarp();
     } else {
         // ------------------------------------------------------------------ softmax + epilogue
-        reg_alloc<216>();
-        const int t = (warp - 4) >> 2;
-        const int r = tid - 128 * (1 + t);                 // row within the tile, 0..127
+        reg_alloc<200>();
+        const int h = (warp - 4) >> 2;                     // which 64 key columns of every block
+        const int r = (tid - 128) & 127;                   // row within the tile = tensor-memory lane
         const uint32_t lane_base = static_cast<uint32_t>(r & ~31) << 16;
-        const uint32_t tS = tmem + lane_base + C::TM_S + t * 128;
-        const uint32_t tO = tmem + lane_base + C::TM_O + t * D;
-        const int i = row0[t] + r;
-        const int nb = nblk[t];
-        float m_ref = -INFINITY, l = 0.f;
+        const uint32_t xchg = base + C::OFF_XCHG;
+        const uint32_t my_x = xchg + (h * 128 + r) * 4, peer_x = xchg + ((h ^ 1) * 128 + r) * 4;
+        float m_ref[2] = {-INFINITY, -INFINITY}, l[2] = {0.f, 0.f};
 
-        for (int n = 0; n < nb; ++n) {
-            mbar_wait(bar(B_SFULL + t), n & 1, status);
-            tc_fence_after();
-            const int j0 = n * BN;
-            const bool masked = (causal && (j0 + BN - 1 > row0[t])) || (j0 + BN > S);
-            const int jmax = min(S - 1, causal ? i : S - 1) - j0;   // columns c <= jmax of this block are visible
+        // barrier over the 256 softmax threads with an OR reduction of `pred`
+        auto bar_or = [](bool pred) -> bool {
+            uint32_t out;
+            asm volatile(
+                "{\n\t.reg .pred P, Q;\n\tsetp.ne.b32 P, %1, 0;\n\t"
+                "barrier.cta.red.or.pred Q, 1, 256, P;\n\tselp.u32 %0, 1, 0, Q;\n\t}"
+                : "=r"(out) : "r"(static_cast<uint32_t>(pred)) : "memory");
+            return out != 0;
+        };
 
-            if (n == 0) {
-                // first block: the reference point is the block maximum of the scaled scores
-                float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+        for (int n = 0; n < n_max; ++n) {
+#pragma unroll
+            for (int t = 0; t < 2; ++t) {
+                if (n >= nblk[t]) continue;
+                const uint32_t tS = tmem + lane_base + C::TM_S + t * 128 + 64 * h;   // this thread's 64 score columns
+                const uint32_t tO = tmem + lane_base + C::TM_O + t * D + (D / 2) * h;
+                const int i = row0[t] + r;
+                mbar_wait(bar(B_SFULL + t), n & 1, status);
+                tc_fence_after();
+                const int j0 = n * BN + 64 * h;
+                const bool masked = (causal && (j0 + 63 > row0[t])) || (j0 + 64 > S);
+                const int jmax = min(S - 1, causal ? i : S - 1) - j0;   // columns c <= jmax of this half are visible
+
+                if (n == 0) {
+                    // first block: the reference point is the row maximum of the scaled scores
+                    float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+#pragma unroll
+                    for (int c = 0; c < 2; ++c) {
+                        uint32_t v[32];
+                        tmem_ld32(tS + 32 * c, v);
+                        tmem_ld_wait();
+                        float x[32];
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) x[e] = __uint_as_float(v[e]) * c2;
+                        if (masked) {
+#pragma unroll
+                            for (int e = 0; e < 32; ++e)
+                                if (32 * c + e > jmax) x[e] = -INFINITY;
+                        }
+#pragma unroll
+                        for (int e = 0; e < 32; e += 4) {
+                            mx0 = fmaxf(mx0, x[e]);
+                            mx1 = fmaxf(mx1, x[e + 1]);
+                            mx2 = fmaxf(mx2, x[e + 2]);
+                            mx3 = fmaxf(mx3, x[e + 3]);
+                        }
+                    }
+                    const float mine = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
+                    sts32(my_x, mine);
+                    bar_or(false);
+                    m_ref[t] = fmaxf(mine, lds32f(peer_x));      // finite: key 0 is visible to every row
+                    bar_or(false);                                // exchange buffer may be reused
+                }
+
+                // One pass: y = s*c2 - m_ref, p = exp2(y), partial row sum, bf16 pack (kept in
+                // registers), and the largest y.  If any row outgrew its reference point by more than
+                // the threshold, move the reference points, rescale O and l, and redo the pass (S is
+                // still intact: P is written over it only afterwards).
+                uint32_t pk[32];
+                float lsum = 0.f;
+                for (int attempt = 0; attempt < 2; ++attempt) {
+                    float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
+                    float y0 = -INFINITY, y1 = -INFINITY, y2 = -INFINITY, y3 = -INFINITY;
+                    const float neg_m = -m_ref[t];
+#pragma unroll
+                    for (int c = 0; c < 2; ++c) {
+                        uint32_t v[32];
+                        tmem_ld32(tS + 32 * c, v);
+                        tmem_ld_wait();
+                        float y[32];
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) y[e] = fmaf(__uint_as_float(v[e]), c2, neg_m);
+                        if (masked) {
+#pragma unroll
+                            for (int e = 0; e < 32; ++e)
+                                if (32 * c + e > jmax) y[e] = -INFINITY;
+                        }
+#pragma unroll
+                        for (int e = 0; e < 32; e += 4) {
+                            y0 = fmaxf(y0, y[e]); y1 = fmaxf(y1, y[e + 1]); y2 = fmaxf(y2, y[e + 2]); y3 = fmaxf(y3, y[e + 3]);
+                            const float p0 = ex2(y[e]), p1 = ex2(y[e + 1]), p2 = ex2(y[e + 2]), p3 = ex2(y[e + 3]);
+                            l0 += p0; l1 += p1; l2 += p2; l3 += p3;
+                            pk[16 * c + e / 2] = pack_bf16(p0, p1);
+                            pk[16 * c + e / 2 + 1] = pack_bf16(p2, p3);
+                        }
+                    }
+                    lsum = (l0 + l1) + (l2 + l3);
+                    const float ymax = fmaxf(fmaxf(y0, y1), fmaxf(y2, y3));
+                    if (attempt == 1) break;
+                    sts32(my_x, ymax);
+                    if (!bar_or(ymax > kRescaleThreshold)) break;
+                    // some row grew: every row moves its reference point to its current maximum
+                    const float ym = fmaxf(ymax, lds32f(peer_x));
+                    const float m_new = fmaxf(m_ref[t], m_ref[t] + ym);
+                    const float alpha = ex2(m_ref[t] - m_new);
+                    m_ref[t] = m_new;
+                    l[t] *= alpha;
 #pragma unroll 1
-                for (int c = 0; c < 4; ++c) {
-                    uint32_t v[32];
-                    tmem_ld32(tS + 32 * c, v);
-                    tmem_ld_wait();
-                    float x[32];
+                    for (int c = 0; c < D / 64; ++c) {
+                        uint32_t v[32];
+                        tmem_ld32(tO + 32 * c, v);
+                        tmem_ld_wait();
 #pragma unroll
-                    for (int e = 0; e < 32; ++e) x[e] = __uint_as_float(v[e]) * c2;
-                    if (masked) {
-#pragma unroll
-                        for (int e = 0; e < 32; ++e)
-                            if (32 * c + e > jmax) x[e] = -INFINITY;
+                        for (int e = 0; e < 32; ++e) v[e] = __float_as_uint(__uint_as_float(v[e]) * alpha);
+                        tmem_st32(tO + 32 * c, v);
                     }
-#pragma unroll
-                    for (int e = 0; e < 32; e += 4) {
-                        mx0 = fmaxf(mx0, x[e]);
-                        mx1 = fmaxf(mx1, x[e + 1]);
-                        mx2 = fmaxf(mx2, x[e + 2]);
-                        mx3 = fmaxf(mx3, x[e + 3]);
-                    }
+                    bar_or(false);                                // everyone has read the exchange buffer
                 }
-                m_ref = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));      // finite: key 0 is visible to every row
-            }
-
-            // One pass: y = s*c2 - m_ref, p = exp2(y), row sum, bf16 pack (kept in registers), and the
-            // largest y.  If some row of the warp outgrew the reference point by more than the
-            // threshold, move the reference, rescale O and l, and redo the pass (S is still intact:
-            // P is written over it only afterwards).
-            uint32_t pk[64];
-            float lsum = 0.f;
-            for (int attempt = 0; attempt < 2; ++attempt) {
-                float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
-                float y0 = -INFINITY, y1 = -INFINITY, y2 = -INFINITY, y3 = -INFINITY;
-                const float neg_m = -m_ref;
+                l[t] += lsum;
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    uint32_t v[32];
-                    tmem_ld32(tS + 32 * c, v);
-                    tmem_ld_wait();
-                    float y[32];
+                for (int c = 0; c < 2; ++c) {
+                    uint32_t u[16];
 #pragma unroll
-                    for (int e = 0; e < 32; ++e) y[e] = fmaf(__uint_as_float(v[e]), c2, neg_m);
-                    if (masked) {
-#pragma unroll
-                        for (int e = 0; e < 32; ++e)
-                            if (32 * c + e > jmax) y[e] = -INFINITY;
-                    }
-#pragma unroll
-                    for (int e = 0; e < 32; e += 4) {
-                        y0 = fmaxf(y0, y[e]); y1 = fmaxf(y1, y[e + 1]); y2 = fmaxf(y2, y[e + 2]); y3 = fmaxf(y3, y[e + 3]);
-                        const float p0 = ex2(y[e]), p1 = ex2(y[e + 1]), p2 = ex2(y[e + 2]), p3 = ex2(y[e + 3]);
-                        l0 += p0; l1 += p1; l2 += p2; l3 += p3;
-                        pk[16 * c + e / 2] = pack_bf16(p0, p1);
-                        pk[16 * c + e / 2 + 1] = pack_bf16(p2, p3);
-                    }
+                    for (int e = 0; e < 16; ++e) u[e] = pk[16 * c + e];
+                    tmem_st16(tS + 16 * c, u);
                 }
-                lsum = (l0 + l1) + (l2 + l3);
-                const float ymax = fmaxf(fmaxf(y0, y1), fmaxf(y2, y3));
-                const bool grow = ymax > kRescaleThreshold;
-                if (attempt == 1 || !__any_sync(0xffffffffu, grow)) break;
-                // move the reference point of every row of this warp
-                const float m_new = fmaxf(m_ref, m_ref + ymax);
-                const float alpha = ex2(m_ref - m_new);
-                m_ref = m_new;
-                l *= alpha;
-#pragma unroll 1
-                for (int c = 0; c < D / 32; ++c) {
-                    uint32_t v[32];
-                    tmem_ld32(tO + 32 * c, v);
-                    tmem_ld_wait();
-#pragma unroll
-                    for (int e = 0; e < 32; ++e) v[e] = __float_as_uint(__uint_as_float(v[e]) * alpha);
-                    tmem_st32(tO + 32 * c, v);
-                }
+                tmem_st_wait();
+                tc_fence_before();
+                mbar_arrive(bar(B_PFULL + t));
             }
-            l += lsum;
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                uint32_t u[16];
-#pragma unroll
-                for (int e = 0; e < 16; ++e) u[e] = pk[16 * c + e];
-                tmem_st16(tS + 16 * c, u);
-            }
-            tmem_st_wait();
-            tc_fence_before();
-            mbar_arrive(bar(B_PFULL + t));
         }
 
-        if (nb > 0) {
-            // ---- epilogue: O / l -> bf16 -> shared (swizzled like the TMA box) -> TMA store; LSE
+        // ---- epilogue per tile: O / l -> bf16 -> shared (swizzled like the TMA box) -> TMA store; LSE
+#pragma unroll
+        for (int t = 0; t < 2; ++t) {
+            if (nblk[t] == 0) continue;
+            const uint32_t tO = tmem + lane_base + C::TM_O + t * D + (D / 2) * h;
+            const int i = row0[t] + r;
+            sts32(my_x, l[t]);
+            bar_or(false);
+            const float lt = l[t] + lds32f(peer_x);
             mbar_wait(bar(B_OFULL + t), 0, status);
             tc_fence_after();
-            const float inv = 1.0f / l;
+            const float inv = 1.0f / lt;
             const uint32_t stage = sQ + t * C::TILE_BYTES;     // Q_t is no longer needed
 #pragma unroll 1
-            for (int c = 0; c < D / 32; ++c) {
+            for (int c = 0; c < D / 64; ++c) {
                 uint32_t v[32];
                 tmem_ld32(tO + 32 * c, v);
                 tmem_ld_wait();
@@ -284,17 +326,18 @@ fast_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
 #pragma unroll
                 for (int e = 0; e < 16; ++e)
                     u[e] = pack_bf16(__uint_as_float(v[2 * e]) * inv, __uint_as_float(v[2 * e + 1]) * inv);
-                const uint32_t rowaddr = stage + (c >> 1) * C::CHUNK_BYTES + r * 128;
+                const int col = (D / 2) * h + 32 * c;          // first output column of this chunk
+                const uint32_t rowaddr = stage + (col >> 6) * C::CHUNK_BYTES + r * 128;
 #pragma unroll
                 for (int q = 0; q < 4; ++q) {
-                    const int piece = (c & 1) * 4 + q;
+                    const int piece = ((col & 63) >> 3) + q;
                     sts128(rowaddr + ((piece ^ (r & 7)) << 4), u[4 * q], u[4 * q + 1], u[4 * q + 2], u[4 * q + 3]);
                 }
             }
-            if (i < S) LSE[static_cast<size_t>(bh) * S + i] = (m_ref + log2f(l)) * kLn2;
+            if (h == 0 && i < S) LSE[static_cast<size_t>(bh) * S + i] = (m_ref[t] + log2f(lt)) * kLn2;
             fence_proxy_async_smem();
-            named_bar_sync(1 + t, 128);
-            if (r == 0) {
+            bar_or(false);
+            if (r == 0 && h == 0) {
 #pragma unroll
                 for (int ch = 0; ch < C::NCH; ++ch)
                     tma_store_3d(&tmO, stage + ch * C::CHUNK_BYTES, ch * 64, row0[t], bh);
