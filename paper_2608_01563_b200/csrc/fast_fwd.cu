@@ -5,8 +5,11 @@
 // One CTA owns two 128-row query tiles of one head and walks over 128-key blocks.
 // Warp roles (384 threads):
 //   warp 0      TMA producer: Q tiles once, then K and V blocks through a 2-stage ring
-//   warp 1      MMA issuer: S_t = Q_t K^T (operands in shared memory) and O_t += P_t V
-//               (P_t read from tensor memory, V as an MN-major shared-memory operand)
+//   warps 1, 2  MMA issuers, one per query tile: S_t = Q_t K^T (operands in shared memory) and
+//               O_t += P_t V (P_t read from tensor memory, V as an MN-major shared-memory
+//               operand).  One lane each; with two issuers the tensor core keeps working on one
+//               tile while the other issuer sits in a barrier wait (a wait costs a few hundred
+//               clocks even when it succeeds at once, and the issue queue is shallow)
 //   warps 4-11  softmax: all 256 threads work on ONE query tile at a time, two threads per row
 //               (64 key columns each), alternating between the two tiles.  A lone warp per
 //               scheduler cannot keep the exp2 unit busy; two can, so a tile's softmax takes half
@@ -79,7 +82,14 @@ fast_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     const int n_max = max(nblk[0], nblk[1]);
 
     if (tid == 0) {
-        for (int i = 0; i < B_COUNT; ++i) mbar_init(bar(i), (i == B_PFULL || i == B_PFULL + 1) ? 256 : 1);
+        const uint32_t issuers = nblk[1] > 0 ? 2 : 1;      // K/V stages are released by every active issuer
+        for (int i = 0; i < B_COUNT; ++i) {
+            uint32_t cnt = 1;
+            if (i == B_PFULL || i == B_PFULL + 1) cnt = 256;
+            if (i >= B_KEMPTY && i < B_KEMPTY + 2) cnt = issuers;
+            if (i >= B_VEMPTY && i < B_VEMPTY + 2) cnt = issuers;
+            mbar_init(bar(i), cnt);
+        }
         fence_mbar_init();
     }
     __syncwarp();
@@ -115,59 +125,59 @@ fast_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                     tma_load_3d(sV + st * C::TILE_BYTES + ch * C::CHUNK_BYTES, &tmV, bar(B_VFULL + st), ch * 64, n * BN, bh);
             }
         }
-        } else if (warp == 1 && lane == 0) {
-        // ------------------------------------------------------------------ MMA issuer
+        } else if ((warp == 1 || warp == 2) && lane == 0 && nblk[warp - 1] > 0) {
+        // ------------------------------------------------------------------ MMA issuer of tile t
         {
+            const int t = warp - 1;
+            const int nb = nblk[t];
             constexpr uint32_t idesc_s = umma_idesc_bf16(BM, BN, false, false);
             constexpr uint32_t idesc_o = umma_idesc_bf16(BM, D, false, true);
             // Descriptors are built once; inside the loops only the start-address field moves (the
             // field holds address >> 4 and cannot carry out of its 14 bits within shared memory).
-            // The issuing thread is a single lane: every instruction it saves shortens the time
-            // between two tensor-core instructions.
-            const uint64_t dQ0 = umma_smem_desc(sQ, 16, 1024), dK0 = umma_smem_desc(sK, 16, 1024);
+            const uint64_t qd = umma_smem_desc(sQ + t * C::TILE_BYTES, 16, 1024);
+            const uint64_t dK0 = umma_smem_desc(sK, 16, 1024);
             const uint64_t dV0 = umma_smem_desc(sV, C::CHUNK_BYTES, 1024);
-            auto issue_s = [&](int t, int n) {   // S_t = Q_t K(n)^T
-                const uint64_t qd = dQ0 + static_cast<uint64_t>((t * C::TILE_BYTES) >> 4);
+            const uint32_t tSd = tmem + C::TM_S + t * 128, tOd = tmem + C::TM_O + t * D;
+            auto issue_s = [&](int n) {   // S_t = Q_t K(n)^T
                 const uint64_t kd = dK0 + static_cast<uint64_t>(((n & 1) * C::TILE_BYTES) >> 4);
-                const uint32_t dst = tmem + C::TM_S + t * 128;
 #pragma unroll
                 for (int kk = 0; kk < D / 16; ++kk) {
                     const uint64_t off = static_cast<uint64_t>(((kk >> 2) * C::CHUNK_BYTES + (kk & 3) * 32) >> 4);
-                    umma_ss(dst, qd + off, kd + off, idesc_s, kk > 0);
+                    umma_ss(tSd, qd + off, kd + off, idesc_s, kk > 0);
                 }
                 umma_commit(bar(B_SFULL + t));
             };
-            auto issue_o = [&](int t, int n) {   // O_t += P_t V(n)
+            auto issue_o = [&](int n) {   // O_t += P_t V(n)
                 const uint64_t vd = dV0 + static_cast<uint64_t>(((n & 1) * C::TILE_BYTES) >> 4);
-                const uint32_t dst = tmem + C::TM_O + t * D, src = tmem + C::TM_S + t * 128;
                 const uint32_t acc0 = n > 0;
 #pragma unroll
                 for (int kk = 0; kk < BN / 16; ++kk)
-                    umma_ts(dst, src + (kk >> 2) * 64 + (kk & 3) * 8, vd + static_cast<uint64_t>((kk * 2048) >> 4), idesc_o,
+                    umma_ts(tOd, tSd + (kk >> 2) * 64 + (kk & 3) * 8, vd + static_cast<uint64_t>((kk * 2048) >> 4), idesc_o,
                             kk > 0 ? 1u : acc0);
             };
             mbar_wait(bar(B_Q), 0, status);
             mbar_wait(bar(B_KFULL + 0), 0, status);
             tc_fence_after();
-            for (int t = 0; t < 2; ++t)
-                if (nblk[t] > 0) issue_s(t, 0);
+            issue_s(0);
             umma_commit(bar(B_KEMPTY + 0));
             for (int n = 0; n < n_max; ++n) {
                 const int st = n & 1;
-                const uint32_t ph = (n >> 1) & 1;
-                mbar_wait(bar(B_VFULL + st), ph, status);
-                if (n + 1 < n_max) mbar_wait(bar(B_KFULL + (st ^ 1)), ((n + 1) >> 1) & 1, status);
-                for (int t = 0; t < 2; ++t) {
-                    if (n < nblk[t]) {
-                        mbar_wait(bar(B_PFULL + t), n & 1, status);
-                        tc_fence_after();
-                        issue_o(t, n);
-                        if (n == nblk[t] - 1) umma_commit(bar(B_OFULL + t));
-                    }
-                    if (n + 1 < nblk[t]) issue_s(t, n + 1);
+                if (n < nb) {
+                    mbar_wait(bar(B_VFULL + st), (n >> 1) & 1, status);
+                    mbar_wait(bar(B_PFULL + t), n & 1, status);
+                    tc_fence_after();
+                    issue_o(n);
+                    if (n == nb - 1) umma_commit(bar(B_OFULL + t));
                 }
-                umma_commit(bar(B_VEMPTY + st));
-                if (n + 1 < n_max) umma_commit(bar(B_KEMPTY + (st ^ 1)));
+                umma_commit(bar(B_VEMPTY + st));          // this issuer is done with V(n)
+                if (n + 1 < n_max) {
+                    if (n + 1 < nb) {
+                        mbar_wait(bar(B_KFULL + (st ^ 1)), ((n + 1) >> 1) & 1, status);
+                        tc_fence_after();
+                        issue_s(n + 1);
+                    }
+                    umma_commit(bar(B_KEMPTY + (st ^ 1)));   // ... and with K(n+1)
+                }
             }
         }
         }
