@@ -89,7 +89,7 @@ class ClockSampler:
             self.fh = open(self.path, "w")
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(self.gpu_index), f"--query-gpu={self.QUERY}",
-                 "--format=csv,noheader,nounits", "-lms", "100"], stdout=self.fh, stderr=subprocess.DEVNULL)
+                 "--format=csv,noheader,nounits", "-lms", "20"], stdout=self.fh, stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
 
@@ -120,6 +120,32 @@ class ClockSampler:
             out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons),
                        samples=len(sm), power_w_max=max(power))
         return out
+
+
+def quick_measure(mgn, w, mode, dtype, steps, warmup):
+    """Device-resident timing of forward and backward calls of one more workload (CUDA events)."""
+    q, k, v, d_o = (t.cuda() for t in synth.make_inputs(w, dtype=dtype))
+    B, H, S, D = q.shape
+    o = torch.empty_like(q)
+    lse = torch.empty(B, H, S, device="cuda", dtype=torch.float32)
+    dq, dk, dv = (torch.empty_like(q) for _ in range(3))
+    ws = mgn.alloc_workspace(B, H, S, D, mode)
+    for _ in range(warmup):
+        mgn.mgn_attn_fwd(q, k, v, o, lse, w.causal, w.scale, mode)
+        mgn.mgn_attn_bwd(q, k, v, o, d_o, lse, dq, dk, dv, ws, w.causal, w.scale, mode)
+    torch.cuda.synchronize()
+    e = [torch.cuda.Event(enable_timing=True) for _ in range(2 * steps + 1)]
+    e[0].record()
+    for i in range(steps):
+        mgn.mgn_attn_fwd(q, k, v, o, lse, w.causal, w.scale, mode)
+        e[2 * i + 1].record()
+        mgn.mgn_attn_bwd(q, k, v, o, d_o, lse, dq, dk, dv, ws, w.causal, w.scale, mode)
+        e[2 * i + 2].record()
+    torch.cuda.synchronize()
+    mgn.mgn_attn_check()
+    fwd_ms = statistics.mean(e[2 * i].elapsed_time(e[2 * i + 1]) for i in range(steps))
+    bwd_ms = statistics.mean(e[2 * i + 1].elapsed_time(e[2 * i + 2]) for i in range(steps))
+    return fwd_ms, bwd_ms
 
 
 def cpu_info():
@@ -214,6 +240,7 @@ def main():
     ap.add_argument("--mode", default="strict", choices=["strict", "fast"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-fast", action="store_true", help="skip the extra fast-mode measurement")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -277,8 +304,12 @@ def main():
             a.record(); b.record()
     torch.cuda.synchronize()
 
-    sampler = ClockSampler(local_rank if "CUDA_VISIBLE_DEVICES" not in os.environ else
-                           int(os.environ["CUDA_VISIBLE_DEVICES"].split(",")[local_rank]))
+    gpu_index = local_rank
+    try:
+        gpu_index = int(os.environ["CUDA_VISIBLE_DEVICES"].split(",")[local_rank])
+    except (KeyError, ValueError, IndexError):
+        pass
+    sampler = ClockSampler(gpu_index)
     if rank == 0:
         sampler.start()
         time.sleep(0.3)
@@ -370,6 +401,18 @@ def main():
             d2h = sum(t_.numel() * t_.element_size() for t_ in host_out)
             line["e2e"] = {"value": whole_job_tflops(w, world, K, e2e_ms_max), "unit": "TFLOP/s",
                            "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+        if world == 1 and args.mode == "strict" and args.workload is None and not args.no_fast:
+            # the other arithmetic mode of the same library on its own target workload, for the record
+            wf = synth.WORKLOADS["long_context"]
+            f_ms, b_ms = quick_measure(mgn, wf, mgn.MODE_FAST_BF16, torch.bfloat16, K, args.warmup)
+            tf = lambda which, ms: flops(wf, which) / (ms * 1e-3) / 1e12
+            line["fast_mode"] = {
+                "workload": wf.name, "dtype": "bf16", "fwd_ms": f_ms, "bwd_ms": b_ms,
+                "fwd_tflops": tf("fwd", f_ms), "bwd_tflops": tf("bwd", b_ms),
+                "sum_tflops": flops(wf, "sum") / ((f_ms + b_ms) * 1e-3) / 1e12,
+                "peak_tflops": peaks["bf16_tflops"], "peak_note": f"{peak_src} dense bf16 burst",
+                "frac_of_peak": flops(wf, "sum") / ((f_ms + b_ms) * 1e-3) / 1e12 / peaks["bf16_tflops"],
+            }
         if world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline(w, dtype)
         print(json.dumps(line))
