@@ -156,7 +156,7 @@ int mgn_attn_check(void* stream)
     if (cudaMemcpy(&h, status, sizeof(h), cudaMemcpyDeviceToHost) != cudaSuccess) return MGN_ERR_CUDA;
     if (h != 0) {
         cudaMemset(status, 0, sizeof(h));
-        return MGN_ERR_DEVICE_TIMEOUT;
+        return h == 8u ? MGN_ERR_CUDA : MGN_ERR_DEVICE_TIMEOUT;   // 8: a kernel found its shared-memory layout short
     }
     return MGN_OK;
 }

@@ -12,6 +12,7 @@ namespace mgn {
 // end (its results are then garbage, but it cannot hang the device).
 constexpr uint32_t kMaxPolls = 1u << 22;
 constexpr unsigned kStatusTimeout = 7u;
+constexpr unsigned kStatusSmemLayout = 8u;   // the dynamic shared-memory base left too little alignment slack
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
     return static_cast<uint32_t>(__cvta_generic_to_shared(p));

@@ -18,14 +18,16 @@
 namespace mgn {
 namespace {
 
-constexpr int kThreads = 256;
 constexpr float kLog2e = 1.4426950408889634f;
 
-template <int D, int BM, int BN>
+// THREADS/16 row groups x 16 column groups; 128-thread CTAs run two per SM so that one CTA's
+// FFMA loops cover the other's barriers and exponentials.
+template <int D, int BM, int BN, int THREADS>
 struct BwdCfg {
-    static constexpr int RM = BM / 16;   // query rows per thread (phases A, C)
+    static constexpr int TR = THREADS / 16;  // row groups
+    static constexpr int RM = BM / TR;   // query rows per thread (phases A, C)
     static constexpr int RN = BN / 16;   // key columns per thread (phase A)
-    static constexpr int JN = BN / 16;   // key rows per thread (phase B), groups of 4 contiguous
+    static constexpr int JN = BN / TR;   // key rows per thread (phase B), groups of 4 contiguous
     static constexpr int DV = D / 16;    // d columns per thread (phases B, C)
     static constexpr int NCH = D / 32;
     static constexpr int PSTR = BN + 4;
@@ -56,16 +58,16 @@ __device__ __forceinline__ float f4_get(const float4& v, int u) {
     return u == 0 ? v.x : u == 1 ? v.y : u == 2 ? v.z : v.w;
 }
 
-template <int D, int BM, int BN>
-__global__ void __launch_bounds__(kThreads, 1)
+template <int D, int BM, int BN, int THREADS>
+__global__ void __launch_bounds__(THREADS, THREADS == 128 ? 2 : 1)
 strict_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                   const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmdO,
                   const float* __restrict__ LSE, const float* __restrict__ DELTA,
                   float* __restrict__ dQ, float* __restrict__ dK, float* __restrict__ dV,
                   int S, int BH, int n_qt, int causal, float scale, unsigned* status)
 {
-    using C = BwdCfg<D, BM, BN>;
-    constexpr int RM = C::RM, RN = C::RN, JN = C::JN, DV = C::DV, NCH = C::NCH, PSTR = C::PSTR;
+    using C = BwdCfg<D, BM, BN, THREADS>;
+    constexpr int RM = C::RM, RN = C::RN, JN = C::JN, DV = C::DV, NCH = C::NCH, PSTR = C::PSTR, TR = C::TR;
 
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -125,7 +127,7 @@ strict_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         float lse2[RM], dl[RM];
 #pragma unroll
         for (int x = 0; x < RM; ++x) {
-            const int i = i0 + tr + 16 * x;
+            const int i = i0 + tr + TR * x;
             const bool ok = i < S;
             lse2[x] = ok ? LSE[static_cast<size_t>(bh) * S + i] * kLog2e : INFINITY;
             dl[x] = ok ? DELTA[static_cast<size_t>(bh) * S + i] : 0.f;
@@ -153,8 +155,8 @@ strict_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 }
 #pragma unroll
                 for (int x = 0; x < RM; ++x) {
-                    const float4 aq = lds128(sQ + oq + x * 16 * 128);
-                    const float4 ad = lds128(sdO + oq + x * 16 * 128);
+                    const float4 aq = lds128(sQ + oq + x * TR * 128);
+                    const float4 ad = lds128(sdO + oq + x * TR * 128);
 #pragma unroll
                     for (int y = 0; y < RN; ++y) {
                         s[x][y] = fmaf(aq.x, bk[y].x, s[x][y]);
@@ -174,8 +176,8 @@ strict_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             const bool need_mask = (causal && (j0 + BN - 1 > i0)) || (j0 + BN > S);
 #pragma unroll
             for (int x = 0; x < RM; ++x) {
-                const int i = i0 + tr + 16 * x;
-                const uint32_t row = ((tr + 16 * x) * PSTR + tc) * 4;
+                const int i = i0 + tr + TR * x;
+                const uint32_t row = ((tr + TR * x) * PSTR + tc) * 4;
 #pragma unroll
                 for (int y = 0; y < RN; ++y) {
                     float p = ex2(fmaf(s[x][y], c2, -lse2[x]));
@@ -204,8 +206,8 @@ strict_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 load_row_cols<D, BM>(sQ, i, iu, tc, qv);
 #pragma unroll
                 for (int g = 0; g < JN / 4; ++g) {
-                    const float4 p4 = lds128(sP + (i * PSTR + 4 * tr + 64 * g) * 4);
-                    const float4 d4 = lds128(sdS + (i * PSTR + 4 * tr + 64 * g) * 4);
+                    const float4 p4 = lds128(sP + (i * PSTR + 4 * tr + 4 * TR * g) * 4);
+                    const float4 d4 = lds128(sdS + (i * PSTR + 4 * tr + 4 * TR * g) * 4);
 #pragma unroll
                     for (int u = 0; u < 4; ++u) {
                         const float pj = f4_get(p4, u), dj = f4_get(d4, u);
@@ -242,7 +244,7 @@ strict_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 for (int hlf = 0; hlf < 2; ++hlf)
 #pragma unroll
                     for (int x = 0; x < RM; ++x)
-                        d4[hlf][x] = lds128(sdS + ((tr + 16 * x) * PSTR + j8 * 8 + hlf * 4) * 4);
+                        d4[hlf][x] = lds128(sdS + ((tr + TR * x) * PSTR + j8 * 8 + hlf * 4) * 4);
 #pragma unroll
                 for (int u = 0; u < 8; ++u) {
                     float kv[DV];
@@ -257,7 +259,7 @@ strict_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             }
 #pragma unroll
             for (int x = 0; x < RM; ++x) {
-                const int i = i0 + tr + 16 * x;
+                const int i = i0 + tr + TR * x;
                 if (i < S) {
                     float* row = dQ + (static_cast<size_t>(bh) * S + i) * D;
                     if constexpr (DV == 2) {
@@ -278,7 +280,7 @@ strict_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     for (int g = 0; g < JN / 4; ++g)
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
-            const int j = j0 + 4 * tr + 64 * g + u;
+            const int j = j0 + 4 * tr + 4 * TR * g + u;
             if (j < S) {
                 const size_t off = (static_cast<size_t>(bh) * S + j) * D;
                 const int a = 4 * g + u;
@@ -299,25 +301,25 @@ strict_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         }
 }
 
-template <int D, int BM, int BN>
+template <int D, int BM, int BN, int THREADS>
 cudaError_t launch(const Problem& p, const float* q, const float* k, const float* v, const float* d_o,
                    const float* lse, const float* delta, float* dq, float* dk, float* dv, unsigned* status,
                    cudaStream_t st)
 {
-    using C = BwdCfg<D, BM, BN>;
+    using C = BwdCfg<D, BM, BN, THREADS>;
     CUtensorMap tq, tk, tv, tdo;
     if (make_tmap_3d(&tq, q, 4, 0, p.BH, p.S, D, 32, BM)) return cudaErrorInvalidValue;
     if (make_tmap_3d(&tdo, d_o, 4, 0, p.BH, p.S, D, 32, BM)) return cudaErrorInvalidValue;
     if (make_tmap_3d(&tk, k, 4, 0, p.BH, p.S, D, 32, BN)) return cudaErrorInvalidValue;
     if (make_tmap_3d(&tv, v, 4, 0, p.BH, p.S, D, 32, BN)) return cudaErrorInvalidValue;
-    auto kern = strict_bwd_kernel<D, BM, BN>;
+    auto kern = strict_bwd_kernel<D, BM, BN, THREADS>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM);
     if (e != cudaSuccess) return e;
     const int n_qt = (p.S + BM - 1) / BM;
     const int n_kt = (p.S + BN - 1) / BN;
     const long long blocks = static_cast<long long>(n_kt) * p.BH;
     if (blocks > 0x7fffffffLL) return cudaErrorInvalidValue;
-    kern<<<static_cast<unsigned>(blocks), kThreads, C::SMEM, st>>>(tq, tk, tv, tdo, lse, delta, dq, dk, dv, p.S, p.BH,
+    kern<<<static_cast<unsigned>(blocks), THREADS, C::SMEM, st>>>(tq, tk, tv, tdo, lse, delta, dq, dk, dv, p.S, p.BH,
                                                                    n_qt, p.causal, p.scale, status);
     return cudaGetLastError();
 }
@@ -329,9 +331,9 @@ cudaError_t launch_strict_bwd(const Problem& p, const float* q, const float* k, 
                               float* dq, float* dk, float* dv, unsigned* status, cudaStream_t st)
 {
     switch (p.D) {
-        case 32:  return launch<32, 64, 128>(p, q, k, v, d_o, lse, delta, dq, dk, dv, status, st);
-        case 64:  return launch<64, 64, 128>(p, q, k, v, d_o, lse, delta, dq, dk, dv, status, st);
-        case 128: return launch<128, 64, 64>(p, q, k, v, d_o, lse, delta, dq, dk, dv, status, st);
+        case 32:  return launch<32, 64, 64, 128>(p, q, k, v, d_o, lse, delta, dq, dk, dv, status, st);
+        case 64:  return launch<64, 64, 64, 128>(p, q, k, v, d_o, lse, delta, dq, dk, dv, status, st);
+        case 128: return launch<128, 64, 64, 256>(p, q, k, v, d_o, lse, delta, dq, dk, dv, status, st);
         default:  return cudaErrorInvalidValue;
     }
 }

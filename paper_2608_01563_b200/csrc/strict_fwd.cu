@@ -18,21 +18,30 @@
 namespace mgn {
 namespace {
 
-constexpr int kThreads = 256;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 
-template <int D, int BM, int BN>
+// THREADS/16 row groups x 16 column groups.  128-thread CTAs fit two per SM (registers and shared
+// memory), which decouples their barriers and softmax phases: one CTA's FFMA loop fills the
+// issue slots the other leaves idle.
+template <int D, int BM, int BN, int THREADS>
 struct FwdCfg {
-    static constexpr int RM = BM / 16;    // query rows per thread
+    static constexpr int TR = THREADS / 16;   // row groups
+    static constexpr int RM = BM / TR;        // query rows per thread
     static constexpr int RN = BN / 16;    // key columns per thread
     static constexpr int DV = D / 16;     // output columns per thread
     static constexpr int NCH = D / 32;    // 128-byte chunks per row
-    static constexpr int PSTR = BN + 4;   // padded row stride of P (floats)
+    static constexpr int PSTR = BN;       // row stride of P (floats); 16-byte pieces XOR-swizzled by row
     static constexpr int Q_BYTES = BM * D * 4;
     static constexpr int KV_BYTES = BN * D * 4;
     static constexpr int P_BYTES = BM * PSTR * 4;
-    static constexpr int SMEM = Q_BYTES + 2 * KV_BYTES + P_BYTES + 64 + 1024;
+    static constexpr int PAYLOAD = Q_BYTES + 2 * KV_BYTES + P_BYTES + 64;
+    // Two 128-thread CTAs per SM must fit 2 x (SMEM + 1 KB reserved) into 228 KB, which leaves less
+    // than the 1023 bytes a worst-case 1024-byte alignment of the tile base could need; the kernel
+    // checks the slack it actually got and reports through the status word if it is short.
+    static constexpr int SLACK = (THREADS == 128 && PAYLOAD + 1024 > 115712) ? 115712 - PAYLOAD : 1024;
+    static constexpr int SMEM = PAYLOAD + SLACK;
+    static_assert(SLACK >= 0, "shared memory budget");
 };
 
 // Byte offset of the 16-byte piece `piece` (0..D/4-1) of row `r` in a swizzled tile of R rows.
@@ -41,14 +50,14 @@ __device__ __forceinline__ uint32_t tile_off(int r, int piece) {
     return static_cast<uint32_t>((piece >> 3) * (R * 128) + r * 128 + (((piece & 7) ^ (r & 7)) << 4));
 }
 
-template <int D, int BM, int BN>
-__global__ void __launch_bounds__(kThreads, 1)
+template <int D, int BM, int BN, int THREADS>
+__global__ void __launch_bounds__(THREADS, THREADS == 128 ? 2 : 1)
 strict_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                   const __grid_constant__ CUtensorMap tmV, float* __restrict__ O, float* __restrict__ LSE,
                   int S, int BH, int n_qt, int causal, float c2, unsigned* status)
 {
-    using C = FwdCfg<D, BM, BN>;
-    constexpr int RM = C::RM, RN = C::RN, DV = C::DV, NCH = C::NCH, PSTR = C::PSTR;
+    using C = FwdCfg<D, BM, BN, THREADS>;
+    constexpr int RM = C::RM, RN = C::RN, DV = C::DV, NCH = C::NCH, PSTR = C::PSTR, TR = C::TR;
 
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -57,6 +66,10 @@ strict_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     const uint32_t sV = sK + C::KV_BYTES;
     const uint32_t sP = sV + C::KV_BYTES;
     const uint32_t barQ = sP + C::P_BYTES, barK = barQ + 8, barV = barQ + 16;
+    if (base + C::PAYLOAD > smem_u32(smem_raw) + C::SMEM) {      // alignment slack ran out
+        if (threadIdx.x == 0) atomicMax(status, kStatusSmemLayout);
+        return;
+    }
 
     const int tid = threadIdx.x;
     const int tr = 2 * (tid >> 5) + ((tid & 31) >> 4);   // 0..15: row group
@@ -123,7 +136,7 @@ strict_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 for (int y = 0; y < RN; ++y) b[y] = lds128(ka + ok + y * 16 * 128);
 #pragma unroll
                 for (int x = 0; x < RM; ++x) {
-                    const float4 a = lds128(qa + oq + x * 16 * 128);
+                    const float4 a = lds128(qa + oq + x * TR * 128);
 #pragma unroll
                     for (int y = 0; y < RN; ++y) {
                         s[x][y] = fmaf(a.x, b[y].x, s[x][y]);
@@ -145,7 +158,7 @@ strict_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         const bool need_mask = (causal && (j0 + BN - 1 > i0)) || (j0 + BN > S);
 #pragma unroll
         for (int x = 0; x < RM; ++x) {
-            const int i = i0 + tr + 16 * x;
+            const int i = i0 + tr + TR * x;
             float mx = -INFINITY;
 #pragma unroll
             for (int y = 0; y < RN; ++y) {
@@ -165,12 +178,13 @@ strict_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             const float alpha = ex2(m[x] - m_new);
             m[x] = m_new;
             float psum = 0.f;
-            const uint32_t prow = sP + ((tr + 16 * x) * PSTR + tc) * 4;
+            // P[i][j] lives at row i, 16-byte piece (j/4) ^ (i & 7); i & 7 == tr & 7 for all of a thread's rows
+            const uint32_t prow = sP + (tr + TR * x) * PSTR * 4 + (tc & 3) * 4;
 #pragma unroll
             for (int y = 0; y < RN; ++y) {
                 const float p = ex2(s[x][y] - m_new);
                 psum += p;
-                sts32(prow + y * 64, p);
+                sts32(prow + ((((tc >> 2) + 4 * y) ^ (tr & 7)) << 4), p);
             }
             l[x] = fmaf(l[x], alpha, psum);
 #pragma unroll
@@ -188,7 +202,8 @@ strict_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
 #pragma unroll
                 for (int hlf = 0; hlf < 2; ++hlf)
 #pragma unroll
-                    for (int x = 0; x < RM; ++x) p[hlf][x] = lds128(pa + (x * 16 * PSTR + j8 * 8 + hlf * 4) * 4);
+                    for (int x = 0; x < RM; ++x)
+                        p[hlf][x] = lds128(pa + x * TR * PSTR * 4 + (((2 * j8 + hlf) ^ (tr & 7)) << 4));
 #pragma unroll
                 for (int u = 0; u < 8; ++u) {
                     const int j = j8 * 8 + u;
@@ -230,7 +245,7 @@ strict_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         lt += __shfl_xor_sync(0xffffffffu, lt, 2);
         lt += __shfl_xor_sync(0xffffffffu, lt, 4);
         lt += __shfl_xor_sync(0xffffffffu, lt, 8);
-        const int i = i0 + tr + 16 * x;
+        const int i = i0 + tr + TR * x;
         if (i < S) {
             const float inv = 1.0f / lt;
             float* orow = O + (static_cast<size_t>(bh) * S + i) * D;
@@ -247,22 +262,22 @@ strict_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     }
 }
 
-template <int D, int BM, int BN>
+template <int D, int BM, int BN, int THREADS>
 cudaError_t launch(const Problem& p, const float* q, const float* k, const float* v, float* o, float* lse,
                    unsigned* status, cudaStream_t st)
 {
-    using C = FwdCfg<D, BM, BN>;
+    using C = FwdCfg<D, BM, BN, THREADS>;
     CUtensorMap tq, tk, tv;
     if (make_tmap_3d(&tq, q, 4, 0, p.BH, p.S, D, 32, BM)) return cudaErrorInvalidValue;
     if (make_tmap_3d(&tk, k, 4, 0, p.BH, p.S, D, 32, BN)) return cudaErrorInvalidValue;
     if (make_tmap_3d(&tv, v, 4, 0, p.BH, p.S, D, 32, BN)) return cudaErrorInvalidValue;
-    auto kern = strict_fwd_kernel<D, BM, BN>;
+    auto kern = strict_fwd_kernel<D, BM, BN, THREADS>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM);
     if (e != cudaSuccess) return e;
     const int n_qt = (p.S + BM - 1) / BM;
     const long long blocks = static_cast<long long>(n_qt) * p.BH;
     if (blocks > 0x7fffffffLL) return cudaErrorInvalidValue;
-    kern<<<static_cast<unsigned>(blocks), kThreads, C::SMEM, st>>>(tq, tk, tv, o, lse, p.S, p.BH, n_qt, p.causal,
+    kern<<<static_cast<unsigned>(blocks), THREADS, C::SMEM, st>>>(tq, tk, tv, o, lse, p.S, p.BH, n_qt, p.causal,
                                                                    p.scale * kLog2e, status);
     return cudaGetLastError();
 }
@@ -273,9 +288,9 @@ cudaError_t launch_strict_fwd(const Problem& p, const float* q, const float* k, 
                               float* o, float* lse, unsigned* status, cudaStream_t st)
 {
     switch (p.D) {
-        case 32:  return launch<32, 128, 128>(p, q, k, v, o, lse, status, st);
-        case 64:  return launch<64, 128, 128>(p, q, k, v, o, lse, status, st);
-        case 128: return launch<128, 128, 64>(p, q, k, v, o, lse, status, st);
+        case 32:  return launch<32, 64, 128, 128>(p, q, k, v, o, lse, status, st);
+        case 64:  return launch<64, 64, 128, 128>(p, q, k, v, o, lse, status, st);
+        case 128: return launch<128, 128, 64, 256>(p, q, k, v, o, lse, status, st);
         default:  return cudaErrorInvalidValue;
     }
 }
