@@ -29,6 +29,9 @@ sys.path.insert(0, ROOT)
 from paper_2608_01563_b200 import inputs as synth  # noqa: E402
 
 METRIC = "attention fwd+bwd TFLOP/s per B200 (strict f32, bf16) and % of matching peak"
+# dram__bytes_read.sum + dram__bytes_write.sum of the backward main kernel, one launch, from the ncu
+# captures summarised under profiles/ (same workload and launch configuration as the bench)
+NCU_TRAFFIC_BYTES = {("strict", "gpt2_small"): 146.9e6 + 45.5e6, ("fast", "long_context"): 455.2e6 + 224.4e6}
 SM_COUNT = 148
 FP32_LANES_PER_SM = 128
 
@@ -389,7 +392,9 @@ def main():
             "bwd_tflops": flops(w, "bwd") / (bwd_call_ms * 1e-3) / 1e12,
             "fwd_ms": fwd_call_ms, "bwd_ms": bwd_call_ms,
             "roofline": {"kernel": "bwd_main (fused dK/dV/dQ)", "bound": bound, "achieved": bwd_main_tflops,
-                         "peak": peak, "unit": "TFLOP/s", "frac": bwd_main_tflops / peak, "traffic": None,
+                         "peak": peak, "unit": "TFLOP/s", "frac": bwd_main_tflops / peak,
+                         "traffic": NCU_TRAFFIC_BYTES.get((args.mode, w.name)),
+                         "traffic_unit": "bytes per launch (ncu dram read+write, see profiles/)",
                          "ms_per_launch": bwd_main_ms, "peak_source": peak_note,
                          "fwd_kernel": {"achieved": fwd_main_tflops, "frac": fwd_main_tflops / peak,
                                         "ms_per_launch": fwd_main_ms}},
