@@ -20,10 +20,14 @@
 //         Global f32 reduce-add runs at about 20 bytes per clock per SM on this part (3300 clocks
 //         for one 64 KB partial), and issued from the load/store unit it stalls every shared-memory
 //         access of the SM; so it goes through TMA and is waited for only by the drain warps.
-// Issue order per pair: MMA4(n), MMA1(n+1), MMA6(n), MMA5(n), MMA2(n+1): the next scores are ready
-// while dQ/dK are still being multiplied, and dP^T(n+1) follows as soon as Y has been drained.
+// Two issuing threads share the tensor core.  Issuer A runs MMA4(n), MMA1(n+1) as soon as P^T(n)
+// is in tensor memory (before dS(n) exists), so the next scores are ready when the compute warps
+// come back for them; issuer B runs MMA6(n), MMA2(n+1), MMA5(n) once dS(n) is in shared memory
+// (the dQ partial first so its drain starts early, dP^T of the next pair as soon as Y has been
+// drained, dK last: nothing waits for it).  The compute warps then never wait for the tensor core
+// in steady state: exp(n+1) and dS(n+1) run back to back.
 // Tensor memory: X [0,128)  Y [128,256)  dK [256,256+D)  dV [256+D,256+2D).
-// Warp roles (512 threads): warp 0 TMA producer, warp 1 MMA issuer, warps 4-11 compute,
+// Warp roles (512 threads): warp 0 TMA producer, warps 1-2 MMA issuers, warps 4-11 compute,
 // warps 12-15 dQ drain; register budgets are rebalanced with setmaxnreg (104 / 128 / 128 / 144).
 #include <cuda_bf16.h>
 
@@ -57,7 +61,7 @@ struct Cfg {
 };
 
 enum { B_KV = 0, B_QFULL = 1, B_QEMPTY = 3, B_DOFULL = 5, B_DOEMPTY = 6, B_SFULL = 7, B_DPFULL = 8,
-       B_PDSFULL = 9, B_DQFULL = 10, B_DQEMPTY = 11, B_DKVFULL = 12, B_COUNT = 13 };
+       B_PDSFULL = 9, B_DQFULL = 10, B_DQEMPTY = 11, B_DKVFULL = 12, B_DSEMPTY = 13, B_PFULL = 14, B_COUNT = 15 };
 
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
@@ -89,7 +93,7 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     const float c2 = scale * kLog2e;
 
     if (tid == 0) {
-        for (int i = 0; i < B_COUNT; ++i) mbar_init(bar(i), i == B_PDSFULL ? 256 : (i == B_DQEMPTY ? 128 : 1));
+        for (int i = 0; i < B_COUNT; ++i) mbar_init(bar(i), (i == B_PDSFULL || i == B_PFULL) ? 256 : (i == B_DQEMPTY ? 128 : (i == B_DKVFULL ? 2 : 1)));
         fence_mbar_init();
     }
     __syncwarp();
@@ -125,73 +129,84 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                     tma_load_3d(sdO + ch * C::CHUNK_BYTES, &tmdO, bar(B_DOFULL), ch * 64, i0, bh);
             }
         }
-        } else if (warp == 1 && lane == 0) {
-        // ------------------------------------------------------------------ MMA issuer
+        } else if ((warp == 1 || warp == 2) && lane == 0) {
+        // ------------------------------------------------------------------ MMA issuers
         {
             constexpr uint32_t idesc_st = umma_idesc_bf16(BLK, BLK, false, false);   // S^T, dP^T
             constexpr uint32_t idesc_dv = umma_idesc_bf16(BLK, D, false, true);      // A tmem / K-major, B MN-major
             constexpr uint32_t idesc_dq = umma_idesc_bf16(BLK, D, true, true);       // A MN-major, B MN-major
             // Descriptors are built once; inside the loops only the start-address field moves (it
-            // holds address >> 4 and cannot carry out of its 14 bits within shared memory).  The
-            // issuing thread is a single lane: every instruction it saves shortens the gap between
-            // two tensor-core instructions.
+            // holds address >> 4 and cannot carry out of its 14 bits within shared memory).
             auto kmajor_off = [](int kk) { return static_cast<uint64_t>(((kk >> 2) * C::CHUNK_BYTES + (kk & 3) * 32) >> 4); };
             auto mn_off = [](int kk) { return static_cast<uint64_t>((kk * 2048) >> 4); };
-            const uint64_t kK = umma_smem_desc(sK, 16, 1024), kV = umma_smem_desc(sV, 16, 1024);
-            const uint64_t kQ = umma_smem_desc(sQ, 16, 1024), kdO = umma_smem_desc(sdO, 16, 1024);
-            const uint64_t kdS = umma_smem_desc(sdS, 16, 1024);
-            const uint64_t mK = umma_smem_desc(sK, C::CHUNK_BYTES, 1024), mQ = umma_smem_desc(sQ, C::CHUNK_BYTES, 1024);
-            const uint64_t mdO = umma_smem_desc(sdO, C::CHUNK_BYTES, 1024), mdS = umma_smem_desc(sdS, C::CHUNK_BYTES, 1024);
             const uint32_t tXa = tmem + C::TM_X, tYa = tmem + C::TM_Y, tDK = tmem + C::TM_DK, tDV = tmem + C::TM_DV;
-            auto mma1 = [&](int n) {   // S^T = K Q(n)^T -> X
-                const uint64_t qd = kQ + static_cast<uint64_t>(((n & 1) * C::TILE_BYTES) >> 4);
-#pragma unroll
-                for (int kk = 0; kk < D / 16; ++kk) umma_ss(tXa, kK + kmajor_off(kk), qd + kmajor_off(kk), idesc_st, kk > 0);
-                umma_commit(bar(B_SFULL));
-            };
-            auto mma2 = [&]() {        // dP^T = V dO^T -> Y
-#pragma unroll
-                for (int kk = 0; kk < D / 16; ++kk) umma_ss(tYa, kV + kmajor_off(kk), kdO + kmajor_off(kk), idesc_st, kk > 0);
-                umma_commit(bar(B_DPFULL));
-            };
             mbar_wait(bar(B_KV), 0, status);
-            mbar_wait(bar(B_QFULL + 0), 0, status);
-            tc_fence_after();
-            mma1(0);
-            mbar_wait(bar(B_DOFULL), 0, status);
-            tc_fence_after();
-            mma2();
-            for (int n = 0; n < N; ++n) {
-                const uint64_t qm = mQ + static_cast<uint64_t>(((n & 1) * C::TILE_BYTES) >> 4);
-                const uint32_t acc0 = n > 0;
-                mbar_wait(bar(B_PDSFULL), n & 1, status);
+            if (warp == 1) {
+                // ---- issuer A: dV += P^T dO (MMA4), then the next S^T = K Q^T (MMA1) into X
+                const uint64_t kK = umma_smem_desc(sK, 16, 1024), kQ = umma_smem_desc(sQ, 16, 1024);
+                const uint64_t mdO = umma_smem_desc(sdO, C::CHUNK_BYTES, 1024);
+                auto mma1 = [&](int n) {
+                    const uint64_t qd = kQ + static_cast<uint64_t>(((n & 1) * C::TILE_BYTES) >> 4);
+#pragma unroll
+                    for (int kk = 0; kk < D / 16; ++kk) umma_ss(tXa, kK + kmajor_off(kk), qd + kmajor_off(kk), idesc_st, kk > 0);
+                    umma_commit(bar(B_SFULL));
+                };
+                mbar_wait(bar(B_QFULL + 0), 0, status);
                 tc_fence_after();
-                // MMA4: dV += P^T dO(n).  P^T: queries 0-63 at X[0,32), queries 64-127 at X[64,96)
-#pragma unroll
-                for (int kk = 0; kk < BLK / 16; ++kk)
-                    umma_ts(tDV, tXa + (kk >> 2) * 64 + (kk & 3) * 8, mdO + mn_off(kk), idesc_dv, kk > 0 ? 1u : acc0);
-                umma_commit(bar(B_DOEMPTY));
-                // MMA1 of the next pair right behind it: X is free once MMA4 has read P^T, and the
-                // compute warps can then exponentiate the next scores while MMA5/MMA6 run
-                if (n + 1 < N) {
-                    mbar_wait(bar(B_QFULL + ((n + 1) & 1)), ((n + 1) >> 1) & 1, status);
+                mma1(0);
+                for (int n = 0; n < N; ++n) {
+                    const uint32_t acc0 = n > 0;
+                    // P^T(n) is complete as soon as the exponentials are done, well before dS(n):
+                    // dV and the next scores are issued at that point, so S^T(n+1) is waiting when
+                    // the compute warps finish dS(n)
+                    // (the operand tiles arrive long before P^T: wait for them first, so that only one
+                    // barrier round trip separates the end of the exponentials from the first MMA)
+                    mbar_wait(bar(B_DOFULL), n & 1, status);
+                    mbar_wait(bar(B_PFULL), n & 1, status);
                     tc_fence_after();
-                    mma1(n + 1);
+                    // P^T: queries 0-63 at X[0,32), queries 64-127 at X[64,96)
+#pragma unroll
+                    for (int kk = 0; kk < BLK / 16; ++kk)
+                        umma_ts(tDV, tXa + (kk >> 2) * 64 + (kk & 3) * 8, mdO + mn_off(kk), idesc_dv, kk > 0 ? 1u : acc0);
+                    umma_commit(bar(B_DOEMPTY));
+                    if (n + 1 < N) {
+                        mbar_wait(bar(B_QFULL + ((n + 1) & 1)), ((n + 1) >> 1) & 1, status);
+                        tc_fence_after();
+                        mma1(n + 1);      // X is free once MMA4 has read P^T (same issuer: in order)
+                    }
                 }
-                // MMA6: dQ partial = dS K -> Y (first, so that the drain can start early)
+            } else {
+                // ---- issuer B: dQ partial (MMA6), dP^T of the next pair (MMA2), dK (MMA5)
+                const uint64_t kV = umma_smem_desc(sV, 16, 1024), kdO = umma_smem_desc(sdO, 16, 1024);
+                const uint64_t kdS = umma_smem_desc(sdS, 16, 1024), mdS = umma_smem_desc(sdS, C::CHUNK_BYTES, 1024);
+                const uint64_t mK = umma_smem_desc(sK, C::CHUNK_BYTES, 1024), mQ = umma_smem_desc(sQ, C::CHUNK_BYTES, 1024);
+                auto mma2 = [&]() {
 #pragma unroll
-                for (int kk = 0; kk < BLK / 16; ++kk) umma_ss(tYa, mdS + mn_off(kk), mK + mn_off(kk), idesc_dq, kk > 0);
-                umma_commit(bar(B_DQFULL));
-                // MMA5: dK += dS^T Q(n)
-#pragma unroll
-                for (int kk = 0; kk < BLK / 16; ++kk)
-                    umma_ss(tDK, kdS + kmajor_off(kk), qm + mn_off(kk), idesc_dv, kk > 0 ? 1u : acc0);
-                umma_commit(bar(B_QEMPTY + (n & 1)));
-                if (n + 1 < N) {
-                    mbar_wait(bar(B_DQEMPTY), n & 1, status);
-                    mbar_wait(bar(B_DOFULL), (n + 1) & 1, status);
+                    for (int kk = 0; kk < D / 16; ++kk) umma_ss(tYa, kV + kmajor_off(kk), kdO + kmajor_off(kk), idesc_st, kk > 0);
+                    umma_commit(bar(B_DPFULL));
+                };
+                mbar_wait(bar(B_DOFULL), 0, status);
+                tc_fence_after();
+                mma2();
+                for (int n = 0; n < N; ++n) {
+                    const uint64_t qm = mQ + static_cast<uint64_t>(((n & 1) * C::TILE_BYTES) >> 4);
+                    const uint32_t acc0 = n > 0;
+                    mbar_wait(bar(B_PDSFULL), n & 1, status);
                     tc_fence_after();
-                    mma2();
+#pragma unroll
+                    for (int kk = 0; kk < BLK / 16; ++kk) umma_ss(tYa, mdS + mn_off(kk), mK + mn_off(kk), idesc_dq, kk > 0);
+                    umma_commit(bar(B_DQFULL));
+                    if (n + 1 < N) {
+                        mbar_wait(bar(B_DOFULL), (n + 1) & 1, status);
+                        mbar_wait(bar(B_DQEMPTY), n & 1, status);            // Y drained
+                        tc_fence_after();
+                        mma2();
+                    }
+#pragma unroll
+                    for (int kk = 0; kk < BLK / 16; ++kk)
+                        umma_ss(tDK, kdS + kmajor_off(kk), qm + mn_off(kk), idesc_dv, kk > 0 ? 1u : acc0);
+                    umma_commit(bar(B_QEMPTY + (n & 1)));
+                    umma_commit(bar(B_DSEMPTY));                             // dS(n) buffer may be rewritten
                 }
             }
             umma_commit(bar(B_DKVFULL));
@@ -287,6 +302,9 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                 }
                 tmem_st16(tX + half * 64 + 16 * c, u);
             }
+            tmem_st_wait();
+            tc_fence_before();
+            mbar_arrive(bar(B_PFULL));
         };
 
         float stat_next = load_stat(0);
@@ -298,6 +316,7 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         for (int n = 0; n < N; ++n) {
             // dS^T = P^T (dP^T - delta) -> bf16 -> shared memory [key][query]
             mbar_wait(bar(B_DPFULL), n & 1, status);
+            if (n > 0) mbar_wait(bar(B_DSEMPTY), (n - 1) & 1, status);     // dK/dQ products of the last pair are done with dS
             tc_fence_after();
 #pragma unroll
             for (int c = 0; c < 2; ++c) {
@@ -321,7 +340,6 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                 for (int q = 0; q < 4; ++q)
                     sts128(rowaddr + (((4 * c + q) ^ (r & 7)) << 4), u[4 * q], u[4 * q + 1], u[4 * q + 2], u[4 * q + 3]);
             }
-            tmem_st_wait();
             fence_proxy_async_smem();
             tc_fence_before();
             mbar_arrive(bar(B_PDSFULL));
