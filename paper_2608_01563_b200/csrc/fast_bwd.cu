@@ -53,15 +53,18 @@ struct Cfg {
     static constexpr int OFF_DO = OFF_Q + 2 * TILE_BYTES;
     static constexpr int OFF_DS = OFF_DO + TILE_BYTES;
     static constexpr int OFF_DQ = OFF_DS + DS_BYTES;           // dQ staging: 2 boxes of 128 rows x 32 f32
-    static constexpr int OFF_STAT = OFF_DQ + 2 * CHUNK_BYTES;  // [lse2 | delta][128] f32
-    static constexpr int OFF_BAR = OFF_STAT + 2 * BLK * 4;
-    static constexpr int SMEM = OFF_BAR + 128 + 1024;
+    static constexpr int OFF_STAT = OFF_DQ + 2 * CHUNK_BYTES;  // [2 stages][lse2 | delta][128] f32
+    static constexpr int OFF_BAR = OFF_STAT + 2 * 2 * BLK * 4;
+    static constexpr int PAYLOAD = OFF_BAR + 160;   // 17 barriers + the tensor-memory slot
+    // Aligning the tile base to 1024 bytes can cost up to 1023 bytes; only 864 are left under the
+    // 227 KB per-block limit at D = 128.  The kernel checks the slack it actually got.
+    static constexpr int SMEM = (PAYLOAD + 1024 <= 232448) ? PAYLOAD + 1024 : 232448;
     static_assert(SMEM <= 232448, "shared memory budget");
     static constexpr uint32_t TM_X = 0, TM_Y = 128, TM_DK = 256, TM_DV = 256 + D, TM_COLS = 512;
 };
 
 enum { B_KV = 0, B_QFULL = 1, B_QEMPTY = 3, B_DOFULL = 5, B_DOEMPTY = 6, B_SFULL = 7, B_DPFULL = 8,
-       B_PDSFULL = 9, B_DQFULL = 10, B_DQEMPTY = 11, B_DKVFULL = 12, B_DSEMPTY = 13, B_PFULL = 14, B_COUNT = 15 };
+       B_PDSFULL = 9, B_DQFULL = 10, B_DQEMPTY = 11, B_DKVFULL = 12, B_DSEMPTY = 13, B_PFULL = 14, B_STATFULL = 15 /* two: one per buffer */, B_COUNT = 17 };
 
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
@@ -82,6 +85,10 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (*reinterpret_cast<volatile unsigned*>(status) != 0) return;   // an earlier wait on this device gave up
+    if (base + C::PAYLOAD > smem_u32(smem_raw) + C::SMEM) {           // alignment slack ran out
+        if (tid == 0) atomicMax(status, kStatusSmemLayout);
+        return;
+    }
 
     // heaviest key blocks (lowest j0) first when causal
     const int kb = static_cast<int>(blockIdx.x) / BH;
@@ -93,7 +100,8 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     const float c2 = scale * kLog2e;
 
     if (tid == 0) {
-        for (int i = 0; i < B_COUNT; ++i) mbar_init(bar(i), (i == B_PDSFULL || i == B_PFULL) ? 256 : (i == B_DQEMPTY ? 128 : (i == B_DKVFULL ? 2 : 1)));
+        for (int i = 0; i < B_COUNT; ++i) mbar_init(bar(i), (i == B_PDSFULL || i == B_PFULL) ? 256
+                                 : ((i == B_DQEMPTY || i == B_STATFULL || i == B_STATFULL + 1) ? 128 : (i == B_DKVFULL ? 2 : 1)));
         fence_mbar_init();
     }
     __syncwarp();
@@ -219,8 +227,27 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         const int r = tid - 384;                           // query row of the block = tensor-memory lane
         const uint32_t tY = tmem + (static_cast<uint32_t>(r & ~31) << 16) + C::TM_Y;
         const uint32_t stage = base + C::OFF_DQ;
+        // These warps also stage the row statistics of the query blocks (log2-domain LSE and delta
+        // of row r) two buffers deep, so the compute warps find them in shared memory without
+        // barriers of their own.  Buffer n&1 may be rewritten once dS(n-2) is complete.
+        auto stage_stats = [&](int n) {
+            const int i = (qb0 + n) * BLK + r;
+            const bool ok = i < S;
+            const float l2 = ok ? LSE[static_cast<size_t>(bh) * S + i] * kLog2e : INFINITY;
+            const float dl = ok ? DELTA[static_cast<size_t>(bh) * S + i] : 0.f;
+            const uint32_t buf = sStat + (n & 1) * (2 * BLK * 4);
+            sts32(buf + r * 4, l2);
+            sts32(buf + BLK * 4 + r * 4, dl);
+            mbar_arrive(bar(B_STATFULL + (n & 1)));
+        };
+        stage_stats(0);
+        if (N > 1) stage_stats(1);
         for (int n = 0; n < N; ++n) {
             const int i0 = (qb0 + n) * BLK;
+            if (n + 2 < N) {
+                mbar_wait(bar(B_PDSFULL), n & 1, status);      // compute warps are done with buffer n&1
+                stage_stats(n + 2);
+            }
             mbar_wait(bar(B_DQFULL), n & 1, status);
             tc_fence_after();
             uint32_t v[D / 32][32];
@@ -258,21 +285,13 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         const uint32_t lane_base = static_cast<uint32_t>(r & ~31) << 16;
         const uint32_t tX = tmem + lane_base + C::TM_X, tY = tmem + lane_base + C::TM_Y;
 
-        // Row statistics of the 64 query columns this warpgroup works on, prefetched one block
-        // ahead: threads 0-63 of the warpgroup fetch LSE (log2 domain), threads 64-127 fetch delta.
-        // Each warpgroup writes only the entries it reads, so the buffer needs no cross-warpgroup sync.
-        const uint32_t statL = sStat, statD = sStat + BLK * 4;
-        const uint32_t my_stat = (r < 64 ? statL : statD) + (half * 64 + (r & 63)) * 4;
-        auto load_stat = [&](int n) -> float {
-            const int i = (qb0 + n) * BLK + half * 64 + (r & 63);
-            if (n >= N || i >= S) return r < 64 ? INFINITY : 0.f;
-            return r < 64 ? LSE[static_cast<size_t>(bh) * S + i] * kLog2e : DELTA[static_cast<size_t>(bh) * S + i];
-        };
         uint32_t pk[32];                                                     // P^T of the current pair, packed bf16
 
         // P^T = exp2(S^T c - lse) of pair n: bf16 into X (A operand of dV) and into pk (for dS)
         auto exp_phase = [&](int n) {
             const bool diag = causal && ((qb0 + n) * BLK == j0);
+            const uint32_t statL = sStat + (n & 1) * (2 * BLK * 4);
+            mbar_wait(bar(B_STATFULL + (n & 1)), (n >> 1) & 1, status);
             mbar_wait(bar(B_SFULL), n & 1, status);
             tc_fence_after();
 #pragma unroll
@@ -307,14 +326,11 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             mbar_arrive(bar(B_PFULL));
         };
 
-        float stat_next = load_stat(0);
-        sts32(my_stat, stat_next);
-        named_bar_sync(2 + half, 128);
-        stat_next = load_stat(1);
         exp_phase(0);
 
         for (int n = 0; n < N; ++n) {
             // dS^T = P^T (dP^T - delta) -> bf16 -> shared memory [key][query]
+            const uint32_t statD = sStat + (n & 1) * (2 * BLK * 4) + BLK * 4;
             mbar_wait(bar(B_DPFULL), n & 1, status);
             if (n > 0) mbar_wait(bar(B_DSEMPTY), (n - 1) & 1, status);     // dK/dQ products of the last pair are done with dS
             tc_fence_after();
@@ -345,13 +361,7 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             mbar_arrive(bar(B_PDSFULL));
 
             // next pair's statistics and exponentials while the dQ/dK products of this pair run
-            if (n + 1 < N) {
-                named_bar_sync(2 + half, 128);     // this warpgroup is done reading the old statistics
-                sts32(my_stat, stat_next);
-                named_bar_sync(2 + half, 128);
-                stat_next = load_stat(n + 2);
-                exp_phase(n + 1);
-            }
+            if (n + 1 < N) exp_phase(n + 1);
         }
 
         // ---- epilogue: dK (scaled) by half 0, dV by half 1 -> bf16 -> shared -> TMA store
