@@ -406,6 +406,10 @@ def main():
             d2h = sum(t_.numel() * t_.element_size() for t_ in host_out)
             line["e2e"] = {"value": whole_job_tflops(w, world, K, e2e_ms_max), "unit": "TFLOP/s",
                            "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+        if args.mode == "strict":
+            measured = mgn.mgn_measure_fp32_ffma_tflops()
+            line["fp32_ffma_measured_tflops"] = measured
+            line["frac_of_measured_ffma_peak"] = value / world / measured if measured > 0 else None
         if world == 1 and args.mode == "strict" and args.workload is None and not args.no_fast:
             # the other arithmetic mode of the same library on its own target workload, for the record
             wf = synth.WORKLOADS["long_context"]

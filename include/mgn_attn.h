@@ -132,6 +132,15 @@ int mgn_attn_bwd_noalloc(const void* q, const void* k, const void* v, const void
 /* The constant above, for callers that bind the library without the header. */
 size_t mgn_attn_bwd_noalloc_max_workspace_bytes(void);
 
+/*
+ * Measures the FP32 FFMA peak of the current device with a register-only fused-multiply-add
+ * loop on every SM (synchronous; a few milliseconds).  `scratch` is a device pointer to at least
+ * one float (never written in practice), `tflops` a HOST pointer that receives the best of three
+ * timed repetitions.  Measurement plumbing for the strict-mode roofline; the paper has no
+ * counterpart.  Returns MGN_OK, MGN_ERR_INVALID_ARG or MGN_ERR_CUDA.
+ */
+int mgn_measure_fp32_ffma_tflops(float* scratch, double* tflops, void* stream);
+
 /* Static string naming a status code. */
 const char* mgn_status_string(int status);
 

@@ -53,6 +53,8 @@ def lib() -> ctypes.CDLL:
         L.mgn_attn_bwd_noalloc.restype = i
         L.mgn_attn_bwd_noalloc_max_workspace_bytes.argtypes = []
         L.mgn_attn_bwd_noalloc_max_workspace_bytes.restype = sz
+        L.mgn_measure_fp32_ffma_tflops.argtypes = [vp, ctypes.POINTER(ctypes.c_double), vp]
+        L.mgn_measure_fp32_ffma_tflops.restype = i
         L.mgn_attn_profile_events.argtypes = [vp, vp]
         L.mgn_attn_profile_events.restype = i
         L.mgn_status_string.argtypes = [i]
@@ -125,6 +127,15 @@ def mgn_attn_profile_events(before_main: Optional[int], after_main: Optional[int
     st = lib().mgn_attn_profile_events(before_main, after_main)
     if st != MGN_OK:
         raise MgnError(st, "mgn_attn_profile_events")
+
+
+def mgn_measure_fp32_ffma_tflops(stream: Optional[int] = None) -> float:
+    scratch = torch.zeros(4, dtype=torch.float32, device="cuda")
+    out = ctypes.c_double(0.0)
+    st = lib().mgn_measure_fp32_ffma_tflops(_ptr(scratch), ctypes.byref(out), _stream(stream))
+    if st != MGN_OK:
+        raise MgnError(st, "mgn_measure_fp32_ffma_tflops")
+    return float(out.value)
 
 
 def mgn_status_string(status: int) -> str:

@@ -32,7 +32,7 @@ def declared_symbols():
 def test_every_declared_symbol_is_exported(lib):
     syms = declared_symbols()
     assert {"mgn_attn_fwd", "mgn_attn_bwd", "mgn_attn_bwd_workspace_bytes", "mgn_attn_check",
-            "mgn_status_string", "mgn_version", "mgn_attn_profile_events"} <= set(syms)
+            "mgn_status_string", "mgn_version", "mgn_attn_profile_events", "mgn_attn_bwd_noalloc", "mgn_measure_fp32_ffma_tflops"} <= set(syms)
     for s in syms:
         assert getattr(lib, s) is not None
 
