@@ -196,9 +196,19 @@ def cpu_baseline(w, dtype, budget_s=15.0):
     heads = min(w.BH, probe_heads * rounds)
     if heads > probe_heads:
         tf, tb, _ = time_oracle(w, dtype, heads)
+    # if even all heads take well under the budget, repeat the pass so that about 10 s of CPU work is timed
+    passes = max(1, min(50, int(10.0 / max(tf + tb, 1e-3))))
+    if passes > 1:
+        acc_f = acc_b = 0.0
+        for _ in range(passes):
+            f1, b1, _ = time_oracle(w, dtype, heads)
+            acc_f += f1
+            acc_b += b1
+        tf, tb = acc_f / passes, acc_b / passes
     fl = flops(w, "sum") * heads / w.BH
     return {"value": fl / (tf + tb) / 1e12, "unit": "TFLOP/s", "cores": threads, "kind": "oracle",
-            "sample": f"first {heads} of {w.BH} heads of {w.name} (f64, fwd {tf:.2f} s + bwd {tb:.2f} s)",
+            "sample": (f"first {heads} of {w.BH} heads of {w.name}, mean of {passes} passes "
+                       f"(f64, fwd {tf:.2f} s + bwd {tb:.2f} s per pass)"),
             "cpu_model": cpu_info()}
 
 
@@ -342,12 +352,41 @@ def main():
     # ---- end to end: host buffers in, host buffers out, copies inside the timed region ----------
     e2e = None
     if not args.no_e2e:
+        # The step is pipelined over batch chunks on three streams (host->device, compute,
+        # device->host), as a caller of a stream-ordered C ABI would do: every byte still crosses
+        # PCIe inside the timed region, but copies overlap the kernels of neighbouring chunks.
+        n_chunks = 4 if B % 4 == 0 else (2 if B % 2 == 0 else 1)
+        bc = B // n_chunks
+        s_cmp = torch.cuda.current_stream()
+        s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
+        ws_c = [mgn.alloc_workspace(bc, H, S, D, mode) for _ in range(n_chunks)]
+        in_done = [torch.cuda.Event() for _ in range(n_chunks)]
+        cmp_done = [torch.cuda.Event() for _ in range(n_chunks)]
+        out_done = [torch.cuda.Event() for _ in range(n_chunks)]
+        outs_dev = (o, lse, dq, dk, dv)
+        for evt in cmp_done + out_done:
+            evt.record(s_cmp)
+
         def e2e_step():
-            for h, d in zip(host, dev):
-                d.copy_(h, non_blocking=True)
-            step()
-            for h, d in zip(host_out, (o, lse, dq, dk, dv)):
-                h.copy_(d, non_blocking=True)
+            for c in range(n_chunks):
+                sl = slice(c * bc, (c + 1) * bc)
+                with torch.cuda.stream(s_in):
+                    s_in.wait_event(cmp_done[c])          # previous step's kernels are done with this chunk's inputs
+                    for h, d in zip(host, dev):
+                        d[sl].copy_(h[sl], non_blocking=True)
+                    in_done[c].record(s_in)
+                s_cmp.wait_event(in_done[c])
+                s_cmp.wait_event(out_done[c])             # previous step's outputs of this chunk have left the device
+                mgn.mgn_attn_fwd(qd[sl], kd[sl], vd[sl], o[sl], lse[sl], w.causal, w.scale, mode)
+                mgn.mgn_attn_bwd(qd[sl], kd[sl], vd[sl], o[sl], dod[sl], lse[sl], dq[sl], dk[sl], dv[sl], ws_c[c],
+                                 w.causal, w.scale, mode)
+                cmp_done[c].record(s_cmp)
+                with torch.cuda.stream(s_out):
+                    s_out.wait_event(cmp_done[c])
+                    for h, d in zip(host_out, outs_dev):
+                        h[sl].copy_(d[sl], non_blocking=True)
+                    out_done[c].record(s_out)
+            s_cmp.wait_event(out_done[n_chunks - 1])      # the step ends when its last bytes are on the host
         for _ in range(3):
             e2e_step()
         barrier()
@@ -385,6 +424,7 @@ def main():
             "dtype": "f32" if args.mode == "strict" else "bf16", "data": "synthetic",
             "config": {"workload": w.name, "B": w.B, "H": w.H, "S": w.S, "D": w.D, "causal": w.causal,
                        "mode": args.mode, "per_rank_batch": "full workload on every rank",
+                       "e2e": "pinned host buffers; batch split in chunks pipelined over H2D / compute / D2H streams",
                        "l2": "no flush: Q,K,V,dO,O,dQ,dK,dV of one step exceed the 126 MB L2"
                        if 8 * qd.numel() * qd.element_size() > 126e6 else "working set fits L2 (compute-bound path)"},
             "frac_of_peak": value / world / peak, "peak_tflops": peak, "peak_note": peak_note,
