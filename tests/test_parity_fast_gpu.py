@@ -87,6 +87,16 @@ def test_decoder_sweep_head_subset(name, heads):
     _workload_parity(name, heads)
 
 
+def test_decoder_sweep_longest_sequence_two_heads():
+    w = synth.WORKLOADS["decoder_sweep_S8192"]
+    heads = [5, 100]
+    q, k, v, d_o = synth.make_inputs(w, dtype=BF)
+    res = hp.run_cuda(q, k, v, d_o, w.causal, w.scale, MODE)
+    ref = hp.run_oracle(q, k, v, d_o, w.causal, w.scale, heads)
+    hp.check_fast(hp.select(res, w.B, w.H, heads), ref, label=w.name + " ")
+    hp.check_invariants(q, k, v, d_o, res, rtol=2e-2, max_heads=16)
+
+
 def test_d32_is_reported_unsupported_in_fast_mode():
     q = torch.zeros(1, 1, 8, 32, device="cuda", dtype=BF)
     lse = torch.zeros(1, 1, 8, device="cuda")

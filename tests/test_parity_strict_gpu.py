@@ -46,6 +46,18 @@ def test_decoder_sweep_outliers_head_subset(name, heads):
     _full_parity(synth.WORKLOADS[name], heads=heads, literal=False)
 
 
+def test_decoder_sweep_longest_sequence_two_heads():
+    """S = 8192 (the largest configured size), in the launch configuration the benchmark times:
+    two heads element by element against the oracle, invariants on 16 heads."""
+    w = synth.WORKLOADS["decoder_sweep_S8192"]
+    heads = [5, 100]
+    q, k, v, d_o = synth.make_inputs(w)
+    res = hp.run_cuda(q, k, v, d_o, w.causal, w.scale, MODE)
+    ref = hp.run_oracle(q, k, v, d_o, w.causal, w.scale, heads)
+    hp.check_strict(hp.select(res, w.B, w.H, heads), ref, literal_max_abs=False, label=w.name + " ")
+    hp.check_invariants(q, k, v, d_o, res, rtol=2e-5, max_heads=16)
+
+
 @pytest.mark.parametrize("D", [32, 64, 128])
 @pytest.mark.parametrize("causal", [False, True])
 @pytest.mark.parametrize("S", [1, 2, 63, 64, 65, 127, 129, 197, 300])
