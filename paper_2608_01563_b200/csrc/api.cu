@@ -125,24 +125,20 @@ int mgn_attn_bwd(const void* q, const void* k, const void* v, const void* o, con
     float* delta = static_cast<float*>(workspace);
     const bool fast = mode == MGN_MODE_FAST_BF16;
 
-    cudaError_t e = mgn::launch_bwd_preprocess(o, d_o, delta, rows, D, fast ? 1 : 0, st);
+    // delta, and the dQ accumulation target cleared in the same pass (dQ is accumulated by
+    // floating-point reductions: in place in strict mode, in an f32 workspace tensor in fast mode)
+    float* dq_acc = fast ? reinterpret_cast<float*>(static_cast<char*>(workspace) + ws_delta_bytes(rows))
+                         : static_cast<float*>(dq);
+    cudaError_t e = mgn::launch_bwd_preprocess(o, d_o, delta, dq_acc, rows, D, fast ? 1 : 0, st);
     if (e != cudaSuccess) return MGN_ERR_CUDA;
-    if (!fast) {
-        // dQ is accumulated in place by floating-point reductions: start from zero.
-        e = cudaMemsetAsync(dq, 0, rows * D * sizeof(float), st);
-        if (e != cudaSuccess) return MGN_ERR_CUDA;
-        MainKernelTimer timer(st);
+    MainKernelTimer timer(st);
+    if (!fast)
         e = mgn::launch_strict_bwd(p, static_cast<const float*>(q), static_cast<const float*>(k),
                                    static_cast<const float*>(v), static_cast<const float*>(d_o), lse, delta,
                                    static_cast<float*>(dq), static_cast<float*>(dk), static_cast<float*>(dv), status,
                                    st);
-    } else {
-        float* dq_acc = reinterpret_cast<float*>(static_cast<char*>(workspace) + ws_delta_bytes(rows));
-        e = cudaMemsetAsync(dq_acc, 0, rows * D * sizeof(float), st);
-        if (e != cudaSuccess) return MGN_ERR_CUDA;
-        MainKernelTimer timer(st);
+    else
         e = mgn::launch_fast_bwd(p, q, k, v, d_o, lse, delta, dq_acc, dq, dk, dv, status, st);
-    }
     return e == cudaSuccess ? MGN_OK : MGN_ERR_CUDA;
 }
 

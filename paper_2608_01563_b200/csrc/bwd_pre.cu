@@ -1,6 +1,7 @@
 // Backward preprocess: delta_i = sum_d dO[i,d] * O[i,d] for every (b,h,i) row.
 // HBM-bound streaming kernel: 128-bit loads, D/4 (f32) or D/8 (bf16) lanes per row,
-// shuffle reduction inside the lane group.  (The paper's backward kernels need this
+// shuffle reduction inside the lane group.  The same pass clears the f32 dQ accumulation target
+// (row r of `zero`, D floats), which saves a separate memset launch.  (The paper's backward kernels need this
 // row statistic; it is the "backward preprocess" step of the attention path.)
 #include <cuda_bf16.h>
 
@@ -11,7 +12,8 @@ namespace {
 
 template <int LANES, bool BF16>
 __global__ void __launch_bounds__(256)
-bwd_preprocess_kernel(const uint4* __restrict__ o, const uint4* __restrict__ d_o, float* __restrict__ delta, size_t rows)
+bwd_preprocess_kernel(const uint4* __restrict__ o, const uint4* __restrict__ d_o, float* __restrict__ delta,
+                      float4* __restrict__ zero, size_t rows)
 {
     constexpr int ROWS_PER_BLOCK = 256 / LANES;
     const int lane = threadIdx.x % LANES;
@@ -21,6 +23,9 @@ bwd_preprocess_kernel(const uint4* __restrict__ o, const uint4* __restrict__ d_o
         const size_t r = r0 + sub;
         float acc = 0.f;
         if (r < rows) {
+            constexpr int ZPL = BF16 ? 2 : 1;      // float4 stores per lane to cover a row of D floats
+#pragma unroll
+            for (int t = 0; t < ZPL; ++t) zero[(r * LANES + lane) * ZPL + t] = make_float4(0.f, 0.f, 0.f, 0.f);
             const uint4 a = __ldg(o + r * LANES + lane);
             const uint4 b = __ldg(d_o + r * LANES + lane);
             if constexpr (BF16) {
@@ -46,33 +51,33 @@ bwd_preprocess_kernel(const uint4* __restrict__ o, const uint4* __restrict__ d_o
 }
 
 template <int LANES, bool BF16>
-cudaError_t run(const void* o, const void* d_o, float* delta, size_t rows, cudaStream_t st)
+cudaError_t run(const void* o, const void* d_o, float* delta, float* zero, size_t rows, cudaStream_t st)
 {
     constexpr int ROWS_PER_BLOCK = 256 / LANES;
     size_t blocks = (rows + ROWS_PER_BLOCK - 1) / ROWS_PER_BLOCK;
     const size_t cap = 148u * 8u * 4u;
     if (blocks > cap) blocks = cap;
     bwd_preprocess_kernel<LANES, BF16><<<static_cast<unsigned>(blocks), 256, 0, st>>>(
-        static_cast<const uint4*>(o), static_cast<const uint4*>(d_o), delta, rows);
+        static_cast<const uint4*>(o), static_cast<const uint4*>(d_o), delta, reinterpret_cast<float4*>(zero), rows);
     return cudaGetLastError();
 }
 
 }  // namespace
 
-cudaError_t launch_bwd_preprocess(const void* o, const void* d_o, float* delta, size_t rows, int D, int is_bf16,
-                                  cudaStream_t st)
+cudaError_t launch_bwd_preprocess(const void* o, const void* d_o, float* delta, float* zero, size_t rows, int D,
+                                  int is_bf16, cudaStream_t st)
 {
     if (is_bf16) {
         switch (D) {
-            case 32:  return run<4, true>(o, d_o, delta, rows, st);
-            case 64:  return run<8, true>(o, d_o, delta, rows, st);
-            case 128: return run<16, true>(o, d_o, delta, rows, st);
+            case 32:  return run<4, true>(o, d_o, delta, zero, rows, st);
+            case 64:  return run<8, true>(o, d_o, delta, zero, rows, st);
+            case 128: return run<16, true>(o, d_o, delta, zero, rows, st);
         }
     } else {
         switch (D) {
-            case 32:  return run<8, false>(o, d_o, delta, rows, st);
-            case 64:  return run<16, false>(o, d_o, delta, rows, st);
-            case 128: return run<32, false>(o, d_o, delta, rows, st);
+            case 32:  return run<8, false>(o, d_o, delta, zero, rows, st);
+            case 64:  return run<16, false>(o, d_o, delta, zero, rows, st);
+            case 128: return run<32, false>(o, d_o, delta, zero, rows, st);
         }
     }
     return cudaErrorInvalidValue;

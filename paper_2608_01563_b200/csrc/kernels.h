@@ -23,8 +23,9 @@ cudaError_t launch_strict_bwd(const Problem& p, const float* q, const float* k, 
                               const float* d_o, const float* lse, const float* delta,
                               float* dq, float* dk, float* dv, unsigned* status, cudaStream_t st);
 
-// delta_i = sum_d dO[i,d] O[i,d]  (f32 or bf16 inputs, f32 output), HBM-bound.
-cudaError_t launch_bwd_preprocess(const void* o, const void* d_o, float* delta,
+// delta_i = sum_d dO[i,d] O[i,d]  (f32 or bf16 inputs, f32 output), HBM-bound; also clears the
+// f32 dQ accumulation target `zero` ([rows][D] floats).
+cudaError_t launch_bwd_preprocess(const void* o, const void* d_o, float* delta, float* zero,
                                   size_t rows, int D, int is_bf16, cudaStream_t st);
 
 // Fast (bf16 tcgen05) kernels.
