@@ -2,7 +2,12 @@
 // accumulation in tensor memory, f32 softmax statistics (paper Section 3.3 "tiled attention
 // forward"; Section 4.2: the validated reduced-input path with f32 accumulation).
 //
-// One CTA owns two 128-row query tiles of one head and walks over 128-key blocks.
+// Persistent kernel: one CTA per SM walks over work items (two 128-row query tiles of one head
+// each, heaviest first, dealt out in snake order so that every CTA gets the same amount of
+// work) and, per item, over 128-key blocks.  All barriers keep counting across items, so the
+// producer prefetches the next item's Q/K/V and the issuers compute its first scores while the
+// softmax warps are still writing the previous item's output: the per-item fill and drain
+// (about 10 us against 2 us per key block) is hidden instead of paid by every CTA.
 // Warp roles (384 threads):
 //   warp 0      TMA producer: Q tiles once, then K and V blocks through a 2-stage ring
 //   warps 1, 2  MMA issuers, one per query tile: S_t = Q_t K^T (operands in shared memory) and
@@ -42,14 +47,41 @@ struct Cfg {
     static constexpr int OFF_Q = 0;
     static constexpr int OFF_K = OFF_Q + 2 * TILE_BYTES;
     static constexpr int OFF_V = OFF_K + kStages * TILE_BYTES;
-    static constexpr int OFF_XCHG = OFF_V + kStages * TILE_BYTES;   // [2 halves][128 rows] f32 exchange
+    static constexpr int OFF_OST = OFF_V + kStages * TILE_BYTES;    // output staging, one tile
+    static constexpr int OFF_XCHG = OFF_OST + TILE_BYTES;           // [2 halves][128 rows] f32 exchange
     static constexpr int OFF_BAR = OFF_XCHG + 2 * 128 * 4;
     static constexpr int SMEM = OFF_BAR + 256 + 1024;
+    static_assert(SMEM <= 232448, "shared memory budget");
     static constexpr uint32_t TM_S = 0, TM_O = 256, TM_COLS = 512;
 };
 
 // barrier slots (8 bytes each)
-enum { B_Q = 0, B_KFULL = 1, B_KEMPTY = 3, B_VFULL = 5, B_VEMPTY = 7, B_SFULL = 9, B_PFULL = 11, B_OFULL = 13, B_COUNT = 15 };
+enum { B_Q = 0, B_KFULL = 1, B_KEMPTY = 3, B_VFULL = 5, B_VEMPTY = 7, B_SFULL = 9, B_PFULL = 11, B_OFULL = 13,
+       B_QEMPTY = 15, B_OEMPTY = 16, B_COUNT = 18 };
+
+// Work item `it` (heaviest first): query-tile pair and head.
+struct Item {
+    int pair, bh, row0[2], nblk[2], n_max;
+};
+__device__ __forceinline__ Item make_item(int it, int BH, int n_pairs, int S, int causal) {
+    Item w;
+    w.pair = n_pairs - 1 - it / BH;
+    w.bh = it % BH;
+    const int n_kb = (S + BN - 1) / BN;
+#pragma unroll
+    for (int t = 0; t < 2; ++t) {
+        w.row0[t] = w.pair * 2 * BM + t * BM;
+        if (w.row0[t] >= S) w.nblk[t] = 0;
+        else w.nblk[t] = causal ? min(n_kb, (min(w.row0[t] + BM, S) - 1) / BN + 1) : n_kb;
+    }
+    w.n_max = max(w.nblk[0], w.nblk[1]);
+    return w;
+}
+// k-th item of CTA c out of G: tiers of G items, odd tiers dealt backwards (snake), -1 past the end.
+__device__ __forceinline__ int item_index(int c, int k, int G, int n_items) {
+    const int it = k * G + ((k & 1) ? (G - 1 - c) : c);
+    return it < n_items ? it : -1;
+}
 
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
@@ -68,26 +100,15 @@ fast_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (*reinterpret_cast<volatile unsigned*>(status) != 0) return;   // an earlier wait on this device gave up
 
-    // heaviest (last) query-tile pairs first when causal
-    const int pair = n_pairs - 1 - static_cast<int>(blockIdx.x) / BH;
-    const int bh = static_cast<int>(blockIdx.x) % BH;
-    const int n_kb = (S + BN - 1) / BN;
-    int row0[2], nblk[2];
-#pragma unroll
-    for (int t = 0; t < 2; ++t) {
-        row0[t] = pair * 2 * BM + t * BM;
-        if (row0[t] >= S) nblk[t] = 0;
-        else nblk[t] = causal ? min(n_kb, (min(row0[t] + BM, S) - 1) / BN + 1) : n_kb;
-    }
-    const int n_max = max(nblk[0], nblk[1]);
+    const int n_items = n_pairs * BH;
+    const int G = static_cast<int>(gridDim.x), cta = static_cast<int>(blockIdx.x);
+    const int n_tiers = (n_items + G - 1) / G;
 
     if (tid == 0) {
-        const uint32_t issuers = nblk[1] > 0 ? 2 : 1;      // K/V stages are released by every active issuer
         for (int i = 0; i < B_COUNT; ++i) {
             uint32_t cnt = 1;
-            if (i == B_PFULL || i == B_PFULL + 1) cnt = 256;
-            if (i >= B_KEMPTY && i < B_KEMPTY + 2) cnt = issuers;
-            if (i >= B_VEMPTY && i < B_VEMPTY + 2) cnt = issuers;
+            if (i == B_PFULL || i == B_PFULL + 1 || i == B_OEMPTY || i == B_OEMPTY + 1) cnt = 256;
+            if ((i >= B_KEMPTY && i < B_KEMPTY + 2) || (i >= B_VEMPTY && i < B_VEMPTY + 2) || i == B_QEMPTY) cnt = 2;
             mbar_init(bar(i), cnt);
         }
         fence_mbar_init();
@@ -104,32 +125,38 @@ fast_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         if (warp == 0 && lane == 0) {
         // ------------------------------------------------------------------ TMA producer
         {
-            const int nq = (nblk[1] > 0) ? 2 : 1;
-            mbar_arrive_expect_tx(bar(B_Q), nq * C::TILE_BYTES);
-            for (int t = 0; t < nq; ++t)
+            int g = 0;                                       // key blocks loaded so far (all items)
+            for (int k = 0; k < n_tiers; ++k) {
+                const int it = item_index(cta, k, G, n_items);
+                if (it < 0) break;
+                const Item w = make_item(it, BH, n_pairs, S, causal);
+                mbar_wait(bar(B_QEMPTY), (k & 1) ^ 1, status);   // both issuers are done with the previous Q tiles
+                const int nq = (w.nblk[1] > 0) ? 2 : 1;
+                mbar_arrive_expect_tx(bar(B_Q), nq * C::TILE_BYTES);
+                for (int t = 0; t < nq; ++t)
 #pragma unroll
-                for (int ch = 0; ch < C::NCH; ++ch)
-                    tma_load_3d(sQ + t * C::TILE_BYTES + ch * C::CHUNK_BYTES, &tmQ, bar(B_Q), ch * 64, row0[t], bh);
-            for (int n = 0; n < n_max; ++n) {
-                const int st = n & 1;
-                const uint32_t ph = (n >> 1) & 1;
-                mbar_wait(bar(B_KEMPTY + st), ph ^ 1, status);
-                mbar_arrive_expect_tx(bar(B_KFULL + st), C::TILE_BYTES);
+                    for (int ch = 0; ch < C::NCH; ++ch)
+                        tma_load_3d(sQ + t * C::TILE_BYTES + ch * C::CHUNK_BYTES, &tmQ, bar(B_Q), ch * 64, w.row0[t], w.bh);
+                for (int n = 0; n < w.n_max; ++n, ++g) {
+                    const int st = g & 1;
+                    const uint32_t ph = (g >> 1) & 1;
+                    mbar_wait(bar(B_KEMPTY + st), ph ^ 1, status);
+                    mbar_arrive_expect_tx(bar(B_KFULL + st), C::TILE_BYTES);
 #pragma unroll
-                for (int ch = 0; ch < C::NCH; ++ch)
-                    tma_load_3d(sK + st * C::TILE_BYTES + ch * C::CHUNK_BYTES, &tmK, bar(B_KFULL + st), ch * 64, n * BN, bh);
-                mbar_wait(bar(B_VEMPTY + st), ph ^ 1, status);
-                mbar_arrive_expect_tx(bar(B_VFULL + st), C::TILE_BYTES);
+                    for (int ch = 0; ch < C::NCH; ++ch)
+                        tma_load_3d(sK + st * C::TILE_BYTES + ch * C::CHUNK_BYTES, &tmK, bar(B_KFULL + st), ch * 64, n * BN, w.bh);
+                    mbar_wait(bar(B_VEMPTY + st), ph ^ 1, status);
+                    mbar_arrive_expect_tx(bar(B_VFULL + st), C::TILE_BYTES);
 #pragma unroll
-                for (int ch = 0; ch < C::NCH; ++ch)
-                    tma_load_3d(sV + st * C::TILE_BYTES + ch * C::CHUNK_BYTES, &tmV, bar(B_VFULL + st), ch * 64, n * BN, bh);
+                    for (int ch = 0; ch < C::NCH; ++ch)
+                        tma_load_3d(sV + st * C::TILE_BYTES + ch * C::CHUNK_BYTES, &tmV, bar(B_VFULL + st), ch * 64, n * BN, w.bh);
+                }
             }
         }
-        } else if ((warp == 1 || warp == 2) && lane == 0 && nblk[warp - 1] > 0) {
+        } else if ((warp == 1 || warp == 2) && lane == 0) {
         // ------------------------------------------------------------------ MMA issuer of tile t
         {
             const int t = warp - 1;
-            const int nb = nblk[t];
             constexpr uint32_t idesc_s = umma_idesc_bf16(BM, BN, false, false);
             constexpr uint32_t idesc_o = umma_idesc_bf16(BM, D, false, true);
             // Descriptors are built once; inside the loops only the start-address field moves (the
@@ -138,8 +165,8 @@ fast_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             const uint64_t dK0 = umma_smem_desc(sK, 16, 1024);
             const uint64_t dV0 = umma_smem_desc(sV, C::CHUNK_BYTES, 1024);
             const uint32_t tSd = tmem + C::TM_S + t * 128, tOd = tmem + C::TM_O + t * D;
-            auto issue_s = [&](int n) {   // S_t = Q_t K(n)^T
-                const uint64_t kd = dK0 + static_cast<uint64_t>(((n & 1) * C::TILE_BYTES) >> 4);
+            auto issue_s = [&](int st) {   // S_t = Q_t K(stage st)^T
+                const uint64_t kd = dK0 + static_cast<uint64_t>((st * C::TILE_BYTES) >> 4);
 #pragma unroll
                 for (int kk = 0; kk < D / 16; ++kk) {
                     const uint64_t off = static_cast<uint64_t>(((kk >> 2) * C::CHUNK_BYTES + (kk & 3) * 32) >> 4);
@@ -147,37 +174,52 @@ fast_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                 }
                 umma_commit(bar(B_SFULL + t));
             };
-            auto issue_o = [&](int n) {   // O_t += P_t V(n)
-                const uint64_t vd = dV0 + static_cast<uint64_t>(((n & 1) * C::TILE_BYTES) >> 4);
-                const uint32_t acc0 = n > 0;
+            auto issue_o = [&](int st, uint32_t acc0) {   // O_t (+)= P_t V(stage st)
+                const uint64_t vd = dV0 + static_cast<uint64_t>((st * C::TILE_BYTES) >> 4);
 #pragma unroll
                 for (int kk = 0; kk < BN / 16; ++kk)
                     umma_ts(tOd, tSd + (kk >> 2) * 64 + (kk & 3) * 8, vd + static_cast<uint64_t>((kk * 2048) >> 4), idesc_o,
                             kk > 0 ? 1u : acc0);
             };
-            mbar_wait(bar(B_Q), 0, status);
-            mbar_wait(bar(B_KFULL + 0), 0, status);
-            tc_fence_after();
-            issue_s(0);
-            umma_commit(bar(B_KEMPTY + 0));
-            for (int n = 0; n < n_max; ++n) {
-                const int st = n & 1;
-                if (n < nb) {
-                    mbar_wait(bar(B_VFULL + st), (n >> 1) & 1, status);
-                    mbar_wait(bar(B_PFULL + t), n & 1, status);
-                    tc_fence_after();
-                    issue_o(n);
-                    if (n == nb - 1) umma_commit(bar(B_OFULL + t));
-                }
-                umma_commit(bar(B_VEMPTY + st));          // this issuer is done with V(n)
-                if (n + 1 < n_max) {
-                    if (n + 1 < nb) {
-                        mbar_wait(bar(B_KFULL + (st ^ 1)), ((n + 1) >> 1) & 1, status);
+            int g = 0;       // key blocks seen so far (all items): stage and phase of the K/V ring
+            int cp = 0;      // P_t blocks consumed so far: phase of P_FULL[t]
+            int co = 0;      // items in which this tile was active: phase of O_EMPTY[t]
+            for (int k = 0; k < n_tiers; ++k) {
+                const int it = item_index(cta, k, G, n_items);
+                if (it < 0) break;
+                const Item w = make_item(it, BH, n_pairs, S, causal);
+                const int nb = w.nblk[t];
+                mbar_wait(bar(B_Q), k & 1, status);
+                mbar_wait(bar(B_KFULL + (g & 1)), (g >> 1) & 1, status);
+                tc_fence_after();
+                if (nb > 0) issue_s(g & 1);
+                umma_commit(bar(B_KEMPTY + (g & 1)));
+                if (nb <= 1) umma_commit(bar(B_QEMPTY));          // no further S products of this item from this issuer
+                if (nb > 0) mbar_wait(bar(B_OEMPTY + t), (co & 1) ^ 1, status);   // the last item's O_t has been read out
+                for (int n = 0; n < w.n_max; ++n, ++g) {
+                    const int st = g & 1;
+                    // Every issuer waits for every block, also the ones its tile does not use: an
+                    // issuer that ran ahead could release a ring slot twice in one phase.
+                    mbar_wait(bar(B_VFULL + st), (g >> 1) & 1, status);
+                    if (n < nb) {
+                        mbar_wait(bar(B_PFULL + t), cp & 1, status);
+                        ++cp;
                         tc_fence_after();
-                        issue_s(n + 1);
+                        issue_o(st, n > 0);
+                        if (n == nb - 1) umma_commit(bar(B_OFULL + t));
                     }
-                    umma_commit(bar(B_KEMPTY + (st ^ 1)));   // ... and with K(n+1)
+                    umma_commit(bar(B_VEMPTY + st));          // this issuer is done with V(n)
+                    if (n + 1 < w.n_max) {
+                        mbar_wait(bar(B_KFULL + (st ^ 1)), ((g + 1) >> 1) & 1, status);
+                        if (n + 1 < nb) {
+                            tc_fence_after();
+                            issue_s(st ^ 1);
+                            if (n + 2 == nb) umma_commit(bar(B_QEMPTY));   // that was this item's last S product
+                        }
+                        umma_commit(bar(B_KEMPTY + (st ^ 1)));   // ... and with K(n+1)
+                    }
                 }
+                if (nb > 0) ++co;
             }
         }
         }
@@ -190,7 +232,9 @@ fast_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         const uint32_t lane_base = static_cast<uint32_t>(r & ~31) << 16;
         const uint32_t xchg = base + C::OFF_XCHG;
         const uint32_t my_x = xchg + (h * 128 + r) * 4, peer_x = xchg + ((h ^ 1) * 128 + r) * 4;
-        float m_ref[2] = {-INFINITY, -INFINITY}, l[2] = {0.f, 0.f};
+        const uint32_t ost = base + C::OFF_OST;
+        int cs[2] = {0, 0};      // S_t blocks consumed so far (all items): phase of S_FULL[t]
+        int co[2] = {0, 0};      // items in which tile t was active: phase of O_FULL[t]
 
         // barrier over the 256 softmax threads with an OR reduction of `pred`
         auto bar_or = [](bool pred) -> bool {
@@ -202,6 +246,14 @@ fast_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             return out != 0;
         };
 
+        for (int k = 0; k < n_tiers; ++k) {
+        const int it = item_index(cta, k, G, n_items);
+        if (it < 0) break;
+        const Item w = make_item(it, BH, n_pairs, S, causal);
+        const int bh = w.bh, n_max = w.n_max;
+        const int row0[2] = {w.row0[0], w.row0[1]}, nblk[2] = {w.nblk[0], w.nblk[1]};
+        float m_ref[2] = {-INFINITY, -INFINITY}, l[2] = {0.f, 0.f};
+
         for (int n = 0; n < n_max; ++n) {
 #pragma unroll
             for (int t = 0; t < 2; ++t) {
@@ -209,7 +261,7 @@ fast_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                 const uint32_t tS = tmem + lane_base + C::TM_S + t * 128 + 64 * h;   // this thread's 64 score columns
                 const uint32_t tO = tmem + lane_base + C::TM_O + t * D + (D / 2) * h;
                 const int i = row0[t] + r;
-                mbar_wait(bar(B_SFULL + t), n & 1, status);
+                mbar_wait(bar(B_SFULL + t), (cs[t] + n) & 1, status);
                 tc_fence_after();
                 const int j0 = n * BN + 64 * h;
                 const bool masked = (causal && (j0 + 63 > row0[t])) || (j0 + 64 > S);
@@ -321,23 +373,26 @@ fast_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             const uint32_t tO = tmem + lane_base + C::TM_O + t * D + (D / 2) * h;
             const int i = row0[t] + r;
             sts32(my_x, l[t]);
+            if (r == 0 && h == 0) bulk_wait_group_read0();     // the previous store has finished reading the staging tile
             bar_or(false);
             const float lt = l[t] + lds32f(peer_x);
-            mbar_wait(bar(B_OFULL + t), 0, status);
+            mbar_wait(bar(B_OFULL + t), co[t] & 1, status);
             tc_fence_after();
             const float inv = 1.0f / lt;
-            const uint32_t stage = sQ + t * C::TILE_BYTES;     // Q_t is no longer needed
-#pragma unroll 1
+            uint32_t v[D / 64][32];
+#pragma unroll
+            for (int c = 0; c < D / 64; ++c) tmem_ld32(tO + 32 * c, v[c]);
+            tmem_ld_wait();
+            tc_fence_before();
+            mbar_arrive(bar(B_OEMPTY + t));                    // the next item may overwrite O_t
+#pragma unroll
             for (int c = 0; c < D / 64; ++c) {
-                uint32_t v[32];
-                tmem_ld32(tO + 32 * c, v);
-                tmem_ld_wait();
                 uint32_t u[16];
 #pragma unroll
                 for (int e = 0; e < 16; ++e)
-                    u[e] = pack_bf16(__uint_as_float(v[2 * e]) * inv, __uint_as_float(v[2 * e + 1]) * inv);
+                    u[e] = pack_bf16(__uint_as_float(v[c][2 * e]) * inv, __uint_as_float(v[c][2 * e + 1]) * inv);
                 const int col = (D / 2) * h + 32 * c;          // first output column of this chunk
-                const uint32_t rowaddr = stage + (col >> 6) * C::CHUNK_BYTES + r * 128;
+                const uint32_t rowaddr = ost + (col >> 6) * C::CHUNK_BYTES + r * 128;
 #pragma unroll
                 for (int q = 0; q < 4; ++q) {
                     const int piece = ((col & 63) >> 3) + q;
@@ -350,10 +405,15 @@ fast_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             if (r == 0 && h == 0) {
 #pragma unroll
                 for (int ch = 0; ch < C::NCH; ++ch)
-                    tma_store_3d(&tmO, stage + ch * C::CHUNK_BYTES, ch * 64, row0[t], bh);
-                tma_store_commit_and_wait_read();
+                    tma_store_3d(&tmO, ost + ch * C::CHUNK_BYTES, ch * 64, row0[t], bh);
+                bulk_commit_group();
             }
+            ++co[t];
         }
+        cs[0] += nblk[0];
+        cs[1] += nblk[1];
+        }   // items
+        if (r == 0 && h == 0) bulk_wait_group_read0();
     }
 
     tc_fence_before();
@@ -375,8 +435,13 @@ cudaError_t launch(const Problem& p, const void* q, const void* k, const void* v
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM);
     if (e != cudaSuccess) return e;
     const int n_pairs = (p.S + 2 * BM - 1) / (2 * BM);
-    const long long blocks = static_cast<long long>(n_pairs) * p.BH;
-    if (blocks > 0x7fffffffLL) return cudaErrorInvalidValue;
+    const long long items = static_cast<long long>(n_pairs) * p.BH;
+    if (items > 0x7fffffffLL) return cudaErrorInvalidValue;
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+        return cudaErrorInvalidValue;
+    const long long blocks = items < sms ? items : sms;       // persistent: one CTA per SM
     kern<<<static_cast<unsigned>(blocks), kThreads, C::SMEM, st>>>(tq, tk, tv, to, lse, p.S, p.BH, n_pairs, p.causal,
                                                                    p.scale * kLog2e, status);
     return cudaGetLastError();
