@@ -2,9 +2,12 @@
 // accumulation in tensor memory (paper Section 3.3 "dQ, and fused dK+dV kernels"; Section 7.3
 // FlashGradKV / FlashGradQ; Section 4.2 for the reduced-input arithmetic contract).
 //
-// Single pass.  One CTA keeps one 128-key block (K, V tiles) resident in shared memory, holds the
-// dK and dV accumulators of that block in tensor memory, and walks over the 128-row query blocks
-// (from the diagonal down when causal).  All score-shaped tiles are computed TRANSPOSED
+// Single pass, persistent: one CTA per SM walks over work items (one 128-key block of one head
+// each, heaviest first, dealt out in snake order).  Per item it keeps the K, V tiles resident in
+// shared memory, holds the dK and dV accumulators of that block in tensor memory, and walks over
+// the 128-row query blocks (from the diagonal down when causal).  Every barrier keeps counting
+// across items (g = running pair count, k = running item count), so the producer and the issuers
+// start the next item (loads, first S^T and dP^T) while the compute warps write out dK/dV.  All score-shaped tiles are computed TRANSPOSED
 // (lanes = keys, columns = queries) so that P^T can feed dV = P^T dO straight from tensor
 // memory.  Per (key block, query block) pair:
 //   MMA1  S^T  = K Q^T            -> X            MMA2  dP^T = V dO^T -> Y
@@ -28,7 +31,7 @@
 // in steady state: exp(n+1) and dS(n+1) run back to back.
 // Tensor memory: X [0,128)  Y [128,256)  dK [256,256+D)  dV [256+D,256+2D).
 // Warp roles (512 threads): warp 0 TMA producer, warps 1-2 MMA issuers, warps 4-11 compute,
-// warps 12-15 dQ drain; register budgets are rebalanced with setmaxnreg (104 / 128 / 128 / 144).
+// warps 12-15 dQ drain; register budgets are rebalanced with setmaxnreg (104 / 128 / 128 / 152).
 #include <cuda_bf16.h>
 
 #include "kernels.h"
@@ -55,7 +58,7 @@ struct Cfg {
     static constexpr int OFF_DQ = OFF_DS + DS_BYTES;           // dQ staging: 2 boxes of 128 rows x 32 f32
     static constexpr int OFF_STAT = OFF_DQ + 2 * CHUNK_BYTES;  // [2 stages][lse2 | delta][128] f32
     static constexpr int OFF_BAR = OFF_STAT + 2 * 2 * BLK * 4;
-    static constexpr int PAYLOAD = OFF_BAR + 160;   // 17 barriers + the tensor-memory slot
+    static constexpr int PAYLOAD = OFF_BAR + 168;   // 20 barriers + the tensor-memory slot
     // Aligning the tile base to 1024 bytes can cost up to 1023 bytes; only 864 are left under the
     // 227 KB per-block limit at D = 128.  The kernel checks the slack it actually got.
     static constexpr int SMEM = (PAYLOAD + 1024 <= 232448) ? PAYLOAD + 1024 : 232448;
@@ -64,7 +67,27 @@ struct Cfg {
 };
 
 enum { B_KV = 0, B_QFULL = 1, B_QEMPTY = 3, B_DOFULL = 5, B_DOEMPTY = 6, B_SFULL = 7, B_DPFULL = 8,
-       B_PDSFULL = 9, B_DQFULL = 10, B_DQEMPTY = 11, B_DKVFULL = 12, B_DSEMPTY = 13, B_PFULL = 14, B_STATFULL = 15 /* two: one per buffer */, B_COUNT = 17 };
+       B_PDSFULL = 9, B_DQFULL = 10, B_DQEMPTY = 11, B_DKVFULL = 12, B_DSEMPTY = 13, B_PFULL = 14, B_STATFULL = 15 /* two: one per buffer */,
+       B_KVEMPTY = 17, B_DKVEMPTY = 18, B_PDSFULL1 = 19 /* dS of odd pairs; B_PDSFULL: even pairs */, B_COUNT = 20 };
+
+// Work item `it` (heaviest first): key block and head.
+struct Item {
+    int kb, bh, j0, qb0, N;
+};
+__device__ __forceinline__ Item make_item(int it, int BH, int S, int causal) {
+    Item w;
+    w.kb = it / BH;
+    w.bh = it % BH;
+    w.j0 = w.kb * BLK;
+    w.qb0 = causal ? w.kb : 0;
+    w.N = (S + BLK - 1) / BLK - w.qb0;        // query blocks visited (>= 1)
+    return w;
+}
+// k-th item of CTA c out of G: tiers of G items, odd tiers dealt backwards (snake), -1 past the end.
+__device__ __forceinline__ int item_index(int c, int k, int G, int n_items) {
+    const int it = k * G + ((k & 1) ? (G - 1 - c) : c);
+    return it < n_items ? it : -1;
+}
 
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
@@ -82,6 +105,8 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     const uint32_t sdS = base + C::OFF_DS, sStat = base + C::OFF_STAT, bars = base + C::OFF_BAR;
     const uint32_t tmem_slot = bars + B_COUNT * 8;
     auto bar = [&](int i) { return bars + 8u * i; };
+    // dS(g) complete: one barrier per parity of g, so that a waiter two pairs behind cannot alias phases
+    auto pds_bar = [&](int g) { return bars + 8u * ((g & 1) ? B_PDSFULL1 : B_PDSFULL); };
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (*reinterpret_cast<volatile unsigned*>(status) != 0) return;   // an earlier wait on this device gave up
@@ -90,18 +115,20 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         return;
     }
 
-    // heaviest key blocks (lowest j0) first when causal
-    const int kb = static_cast<int>(blockIdx.x) / BH;
-    const int bh = static_cast<int>(blockIdx.x) % BH;
-    const int j0 = kb * BLK;
-    const int n_qb = (S + BLK - 1) / BLK;
-    const int qb0 = causal ? kb : 0;
-    const int N = n_qb - qb0;                 // query blocks this CTA visits (>= 1)
+    const int n_items = ((S + BLK - 1) / BLK) * BH;
+    const int G = static_cast<int>(gridDim.x), cta = static_cast<int>(blockIdx.x);
+    const int n_tiers = (n_items + G - 1) / G;
     const float c2 = scale * kLog2e;
 
     if (tid == 0) {
-        for (int i = 0; i < B_COUNT; ++i) mbar_init(bar(i), (i == B_PDSFULL || i == B_PFULL) ? 256
-                                 : ((i == B_DQEMPTY || i == B_STATFULL || i == B_STATFULL + 1) ? 128 : (i == B_DKVFULL ? 2 : 1)));
+        for (int i = 0; i < B_COUNT; ++i) {
+            uint32_t cnt = 1;
+            if (i == B_PDSFULL || i == B_PDSFULL1 || i == B_PFULL || i == B_DKVEMPTY) cnt = 256;
+            if (i == B_DQEMPTY) cnt = 128;
+            if (i == B_STATFULL || i == B_STATFULL + 1) cnt = 32;
+            if (i == B_DKVFULL || i == B_KVEMPTY || i == B_DOEMPTY) cnt = 2;   // one arrival per issuer
+            mbar_init(bar(i), cnt);
+        }
         fence_mbar_init();
     }
     __syncwarp();
@@ -116,25 +143,32 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         if (warp == 0 && lane == 0) {
         // ------------------------------------------------------------------ TMA producer
         {
-            mbar_arrive_expect_tx(bar(B_KV), 2 * C::TILE_BYTES);
+            int g = 0;                                          // pairs loaded so far (all items)
+            for (int k = 0; k < n_tiers; ++k) {
+                const int it = item_index(cta, k, G, n_items);
+                if (it < 0) break;
+                const Item w = make_item(it, BH, S, causal);
+                mbar_wait(bar(B_KVEMPTY), (k & 1) ^ 1, status);  // both issuers are done with the previous K, V
+                mbar_arrive_expect_tx(bar(B_KV), 2 * C::TILE_BYTES);
 #pragma unroll
-            for (int ch = 0; ch < C::NCH; ++ch) {
-                tma_load_3d(sK + ch * C::CHUNK_BYTES, &tmK, bar(B_KV), ch * 64, j0, bh);
-                tma_load_3d(sV + ch * C::CHUNK_BYTES, &tmV, bar(B_KV), ch * 64, j0, bh);
-            }
-            for (int n = 0; n < N; ++n) {
-                const int st = n & 1;
-                const int i0 = (qb0 + n) * BLK;
-                mbar_wait(bar(B_QEMPTY + st), ((n >> 1) & 1) ^ 1, status);
-                mbar_arrive_expect_tx(bar(B_QFULL + st), C::TILE_BYTES);
+                for (int ch = 0; ch < C::NCH; ++ch) {
+                    tma_load_3d(sK + ch * C::CHUNK_BYTES, &tmK, bar(B_KV), ch * 64, w.j0, w.bh);
+                    tma_load_3d(sV + ch * C::CHUNK_BYTES, &tmV, bar(B_KV), ch * 64, w.j0, w.bh);
+                }
+                for (int n = 0; n < w.N; ++n, ++g) {
+                    const int st = g & 1;
+                    const int i0 = (w.qb0 + n) * BLK;
+                    mbar_wait(bar(B_QEMPTY + st), ((g >> 1) & 1) ^ 1, status);
+                    mbar_arrive_expect_tx(bar(B_QFULL + st), C::TILE_BYTES);
 #pragma unroll
-                for (int ch = 0; ch < C::NCH; ++ch)
-                    tma_load_3d(sQ + st * C::TILE_BYTES + ch * C::CHUNK_BYTES, &tmQ, bar(B_QFULL + st), ch * 64, i0, bh);
-                mbar_wait(bar(B_DOEMPTY), (n & 1) ^ 1, status);
-                mbar_arrive_expect_tx(bar(B_DOFULL), C::TILE_BYTES);
+                    for (int ch = 0; ch < C::NCH; ++ch)
+                        tma_load_3d(sQ + st * C::TILE_BYTES + ch * C::CHUNK_BYTES, &tmQ, bar(B_QFULL + st), ch * 64, i0, w.bh);
+                    mbar_wait(bar(B_DOEMPTY), (g & 1) ^ 1, status);
+                    mbar_arrive_expect_tx(bar(B_DOFULL), C::TILE_BYTES);
 #pragma unroll
-                for (int ch = 0; ch < C::NCH; ++ch)
-                    tma_load_3d(sdO + ch * C::CHUNK_BYTES, &tmdO, bar(B_DOFULL), ch * 64, i0, bh);
+                    for (int ch = 0; ch < C::NCH; ++ch)
+                        tma_load_3d(sdO + ch * C::CHUNK_BYTES, &tmdO, bar(B_DOFULL), ch * 64, i0, w.bh);
+                }
             }
         }
         } else if ((warp == 1 || warp == 2) && lane == 0) {
@@ -148,40 +182,47 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             auto kmajor_off = [](int kk) { return static_cast<uint64_t>(((kk >> 2) * C::CHUNK_BYTES + (kk & 3) * 32) >> 4); };
             auto mn_off = [](int kk) { return static_cast<uint64_t>((kk * 2048) >> 4); };
             const uint32_t tXa = tmem + C::TM_X, tYa = tmem + C::TM_Y, tDK = tmem + C::TM_DK, tDV = tmem + C::TM_DV;
-            mbar_wait(bar(B_KV), 0, status);
             if (warp == 1) {
                 // ---- issuer A: dV += P^T dO (MMA4), then the next S^T = K Q^T (MMA1) into X
                 const uint64_t kK = umma_smem_desc(sK, 16, 1024), kQ = umma_smem_desc(sQ, 16, 1024);
                 const uint64_t mdO = umma_smem_desc(sdO, C::CHUNK_BYTES, 1024);
-                auto mma1 = [&](int n) {
-                    const uint64_t qd = kQ + static_cast<uint64_t>(((n & 1) * C::TILE_BYTES) >> 4);
+                auto mma1 = [&](int g) {
+                    const uint64_t qd = kQ + static_cast<uint64_t>(((g & 1) * C::TILE_BYTES) >> 4);
 #pragma unroll
                     for (int kk = 0; kk < D / 16; ++kk) umma_ss(tXa, kK + kmajor_off(kk), qd + kmajor_off(kk), idesc_st, kk > 0);
                     umma_commit(bar(B_SFULL));
                 };
-                mbar_wait(bar(B_QFULL + 0), 0, status);
-                tc_fence_after();
-                mma1(0);
-                for (int n = 0; n < N; ++n) {
-                    const uint32_t acc0 = n > 0;
-                    // P^T(n) is complete as soon as the exponentials are done, well before dS(n):
-                    // dV and the next scores are issued at that point, so S^T(n+1) is waiting when
-                    // the compute warps finish dS(n)
-                    // (the operand tiles arrive long before P^T: wait for them first, so that only one
-                    // barrier round trip separates the end of the exponentials from the first MMA)
-                    mbar_wait(bar(B_DOFULL), n & 1, status);
-                    mbar_wait(bar(B_PFULL), n & 1, status);
+                int g = 0;
+                for (int k = 0; k < n_tiers; ++k) {
+                    const int it = item_index(cta, k, G, n_items);
+                    if (it < 0) break;
+                    const Item w = make_item(it, BH, S, causal);
+                    mbar_wait(bar(B_KV), k & 1, status);
+                    mbar_wait(bar(B_QFULL + (g & 1)), (g >> 1) & 1, status);
                     tc_fence_after();
-                    // P^T: queries 0-63 at X[0,32), queries 64-127 at X[64,96)
-#pragma unroll
-                    for (int kk = 0; kk < BLK / 16; ++kk)
-                        umma_ts(tDV, tXa + (kk >> 2) * 64 + (kk & 3) * 8, mdO + mn_off(kk), idesc_dv, kk > 0 ? 1u : acc0);
-                    umma_commit(bar(B_DOEMPTY));
-                    if (n + 1 < N) {
-                        mbar_wait(bar(B_QFULL + ((n + 1) & 1)), ((n + 1) >> 1) & 1, status);
+                    mma1(g);             // X: P^T of the previous item was read by its last MMA4 (same issuer)
+                    for (int n = 0; n < w.N; ++n, ++g) {
+                        // P^T(n) is complete as soon as the exponentials are done, well before dS(n):
+                        // dV and the next scores are issued at that point, so S^T(n+1) is waiting when
+                        // the compute warps finish dS(n).  The operand tile arrives long before P^T.
+                        mbar_wait(bar(B_DOFULL), g & 1, status);
+                        mbar_wait(bar(B_PFULL), g & 1, status);
+                        if (n == 0) mbar_wait(bar(B_DKVEMPTY), (k & 1) ^ 1, status);   // last item's dV has been read out
                         tc_fence_after();
-                        mma1(n + 1);      // X is free once MMA4 has read P^T (same issuer: in order)
+                        // P^T: queries 0-63 at X[0,32), queries 64-127 at X[64,96)
+#pragma unroll
+                        for (int kk = 0; kk < BLK / 16; ++kk)
+                            umma_ts(tDV, tXa + (kk >> 2) * 64 + (kk & 3) * 8, mdO + mn_off(kk), idesc_dv,
+                                    (kk > 0 || n > 0) ? 1u : 0u);
+                        umma_commit(bar(B_DOEMPTY));
+                        if (n + 1 < w.N) {
+                            mbar_wait(bar(B_QFULL + ((g + 1) & 1)), ((g + 1) >> 1) & 1, status);
+                            tc_fence_after();
+                            mma1(g + 1);      // X is free once MMA4 has read P^T (same issuer: in order)
+                        }
                     }
+                    umma_commit(bar(B_DKVFULL));
+                    umma_commit(bar(B_KVEMPTY));      // this issuer's last product with K of this item is done
                 }
             } else {
                 // ---- issuer B: dQ partial (MMA6), dP^T of the next pair (MMA2), dK (MMA5)
@@ -192,63 +233,87 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
 #pragma unroll
                     for (int kk = 0; kk < D / 16; ++kk) umma_ss(tYa, kV + kmajor_off(kk), kdO + kmajor_off(kk), idesc_st, kk > 0);
                     umma_commit(bar(B_DPFULL));
+                    umma_commit(bar(B_DOEMPTY));     // with issuer A's arrival after dV: both readers of dO are done
                 };
-                mbar_wait(bar(B_DOFULL), 0, status);
-                tc_fence_after();
-                mma2();
-                for (int n = 0; n < N; ++n) {
-                    const uint64_t qm = mQ + static_cast<uint64_t>(((n & 1) * C::TILE_BYTES) >> 4);
-                    const uint32_t acc0 = n > 0;
-                    mbar_wait(bar(B_PDSFULL), n & 1, status);
+                int g = 0;
+                for (int k = 0; k < n_tiers; ++k) {
+                    const int it = item_index(cta, k, G, n_items);
+                    if (it < 0) break;
+                    const Item w = make_item(it, BH, S, causal);
+                    mbar_wait(bar(B_KV), k & 1, status);
+                    mbar_wait(bar(B_DOFULL), g & 1, status);
+                    if (g > 0) mbar_wait(bar(B_DQEMPTY), (g - 1) & 1, status);   // Y: last item's final dQ partial drained
                     tc_fence_after();
-#pragma unroll
-                    for (int kk = 0; kk < BLK / 16; ++kk) umma_ss(tYa, mdS + mn_off(kk), mK + mn_off(kk), idesc_dq, kk > 0);
-                    umma_commit(bar(B_DQFULL));
-                    if (n + 1 < N) {
-                        mbar_wait(bar(B_DOFULL), (n + 1) & 1, status);
-                        mbar_wait(bar(B_DQEMPTY), n & 1, status);            // Y drained
+                    mma2();
+                    for (int n = 0; n < w.N; ++n, ++g) {
+                        const uint64_t qm = mQ + static_cast<uint64_t>(((g & 1) * C::TILE_BYTES) >> 4);
+                        mbar_wait(pds_bar(g), (g >> 1) & 1, status);
                         tc_fence_after();
-                        mma2();
-                    }
 #pragma unroll
-                    for (int kk = 0; kk < BLK / 16; ++kk)
-                        umma_ss(tDK, kdS + kmajor_off(kk), qm + mn_off(kk), idesc_dv, kk > 0 ? 1u : acc0);
-                    umma_commit(bar(B_QEMPTY + (n & 1)));
-                    umma_commit(bar(B_DSEMPTY));                             // dS(n) buffer may be rewritten
+                        for (int kk = 0; kk < BLK / 16; ++kk) umma_ss(tYa, mdS + mn_off(kk), mK + mn_off(kk), idesc_dq, kk > 0);
+                        umma_commit(bar(B_DQFULL));
+                        if (n + 1 < w.N) {
+                            mbar_wait(bar(B_DOFULL), (g + 1) & 1, status);
+                            mbar_wait(bar(B_DQEMPTY), g & 1, status);            // Y drained
+                            tc_fence_after();
+                            mma2();
+                        }
+                        if (n == 0) mbar_wait(bar(B_DKVEMPTY), (k & 1) ^ 1, status);   // last item's dK has been read out
+#pragma unroll
+                        for (int kk = 0; kk < BLK / 16; ++kk)
+                            umma_ss(tDK, kdS + kmajor_off(kk), qm + mn_off(kk), idesc_dv, (kk > 0 || n > 0) ? 1u : 0u);
+                        umma_commit(bar(B_QEMPTY + (g & 1)));
+                        umma_commit(bar(B_DSEMPTY));                             // dS(n) buffer may be rewritten
+                    }
+                    umma_commit(bar(B_DKVFULL));
+                    umma_commit(bar(B_KVEMPTY));
                 }
             }
-            umma_commit(bar(B_DKVFULL));
         }
+        } else if (warp == 3) {
+        // ------------------------------------------------------------------ row statistics
+        // Stages the log2-domain LSE and delta of each query block in shared memory, two pairs
+        // ahead of the compute warps (across item boundaries), so that they find them there
+        // without global loads of their own.  Buffer g&1 may be rewritten once dS(g-2) is complete.
+            int g = 0;
+            for (int k = 0; k < n_tiers; ++k) {
+                const int it = item_index(cta, k, G, n_items);
+                if (it < 0) break;
+                const Item w = make_item(it, BH, S, causal);
+                for (int n = 0; n < w.N; ++n, ++g) {
+                    if (g >= 2) mbar_wait(pds_bar(g), ((g - 2) >> 1) & 1, status);
+                    const uint32_t buf = sStat + (g & 1) * (2 * BLK * 4);
+                    const int i = (w.qb0 + n) * BLK + 4 * lane;        // rows i..i+3 of the head
+                    float l2[4], dl[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const bool ok = i + e < S;
+                        l2[e] = ok ? LSE[static_cast<size_t>(w.bh) * S + i + e] * kLog2e : INFINITY;
+                        dl[e] = ok ? DELTA[static_cast<size_t>(w.bh) * S + i + e] : 0.f;
+                    }
+                    sts128(buf + lane * 16, __float_as_uint(l2[0]), __float_as_uint(l2[1]), __float_as_uint(l2[2]),
+                           __float_as_uint(l2[3]));
+                    sts128(buf + BLK * 4 + lane * 16, __float_as_uint(dl[0]), __float_as_uint(dl[1]),
+                           __float_as_uint(dl[2]), __float_as_uint(dl[3]));
+                    mbar_arrive(bar(B_STATFULL + (g & 1)));
+                }
+            }
         }
         __syncwarp();
     } else if (warp >= 12) {
         // ------------------------------------------------------------------ dQ drain warps
-        reg_alloc<144>();
+        reg_alloc<152>();
         const int r = tid - 384;                           // query row of the block = tensor-memory lane
         const uint32_t tY = tmem + (static_cast<uint32_t>(r & ~31) << 16) + C::TM_Y;
         const uint32_t stage = base + C::OFF_DQ;
-        // These warps also stage the row statistics of the query blocks (log2-domain LSE and delta
-        // of row r) two buffers deep, so the compute warps find them in shared memory without
-        // barriers of their own.  Buffer n&1 may be rewritten once dS(n-2) is complete.
-        auto stage_stats = [&](int n) {
-            const int i = (qb0 + n) * BLK + r;
-            const bool ok = i < S;
-            const float l2 = ok ? LSE[static_cast<size_t>(bh) * S + i] * kLog2e : INFINITY;
-            const float dl = ok ? DELTA[static_cast<size_t>(bh) * S + i] : 0.f;
-            const uint32_t buf = sStat + (n & 1) * (2 * BLK * 4);
-            sts32(buf + r * 4, l2);
-            sts32(buf + BLK * 4 + r * 4, dl);
-            mbar_arrive(bar(B_STATFULL + (n & 1)));
-        };
-        stage_stats(0);
-        if (N > 1) stage_stats(1);
-        for (int n = 0; n < N; ++n) {
-            const int i0 = (qb0 + n) * BLK;
-            if (n + 2 < N) {
-                mbar_wait(bar(B_PDSFULL), n & 1, status);      // compute warps are done with buffer n&1
-                stage_stats(n + 2);
-            }
-            mbar_wait(bar(B_DQFULL), n & 1, status);
+        int g = 0;
+        for (int k = 0; k < n_tiers; ++k) {
+        const int it = item_index(cta, k, G, n_items);
+        if (it < 0) break;
+        const Item w = make_item(it, BH, S, causal);
+        for (int n = 0; n < w.N; ++n, ++g) {
+            const int i0 = (w.qb0 + n) * BLK;
+            mbar_wait(bar(B_DQFULL), g & 1, status);
             tc_fence_after();
             uint32_t v[D / 32][32];
 #pragma unroll
@@ -270,11 +335,12 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                 fence_proxy_async_smem();
                 named_bar_sync(4, 128);
                 if (r == 0) {
-                    tma_reduce_add_3d(&tmdQ, stage, 64 * round, i0, bh);
-                    tma_reduce_add_3d(&tmdQ, stage + C::CHUNK_BYTES, 64 * round + 32, i0, bh);
+                    tma_reduce_add_3d(&tmdQ, stage, 64 * round, i0, w.bh);
+                    tma_reduce_add_3d(&tmdQ, stage + C::CHUNK_BYTES, 64 * round + 32, i0, w.bh);
                     bulk_commit_group();
                 }
             }
+        }
         }
         if (r == 0) bulk_wait_group_read0();
     } else {
@@ -288,11 +354,11 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         uint32_t pk[32];                                                     // P^T of the current pair, packed bf16
 
         // P^T = exp2(S^T c - lse) of pair n: bf16 into X (A operand of dV) and into pk (for dS)
-        auto exp_phase = [&](int n) {
-            const bool diag = causal && ((qb0 + n) * BLK == j0);
-            const uint32_t statL = sStat + (n & 1) * (2 * BLK * 4);
-            mbar_wait(bar(B_STATFULL + (n & 1)), (n >> 1) & 1, status);
-            mbar_wait(bar(B_SFULL), n & 1, status);
+        auto exp_phase = [&](const Item& w, int n, int g) {
+            const bool diag = causal && ((w.qb0 + n) * BLK == w.j0);
+            const uint32_t statL = sStat + (g & 1) * (2 * BLK * 4);
+            mbar_wait(bar(B_STATFULL + (g & 1)), (g >> 1) & 1, status);
+            mbar_wait(bar(B_SFULL), g & 1, status);
             tc_fence_after();
 #pragma unroll
             for (int c = 0; c < 2; ++c) {
@@ -326,13 +392,18 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             mbar_arrive(bar(B_PFULL));
         };
 
-        exp_phase(0);
+        int g = 0;
+        for (int k = 0; k < n_tiers; ++k) {
+        const int it = item_index(cta, k, G, n_items);
+        if (it < 0) break;
+        const Item w = make_item(it, BH, S, causal);
+        exp_phase(w, 0, g);
 
-        for (int n = 0; n < N; ++n) {
+        for (int n = 0; n < w.N; ++n, ++g) {
             // dS^T = P^T (dP^T - delta) -> bf16 -> shared memory [key][query]
-            const uint32_t statD = sStat + (n & 1) * (2 * BLK * 4) + BLK * 4;
-            mbar_wait(bar(B_DPFULL), n & 1, status);
-            if (n > 0) mbar_wait(bar(B_DSEMPTY), (n - 1) & 1, status);     // dK/dQ products of the last pair are done with dS
+            const uint32_t statD = sStat + (g & 1) * (2 * BLK * 4) + BLK * 4;
+            mbar_wait(bar(B_DPFULL), g & 1, status);
+            if (g > 0) mbar_wait(bar(B_DSEMPTY), (g - 1) & 1, status);     // dK/dQ products of the last pair are done with dS
             tc_fence_after();
 #pragma unroll
             for (int c = 0; c < 2; ++c) {
@@ -358,43 +429,49 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             }
             fence_proxy_async_smem();
             tc_fence_before();
-            mbar_arrive(bar(B_PDSFULL));
+            mbar_arrive(pds_bar(g));
 
             // next pair's statistics and exponentials while the dQ/dK products of this pair run
-            if (n + 1 < N) exp_phase(n + 1);
+            if (n + 1 < w.N) exp_phase(w, n + 1, g + 1);
         }
 
-        // ---- epilogue: dK (scaled) by half 0, dV by half 1 -> bf16 -> shared -> TMA store
-        mbar_wait(bar(B_DKVFULL), 0, status);
+        // ---- item epilogue: dK (scaled) by half 0, dV by half 1 -> bf16 registers (the accumulators
+        // are released at that point) -> this half's 16 KB of the dS buffer, one 64-column box at a
+        // time -> TMA store.  The dS buffer is idle here: the last dK product has completed.
+        mbar_wait(bar(B_DKVFULL), k & 1, status);
         tc_fence_after();
         {
             const uint32_t tAcc = tmem + lane_base + (half == 0 ? C::TM_DK : C::TM_DV);
             const float mul = half == 0 ? scale : 1.0f;
-            const uint32_t stage = sQ + half * C::TILE_BYTES;
-#pragma unroll 1
+            const uint32_t stage = sdS + half * C::CHUNK_BYTES;
+            uint32_t u[D / 32][16];
+#pragma unroll
             for (int c = 0; c < D / 32; ++c) {
                 uint32_t v[32];
                 tmem_ld32(tAcc + 32 * c, v);
                 tmem_ld_wait();
-                uint32_t u[16];
 #pragma unroll
                 for (int e = 0; e < 16; ++e)
-                    u[e] = pack_bf16(__uint_as_float(v[2 * e]) * mul, __uint_as_float(v[2 * e + 1]) * mul);
-                const uint32_t rowaddr = stage + (c >> 1) * C::CHUNK_BYTES + r * 128;
+                    u[c][e] = pack_bf16(__uint_as_float(v[2 * e]) * mul, __uint_as_float(v[2 * e + 1]) * mul);
+            }
+            tc_fence_before();
+            mbar_arrive(bar(B_DKVEMPTY));                  // the next item may accumulate into dK, dV
 #pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    const int piece = (c & 1) * 4 + q;
-                    sts128(rowaddr + ((piece ^ (r & 7)) << 4), u[4 * q], u[4 * q + 1], u[4 * q + 2], u[4 * q + 3]);
+            for (int ch = 0; ch < C::NCH; ++ch) {
+                const uint32_t rowaddr = stage + r * 128;
+#pragma unroll
+                for (int q = 0; q < 8; ++q)
+                    sts128(rowaddr + ((q ^ (r & 7)) << 4), u[2 * ch + (q >> 2)][4 * (q & 3)], u[2 * ch + (q >> 2)][4 * (q & 3) + 1],
+                           u[2 * ch + (q >> 2)][4 * (q & 3) + 2], u[2 * ch + (q >> 2)][4 * (q & 3) + 3]);
+                fence_proxy_async_smem();
+                named_bar_sync(2 + half, 128);
+                if (r == 0) {
+                    tma_store_3d(half == 0 ? &tmdK : &tmdV, stage, ch * 64, w.j0, w.bh);
+                    tma_store_commit_and_wait_read();
                 }
+                named_bar_sync(2 + half, 128);             // the box has been read: the buffer may be rewritten
             }
-            fence_proxy_async_smem();
-            named_bar_sync(2 + half, 128);
-            if (r == 0) {
-#pragma unroll
-                for (int ch = 0; ch < C::NCH; ++ch)
-                    tma_store_3d(half == 0 ? &tmdK : &tmdV, stage + ch * C::CHUNK_BYTES, ch * 64, j0, bh);
-                tma_store_commit_and_wait_read();
-            }
+        }
         }
     }
 
@@ -435,8 +512,13 @@ cudaError_t launch(const Problem& p, const void* q, const void* k, const void* v
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM);
     if (e != cudaSuccess) return e;
     const int n_kb = (p.S + BLK - 1) / BLK;
-    const long long blocks = static_cast<long long>(n_kb) * p.BH;
-    if (blocks > 0x7fffffffLL) return cudaErrorInvalidValue;
+    const long long items = static_cast<long long>(n_kb) * p.BH;
+    if (items > 0x7fffffffLL) return cudaErrorInvalidValue;
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+        return cudaErrorInvalidValue;
+    const long long blocks = items < sms ? items : sms;       // persistent: one CTA per SM
     kern<<<static_cast<unsigned>(blocks), kThreads, C::SMEM, st>>>(tq, tk, tv, tdo, tdk, tdv, tdq, lse, delta, p.S,
                                                                    p.BH, p.causal, p.scale, status);
     e = cudaGetLastError();
