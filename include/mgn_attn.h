@@ -100,6 +100,18 @@ int mgn_attn_check(void* stream);
 int mgn_attn_profile_events(void* before_main, void* after_main);
 
 /*
+ * Tuning hook (library plumbing; the paper has no counterpart).  The fast-mode kernels are
+ * persistent: each CTA walks a fixed list of work items (a block of keys or queries of one head).
+ * Two item orders exist: 0, block-major (balanced for any size, but the CTAs running at one time
+ * touch every head), and 1, head-major (the CTAs running at one time share a few heads, whose
+ * tensors stay in L2; balanced only with many items per CTA).  By default (-1) each call picks the
+ * order from the problem size; 0 or 1 forces it for all later fast-mode calls of the process.
+ * Results are the same in either order up to the summation order of dq.  Returns MGN_OK, or
+ * MGN_ERR_INVALID_ARG for any other value.
+ */
+int mgn_attn_fast_item_order(int order);
+
+/*
  * Backward for callers that cannot allocate device memory.  (The paper has no counterpart:
  * this is a convenience of this library.)
  *

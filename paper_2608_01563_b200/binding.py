@@ -57,6 +57,8 @@ def lib() -> ctypes.CDLL:
         L.mgn_measure_fp32_ffma_tflops.restype = i
         L.mgn_attn_profile_events.argtypes = [vp, vp]
         L.mgn_attn_profile_events.restype = i
+        L.mgn_attn_fast_item_order.argtypes = [i]
+        L.mgn_attn_fast_item_order.restype = i
         L.mgn_status_string.argtypes = [i]
         L.mgn_status_string.restype = ctypes.c_char_p
         L.mgn_version.argtypes = []
@@ -127,6 +129,12 @@ def mgn_attn_profile_events(before_main: Optional[int], after_main: Optional[int
     st = lib().mgn_attn_profile_events(before_main, after_main)
     if st != MGN_OK:
         raise MgnError(st, "mgn_attn_profile_events")
+
+
+def mgn_attn_fast_item_order(order: int) -> None:
+    st = lib().mgn_attn_fast_item_order(int(order))
+    if st != MGN_OK:
+        raise MgnError(st, "mgn_attn_fast_item_order")
 
 
 def mgn_measure_fp32_ffma_tflops(stream: Optional[int] = None) -> float:

@@ -7,6 +7,10 @@
 #include "../../include/mgn_attn.h"
 #include "kernels.h"
 
+namespace mgn {
+int g_forced_item_order = -1;
+}
+
 namespace {
 
 // Device status word set by kernels whose bounded waits ran out.
@@ -162,6 +166,13 @@ int mgn_attn_profile_events(void* before_main, void* after_main)
     if ((before_main == nullptr) != (after_main == nullptr)) return MGN_ERR_INVALID_ARG;
     g_ev_before = static_cast<cudaEvent_t>(before_main);
     g_ev_after = static_cast<cudaEvent_t>(after_main);
+    return MGN_OK;
+}
+
+int mgn_attn_fast_item_order(int order)
+{
+    if (order < -1 || order > 1) return MGN_ERR_INVALID_ARG;
+    mgn::g_forced_item_order = order;
     return MGN_OK;
 }
 

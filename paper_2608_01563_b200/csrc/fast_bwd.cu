@@ -58,7 +58,7 @@ struct Cfg {
     static constexpr int OFF_DQ = OFF_DS + DS_BYTES;           // dQ staging: 2 boxes of 128 rows x 32 f32
     static constexpr int OFF_STAT = OFF_DQ + 2 * CHUNK_BYTES;  // [2 stages][lse2 | delta][128] f32
     static constexpr int OFF_BAR = OFF_STAT + 2 * 2 * BLK * 4;
-    static constexpr int PAYLOAD = OFF_BAR + 168;   // 20 barriers + the tensor-memory slot
+    static constexpr int PAYLOAD = OFF_BAR + 176;   // 21 barriers + the tensor-memory slot
     // Aligning the tile base to 1024 bytes can cost up to 1023 bytes; only 864 are left under the
     // 227 KB per-block limit at D = 128.  The kernel checks the slack it actually got.
     static constexpr int SMEM = (PAYLOAD + 1024 <= 232448) ? PAYLOAD + 1024 : 232448;
@@ -67,25 +67,39 @@ struct Cfg {
 };
 
 enum { B_KV = 0, B_QFULL = 1, B_QEMPTY = 3, B_DOFULL = 5, B_DOEMPTY = 6, B_SFULL = 7, B_DPFULL = 8,
-       B_PDSFULL = 9, B_DQFULL = 10, B_DQEMPTY = 11, B_DKVFULL = 12, B_DSEMPTY = 13, B_PFULL = 14, B_STATFULL = 15 /* two: one per buffer */,
-       B_KVEMPTY = 17, B_DKVEMPTY = 18, B_PDSFULL1 = 19 /* dS of odd pairs; B_PDSFULL: even pairs */, B_COUNT = 20 };
+       B_PDSFULL = 9, B_DQFULL = 10, B_DQEMPTY = 11, B_DVFULL = 12, B_DSEMPTY = 13, B_PFULL = 14, B_STATFULL = 15 /* two: one per buffer */,
+       B_KVEMPTY = 17, B_DKVEMPTY = 18, B_PDSFULL1 = 19 /* dS of odd pairs; B_PDSFULL: even pairs */, B_DKFULL = 20, B_COUNT = 21 };
 
-// Work item `it` (heaviest first): key block and head.
+// Work items are (key block, head).  Two orders, chosen by the launcher (pick_schedule):
+//   order 0, block-major: items sorted heaviest first (key block 0 of every head, then block 1, ...),
+//     dealt to the CTAs in tiers of G, odd tiers backwards (snake).  Balanced for any item count,
+//     but the CTAs running at one time touch every head.
+//   order 1, head-major: all blocks of a head are consecutive, alternating heaviest / lightest
+//     remaining block, so that two consecutive items always weigh the same; CTA c takes the item
+//     pairs c, c+G, c+2G, ...  The CTAs running at one time share a few heads, whose dQ accumulator,
+//     Q and dO stay in L2.  Balanced only when there are many item pairs per CTA.
 struct Item {
     int kb, bh, j0, qb0, N;
 };
-__device__ __forceinline__ Item make_item(int it, int BH, int S, int causal) {
+__device__ __forceinline__ Item make_item(int it, int BH, int S, int causal, int order) {
     Item w;
-    w.kb = it / BH;
-    w.bh = it % BH;
+    const int nb = (S + BLK - 1) / BLK;
+    if (order == 0) {
+        w.kb = it / BH;
+        w.bh = it % BH;
+    } else {
+        w.bh = it / nb;
+        const int j = it % nb;
+        w.kb = (j & 1) ? nb - 1 - (j >> 1) : (j >> 1);
+    }
     w.j0 = w.kb * BLK;
     w.qb0 = causal ? w.kb : 0;
-    w.N = (S + BLK - 1) / BLK - w.qb0;        // query blocks visited (>= 1)
+    w.N = nb - w.qb0;                          // query blocks visited (>= 1)
     return w;
 }
-// k-th item of CTA c out of G: tiers of G items, odd tiers dealt backwards (snake), -1 past the end.
-__device__ __forceinline__ int item_index(int c, int k, int G, int n_items) {
-    const int it = k * G + ((k & 1) ? (G - 1 - c) : c);
+// k-th item of CTA c out of G, -1 past the end (then also for every larger k).
+__device__ __forceinline__ int item_index(int c, int k, int G, int n_items, int order) {
+    const int it = order == 0 ? k * G + ((k & 1) ? (G - 1 - c) : c) : 2 * (c + G * (k >> 1)) + (k & 1);
     return it < n_items ? it : -1;
 }
 
@@ -93,10 +107,10 @@ template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
 fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                 const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmdO,
-                const __grid_constant__ CUtensorMap tmdK, const __grid_constant__ CUtensorMap tmdV,
                 const __grid_constant__ CUtensorMap tmdQ,
                 const float* __restrict__ LSE, const float* __restrict__ DELTA,
-                int S, int BH, int causal, float scale, unsigned* status)
+                __nv_bfloat16* __restrict__ dK, __nv_bfloat16* __restrict__ dV,
+                int S, int BH, int causal, int order, float scale, unsigned* status)
 {
     using C = Cfg<D>;
     extern __shared__ uint8_t smem_raw[];
@@ -117,7 +131,7 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
 
     const int n_items = ((S + BLK - 1) / BLK) * BH;
     const int G = static_cast<int>(gridDim.x), cta = static_cast<int>(blockIdx.x);
-    const int n_tiers = (n_items + G - 1) / G;
+    const int n_tiers = 2 * ((n_items + 2 * G - 1) / (2 * G));   // upper bound on items per CTA in either order
     const float c2 = scale * kLog2e;
 
     if (tid == 0) {
@@ -126,7 +140,7 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             if (i == B_PDSFULL || i == B_PDSFULL1 || i == B_PFULL || i == B_DKVEMPTY) cnt = 256;
             if (i == B_DQEMPTY) cnt = 128;
             if (i == B_STATFULL || i == B_STATFULL + 1) cnt = 32;
-            if (i == B_DKVFULL || i == B_KVEMPTY || i == B_DOEMPTY) cnt = 2;   // one arrival per issuer
+            if (i == B_KVEMPTY || i == B_DOEMPTY) cnt = 2;   // one arrival per issuer
             mbar_init(bar(i), cnt);
         }
         fence_mbar_init();
@@ -145,9 +159,9 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         {
             int g = 0;                                          // pairs loaded so far (all items)
             for (int k = 0; k < n_tiers; ++k) {
-                const int it = item_index(cta, k, G, n_items);
+                const int it = item_index(cta, k, G, n_items, order);
                 if (it < 0) break;
-                const Item w = make_item(it, BH, S, causal);
+                const Item w = make_item(it, BH, S, causal, order);
                 mbar_wait(bar(B_KVEMPTY), (k & 1) ^ 1, status);  // both issuers are done with the previous K, V
                 mbar_arrive_expect_tx(bar(B_KV), 2 * C::TILE_BYTES);
 #pragma unroll
@@ -194,9 +208,9 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                 };
                 int g = 0;
                 for (int k = 0; k < n_tiers; ++k) {
-                    const int it = item_index(cta, k, G, n_items);
+                    const int it = item_index(cta, k, G, n_items, order);
                     if (it < 0) break;
-                    const Item w = make_item(it, BH, S, causal);
+                    const Item w = make_item(it, BH, S, causal, order);
                     mbar_wait(bar(B_KV), k & 1, status);
                     mbar_wait(bar(B_QFULL + (g & 1)), (g >> 1) & 1, status);
                     tc_fence_after();
@@ -221,7 +235,7 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                             mma1(g + 1);      // X is free once MMA4 has read P^T (same issuer: in order)
                         }
                     }
-                    umma_commit(bar(B_DKVFULL));
+                    umma_commit(bar(B_DVFULL));
                     umma_commit(bar(B_KVEMPTY));      // this issuer's last product with K of this item is done
                 }
             } else {
@@ -237,9 +251,9 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                 };
                 int g = 0;
                 for (int k = 0; k < n_tiers; ++k) {
-                    const int it = item_index(cta, k, G, n_items);
+                    const int it = item_index(cta, k, G, n_items, order);
                     if (it < 0) break;
-                    const Item w = make_item(it, BH, S, causal);
+                    const Item w = make_item(it, BH, S, causal, order);
                     mbar_wait(bar(B_KV), k & 1, status);
                     mbar_wait(bar(B_DOFULL), g & 1, status);
                     if (g > 0) mbar_wait(bar(B_DQEMPTY), (g - 1) & 1, status);   // Y: last item's final dQ partial drained
@@ -265,7 +279,7 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                         umma_commit(bar(B_QEMPTY + (g & 1)));
                         umma_commit(bar(B_DSEMPTY));                             // dS(n) buffer may be rewritten
                     }
-                    umma_commit(bar(B_DKVFULL));
+                    umma_commit(bar(B_DKFULL));
                     umma_commit(bar(B_KVEMPTY));
                 }
             }
@@ -277,9 +291,9 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         // without global loads of their own.  Buffer g&1 may be rewritten once dS(g-2) is complete.
             int g = 0;
             for (int k = 0; k < n_tiers; ++k) {
-                const int it = item_index(cta, k, G, n_items);
+                const int it = item_index(cta, k, G, n_items, order);
                 if (it < 0) break;
-                const Item w = make_item(it, BH, S, causal);
+                const Item w = make_item(it, BH, S, causal, order);
                 for (int n = 0; n < w.N; ++n, ++g) {
                     if (g >= 2) mbar_wait(pds_bar(g), ((g - 2) >> 1) & 1, status);
                     const uint32_t buf = sStat + (g & 1) * (2 * BLK * 4);
@@ -308,9 +322,9 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         const uint32_t stage = base + C::OFF_DQ;
         int g = 0;
         for (int k = 0; k < n_tiers; ++k) {
-        const int it = item_index(cta, k, G, n_items);
+        const int it = item_index(cta, k, G, n_items, order);
         if (it < 0) break;
-        const Item w = make_item(it, BH, S, causal);
+        const Item w = make_item(it, BH, S, causal, order);
         for (int n = 0; n < w.N; ++n, ++g) {
             const int i0 = (w.qb0 + n) * BLK;
             mbar_wait(bar(B_DQFULL), g & 1, status);
@@ -394,9 +408,9 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
 
         int g = 0;
         for (int k = 0; k < n_tiers; ++k) {
-        const int it = item_index(cta, k, G, n_items);
+        const int it = item_index(cta, k, G, n_items, order);
         if (it < 0) break;
-        const Item w = make_item(it, BH, S, causal);
+        const Item w = make_item(it, BH, S, causal, order);
         exp_phase(w, 0, g);
 
         for (int n = 0; n < w.N; ++n, ++g) {
@@ -435,42 +449,55 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             if (n + 1 < w.N) exp_phase(w, n + 1, g + 1);
         }
 
-        // ---- item epilogue: dK (scaled) by half 0, dV by half 1 -> bf16 registers (the accumulators
-        // are released at that point) -> this half's 16 KB of the dS buffer, one 64-column box at a
-        // time -> TMA store.  The dS buffer is idle here: the last dK product has completed.
-        mbar_wait(bar(B_DKVFULL), k & 1, status);
-        tc_fence_after();
+        // ---- item epilogue.  Each warpgroup writes D/2 columns of dV, then D/2 columns of dK (scaled):
+        // tensor memory -> bf16 registers -> this warpgroup's half of the dS buffer (idle here) ->
+        // coalesced 16-byte global stores.  Not a TMA store: it would queue behind the dQ reductions
+        // of the last pairs in the copy engine.
         {
-            const uint32_t tAcc = tmem + lane_base + (half == 0 ? C::TM_DK : C::TM_DV);
-            const float mul = half == 0 ? scale : 1.0f;
+            constexpr int HC = D / 2;                      // columns per warpgroup and tensor
+            constexpr int PCS = HC / 8;                    // 16-byte pieces per staged row
             const uint32_t stage = sdS + half * C::CHUNK_BYTES;
-            uint32_t u[D / 32][16];
+            auto swz = [](int piece, int row) { return D == 128 ? (piece ^ (row & 7)) : (piece ^ ((row >> 1) & 3)); };
+            auto emit = [&](uint32_t tAcc, float mul, __nv_bfloat16* out, bool last) {
+                uint32_t u[HC / 2];
 #pragma unroll
-            for (int c = 0; c < D / 32; ++c) {
-                uint32_t v[32];
-                tmem_ld32(tAcc + 32 * c, v);
-                tmem_ld_wait();
+                for (int c = 0; c < HC / 32; ++c) {
+                    uint32_t v[32];
+                    tmem_ld32(tAcc + half * HC + 32 * c, v);
+                    tmem_ld_wait();
 #pragma unroll
-                for (int e = 0; e < 16; ++e)
-                    u[c][e] = pack_bf16(__uint_as_float(v[2 * e]) * mul, __uint_as_float(v[2 * e + 1]) * mul);
-            }
-            tc_fence_before();
-            mbar_arrive(bar(B_DKVEMPTY));                  // the next item may accumulate into dK, dV
-#pragma unroll
-            for (int ch = 0; ch < C::NCH; ++ch) {
-                const uint32_t rowaddr = stage + r * 128;
-#pragma unroll
-                for (int q = 0; q < 8; ++q)
-                    sts128(rowaddr + ((q ^ (r & 7)) << 4), u[2 * ch + (q >> 2)][4 * (q & 3)], u[2 * ch + (q >> 2)][4 * (q & 3) + 1],
-                           u[2 * ch + (q >> 2)][4 * (q & 3) + 2], u[2 * ch + (q >> 2)][4 * (q & 3) + 3]);
-                fence_proxy_async_smem();
-                named_bar_sync(2 + half, 128);
-                if (r == 0) {
-                    tma_store_3d(half == 0 ? &tmdK : &tmdV, stage, ch * 64, w.j0, w.bh);
-                    tma_store_commit_and_wait_read();
+                    for (int e = 0; e < 16; ++e)
+                        u[16 * c + e] = pack_bf16(__uint_as_float(v[2 * e]) * mul, __uint_as_float(v[2 * e + 1]) * mul);
                 }
-                named_bar_sync(2 + half, 128);             // the box has been read: the buffer may be rewritten
-            }
+                if (last) {
+                    tc_fence_before();
+                    mbar_arrive(bar(B_DKVEMPTY));          // the next item may accumulate into dK, dV
+                }
+#pragma unroll
+                for (int q = 0; q < PCS; ++q)
+                    sts128(stage + r * (HC * 2) + (swz(q, r) << 4), u[4 * q], u[4 * q + 1], u[4 * q + 2], u[4 * q + 3]);
+                named_bar_sync(2 + half, 128);
+                out += (static_cast<size_t>(w.bh) * S + w.j0) * D + half * HC;
+                float4 val[PCS];
+#pragma unroll
+                for (int i = 0; i < PCS; ++i) {
+                    const int idx = i * 128 + r, row = idx / PCS, piece = idx % PCS;   // a warp covers whole rows
+                    val[i] = lds128(stage + row * (HC * 2) + (swz(piece, row) << 4));
+                }
+#pragma unroll
+                for (int i = 0; i < PCS; ++i) {
+                    const int idx = i * 128 + r, row = idx / PCS, piece = idx % PCS;
+                    if (w.j0 + row < S) *reinterpret_cast<float4*>(out + static_cast<size_t>(row) * D + piece * 8) = val[i];
+                }
+                named_bar_sync(2 + half, 128);             // the slab has been read: the buffer may be rewritten
+            };
+            // Both accumulators complete: then the last dK and dQ products have also finished reading
+            // the dS buffer that the slabs are staged in.
+            mbar_wait(bar(B_DVFULL), k & 1, status);
+            mbar_wait(bar(B_DKFULL), k & 1, status);
+            tc_fence_after();
+            emit(tmem + lane_base + C::TM_DV, 1.0f, dV, false);
+            emit(tmem + lane_base + C::TM_DK, scale, dK, true);
         }
         }
     }
@@ -500,14 +527,12 @@ cudaError_t launch(const Problem& p, const void* q, const void* k, const void* v
                    unsigned* status, cudaStream_t st)
 {
     using C = Cfg<D>;
-    CUtensorMap tq, tk, tv, tdo, tdk, tdv, tdq;
+    CUtensorMap tq, tk, tv, tdo, tdq;
     if (make_tmap_3d(&tdq, dq_acc, 4, 0, p.BH, p.S, D, 32, BLK)) return cudaErrorInvalidValue;
     if (make_tmap_3d(&tq, q, 2, 1, p.BH, p.S, D, 64, BLK)) return cudaErrorInvalidValue;
     if (make_tmap_3d(&tk, k, 2, 1, p.BH, p.S, D, 64, BLK)) return cudaErrorInvalidValue;
     if (make_tmap_3d(&tv, v, 2, 1, p.BH, p.S, D, 64, BLK)) return cudaErrorInvalidValue;
     if (make_tmap_3d(&tdo, d_o, 2, 1, p.BH, p.S, D, 64, BLK)) return cudaErrorInvalidValue;
-    if (make_tmap_3d(&tdk, dk, 2, 1, p.BH, p.S, D, 64, BLK)) return cudaErrorInvalidValue;
-    if (make_tmap_3d(&tdv, dv, 2, 1, p.BH, p.S, D, 64, BLK)) return cudaErrorInvalidValue;
     auto kern = fast_bwd_kernel<D>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM);
     if (e != cudaSuccess) return e;
@@ -519,8 +544,12 @@ cudaError_t launch(const Problem& p, const void* q, const void* k, const void* v
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
         return cudaErrorInvalidValue;
     const long long blocks = items < sms ? items : sms;       // persistent: one CTA per SM
-    kern<<<static_cast<unsigned>(blocks), kThreads, C::SMEM, st>>>(tq, tk, tv, tdo, tdk, tdv, tdq, lse, delta, p.S,
-                                                                   p.BH, p.causal, p.scale, status);
+    // streamed per pair and shared between the key blocks of a head: dQ accumulator (f32), Q, dO
+    const int order = pick_schedule(items, sms, static_cast<double>(p.BH) * p.S * D * (4 + 2 + 2), dev);
+    kern<<<static_cast<unsigned>(blocks), kThreads, C::SMEM, st>>>(tq, tk, tv, tdo, tdq, lse, delta,
+                                                                   static_cast<__nv_bfloat16*>(dk),
+                                                                   static_cast<__nv_bfloat16*>(dv), p.S, p.BH, p.causal,
+                                                                   order, p.scale, status);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     const size_t n4 = static_cast<size_t>(p.BH) * p.S * D / 4;

@@ -59,14 +59,24 @@ struct Cfg {
 enum { B_Q = 0, B_KFULL = 1, B_KEMPTY = 3, B_VFULL = 5, B_VEMPTY = 7, B_SFULL = 9, B_PFULL = 11, B_OFULL = 13,
        B_QEMPTY = 15, B_OEMPTY = 16, B_COUNT = 18 };
 
-// Work item `it` (heaviest first): query-tile pair and head.
+// Work item `it`: query-tile pair and head.  Order 0 (block-major): heaviest tiles of every head
+// first, dealt in snake order -- balanced for any item count, but the CTAs running at one time touch
+// every head.  Order 1 (head-major): the tile pairs of a head are consecutive, heaviest and lightest
+// remaining in turn, and CTA c takes the item pairs c, c+G, ... -- the CTAs running at one time
+// share the K, V of a few heads, which then stay in L2.  The launcher chooses (pick_schedule).
 struct Item {
     int pair, bh, row0[2], nblk[2], n_max;
 };
-__device__ __forceinline__ Item make_item(int it, int BH, int n_pairs, int S, int causal) {
+__device__ __forceinline__ Item make_item(int it, int BH, int n_pairs, int S, int causal, int order) {
     Item w;
-    w.pair = n_pairs - 1 - it / BH;
-    w.bh = it % BH;
+    if (order == 0) {                          // block-major, heaviest (last) query tiles first
+        w.pair = n_pairs - 1 - it / BH;
+        w.bh = it % BH;
+    } else {                                   // head-major, heaviest / lightest remaining tile pair in turn
+        w.bh = it / n_pairs;
+        const int j = it % n_pairs;
+        w.pair = (j & 1) ? (j >> 1) : n_pairs - 1 - (j >> 1);
+    }
     const int n_kb = (S + BN - 1) / BN;
 #pragma unroll
     for (int t = 0; t < 2; ++t) {
@@ -78,8 +88,8 @@ __device__ __forceinline__ Item make_item(int it, int BH, int n_pairs, int S, in
     return w;
 }
 // k-th item of CTA c out of G: tiers of G items, odd tiers dealt backwards (snake), -1 past the end.
-__device__ __forceinline__ int item_index(int c, int k, int G, int n_items) {
-    const int it = k * G + ((k & 1) ? (G - 1 - c) : c);
+__device__ __forceinline__ int item_index(int c, int k, int G, int n_items, int order) {
+    const int it = order == 0 ? k * G + ((k & 1) ? (G - 1 - c) : c) : 2 * (c + G * (k >> 1)) + (k & 1);
     return it < n_items ? it : -1;
 }
 
@@ -87,7 +97,7 @@ template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
 fast_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                 const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO,
-                float* __restrict__ LSE, int S, int BH, int n_pairs, int causal, float c2, unsigned* status)
+                float* __restrict__ LSE, int S, int BH, int n_pairs, int causal, int order, float c2, unsigned* status)
 {
     using C = Cfg<D>;
     extern __shared__ uint8_t smem_raw[];
@@ -102,7 +112,7 @@ fast_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
 
     const int n_items = n_pairs * BH;
     const int G = static_cast<int>(gridDim.x), cta = static_cast<int>(blockIdx.x);
-    const int n_tiers = (n_items + G - 1) / G;
+    const int n_tiers = 2 * ((n_items + 2 * G - 1) / (2 * G));   // upper bound on items per CTA in either order
 
     if (tid == 0) {
         for (int i = 0; i < B_COUNT; ++i) {
@@ -127,9 +137,9 @@ fast_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         {
             int g = 0;                                       // key blocks loaded so far (all items)
             for (int k = 0; k < n_tiers; ++k) {
-                const int it = item_index(cta, k, G, n_items);
+                const int it = item_index(cta, k, G, n_items, order);
                 if (it < 0) break;
-                const Item w = make_item(it, BH, n_pairs, S, causal);
+                const Item w = make_item(it, BH, n_pairs, S, causal, order);
                 mbar_wait(bar(B_QEMPTY), (k & 1) ^ 1, status);   // both issuers are done with the previous Q tiles
                 const int nq = (w.nblk[1] > 0) ? 2 : 1;
                 mbar_arrive_expect_tx(bar(B_Q), nq * C::TILE_BYTES);
@@ -185,9 +195,9 @@ fast_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             int cp = 0;      // P_t blocks consumed so far: phase of P_FULL[t]
             int co = 0;      // items in which this tile was active: phase of O_EMPTY[t]
             for (int k = 0; k < n_tiers; ++k) {
-                const int it = item_index(cta, k, G, n_items);
+                const int it = item_index(cta, k, G, n_items, order);
                 if (it < 0) break;
-                const Item w = make_item(it, BH, n_pairs, S, causal);
+                const Item w = make_item(it, BH, n_pairs, S, causal, order);
                 const int nb = w.nblk[t];
                 mbar_wait(bar(B_Q), k & 1, status);
                 mbar_wait(bar(B_KFULL + (g & 1)), (g >> 1) & 1, status);
@@ -247,9 +257,9 @@ fast_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         };
 
         for (int k = 0; k < n_tiers; ++k) {
-        const int it = item_index(cta, k, G, n_items);
+        const int it = item_index(cta, k, G, n_items, order);
         if (it < 0) break;
-        const Item w = make_item(it, BH, n_pairs, S, causal);
+        const Item w = make_item(it, BH, n_pairs, S, causal, order);
         const int bh = w.bh, n_max = w.n_max;
         const int row0[2] = {w.row0[0], w.row0[1]}, nblk[2] = {w.nblk[0], w.nblk[1]};
         float m_ref[2] = {-INFINITY, -INFINITY}, l[2] = {0.f, 0.f};
@@ -442,7 +452,9 @@ cudaError_t launch(const Problem& p, const void* q, const void* k, const void* v
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
         return cudaErrorInvalidValue;
     const long long blocks = items < sms ? items : sms;       // persistent: one CTA per SM
-    kern<<<static_cast<unsigned>(blocks), kThreads, C::SMEM, st>>>(tq, tk, tv, to, lse, p.S, p.BH, n_pairs, p.causal,
+    // streamed per block and shared between the query tiles of a head: K, V
+    const int order = pick_schedule(items, sms, static_cast<double>(p.BH) * p.S * D * (2 + 2), dev);
+    kern<<<static_cast<unsigned>(blocks), kThreads, C::SMEM, st>>>(tq, tk, tv, to, lse, p.S, p.BH, n_pairs, p.causal, order,
                                                                    p.scale * kLog2e, status);
     return cudaGetLastError();
 }

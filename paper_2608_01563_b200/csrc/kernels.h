@@ -28,6 +28,21 @@ cudaError_t launch_strict_bwd(const Problem& p, const float* q, const float* k, 
 cudaError_t launch_bwd_preprocess(const void* o, const void* d_o, float* delta, float* zero,
                                   size_t rows, int D, int is_bf16, cudaStream_t st);
 
+// Work-item order of the persistent fast kernels (see the kernels for the two orders).  Head-major
+// order (1) is chosen when the data that the items of one head share (`shared_bytes`, over all
+// heads) would not stay in L2 under block-major order, and there are enough item pairs per CTA
+// for its static assignment to be balanced within 4 %.
+extern int g_forced_item_order;   // -1: choose per call (set by mgn_attn_fast_item_order)
+inline int pick_schedule(long long n_items, int sms, double shared_bytes, int device) {
+    if (g_forced_item_order >= 0) return g_forced_item_order;
+    int l2 = 0;
+    if (cudaDeviceGetAttribute(&l2, cudaDevAttrL2CacheSize, device) != cudaSuccess || l2 <= 0) return 0;
+    const double x = static_cast<double>(n_items) / (2.0 * sms);
+    if (x < 1.0) return 0;
+    const double tiers = static_cast<double>((n_items + 2LL * sms - 1) / (2LL * sms));
+    return (shared_bytes > 0.75 * l2 && tiers / x <= 1.04) ? 1 : 0;
+}
+
 // Fast (bf16 tcgen05) kernels.
 cudaError_t launch_fast_fwd(const Problem& p, const void* q, const void* k, const void* v,
                             void* o, float* lse, unsigned* status, cudaStream_t st);

@@ -32,9 +32,17 @@ def declared_symbols():
 def test_every_declared_symbol_is_exported(lib):
     syms = declared_symbols()
     assert {"mgn_attn_fwd", "mgn_attn_bwd", "mgn_attn_bwd_workspace_bytes", "mgn_attn_check",
-            "mgn_status_string", "mgn_version", "mgn_attn_profile_events", "mgn_attn_bwd_noalloc", "mgn_measure_fp32_ffma_tflops"} <= set(syms)
+            "mgn_status_string", "mgn_version", "mgn_attn_profile_events", "mgn_attn_bwd_noalloc", "mgn_measure_fp32_ffma_tflops",
+            "mgn_attn_fast_item_order"} <= set(syms)
     for s in syms:
         assert getattr(lib, s) is not None
+
+
+def test_item_order_hook_validates_its_argument(lib):
+    assert lib.mgn_attn_fast_item_order(2) == 1       # MGN_ERR_INVALID_ARG
+    assert lib.mgn_attn_fast_item_order(-2) == 1
+    for order in (0, 1, -1):
+        assert lib.mgn_attn_fast_item_order(order) == 0
 
 
 def test_version_and_status_strings(lib):

@@ -42,6 +42,29 @@ def test_forward_backward_edge_shapes(S, D, causal):
     hp.check_fast(hp.select(res, B, H), ref, label=f"S={S} D={D} causal={causal} ")
 
 
+@pytest.mark.parametrize("order", [0, 1])
+@pytest.mark.parametrize("B,H,S,D,causal", [
+    (1, 3, 300, 64, True),       # ragged tail, odd number of blocks, fewer items than CTAs
+    (2, 40, 700, 128, True),     # several items per CTA, odd number of key blocks and of tile pairs
+    (2, 40, 640, 128, False),    # non-causal: equal weights
+    (1, 150, 257, 64, True),     # one more item pair than CTAs can share evenly
+])
+def test_both_item_orders_match_the_oracle(order, B, H, S, D, causal):
+    """The two work-item orders of the persistent kernels (block-major and head-major) visit the
+    same items; both are forced here at sizes where the default would pick only one of them."""
+    scale = 1.0 / math.sqrt(D)
+    q, k, v, d_o = synth.random_inputs(77 + order, B, H, S, D, dtype=BF)
+    heads = sorted({0, (B * H) // 2, B * H - 1})
+    mgn.mgn_attn_fast_item_order(order)
+    try:
+        res = hp.run_cuda(q, k, v, d_o, causal, scale, MODE)
+    finally:
+        mgn.mgn_attn_fast_item_order(-1)
+    ref = hp.run_oracle(q, k, v, d_o, causal, scale, heads)
+    hp.check_fast(hp.select(res, B, H, heads), ref, label=f"order={order} ")
+    hp.check_invariants(q, k, v, d_o, res, rtol=2e-2)
+
+
 def test_forward_large_max_growth_triggers_rescale():
     """Keys grow along the sequence so the running maximum moves by far more than the lazy threshold."""
     B, H, S, D = 1, 2, 1024, 128
