@@ -18,6 +18,7 @@ import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "attn_ref.c")
+_SRC_EXT = os.path.join(_HERE, "attn_ref_ext.c")      # separate query/key lengths, grouped K/V heads
 _LIB = os.path.join(_HERE, "libmgn_oracle.so")
 _lib = None
 
@@ -26,10 +27,11 @@ _dp = ctypes.POINTER(ctypes.c_double)
 
 def build(force: bool = False) -> str:
     """Compile the oracle with gcc (-O2, OpenMP, no fast-math). Returns the .so path."""
-    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+    newest = max(os.path.getmtime(_SRC), os.path.getmtime(_SRC_EXT))
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < newest:
         tmp = _LIB + f".tmp{os.getpid()}"
         subprocess.check_call(
-            ["gcc", "-O2", "-std=c11", "-fopenmp", "-fPIC", "-shared", "-o", tmp, _SRC, "-lm"]
+            ["gcc", "-O2", "-std=c11", "-fopenmp", "-fPIC", "-shared", "-o", tmp, _SRC, _SRC_EXT, "-lm"]
         )
         os.replace(tmp, _LIB)
     return _LIB
@@ -48,6 +50,10 @@ def _load():
         lib.ref_attn_head_matrices.restype = None
         lib.ref_grads_from_ds.argtypes = [_dp] * 5 + [i, i, d]
         lib.ref_grads_from_ds.restype = None
+        lib.ref_attn_fwd_ext.argtypes = [_dp] * 5 + [i] * 7 + [d, i]
+        lib.ref_attn_fwd_ext.restype = i
+        lib.ref_attn_bwd_ext.argtypes = [_dp] * 9 + [i] * 7 + [d, i]
+        lib.ref_attn_bwd_ext.restype = i
         lib.ref_max_threads.argtypes = []
         lib.ref_max_threads.restype = i
         _lib = lib
@@ -108,3 +114,41 @@ def grads_from_ds(dS, q, k, scale: float):
     dq = np.empty_like(q); dk = np.empty_like(q)
     _load().ref_grads_from_ds(_p(dS), _p(q), _p(k), _p(dq), _p(dk), S, D, float(scale))
     return dq, dk
+
+
+def _ext_dims(q, k):
+    B, H, Sq, D = q.shape
+    Bk, Hkv, Sk, Dk = k.shape
+    assert Bk == B and Dk == D and H % Hkv == 0
+    return B, H, Hkv, Sq, Sk, D
+
+
+def attn_fwd_ext(q, k, v, causal: bool, scale: float, nthreads: int = 0):
+    """Separate query/key lengths and grouped key/value heads: q [B,H,Sq,D], k, v [B,Hkv,Sk,D].
+    Causal masks are aligned bottom-right (key j visible to query i iff j <= i + Sk - Sq).
+    Returns (O [B,H,Sq,D], LSE [B,H,Sq]) in float64."""
+    q, k, v = _c(q), _c(k), _c(v)
+    B, H, Hkv, Sq, Sk, D = _ext_dims(q, k)
+    assert v.shape == k.shape
+    o = np.empty_like(q)
+    lse = np.empty((B, H, Sq), dtype=np.float64)
+    rc = _load().ref_attn_fwd_ext(_p(q), _p(k), _p(v), _p(o), _p(lse), B, H, Hkv, Sq, Sk, D,
+                                  int(bool(causal)), float(scale), int(nthreads))
+    if rc != 0:
+        raise ValueError("shapes outside the definition (H % Hkv != 0, or causal with Sq > Sk)")
+    return o, lse
+
+
+def attn_bwd_ext(q, k, v, d_o, causal: bool, scale: float, nthreads: int = 0):
+    """Returns (O, LSE, dQ [B,H,Sq,D], dK, dV [B,Hkv,Sk,D]) in float64; O and LSE are recomputed here."""
+    q, k, v, d_o = _c(q), _c(k), _c(v), _c(d_o)
+    B, H, Hkv, Sq, Sk, D = _ext_dims(q, k)
+    assert v.shape == k.shape and d_o.shape == q.shape
+    o = np.empty_like(q)
+    lse = np.empty((B, H, Sq), dtype=np.float64)
+    dq, dk, dv = np.empty_like(q), np.empty_like(k), np.empty_like(k)
+    rc = _load().ref_attn_bwd_ext(_p(q), _p(k), _p(v), _p(d_o), _p(o), _p(lse), _p(dq), _p(dk), _p(dv),
+                                  B, H, Hkv, Sq, Sk, D, int(bool(causal)), float(scale), int(nthreads))
+    if rc != 0:
+        raise ValueError("shapes outside the definition (H % Hkv != 0, or causal with Sq > Sk)")
+    return o, lse, dq, dk, dv
