@@ -151,6 +151,35 @@ def quick_measure(mgn, w, mode, dtype, steps, warmup):
     return fwd_ms, bwd_ms
 
 
+def quick_measure_ext(mgn, w, mode, dtype, steps, warmup):
+    """Device-resident timing of one cross-attention / grouped-head workload (CUDA events)."""
+    q, k, v, d_o = (t.cuda() for t in synth.make_inputs_ext(w, dtype=dtype))
+    o = torch.empty_like(q)
+    lse = torch.empty(w.B, w.H, w.Sq, device="cuda", dtype=torch.float32)
+    dq, dk, dv = torch.empty_like(q), torch.empty_like(k), torch.empty_like(v)
+    ws = mgn.alloc_workspace(w.B, w.H, w.Sq, w.D, mode)
+    for _ in range(warmup):
+        mgn.mgn_attn_fwd_ext(q, k, v, o, lse, w.causal, w.scale, mode)
+        mgn.mgn_attn_bwd_ext(q, k, v, o, d_o, lse, dq, dk, dv, ws, w.causal, w.scale, mode)
+    torch.cuda.synchronize()
+    e = [torch.cuda.Event(enable_timing=True) for _ in range(2 * steps + 1)]
+    e[0].record()
+    for i in range(steps):
+        mgn.mgn_attn_fwd_ext(q, k, v, o, lse, w.causal, w.scale, mode)
+        e[2 * i + 1].record()
+        mgn.mgn_attn_bwd_ext(q, k, v, o, d_o, lse, dq, dk, dv, ws, w.causal, w.scale, mode)
+        e[2 * i + 2].record()
+    torch.cuda.synchronize()
+    mgn.mgn_attn_check()
+    fwd_ms = statistics.mean(e[2 * i].elapsed_time(e[2 * i + 1]) for i in range(steps))
+    bwd_ms = statistics.mean(e[2 * i + 1].elapsed_time(e[2 * i + 2]) for i in range(steps))
+    unit = w.B * w.H * w.pairs * w.D
+    return {"B": w.B, "H": w.H, "H_kv": w.Hkv, "S_q": w.Sq, "S_k": w.Sk, "D": w.D, "causal": w.causal,
+            "fwd_ms": fwd_ms, "bwd_ms": bwd_ms, "fwd_tflops": 4.0 * unit / (fwd_ms * 1e-3) / 1e12,
+            "bwd_tflops": 10.0 * unit / (bwd_ms * 1e-3) / 1e12,
+            "sum_tflops": 14.0 * unit / ((fwd_ms + bwd_ms) * 1e-3) / 1e12}
+
+
 def cpu_info():
     model = "unknown"
     try:
@@ -462,6 +491,15 @@ def main():
                 "peak_tflops": peaks["bf16_tflops"], "peak_note": f"{peak_src} dense bf16 burst",
                 "frac_of_peak": flops(wf, "sum") / ((f_ms + b_ms) * 1e-3) / 1e12 / peaks["bf16_tflops"],
             }
+        if world == 1 and args.workload is None and not args.no_fast:
+            # cross-attention and grouped key/value heads (mgn_attn_*_ext), in this run's arithmetic mode
+            mode_peak = peak if args.mode == "strict" else peaks["bf16_tflops"]
+            ext = {}
+            for name in ("gqa_decoder", "gqa_suffix", "cross_attn_text", "cross_attn_action"):
+                r = quick_measure_ext(mgn, synth.EXT_WORKLOADS[name], mode, dtype, K, args.warmup)
+                r["frac_of_peak"] = r["sum_tflops"] / mode_peak
+                ext[name] = r
+            line["ext_shapes"] = ext
         if world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline(w, dtype)
         print(json.dumps(line))

@@ -81,6 +81,31 @@ int mgn_attn_bwd(const void* q, const void* k, const void* v, const void* o, con
 size_t mgn_attn_bwd_workspace_bytes(int B, int H, int S, int D, int mode);
 
 /*
+ * Cross-attention and grouped key/value heads.  The paper's matched workloads (Section 4.1,
+ * workload table) contain attention between sequences of different length (50 action tokens over
+ * 16 context tokens; 77-token text cross-attention); it prints no formula for them, so these entry
+ * points compute the textbook generalisation of the two above:
+ *   q, o, d_o, dq : [B, H, S_q, D]      k, v, dk, dv : [B, H_kv, S_k, D]      lse : [B, H, S_q]
+ *   H must be a multiple of H_kv; query head h reads key/value head h / (H / H_kv), and dk, dv of
+ *   a key/value head sum the contributions of all its query heads;
+ *   causal != 0 keeps key j for query i iff j <= i + (S_k - S_q): the mask is aligned to the
+ *   bottom-right corner (the last query sees every key) and needs S_q <= S_k, else the call
+ *   returns MGN_ERR_UNSUPPORTED (a query row without a visible key has no softmax).
+ * Everything else -- element types per mode, alignment, ownership, stream semantics, error
+ * order, dq accumulated with floating-point atomics -- is as for mgn_attn_fwd / mgn_attn_bwd,
+ * which are these functions with H_kv = H and S_q = S_k = S.  H % H_kv != 0 is MGN_ERR_INVALID_ARG.
+ * The workspace of mgn_attn_bwd_ext is mgn_attn_bwd_workspace_bytes(B, H, S_q, D, mode) bytes.
+ */
+int mgn_attn_fwd_ext(const void* q, const void* k, const void* v, void* o, float* lse,
+                     int B, int H, int H_kv, int S_q, int S_k, int D, int causal, float scale, int mode,
+                     void* stream);
+int mgn_attn_bwd_ext(const void* q, const void* k, const void* v, const void* o, const void* d_o,
+                     const float* lse, void* dq, void* dk, void* dv,
+                     void* workspace, size_t workspace_bytes,
+                     int B, int H, int H_kv, int S_q, int S_k, int D, int causal, float scale, int mode,
+                     void* stream);
+
+/*
  * Synchronises `stream`, then reads and clears the device-side status word that
  * kernels set when one of their bounded waits (TMA / tensor-core completion
  * barriers) ran out.  Returns MGN_OK, MGN_ERR_DEVICE_TIMEOUT or MGN_ERR_CUDA.

@@ -45,6 +45,10 @@ def lib() -> ctypes.CDLL:
         L.mgn_attn_fwd.restype = i
         L.mgn_attn_bwd.argtypes = [vp] * 9 + [vp, sz, i, i, i, i, i, f, i, vp]
         L.mgn_attn_bwd.restype = i
+        L.mgn_attn_fwd_ext.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, i, i, i, f, i, vp]
+        L.mgn_attn_fwd_ext.restype = i
+        L.mgn_attn_bwd_ext.argtypes = [vp] * 9 + [vp, sz, i, i, i, i, i, i, i, f, i, vp]
+        L.mgn_attn_bwd_ext.restype = i
         L.mgn_attn_bwd_workspace_bytes.argtypes = [i, i, i, i, i]
         L.mgn_attn_bwd_workspace_bytes.restype = sz
         L.mgn_attn_check.argtypes = [vp]
@@ -102,6 +106,31 @@ def mgn_attn_bwd(q, k, v, o, d_o, lse, dq, dk, dv, workspace, causal: bool, scal
                             B, H, S, D, int(causal), float(scale), int(mode), _stream(stream))
     if st != MGN_OK:
         raise MgnError(st, "mgn_attn_bwd")
+
+
+def _ext_dims(q: torch.Tensor, k: torch.Tensor):
+    B, H, Sq, D = q.shape
+    _, Hkv, Sk, _ = k.shape
+    return int(B), int(H), int(Hkv), int(Sq), int(Sk), int(D)
+
+
+def mgn_attn_fwd_ext(q, k, v, o, lse, causal: bool, scale: float, mode: int, stream: Optional[int] = None) -> None:
+    """q, o: [B,H,Sq,D]; k, v: [B,Hkv,Sk,D] (cross-attention, grouped key/value heads)."""
+    B, H, Hkv, Sq, Sk, D = _ext_dims(q, k)
+    st = lib().mgn_attn_fwd_ext(_ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse), B, H, Hkv, Sq, Sk, D,
+                                int(causal), float(scale), int(mode), _stream(stream))
+    if st != MGN_OK:
+        raise MgnError(st, "mgn_attn_fwd_ext")
+
+
+def mgn_attn_bwd_ext(q, k, v, o, d_o, lse, dq, dk, dv, workspace, causal: bool, scale: float, mode: int,
+                     stream: Optional[int] = None) -> None:
+    B, H, Hkv, Sq, Sk, D = _ext_dims(q, k)
+    st = lib().mgn_attn_bwd_ext(_ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(d_o), _ptr(lse), _ptr(dq), _ptr(dk),
+                                _ptr(dv), _ptr(workspace), workspace.numel() * workspace.element_size(),
+                                B, H, Hkv, Sq, Sk, D, int(causal), float(scale), int(mode), _stream(stream))
+    if st != MGN_OK:
+        raise MgnError(st, "mgn_attn_bwd_ext")
 
 
 def mgn_attn_bwd_noalloc(q, k, v, o, d_o, lse, dq, dk, dv, causal: bool, scale: float, mode: int,

@@ -48,6 +48,16 @@ int check_common(int B, int H, int S, int D, int causal, float scale, int mode)
     return MGN_OK;
 }
 
+// Extended shapes: separate query/key lengths, grouped key/value heads.
+int check_ext(int B, int H, int Hkv, int Sq, int Sk, int D, int causal, float scale, int mode)
+{
+    if (Hkv <= 0 || Sq <= 0 || Sk <= 0) return MGN_ERR_INVALID_ARG;
+    if (int r = check_common(B, H, Sq > Sk ? Sq : Sk, D, causal, scale, mode)) return r;
+    if (H % Hkv != 0) return MGN_ERR_INVALID_ARG;
+    if (causal && Sq > Sk) return MGN_ERR_UNSUPPORTED;   // a query row would see no key
+    return MGN_OK;
+}
+
 // Per-device set-up: architecture check and the address of the status word.
 int device_setup(unsigned** status)
 {
@@ -87,15 +97,16 @@ size_t mgn_attn_bwd_workspace_bytes(int B, int H, int S, int D, int mode)
     return bytes;
 }
 
-int mgn_attn_fwd(const void* q, const void* k, const void* v, void* o, float* lse,
-                 int B, int H, int S, int D, int causal, float scale, int mode, void* stream)
+int mgn_attn_fwd_ext(const void* q, const void* k, const void* v, void* o, float* lse,
+                     int B, int H, int H_kv, int S_q, int S_k, int D, int causal, float scale, int mode,
+                     void* stream)
 {
     if (!q || !k || !v || !o || !lse) return MGN_ERR_INVALID_ARG;
-    if (int r = check_common(B, H, S, D, causal, scale, mode)) return r;
+    if (int r = check_ext(B, H, H_kv, S_q, S_k, D, causal, scale, mode)) return r;
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(lse)) return MGN_ERR_MISALIGNED;
     unsigned* status = nullptr;
     if (int r = device_setup(&status)) return r;
-    const mgn::Problem p{B * H, S, D, causal, scale};
+    const mgn::Problem p{B, H, H_kv, S_q, S_k, D, causal, scale};
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     cudaError_t e;
     MainKernelTimer timer(st);
@@ -107,25 +118,32 @@ int mgn_attn_fwd(const void* q, const void* k, const void* v, void* o, float* ls
     return e == cudaSuccess ? MGN_OK : MGN_ERR_CUDA;
 }
 
-int mgn_attn_bwd(const void* q, const void* k, const void* v, const void* o, const void* d_o,
-                 const float* lse, void* dq, void* dk, void* dv,
-                 void* workspace, size_t workspace_bytes,
+int mgn_attn_fwd(const void* q, const void* k, const void* v, void* o, float* lse,
                  int B, int H, int S, int D, int causal, float scale, int mode, void* stream)
 {
+    return mgn_attn_fwd_ext(q, k, v, o, lse, B, H, H, S, S, D, causal, scale, mode, stream);
+}
+
+int mgn_attn_bwd_ext(const void* q, const void* k, const void* v, const void* o, const void* d_o,
+                     const float* lse, void* dq, void* dk, void* dv,
+                     void* workspace, size_t workspace_bytes,
+                     int B, int H, int H_kv, int S_q, int S_k, int D, int causal, float scale, int mode,
+                     void* stream)
+{
     if (!q || !k || !v || !o || !d_o || !lse || !dq || !dk || !dv) return MGN_ERR_INVALID_ARG;
-    if (int r = check_common(B, H, S, D, causal, scale, mode)) return r;
+    if (int r = check_ext(B, H, H_kv, S_q, S_k, D, causal, scale, mode)) return r;
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(d_o) || !aligned16(lse) ||
         !aligned16(dq) || !aligned16(dk) || !aligned16(dv))
         return MGN_ERR_MISALIGNED;
-    const size_t need = mgn_attn_bwd_workspace_bytes(B, H, S, D, mode);
+    const size_t need = mgn_attn_bwd_workspace_bytes(B, H, S_q, D, mode);
     if (!workspace || workspace_bytes < need) return MGN_ERR_WORKSPACE;
     if (reinterpret_cast<uintptr_t>(workspace) & 255u) return MGN_ERR_WORKSPACE;
     unsigned* status = nullptr;
     if (int r = device_setup(&status)) return r;
 
-    const mgn::Problem p{B * H, S, D, causal, scale};
+    const mgn::Problem p{B, H, H_kv, S_q, S_k, D, causal, scale};
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const size_t rows = static_cast<size_t>(B) * H * S;
+    const size_t rows = static_cast<size_t>(B) * H * S_q;
     float* delta = static_cast<float*>(workspace);
     const bool fast = mode == MGN_MODE_FAST_BF16;
 
@@ -144,6 +162,15 @@ int mgn_attn_bwd(const void* q, const void* k, const void* v, const void* o, con
     else
         e = mgn::launch_fast_bwd(p, q, k, v, d_o, lse, delta, dq_acc, dq, dk, dv, status, st);
     return e == cudaSuccess ? MGN_OK : MGN_ERR_CUDA;
+}
+
+int mgn_attn_bwd(const void* q, const void* k, const void* v, const void* o, const void* d_o,
+                 const float* lse, void* dq, void* dk, void* dv,
+                 void* workspace, size_t workspace_bytes,
+                 int B, int H, int S, int D, int causal, float scale, int mode, void* stream)
+{
+    return mgn_attn_bwd_ext(q, k, v, o, d_o, lse, dq, dk, dv, workspace, workspace_bytes, B, H, H, S, S, D, causal,
+                            scale, mode, stream);
 }
 
 int mgn_attn_check(void* stream)

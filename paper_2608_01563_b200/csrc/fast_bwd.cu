@@ -78,23 +78,40 @@ enum { B_KV = 0, B_QFULL = 1, B_QEMPTY = 3, B_DOFULL = 5, B_DOEMPTY = 6, B_SFULL
 //     remaining block, so that two consecutive items always weigh the same; CTA c takes the item
 //     pairs c, c+G, c+2G, ...  The CTAs running at one time share a few heads, whose dQ accumulator,
 //     Q and dO stay in L2.  Balanced only when there are many item pairs per CTA.
-struct Item {
-    int kb, bh, j0, qb0, N;
+// Shapes: q, d_o, dq [BH = B*H, Sq, D]; k, v, dk, dv [BHkv = B*H/G, Sk, D]; query head h reads
+// key/value head h / G; causal: key j is visible to query i iff j <= i + off, off = Sk - Sq >= 0.
+struct Dims {
+    int Sq, Sk, BH, H, G, off;
 };
-__device__ __forceinline__ Item make_item(int it, int BH, int S, int causal, int order) {
-    Item w;
-    const int nb = (S + BLK - 1) / BLK;
+// An item is one key block of one key/value head; its pairs run over the query heads of the group
+// and, for each, over the query blocks that see the key block.
+// GEN = false is the square multi-head case (Sk == Sq, G == 1): the head mapping, the offset and the
+// divisions by the number of query blocks fold away.
+template <bool GEN>
+struct Item {
+    int kb, bhk, bhq0, j0, qb0, nq, N;
+    __device__ __forceinline__ int bh(int n) const { return GEN ? bhq0 + n / nq : bhq0; }          // query head of pair n
+    __device__ __forceinline__ int i0(int n) const { return (qb0 + (GEN ? n % nq : n)) * BLK; }   // first query row of pair n
+};
+template <bool GEN>
+__device__ __forceinline__ Item<GEN> make_item(int it, const Dims& dm, int causal, int order) {
+    Item<GEN> w;
+    const int Sk = GEN ? dm.Sk : dm.Sq, G = GEN ? dm.G : 1, off = GEN ? dm.off : 0;
+    const int nb = (Sk + BLK - 1) / BLK, nqb = (dm.Sq + BLK - 1) / BLK;
+    const int Hkv = dm.H / G, BHkv = dm.BH / G;
     if (order == 0) {
-        w.kb = it / BH;
-        w.bh = it % BH;
+        w.kb = it / BHkv;
+        w.bhk = it % BHkv;
     } else {
-        w.bh = it / nb;
+        w.bhk = it / nb;
         const int j = it % nb;
         w.kb = (j & 1) ? nb - 1 - (j >> 1) : (j >> 1);
     }
+    w.bhq0 = GEN ? (w.bhk / Hkv) * dm.H + (w.bhk % Hkv) * G : w.bhk;
     w.j0 = w.kb * BLK;
-    w.qb0 = causal ? w.kb : 0;
-    w.N = nb - w.qb0;                          // query blocks visited (>= 1)
+    w.qb0 = causal ? max(w.j0 - off, 0) / BLK : 0;       // first query block with a row that sees key j0
+    w.nq = nqb - w.qb0;                                   // query blocks visited per head (>= 1)
+    w.N = G * w.nq;
     return w;
 }
 // k-th item of CTA c out of G, -1 past the end (then also for every larger k).
@@ -103,14 +120,14 @@ __device__ __forceinline__ int item_index(int c, int k, int G, int n_items, int 
     return it < n_items ? it : -1;
 }
 
-template <int D>
+template <int D, bool GEN>
 __global__ void __launch_bounds__(kThreads, 1)
 fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                 const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmdO,
                 const __grid_constant__ CUtensorMap tmdQ,
                 const float* __restrict__ LSE, const float* __restrict__ DELTA,
                 __nv_bfloat16* __restrict__ dK, __nv_bfloat16* __restrict__ dV,
-                int S, int BH, int causal, int order, float scale, unsigned* status)
+                const Dims dm, int causal, int order, float scale, unsigned* status)
 {
     using C = Cfg<D>;
     extern __shared__ uint8_t smem_raw[];
@@ -129,7 +146,8 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         return;
     }
 
-    const int n_items = ((S + BLK - 1) / BLK) * BH;
+    const int Sq = dm.Sq, Sk = GEN ? dm.Sk : dm.Sq, coff = GEN ? dm.off : 0;
+    const int n_items = ((Sk + BLK - 1) / BLK) * (dm.BH / (GEN ? dm.G : 1));
     const int G = static_cast<int>(gridDim.x), cta = static_cast<int>(blockIdx.x);
     const int n_tiers = 2 * ((n_items + 2 * G - 1) / (2 * G));   // upper bound on items per CTA in either order
     const float c2 = scale * kLog2e;
@@ -161,27 +179,27 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             for (int k = 0; k < n_tiers; ++k) {
                 const int it = item_index(cta, k, G, n_items, order);
                 if (it < 0) break;
-                const Item w = make_item(it, BH, S, causal, order);
+                const Item<GEN> w = make_item<GEN>(it, dm, causal, order);
                 mbar_wait(bar(B_KVEMPTY), (k & 1) ^ 1, status);  // both issuers are done with the previous K, V
                 mbar_arrive_expect_tx(bar(B_KV), 2 * C::TILE_BYTES);
 #pragma unroll
                 for (int ch = 0; ch < C::NCH; ++ch) {
-                    tma_load_3d(sK + ch * C::CHUNK_BYTES, &tmK, bar(B_KV), ch * 64, w.j0, w.bh);
-                    tma_load_3d(sV + ch * C::CHUNK_BYTES, &tmV, bar(B_KV), ch * 64, w.j0, w.bh);
+                    tma_load_3d(sK + ch * C::CHUNK_BYTES, &tmK, bar(B_KV), ch * 64, w.j0, w.bhk);
+                    tma_load_3d(sV + ch * C::CHUNK_BYTES, &tmV, bar(B_KV), ch * 64, w.j0, w.bhk);
                 }
                 for (int n = 0; n < w.N; ++n, ++g) {
                     const int st = g & 1;
-                    const int i0 = (w.qb0 + n) * BLK;
+                    const int i0 = w.i0(n), bh = w.bh(n);
                     mbar_wait(bar(B_QEMPTY + st), ((g >> 1) & 1) ^ 1, status);
                     mbar_arrive_expect_tx(bar(B_QFULL + st), C::TILE_BYTES);
 #pragma unroll
                     for (int ch = 0; ch < C::NCH; ++ch)
-                        tma_load_3d(sQ + st * C::TILE_BYTES + ch * C::CHUNK_BYTES, &tmQ, bar(B_QFULL + st), ch * 64, i0, w.bh);
+                        tma_load_3d(sQ + st * C::TILE_BYTES + ch * C::CHUNK_BYTES, &tmQ, bar(B_QFULL + st), ch * 64, i0, bh);
                     mbar_wait(bar(B_DOEMPTY), (g & 1) ^ 1, status);
                     mbar_arrive_expect_tx(bar(B_DOFULL), C::TILE_BYTES);
 #pragma unroll
                     for (int ch = 0; ch < C::NCH; ++ch)
-                        tma_load_3d(sdO + ch * C::CHUNK_BYTES, &tmdO, bar(B_DOFULL), ch * 64, i0, w.bh);
+                        tma_load_3d(sdO + ch * C::CHUNK_BYTES, &tmdO, bar(B_DOFULL), ch * 64, i0, bh);
                 }
             }
         }
@@ -210,7 +228,7 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                 for (int k = 0; k < n_tiers; ++k) {
                     const int it = item_index(cta, k, G, n_items, order);
                     if (it < 0) break;
-                    const Item w = make_item(it, BH, S, causal, order);
+                    const Item<GEN> w = make_item<GEN>(it, dm, causal, order);
                     mbar_wait(bar(B_KV), k & 1, status);
                     mbar_wait(bar(B_QFULL + (g & 1)), (g >> 1) & 1, status);
                     tc_fence_after();
@@ -253,7 +271,7 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                 for (int k = 0; k < n_tiers; ++k) {
                     const int it = item_index(cta, k, G, n_items, order);
                     if (it < 0) break;
-                    const Item w = make_item(it, BH, S, causal, order);
+                    const Item<GEN> w = make_item<GEN>(it, dm, causal, order);
                     mbar_wait(bar(B_KV), k & 1, status);
                     mbar_wait(bar(B_DOFULL), g & 1, status);
                     if (g > 0) mbar_wait(bar(B_DQEMPTY), (g - 1) & 1, status);   // Y: last item's final dQ partial drained
@@ -293,17 +311,18 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             for (int k = 0; k < n_tiers; ++k) {
                 const int it = item_index(cta, k, G, n_items, order);
                 if (it < 0) break;
-                const Item w = make_item(it, BH, S, causal, order);
+                const Item<GEN> w = make_item<GEN>(it, dm, causal, order);
                 for (int n = 0; n < w.N; ++n, ++g) {
                     if (g >= 2) mbar_wait(pds_bar(g), ((g - 2) >> 1) & 1, status);
                     const uint32_t buf = sStat + (g & 1) * (2 * BLK * 4);
-                    const int i = (w.qb0 + n) * BLK + 4 * lane;        // rows i..i+3 of the head
+                    const int i = w.i0(n) + 4 * lane;                  // rows i..i+3 of the query head
+                    const size_t row0 = static_cast<size_t>(w.bh(n)) * Sq;
                     float l2[4], dl[4];
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
-                        const bool ok = i + e < S;
-                        l2[e] = ok ? LSE[static_cast<size_t>(w.bh) * S + i + e] * kLog2e : INFINITY;
-                        dl[e] = ok ? DELTA[static_cast<size_t>(w.bh) * S + i + e] : 0.f;
+                        const bool ok = i + e < Sq;
+                        l2[e] = ok ? LSE[row0 + i + e] * kLog2e : INFINITY;
+                        dl[e] = ok ? DELTA[row0 + i + e] : 0.f;
                     }
                     sts128(buf + lane * 16, __float_as_uint(l2[0]), __float_as_uint(l2[1]), __float_as_uint(l2[2]),
                            __float_as_uint(l2[3]));
@@ -324,9 +343,9 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         for (int k = 0; k < n_tiers; ++k) {
         const int it = item_index(cta, k, G, n_items, order);
         if (it < 0) break;
-        const Item w = make_item(it, BH, S, causal, order);
+        const Item<GEN> w = make_item<GEN>(it, dm, causal, order);
         for (int n = 0; n < w.N; ++n, ++g) {
-            const int i0 = (w.qb0 + n) * BLK;
+            const int i0 = w.i0(n), bh = w.bh(n);
             mbar_wait(bar(B_DQFULL), g & 1, status);
             tc_fence_after();
             uint32_t v[D / 32][32];
@@ -349,8 +368,8 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                 fence_proxy_async_smem();
                 named_bar_sync(4, 128);
                 if (r == 0) {
-                    tma_reduce_add_3d(&tmdQ, stage, 64 * round, i0, w.bh);
-                    tma_reduce_add_3d(&tmdQ, stage + C::CHUNK_BYTES, 64 * round + 32, i0, w.bh);
+                    tma_reduce_add_3d(&tmdQ, stage, 64 * round, i0, bh);
+                    tma_reduce_add_3d(&tmdQ, stage + C::CHUNK_BYTES, 64 * round + 32, i0, bh);
                     bulk_commit_group();
                 }
             }
@@ -368,8 +387,10 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         uint32_t pk[32];                                                     // P^T of the current pair, packed bf16
 
         // P^T = exp2(S^T c - lse) of pair n: bf16 into X (A operand of dV) and into pk (for dS)
-        auto exp_phase = [&](const Item& w, int n, int g) {
-            const bool diag = causal && ((w.qb0 + n) * BLK == w.j0);
+        auto exp_phase = [&](const Item<GEN>& w, int n, int g) {
+            // key lane r (key j0 + r) is visible to query column c (query i0 + c) iff r <= c + dlt
+            const int dlt = w.i0(n) + coff - w.j0;
+            const bool diag = causal && dlt < BLK - 1;
             const uint32_t statL = sStat + (g & 1) * (2 * BLK * 4);
             mbar_wait(bar(B_STATFULL + (g & 1)), (g >> 1) & 1, status);
             mbar_wait(bar(B_SFULL), g & 1, status);
@@ -391,7 +412,7 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                 if (diag) {   // keep key j <= query i, i.e. lane r <= column
 #pragma unroll
                     for (int e = 0; e < 32; ++e)
-                        if (r > half * 64 + 32 * c + e) p[e] = 0.f;
+                        if (r > half * 64 + 32 * c + e + dlt) p[e] = 0.f;
                 }
                 uint32_t u[16];
 #pragma unroll
@@ -410,7 +431,7 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         for (int k = 0; k < n_tiers; ++k) {
         const int it = item_index(cta, k, G, n_items, order);
         if (it < 0) break;
-        const Item w = make_item(it, BH, S, causal, order);
+        const Item<GEN> w = make_item<GEN>(it, dm, causal, order);
         exp_phase(w, 0, g);
 
         for (int n = 0; n < w.N; ++n, ++g) {
@@ -477,7 +498,7 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                 for (int q = 0; q < PCS; ++q)
                     sts128(stage + r * (HC * 2) + (swz(q, r) << 4), u[4 * q], u[4 * q + 1], u[4 * q + 2], u[4 * q + 3]);
                 named_bar_sync(2 + half, 128);
-                out += (static_cast<size_t>(w.bh) * S + w.j0) * D + half * HC;
+                out += (static_cast<size_t>(w.bhk) * Sk + w.j0) * D + half * HC;
                 float4 val[PCS];
 #pragma unroll
                 for (int i = 0; i < PCS; ++i) {
@@ -487,7 +508,7 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
 #pragma unroll
                 for (int i = 0; i < PCS; ++i) {
                     const int idx = i * 128 + r, row = idx / PCS, piece = idx % PCS;
-                    if (w.j0 + row < S) *reinterpret_cast<float4*>(out + static_cast<size_t>(row) * D + piece * 8) = val[i];
+                    if (w.j0 + row < Sk) *reinterpret_cast<float4*>(out + static_cast<size_t>(row) * D + piece * 8) = val[i];
                 }
                 named_bar_sync(2 + half, 128);             // the slab has been read: the buffer may be rewritten
             };
@@ -521,23 +542,23 @@ dq_convert_kernel(const float4* __restrict__ acc, uint2* __restrict__ out, size_
     }
 }
 
-template <int D>
-cudaError_t launch(const Problem& p, const void* q, const void* k, const void* v, const void* d_o,
-                   const float* lse, const float* delta, float* dq_acc, void* dq, void* dk, void* dv,
-                   unsigned* status, cudaStream_t st)
+template <int D, bool GEN>
+cudaError_t launch_gen(const Problem& p, const void* q, const void* k, const void* v, const void* d_o,
+                       const float* lse, const float* delta, float* dq_acc, void* dq, void* dk, void* dv,
+                       unsigned* status, cudaStream_t st)
 {
     using C = Cfg<D>;
     CUtensorMap tq, tk, tv, tdo, tdq;
-    if (make_tmap_3d(&tdq, dq_acc, 4, 0, p.BH, p.S, D, 32, BLK)) return cudaErrorInvalidValue;
-    if (make_tmap_3d(&tq, q, 2, 1, p.BH, p.S, D, 64, BLK)) return cudaErrorInvalidValue;
-    if (make_tmap_3d(&tk, k, 2, 1, p.BH, p.S, D, 64, BLK)) return cudaErrorInvalidValue;
-    if (make_tmap_3d(&tv, v, 2, 1, p.BH, p.S, D, 64, BLK)) return cudaErrorInvalidValue;
-    if (make_tmap_3d(&tdo, d_o, 2, 1, p.BH, p.S, D, 64, BLK)) return cudaErrorInvalidValue;
-    auto kern = fast_bwd_kernel<D>;
+    if (make_tmap_3d(&tdq, dq_acc, 4, 0, p.BH(), p.Sq, D, 32, BLK)) return cudaErrorInvalidValue;
+    if (make_tmap_3d(&tq, q, 2, 1, p.BH(), p.Sq, D, 64, BLK)) return cudaErrorInvalidValue;
+    if (make_tmap_3d(&tk, k, 2, 1, p.BHkv(), p.Sk, D, 64, BLK)) return cudaErrorInvalidValue;
+    if (make_tmap_3d(&tv, v, 2, 1, p.BHkv(), p.Sk, D, 64, BLK)) return cudaErrorInvalidValue;
+    if (make_tmap_3d(&tdo, d_o, 2, 1, p.BH(), p.Sq, D, 64, BLK)) return cudaErrorInvalidValue;
+    auto kern = fast_bwd_kernel<D, GEN>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM);
     if (e != cudaSuccess) return e;
-    const int n_kb = (p.S + BLK - 1) / BLK;
-    const long long items = static_cast<long long>(n_kb) * p.BH;
+    const int n_kb = (p.Sk + BLK - 1) / BLK;
+    const long long items = static_cast<long long>(n_kb) * p.BHkv();
     if (items > 0x7fffffffLL) return cudaErrorInvalidValue;
     int dev = 0, sms = 0;
     if (cudaGetDevice(&dev) != cudaSuccess ||
@@ -545,18 +566,29 @@ cudaError_t launch(const Problem& p, const void* q, const void* k, const void* v
         return cudaErrorInvalidValue;
     const long long blocks = items < sms ? items : sms;       // persistent: one CTA per SM
     // streamed per pair and shared between the key blocks of a head: dQ accumulator (f32), Q, dO
-    const int order = pick_schedule(items, sms, static_cast<double>(p.BH) * p.S * D * (4 + 2 + 2), dev);
+    const int order = pick_schedule(items, sms, static_cast<double>(p.BH()) * p.Sq * D * (4 + 2 + 2), dev);
+    const Dims dm{p.Sq, p.Sk, p.BH(), p.H, p.group(), p.off()};
     kern<<<static_cast<unsigned>(blocks), kThreads, C::SMEM, st>>>(tq, tk, tv, tdo, tdq, lse, delta,
                                                                    static_cast<__nv_bfloat16*>(dk),
-                                                                   static_cast<__nv_bfloat16*>(dv), p.S, p.BH, p.causal,
+                                                                   static_cast<__nv_bfloat16*>(dv), dm, p.causal,
                                                                    order, p.scale, status);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    const size_t n4 = static_cast<size_t>(p.BH) * p.S * D / 4;
+    const size_t n4 = static_cast<size_t>(p.BH()) * p.Sq * D / 4;
     const unsigned cblocks = static_cast<unsigned>(n4 / 256 + 1 < 148u * 16u ? n4 / 256 + 1 : 148u * 16u);
     dq_convert_kernel<<<cblocks, 256, 0, st>>>(reinterpret_cast<const float4*>(dq_acc), reinterpret_cast<uint2*>(dq), n4,
                                                p.scale);
     return cudaGetLastError();
+}
+
+template <int D>
+cudaError_t launch(const Problem& p, const void* q, const void* k, const void* v, const void* d_o,
+                   const float* lse, const float* delta, float* dq_acc, void* dq, void* dk, void* dv,
+                   unsigned* status, cudaStream_t st)
+{
+    return (p.Hkv != p.H || p.Sq != p.Sk)
+               ? launch_gen<D, true>(p, q, k, v, d_o, lse, delta, dq_acc, dq, dk, dv, status, st)
+               : launch_gen<D, false>(p, q, k, v, d_o, lse, delta, dq_acc, dq, dk, dv, status, st);
 }
 
 }  // namespace

@@ -64,10 +64,19 @@ enum { B_Q = 0, B_KFULL = 1, B_KEMPTY = 3, B_VFULL = 5, B_VEMPTY = 7, B_SFULL = 
 // every head.  Order 1 (head-major): the tile pairs of a head are consecutive, heaviest and lightest
 // remaining in turn, and CTA c takes the item pairs c, c+G, ... -- the CTAs running at one time
 // share the K, V of a few heads, which then stay in L2.  The launcher chooses (pick_schedule).
-struct Item {
-    int pair, bh, row0[2], nblk[2], n_max;
+// Shapes: q, o [BH = B*H, Sq, D]; k, v [B*H/G, Sk, D]; query head h reads key/value head h / G;
+// causal: key j is visible to query i iff j <= i + off, off = Sk - Sq >= 0.
+struct Dims {
+    int Sq, Sk, BH, H, G, off;
 };
-__device__ __forceinline__ Item make_item(int it, int BH, int n_pairs, int S, int causal, int order) {
+struct Item {
+    int pair, bh, bhk, row0[2], nblk[2], n_max;
+};
+// GEN = false is the square multi-head case (Sk == Sq, G == 1): offsets and the head mapping fold away.
+template <bool GEN>
+__device__ __forceinline__ Item make_item(int it, const Dims& dm, int n_pairs, int causal, int order) {
+    const int BH = dm.BH;
+    const int Sk = GEN ? dm.Sk : dm.Sq, off = GEN ? dm.off : 0;
     Item w;
     if (order == 0) {                          // block-major, heaviest (last) query tiles first
         w.pair = n_pairs - 1 - it / BH;
@@ -77,12 +86,13 @@ __device__ __forceinline__ Item make_item(int it, int BH, int n_pairs, int S, in
         const int j = it % n_pairs;
         w.pair = (j & 1) ? (j >> 1) : n_pairs - 1 - (j >> 1);
     }
-    const int n_kb = (S + BN - 1) / BN;
+    w.bhk = GEN ? (w.bh / dm.H) * (dm.H / dm.G) + (w.bh % dm.H) / dm.G : w.bh;
+    const int n_kb = (Sk + BN - 1) / BN;
 #pragma unroll
     for (int t = 0; t < 2; ++t) {
         w.row0[t] = w.pair * 2 * BM + t * BM;
-        if (w.row0[t] >= S) w.nblk[t] = 0;
-        else w.nblk[t] = causal ? min(n_kb, (min(w.row0[t] + BM, S) - 1) / BN + 1) : n_kb;
+        if (w.row0[t] >= dm.Sq) w.nblk[t] = 0;
+        else w.nblk[t] = causal ? min(n_kb, (min(w.row0[t] + BM, dm.Sq) - 1 + off) / BN + 1) : n_kb;
     }
     w.n_max = max(w.nblk[0], w.nblk[1]);
     return w;
@@ -93,11 +103,11 @@ __device__ __forceinline__ int item_index(int c, int k, int G, int n_items, int 
     return it < n_items ? it : -1;
 }
 
-template <int D>
+template <int D, bool GEN>
 __global__ void __launch_bounds__(kThreads, 1)
 fast_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                 const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO,
-                float* __restrict__ LSE, int S, int BH, int n_pairs, int causal, int order, float c2, unsigned* status)
+                float* __restrict__ LSE, const Dims dm, int n_pairs, int causal, int order, float c2, unsigned* status)
 {
     using C = Cfg<D>;
     extern __shared__ uint8_t smem_raw[];
@@ -110,7 +120,8 @@ fast_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (*reinterpret_cast<volatile unsigned*>(status) != 0) return;   // an earlier wait on this device gave up
 
-    const int n_items = n_pairs * BH;
+    const int n_items = n_pairs * dm.BH;
+    const int Sq = dm.Sq, Sk = GEN ? dm.Sk : dm.Sq, coff = GEN ? dm.off : 0;
     const int G = static_cast<int>(gridDim.x), cta = static_cast<int>(blockIdx.x);
     const int n_tiers = 2 * ((n_items + 2 * G - 1) / (2 * G));   // upper bound on items per CTA in either order
 
@@ -139,7 +150,7 @@ fast_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             for (int k = 0; k < n_tiers; ++k) {
                 const int it = item_index(cta, k, G, n_items, order);
                 if (it < 0) break;
-                const Item w = make_item(it, BH, n_pairs, S, causal, order);
+                const Item w = make_item<GEN>(it, dm, n_pairs, causal, order);
                 mbar_wait(bar(B_QEMPTY), (k & 1) ^ 1, status);   // both issuers are done with the previous Q tiles
                 const int nq = (w.nblk[1] > 0) ? 2 : 1;
                 mbar_arrive_expect_tx(bar(B_Q), nq * C::TILE_BYTES);
@@ -154,12 +165,12 @@ fast_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                     mbar_arrive_expect_tx(bar(B_KFULL + st), C::TILE_BYTES);
 #pragma unroll
                     for (int ch = 0; ch < C::NCH; ++ch)
-                        tma_load_3d(sK + st * C::TILE_BYTES + ch * C::CHUNK_BYTES, &tmK, bar(B_KFULL + st), ch * 64, n * BN, w.bh);
+                        tma_load_3d(sK + st * C::TILE_BYTES + ch * C::CHUNK_BYTES, &tmK, bar(B_KFULL + st), ch * 64, n * BN, w.bhk);
                     mbar_wait(bar(B_VEMPTY + st), ph ^ 1, status);
                     mbar_arrive_expect_tx(bar(B_VFULL + st), C::TILE_BYTES);
 #pragma unroll
                     for (int ch = 0; ch < C::NCH; ++ch)
-                        tma_load_3d(sV + st * C::TILE_BYTES + ch * C::CHUNK_BYTES, &tmV, bar(B_VFULL + st), ch * 64, n * BN, w.bh);
+                        tma_load_3d(sV + st * C::TILE_BYTES + ch * C::CHUNK_BYTES, &tmV, bar(B_VFULL + st), ch * 64, n * BN, w.bhk);
                 }
             }
         }
@@ -197,7 +208,7 @@ fast_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             for (int k = 0; k < n_tiers; ++k) {
                 const int it = item_index(cta, k, G, n_items, order);
                 if (it < 0) break;
-                const Item w = make_item(it, BH, n_pairs, S, causal, order);
+                const Item w = make_item<GEN>(it, dm, n_pairs, causal, order);
                 const int nb = w.nblk[t];
                 mbar_wait(bar(B_Q), k & 1, status);
                 mbar_wait(bar(B_KFULL + (g & 1)), (g >> 1) & 1, status);
@@ -259,7 +270,7 @@ fast_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         for (int k = 0; k < n_tiers; ++k) {
         const int it = item_index(cta, k, G, n_items, order);
         if (it < 0) break;
-        const Item w = make_item(it, BH, n_pairs, S, causal, order);
+        const Item w = make_item<GEN>(it, dm, n_pairs, causal, order);
         const int bh = w.bh, n_max = w.n_max;
         const int row0[2] = {w.row0[0], w.row0[1]}, nblk[2] = {w.nblk[0], w.nblk[1]};
         float m_ref[2] = {-INFINITY, -INFINITY}, l[2] = {0.f, 0.f};
@@ -274,8 +285,8 @@ fast_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                 mbar_wait(bar(B_SFULL + t), (cs[t] + n) & 1, status);
                 tc_fence_after();
                 const int j0 = n * BN + 64 * h;
-                const bool masked = (causal && (j0 + 63 > row0[t])) || (j0 + 64 > S);
-                const int jmax = min(S - 1, causal ? i : S - 1) - j0;   // columns c <= jmax of this half are visible
+                const bool masked = (causal && (j0 + 63 > row0[t] + coff)) || (j0 + 64 > Sk);
+                const int jmax = min(Sk - 1, causal ? i + coff : Sk - 1) - j0;   // columns c <= jmax of this half are visible
 
                 if (n == 0) {
                     // first block: the reference point is the row maximum of the scaled scores
@@ -409,7 +420,7 @@ fast_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                     sts128(rowaddr + ((piece ^ (r & 7)) << 4), u[4 * q], u[4 * q + 1], u[4 * q + 2], u[4 * q + 3]);
                 }
             }
-            if (h == 0 && i < S) LSE[static_cast<size_t>(bh) * S + i] = (m_ref[t] + log2f(lt)) * kLn2;
+            if (h == 0 && i < Sq) LSE[static_cast<size_t>(bh) * Sq + i] = (m_ref[t] + log2f(lt)) * kLn2;
             fence_proxy_async_smem();
             bar_or(false);
             if (r == 0 && h == 0) {
@@ -431,32 +442,41 @@ fast_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     if (warp == 0) tmem_dealloc(tmem, C::TM_COLS);
 }
 
-template <int D>
-cudaError_t launch(const Problem& p, const void* q, const void* k, const void* v, void* o, float* lse,
-                   unsigned* status, cudaStream_t st)
+template <int D, bool GEN>
+cudaError_t launch_gen(const Problem& p, const void* q, const void* k, const void* v, void* o, float* lse,
+                       unsigned* status, cudaStream_t st)
 {
     using C = Cfg<D>;
     CUtensorMap tq, tk, tv, to;
-    if (make_tmap_3d(&tq, q, 2, 1, p.BH, p.S, D, 64, 128)) return cudaErrorInvalidValue;
-    if (make_tmap_3d(&tk, k, 2, 1, p.BH, p.S, D, 64, 128)) return cudaErrorInvalidValue;
-    if (make_tmap_3d(&tv, v, 2, 1, p.BH, p.S, D, 64, 128)) return cudaErrorInvalidValue;
-    if (make_tmap_3d(&to, o, 2, 1, p.BH, p.S, D, 64, 128)) return cudaErrorInvalidValue;
-    auto kern = fast_fwd_kernel<D>;
+    if (make_tmap_3d(&tq, q, 2, 1, p.BH(), p.Sq, D, 64, 128)) return cudaErrorInvalidValue;
+    if (make_tmap_3d(&tk, k, 2, 1, p.BHkv(), p.Sk, D, 64, 128)) return cudaErrorInvalidValue;
+    if (make_tmap_3d(&tv, v, 2, 1, p.BHkv(), p.Sk, D, 64, 128)) return cudaErrorInvalidValue;
+    if (make_tmap_3d(&to, o, 2, 1, p.BH(), p.Sq, D, 64, 128)) return cudaErrorInvalidValue;
+    auto kern = fast_fwd_kernel<D, GEN>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM);
     if (e != cudaSuccess) return e;
-    const int n_pairs = (p.S + 2 * BM - 1) / (2 * BM);
-    const long long items = static_cast<long long>(n_pairs) * p.BH;
+    const int n_pairs = (p.Sq + 2 * BM - 1) / (2 * BM);
+    const long long items = static_cast<long long>(n_pairs) * p.BH();
     if (items > 0x7fffffffLL) return cudaErrorInvalidValue;
     int dev = 0, sms = 0;
     if (cudaGetDevice(&dev) != cudaSuccess ||
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
         return cudaErrorInvalidValue;
     const long long blocks = items < sms ? items : sms;       // persistent: one CTA per SM
+    const Dims dm{p.Sq, p.Sk, p.BH(), p.H, p.group(), p.off()};
     // streamed per block and shared between the query tiles of a head: K, V
-    const int order = pick_schedule(items, sms, static_cast<double>(p.BH) * p.S * D * (2 + 2), dev);
-    kern<<<static_cast<unsigned>(blocks), kThreads, C::SMEM, st>>>(tq, tk, tv, to, lse, p.S, p.BH, n_pairs, p.causal, order,
+    const int order = pick_schedule(items, sms, static_cast<double>(p.BHkv()) * p.Sk * D * (2 + 2), dev);
+    kern<<<static_cast<unsigned>(blocks), kThreads, C::SMEM, st>>>(tq, tk, tv, to, lse, dm, n_pairs, p.causal, order,
                                                                    p.scale * kLog2e, status);
     return cudaGetLastError();
+}
+
+template <int D>
+cudaError_t launch(const Problem& p, const void* q, const void* k, const void* v, void* o, float* lse,
+                   unsigned* status, cudaStream_t st)
+{
+    return (p.Hkv != p.H || p.Sq != p.Sk) ? launch_gen<D, true>(p, q, k, v, o, lse, status, st)
+                                          : launch_gen<D, false>(p, q, k, v, o, lse, status, st);
 }
 
 }  // namespace

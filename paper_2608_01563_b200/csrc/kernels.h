@@ -6,9 +6,16 @@
 
 namespace mgn {
 
+// q, o, d_o, dq: [B,H,Sq,D]; k, v, dk, dv: [B,Hkv,Sk,D]; query head h reads key/value head
+// h / (H/Hkv).  With a causal mask key j is visible to query i iff j <= i + (Sk - Sq)
+// (bottom-right aligned; the launchers are only given Sq <= Sk then).
 struct Problem {
-    int BH, S, D, causal;
+    int B, H, Hkv, Sq, Sk, D, causal;
     float scale;
+    int BH() const { return B * H; }
+    int BHkv() const { return B * Hkv; }
+    int group() const { return H / Hkv; }
+    int off() const { return Sk - Sq; }
 };
 
 // Tensor maps (host side).  rank-3 view (D, S, BH) of a dense [BH,S,D] tensor with

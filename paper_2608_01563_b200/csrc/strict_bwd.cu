@@ -11,7 +11,9 @@
 //   C. forms the partial dQ = dS K of this pair and adds it to global dQ with 128-bit
 //      floating-point reductions (the "atomic accumulation" variant of the dQ kernel),
 // so exactly the five counted matrix products are executed.  Tiles arrive by TMA in the
-// swizzled layout described in strict_fwd.cu.
+// swizzled layout described in strict_fwd.cu.  With grouped key/value heads the CTA walks over the
+// query tiles of every query head of its group in turn (dK, dV sum over the group in registers);
+// with separate query and key lengths the causal mask is aligned bottom-right.
 #include "kernels.h"
 #include "ptx.cuh"
 
@@ -58,14 +60,18 @@ __device__ __forceinline__ float f4_get(const float4& v, int u) {
     return u == 0 ? v.x : u == 1 ? v.y : u == 2 ? v.z : v.w;
 }
 
-template <int D, int BM, int BN, int THREADS>
+// GEN = false is the square multi-head case (Sk == Sq, one key/value head per query head): the
+// offset, the group loop and the second length fold away at compile time.
+template <int D, int BM, int BN, int THREADS, bool GEN>
 __global__ void __launch_bounds__(THREADS, THREADS == 128 ? 2 : 1)
 strict_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                   const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmdO,
                   const float* __restrict__ LSE, const float* __restrict__ DELTA,
                   float* __restrict__ dQ, float* __restrict__ dK, float* __restrict__ dV,
-                  int S, int BH, int n_qt, int causal, float scale, unsigned* status)
+                  int Sq, int Sk_, int BHkv, int H, int G_, int n_qt, int causal, float scale, unsigned* status)
 {
+    const int Sk = GEN ? Sk_ : Sq;
+    const int G = GEN ? G_ : 1;
     using C = BwdCfg<D, BM, BN, THREADS>;
     constexpr int RM = C::RM, RN = C::RN, JN = C::JN, DV = C::DV, NCH = C::NCH, PSTR = C::PSTR, TR = C::TR;
 
@@ -84,10 +90,15 @@ strict_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     const int tc = tid & 15;                             // 0..15
 
     // Heaviest key tiles (lowest j0) first when causal.
-    const int kt = static_cast<int>(blockIdx.x) / BH;
-    const int bh = static_cast<int>(blockIdx.x) % BH;
+    const int kt = static_cast<int>(blockIdx.x) / BHkv;
+    const int bhk = static_cast<int>(blockIdx.x) % BHkv;          // (batch, key/value head)
+    const int Hkv = H / G;
+    const int bhq0 = GEN ? (bhk / Hkv) * H + (bhk % Hkv) * G : bhk;   // first query head of the group
+    const int coff = GEN ? Sk - Sq : 0;                           // causal: key j visible to query i iff j <= i + coff
     const int j0 = kt * BN;
-    const int qt0 = causal ? (j0 / BM) : 0;
+    const int qt0 = causal ? (max(j0 - coff, 0) / BM) : 0;         // first query tile that sees this key tile
+    const int nq = n_qt - qt0;                                    // query tiles per head (>= 1)
+    const int steps = G * nq;                                     // (query head of the group, query tile) pairs
     const float c2 = scale * kLog2e;
 
     if (tid == 0) {
@@ -100,14 +111,14 @@ strict_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         mbar_arrive_expect_tx(barKV, 2 * C::KV_BYTES);
 #pragma unroll
         for (int ch = 0; ch < NCH; ++ch) {
-            tma_load_3d(sK + ch * BN * 128, &tmK, barKV, ch * 32, j0, bh);
-            tma_load_3d(sV + ch * BN * 128, &tmV, barKV, ch * 32, j0, bh);
+            tma_load_3d(sK + ch * BN * 128, &tmK, barKV, ch * 32, j0, bhk);
+            tma_load_3d(sV + ch * BN * 128, &tmV, barKV, ch * 32, j0, bhk);
         }
         mbar_arrive_expect_tx(barQ, 2 * C::Q_BYTES);
 #pragma unroll
         for (int ch = 0; ch < NCH; ++ch) {
-            tma_load_3d(sQ + ch * BM * 128, &tmQ, barQ, ch * 32, qt0 * BM, bh);
-            tma_load_3d(sdO + ch * BM * 128, &tmdO, barQ, ch * 32, qt0 * BM, bh);
+            tma_load_3d(sQ + ch * BM * 128, &tmQ, barQ, ch * 32, qt0 * BM, bhq0);
+            tma_load_3d(sdO + ch * BM * 128, &tmdO, barQ, ch * 32, qt0 * BM, bhq0);
         }
     }
 
@@ -119,18 +130,21 @@ strict_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
 
     mbar_wait(barKV, 0, status);
 
-    for (int qt = qt0; qt < n_qt; ++qt) {
-        const int i0 = qt * BM;
-        const uint32_t ph = (qt - qt0) & 1;
+    // Step counter: the general case counts (head, tile) pairs from 0; the square case counts
+    // query tiles from qt0 as the loop always did (the two forms compile to different schedules).
+    for (int t = GEN ? 0 : qt0; t < (GEN ? steps : n_qt); ++t) {
+        const int bh = GEN ? bhq0 + t / nq : bhq0;    // query head
+        const int i0 = (GEN ? qt0 + t % nq : t) * BM;
+        const uint32_t ph = (GEN ? t : t - qt0) & 1;
 
         // row statistics of this thread's query rows (rows past S: P = 0 via lse = +inf)
         float lse2[RM], dl[RM];
 #pragma unroll
         for (int x = 0; x < RM; ++x) {
             const int i = i0 + tr + TR * x;
-            const bool ok = i < S;
-            lse2[x] = ok ? LSE[static_cast<size_t>(bh) * S + i] * kLog2e : INFINITY;
-            dl[x] = ok ? DELTA[static_cast<size_t>(bh) * S + i] : 0.f;
+            const bool ok = i < Sq;
+            lse2[x] = ok ? LSE[static_cast<size_t>(bh) * Sq + i] * kLog2e : INFINITY;
+            dl[x] = ok ? DELTA[static_cast<size_t>(bh) * Sq + i] : 0.f;
         }
 
         mbar_wait(barQ, ph, status);
@@ -173,7 +187,7 @@ strict_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         }
         __syncthreads();   // phase C of the previous pair has finished reading dS
         {
-            const bool need_mask = (causal && (j0 + BN - 1 > i0)) || (j0 + BN > S);
+            const bool need_mask = (causal && (j0 + BN - 1 > i0 + coff)) || (j0 + BN > Sk);
 #pragma unroll
             for (int x = 0; x < RM; ++x) {
                 const int i = i0 + tr + TR * x;
@@ -183,7 +197,7 @@ strict_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                     float p = ex2(fmaf(s[x][y], c2, -lse2[x]));
                     if (need_mask) {
                         const int j = j0 + tc + 16 * y;
-                        if (j >= S || (causal && j > i)) p = 0.f;
+                        if (j >= Sk || (causal && j > i + coff)) p = 0.f;
                     }
                     const float ds = p * (dp[x][y] - dl[x]);
                     sts32(sP + row + y * 64, p);
@@ -221,12 +235,13 @@ strict_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             }
         }
         __syncthreads();   // Q and dO tiles are free
-        if (tid == 0 && qt + 1 < n_qt) {
+        if (tid == 0 && t + 1 < (GEN ? steps : n_qt)) {
+            const int bh1 = GEN ? bhq0 + (t + 1) / nq : bhq0, i1 = (GEN ? qt0 + (t + 1) % nq : t + 1) * BM;
             mbar_arrive_expect_tx(barQ, 2 * C::Q_BYTES);
 #pragma unroll
             for (int ch = 0; ch < NCH; ++ch) {
-                tma_load_3d(sQ + ch * BM * 128, &tmQ, barQ, ch * 32, i0 + BM, bh);
-                tma_load_3d(sdO + ch * BM * 128, &tmdO, barQ, ch * 32, i0 + BM, bh);
+                tma_load_3d(sQ + ch * BM * 128, &tmQ, barQ, ch * 32, i1, bh1);
+                tma_load_3d(sdO + ch * BM * 128, &tmdO, barQ, ch * 32, i1, bh1);
             }
         }
 
@@ -260,8 +275,8 @@ strict_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
 #pragma unroll
             for (int x = 0; x < RM; ++x) {
                 const int i = i0 + tr + TR * x;
-                if (i < S) {
-                    float* row = dQ + (static_cast<size_t>(bh) * S + i) * D;
+                if (i < Sq) {
+                    float* row = dQ + (static_cast<size_t>(bh) * Sq + i) * D;
                     if constexpr (DV == 2) {
                         red_add_v2(row + 2 * tc, dq[x][0] * scale, dq[x][1] * scale);
                     } else {
@@ -281,8 +296,8 @@ strict_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
             const int j = j0 + 4 * tr + 4 * TR * g + u;
-            if (j < S) {
-                const size_t off = (static_cast<size_t>(bh) * S + j) * D;
+            if (j < Sk) {
+                const size_t off = (static_cast<size_t>(bhk) * Sk + j) * D;
                 const int a = 4 * g + u;
                 if constexpr (DV == 2) {
                     *reinterpret_cast<float2*>(dK + off + 2 * tc) = make_float2(dk[a][0] * scale, dk[a][1] * scale);
@@ -301,27 +316,38 @@ strict_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         }
 }
 
+template <int D, int BM, int BN, int THREADS, bool GEN>
+cudaError_t launch_gen(const Problem& p, const float* q, const float* k, const float* v, const float* d_o,
+                       const float* lse, const float* delta, float* dq, float* dk, float* dv, unsigned* status,
+                       cudaStream_t st)
+{
+    using C = BwdCfg<D, BM, BN, THREADS>;
+    CUtensorMap tq, tk, tv, tdo;
+    if (make_tmap_3d(&tq, q, 4, 0, p.BH(), p.Sq, D, 32, BM)) return cudaErrorInvalidValue;
+    if (make_tmap_3d(&tdo, d_o, 4, 0, p.BH(), p.Sq, D, 32, BM)) return cudaErrorInvalidValue;
+    if (make_tmap_3d(&tk, k, 4, 0, p.BHkv(), p.Sk, D, 32, BN)) return cudaErrorInvalidValue;
+    if (make_tmap_3d(&tv, v, 4, 0, p.BHkv(), p.Sk, D, 32, BN)) return cudaErrorInvalidValue;
+    auto kern = strict_bwd_kernel<D, BM, BN, THREADS, GEN>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM);
+    if (e != cudaSuccess) return e;
+    const int n_qt = (p.Sq + BM - 1) / BM;
+    const int n_kt = (p.Sk + BN - 1) / BN;
+    const long long blocks = static_cast<long long>(n_kt) * p.BHkv();
+    if (blocks > 0x7fffffffLL) return cudaErrorInvalidValue;
+    kern<<<static_cast<unsigned>(blocks), THREADS, C::SMEM, st>>>(tq, tk, tv, tdo, lse, delta, dq, dk, dv, p.Sq, p.Sk,
+                                                                   p.BHkv(), p.H, p.group(), n_qt, p.causal, p.scale,
+                                                                   status);
+    return cudaGetLastError();
+}
+
 template <int D, int BM, int BN, int THREADS>
 cudaError_t launch(const Problem& p, const float* q, const float* k, const float* v, const float* d_o,
                    const float* lse, const float* delta, float* dq, float* dk, float* dv, unsigned* status,
                    cudaStream_t st)
 {
-    using C = BwdCfg<D, BM, BN, THREADS>;
-    CUtensorMap tq, tk, tv, tdo;
-    if (make_tmap_3d(&tq, q, 4, 0, p.BH, p.S, D, 32, BM)) return cudaErrorInvalidValue;
-    if (make_tmap_3d(&tdo, d_o, 4, 0, p.BH, p.S, D, 32, BM)) return cudaErrorInvalidValue;
-    if (make_tmap_3d(&tk, k, 4, 0, p.BH, p.S, D, 32, BN)) return cudaErrorInvalidValue;
-    if (make_tmap_3d(&tv, v, 4, 0, p.BH, p.S, D, 32, BN)) return cudaErrorInvalidValue;
-    auto kern = strict_bwd_kernel<D, BM, BN, THREADS>;
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM);
-    if (e != cudaSuccess) return e;
-    const int n_qt = (p.S + BM - 1) / BM;
-    const int n_kt = (p.S + BN - 1) / BN;
-    const long long blocks = static_cast<long long>(n_kt) * p.BH;
-    if (blocks > 0x7fffffffLL) return cudaErrorInvalidValue;
-    kern<<<static_cast<unsigned>(blocks), THREADS, C::SMEM, st>>>(tq, tk, tv, tdo, lse, delta, dq, dk, dv, p.S, p.BH,
-                                                                   n_qt, p.causal, p.scale, status);
-    return cudaGetLastError();
+    return (p.Hkv != p.H || p.Sq != p.Sk)
+               ? launch_gen<D, BM, BN, THREADS, true>(p, q, k, v, d_o, lse, delta, dq, dk, dv, status, st)
+               : launch_gen<D, BM, BN, THREADS, false>(p, q, k, v, d_o, lse, delta, dq, dk, dv, status, st);
 }
 
 }  // namespace

@@ -5,7 +5,8 @@
 // K and V through shared memory with TMA.  Scores live in registers (each thread an
 // (BM/16)x(BN/16) micro-tile), the softmax is the online form (running row max in
 // the log2 domain, thread-local partial row sums), P goes through shared memory
-// once to become the A operand of O += P V.
+// once to become the A operand of O += P V.  Query head h reads key/value head h / G (grouped
+// heads); queries and keys may differ in length, the causal mask then being aligned bottom-right.
 //
 // Shared-memory tile layout (as TMA writes it with the 128-byte swizzle): a tile of
 // R rows x D floats is stored as D/32 chunks; chunk c holds, for every row, the 32
@@ -50,12 +51,16 @@ __device__ __forceinline__ uint32_t tile_off(int r, int piece) {
     return static_cast<uint32_t>((piece >> 3) * (R * 128) + r * 128 + (((piece & 7) ^ (r & 7)) << 4));
 }
 
-template <int D, int BM, int BN, int THREADS>
+// GEN = false is the square multi-head case (Sk == Sq, one key/value head per query head): the
+// offset, the group size and the second length fold away at compile time.
+template <int D, int BM, int BN, int THREADS, bool GEN>
 __global__ void __launch_bounds__(THREADS, THREADS == 128 ? 2 : 1)
 strict_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                   const __grid_constant__ CUtensorMap tmV, float* __restrict__ O, float* __restrict__ LSE,
-                  int S, int BH, int n_qt, int causal, float c2, unsigned* status)
+                  int Sq, int Sk_, int BH, int H, int G_, int n_qt, int causal, float c2, unsigned* status)
 {
+    const int Sk = GEN ? Sk_ : Sq;
+    const int G = GEN ? G_ : 1;
     using C = FwdCfg<D, BM, BN, THREADS>;
     constexpr int RM = C::RM, RN = C::RN, DV = C::DV, NCH = C::NCH, PSTR = C::PSTR, TR = C::TR;
 
@@ -78,9 +83,11 @@ strict_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     // Heaviest (last) query tiles first when causal.
     const int qt = n_qt - 1 - static_cast<int>(blockIdx.x) / BH;
     const int bh = static_cast<int>(blockIdx.x) % BH;
+    const int bhk = GEN ? (bh / H) * (H / G) + (bh % H) / G : bh;   // key/value head of this query head
+    const int off = GEN ? Sk - Sq : 0;                   // causal: key j visible to query i iff j <= i + off
     const int i0 = qt * BM;
-    const int i_last = min(i0 + BM, S) - 1;
-    const int n_kt = causal ? (i_last / BN + 1) : ((S + BN - 1) / BN);
+    const int i_last = min(i0 + BM, Sq) - 1;
+    const int n_kt = causal ? ((i_last + off) / BN + 1) : ((Sk + BN - 1) / BN);
 
     if (tid == 0) {
         mbar_init(barQ, 1);
@@ -95,10 +102,10 @@ strict_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         for (int ch = 0; ch < NCH; ++ch) tma_load_3d(sQ + ch * BM * 128, &tmQ, barQ, ch * 32, i0, bh);
         mbar_arrive_expect_tx(barK, C::KV_BYTES);
 #pragma unroll
-        for (int ch = 0; ch < NCH; ++ch) tma_load_3d(sK + ch * BN * 128, &tmK, barK, ch * 32, 0, bh);
+        for (int ch = 0; ch < NCH; ++ch) tma_load_3d(sK + ch * BN * 128, &tmK, barK, ch * 32, 0, bhk);
         mbar_arrive_expect_tx(barV, C::KV_BYTES);
 #pragma unroll
-        for (int ch = 0; ch < NCH; ++ch) tma_load_3d(sV + ch * BN * 128, &tmV, barV, ch * 32, 0, bh);
+        for (int ch = 0; ch < NCH; ++ch) tma_load_3d(sV + ch * BN * 128, &tmV, barV, ch * 32, 0, bhk);
     }
 
     float o[RM][DV];
@@ -151,11 +158,11 @@ strict_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         if (tid == 0 && kt + 1 < n_kt) {
             mbar_arrive_expect_tx(barK, C::KV_BYTES);
 #pragma unroll
-            for (int ch = 0; ch < NCH; ++ch) tma_load_3d(sK + ch * BN * 128, &tmK, barK, ch * 32, j0 + BN, bh);
+            for (int ch = 0; ch < NCH; ++ch) tma_load_3d(sK + ch * BN * 128, &tmK, barK, ch * 32, j0 + BN, bhk);
         }
 
         // ---- scale into the log2 domain, mask, online softmax ------------------------------
-        const bool need_mask = (causal && (j0 + BN - 1 > i0)) || (j0 + BN > S);
+        const bool need_mask = (causal && (j0 + BN - 1 > i0 + off)) || (j0 + BN > Sk);
 #pragma unroll
         for (int x = 0; x < RM; ++x) {
             const int i = i0 + tr + TR * x;
@@ -165,7 +172,7 @@ strict_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 float v = s[x][y] * c2;
                 if (need_mask) {
                     const int j = j0 + tc + 16 * y;
-                    if (j >= S || (causal && j > i)) v = -INFINITY;
+                    if (j >= Sk || (causal && j > i + off)) v = -INFINITY;
                 }
                 s[x][y] = v;
                 mx = fmaxf(mx, v);
@@ -233,7 +240,7 @@ strict_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         if (tid == 0 && kt + 1 < n_kt) {
             mbar_arrive_expect_tx(barV, C::KV_BYTES);
 #pragma unroll
-            for (int ch = 0; ch < NCH; ++ch) tma_load_3d(sV + ch * BN * 128, &tmV, barV, ch * 32, j0 + BN, bh);
+            for (int ch = 0; ch < NCH; ++ch) tma_load_3d(sV + ch * BN * 128, &tmV, barV, ch * 32, j0 + BN, bhk);
         }
     }
 
@@ -246,9 +253,9 @@ strict_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         lt += __shfl_xor_sync(0xffffffffu, lt, 4);
         lt += __shfl_xor_sync(0xffffffffu, lt, 8);
         const int i = i0 + tr + TR * x;
-        if (i < S) {
+        if (i < Sq) {
             const float inv = 1.0f / lt;
-            float* orow = O + (static_cast<size_t>(bh) * S + i) * D;
+            float* orow = O + (static_cast<size_t>(bh) * Sq + i) * D;
             if constexpr (DV == 2) {
                 *reinterpret_cast<float2*>(orow + 2 * tc) = make_float2(o[x][0] * inv, o[x][1] * inv);
             } else {
@@ -257,29 +264,38 @@ strict_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                     *reinterpret_cast<float4*>(orow + 4 * tc + 64 * e) =
                         make_float4(o[x][4 * e] * inv, o[x][4 * e + 1] * inv, o[x][4 * e + 2] * inv, o[x][4 * e + 3] * inv);
             }
-            if (tc == 0) LSE[static_cast<size_t>(bh) * S + i] = (m[x] + log2f(lt)) * kLn2;
+            if (tc == 0) LSE[static_cast<size_t>(bh) * Sq + i] = (m[x] + log2f(lt)) * kLn2;
         }
     }
+}
+
+template <int D, int BM, int BN, int THREADS, bool GEN>
+cudaError_t launch_gen(const Problem& p, const float* q, const float* k, const float* v, float* o, float* lse,
+                   unsigned* status, cudaStream_t st)
+{
+    using C = FwdCfg<D, BM, BN, THREADS>;
+    CUtensorMap tq, tk, tv;
+    if (make_tmap_3d(&tq, q, 4, 0, p.BH(), p.Sq, D, 32, BM)) return cudaErrorInvalidValue;
+    if (make_tmap_3d(&tk, k, 4, 0, p.BHkv(), p.Sk, D, 32, BN)) return cudaErrorInvalidValue;
+    if (make_tmap_3d(&tv, v, 4, 0, p.BHkv(), p.Sk, D, 32, BN)) return cudaErrorInvalidValue;
+    auto kern = strict_fwd_kernel<D, BM, BN, THREADS, GEN>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM);
+    if (e != cudaSuccess) return e;
+    const int n_qt = (p.Sq + BM - 1) / BM;
+    const long long blocks = static_cast<long long>(n_qt) * p.BH();
+    if (blocks > 0x7fffffffLL) return cudaErrorInvalidValue;
+    kern<<<static_cast<unsigned>(blocks), THREADS, C::SMEM, st>>>(tq, tk, tv, o, lse, p.Sq, p.Sk, p.BH(), p.H, p.group(), n_qt,
+                                                                   p.causal,
+                                                                   p.scale * kLog2e, status);
+    return cudaGetLastError();
 }
 
 template <int D, int BM, int BN, int THREADS>
 cudaError_t launch(const Problem& p, const float* q, const float* k, const float* v, float* o, float* lse,
                    unsigned* status, cudaStream_t st)
 {
-    using C = FwdCfg<D, BM, BN, THREADS>;
-    CUtensorMap tq, tk, tv;
-    if (make_tmap_3d(&tq, q, 4, 0, p.BH, p.S, D, 32, BM)) return cudaErrorInvalidValue;
-    if (make_tmap_3d(&tk, k, 4, 0, p.BH, p.S, D, 32, BN)) return cudaErrorInvalidValue;
-    if (make_tmap_3d(&tv, v, 4, 0, p.BH, p.S, D, 32, BN)) return cudaErrorInvalidValue;
-    auto kern = strict_fwd_kernel<D, BM, BN, THREADS>;
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM);
-    if (e != cudaSuccess) return e;
-    const int n_qt = (p.S + BM - 1) / BM;
-    const long long blocks = static_cast<long long>(n_qt) * p.BH;
-    if (blocks > 0x7fffffffLL) return cudaErrorInvalidValue;
-    kern<<<static_cast<unsigned>(blocks), THREADS, C::SMEM, st>>>(tq, tk, tv, o, lse, p.S, p.BH, n_qt, p.causal,
-                                                                   p.scale * kLog2e, status);
-    return cudaGetLastError();
+    return (p.Hkv != p.H || p.Sq != p.Sk) ? launch_gen<D, BM, BN, THREADS, true>(p, q, k, v, o, lse, status, st)
+                                          : launch_gen<D, BM, BN, THREADS, false>(p, q, k, v, o, lse, status, st);
 }
 
 }  // namespace

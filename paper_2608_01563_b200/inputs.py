@@ -104,3 +104,58 @@ def random_inputs(seed: int, B: int, H: int, S: int, D: int,
         (torch.randn((B, H, S, D), generator=g, dtype=torch.float32) * std).to(dtype).contiguous()
         for _ in range(4)
     )
+
+
+# ---------------------------------------------------------------------------------------------
+# Cross-attention and grouped key/value heads: q, dO are [B,H,Sq,D]; k, v are [B,Hkv,Sk,D].
+@dataclasses.dataclass(frozen=True)
+class ExtWorkload:
+    name: str
+    number: int          # enters the seed like Workload.number
+    B: int
+    H: int
+    Hkv: int
+    Sq: int
+    Sk: int
+    D: int
+    causal: bool
+
+    @property
+    def scale(self) -> float:
+        return 1.0 / math.sqrt(self.D)
+
+    @property
+    def seed(self) -> int:
+        return BASE_SEED + 100 * self.number
+
+    @property
+    def pairs(self) -> float:
+        """Score pairs per (batch, query head), counted like the square workloads: a causal
+        triangle of side Sq counts Sq^2/2, the rectangle of always-visible keys in front of it fully."""
+        return self.Sq * (self.Sk - self.Sq) + self.Sq * self.Sq / 2.0 if self.causal else float(self.Sq * self.Sk)
+
+
+EXT_WORKLOADS: Dict[str, ExtWorkload] = {
+    w.name: w
+    for w in [
+        # decoder block with grouped key/value heads at the size of the decoder sweep (S = 2048)
+        ExtWorkload("gqa_decoder", 6, 4, 32, 8, 2048, 2048, 128, True),
+        # text cross-attention of a latent-diffusion U-Net: a 32x32 latent (1024 queries) over 77 text tokens
+        ExtWorkload("cross_attn_text", 7, 16, 8, 8, 1024, 77, 64, False),
+        # action tokens over vision-language context tokens, batched
+        ExtWorkload("cross_attn_action", 8, 64, 8, 8, 50, 16, 64, False),
+        # chunked causal continuation: 512 new queries at the end of a 4096-token context, grouped heads
+        ExtWorkload("gqa_suffix", 9, 2, 16, 4, 512, 4096, 128, True),
+    ]
+}
+
+
+def make_inputs_ext(w: ExtWorkload, dtype: torch.dtype = torch.float32) -> Tuple[torch.Tensor, ...]:
+    """Host tensors (Q [B,H,Sq,D], K, V [B,Hkv,Sk,D], dO [B,H,Sq,D]) ~ N(0,1), drawn in that order
+    with ``torch.randn`` in float32 from ``torch.Generator("cpu").manual_seed(w.seed)``."""
+    g = torch.Generator(device="cpu").manual_seed(w.seed)
+    q = torch.randn((w.B, w.H, w.Sq, w.D), generator=g, dtype=torch.float32)
+    k = torch.randn((w.B, w.Hkv, w.Sk, w.D), generator=g, dtype=torch.float32)
+    v = torch.randn((w.B, w.Hkv, w.Sk, w.D), generator=g, dtype=torch.float32)
+    d_o = torch.randn((w.B, w.H, w.Sq, w.D), generator=g, dtype=torch.float32)
+    return tuple(t.to(dtype).contiguous() for t in (q, k, v, d_o))

@@ -143,3 +143,36 @@ def check_invariants(q, k, v, d_o, res, rtol, max_heads=None):
     assert e1 <= rtol, f"<dQ,Q> vs <dK,K>: {e1:.3e}"
     assert e2 <= rtol, f"<dV,V> vs <dO,O>: {e2:.3e}"
     return e1, e2
+
+
+def run_cuda_ext(q, k, v, d_o, causal, scale, mode, run_bwd=True):
+    """Extended shapes: q, d_o [B,H,Sq,D]; k, v [B,Hkv,Sk,D] (host tensors). Returns host tensors."""
+    dev = "cuda"
+    dt = q.dtype
+    B, H, Sq, D = q.shape
+    _, Hkv, Sk, _ = k.shape
+    qd, kd, vd, dod = (t.to(dev) for t in (q, k, v, d_o))
+    o = Guarded((B, H, Sq, D), dt)
+    lse = Guarded((B, H, Sq), torch.float32)
+    mgn.mgn_attn_fwd_ext(qd, kd, vd, o.view, lse.view, causal, scale, mode)
+    res = {}
+    if run_bwd:
+        dq = Guarded((B, H, Sq, D), dt)
+        dk, dv = (Guarded((B, Hkv, Sk, D), dt) for _ in range(2))
+        ws = mgn.alloc_workspace(B, H, Sq, D, mode)
+        ws.fill_(0xFF)
+        mgn.mgn_attn_bwd_ext(qd, kd, vd, o.view, dod, lse.view, dq.view, dk.view, dv.view, ws, causal, scale, mode)
+    mgn.mgn_attn_check()
+    res["O"] = o.check("O")
+    res["LSE"] = lse.check("LSE")
+    if run_bwd:
+        res["dQ"] = dq.check("dQ")
+        res["dK"] = dk.check("dK")
+        res["dV"] = dv.check("dV")
+    return {n: t.double().numpy() for n, t in res.items()}
+
+
+def run_oracle_ext(q, k, v, d_o, causal, scale):
+    o, lse, dq, dk, dv = orc.attn_bwd_ext(q.double().numpy(), k.double().numpy(), v.double().numpy(),
+                                          d_o.double().numpy(), causal, scale)
+    return {"O": o, "LSE": lse, "dQ": dq, "dK": dk, "dV": dv}

@@ -33,7 +33,7 @@ def test_every_declared_symbol_is_exported(lib):
     syms = declared_symbols()
     assert {"mgn_attn_fwd", "mgn_attn_bwd", "mgn_attn_bwd_workspace_bytes", "mgn_attn_check",
             "mgn_status_string", "mgn_version", "mgn_attn_profile_events", "mgn_attn_bwd_noalloc", "mgn_measure_fp32_ffma_tflops",
-            "mgn_attn_fast_item_order"} <= set(syms)
+            "mgn_attn_fast_item_order", "mgn_attn_fwd_ext", "mgn_attn_bwd_ext"} <= set(syms)
     for s in syms:
         assert getattr(lib, s) is not None
 
@@ -123,3 +123,31 @@ def test_binding_fails_loudly_without_library(monkeypatch, tmp_path):
     monkeypatch.setattr(binding, "LIB_PATH", str(tmp_path / "nope.so"))
     with pytest.raises(RuntimeError):
         binding.mgn_version()
+
+
+def test_extended_shape_argument_validation(lib):
+    """mgn_attn_fwd_ext / mgn_attn_bwd_ext refuse bad head groups and causal S_q > S_k before any launch."""
+    INVALID, UNSUPPORTED, MISALIGNED, WORKSPACE = 1, 2, 3, 4
+    vp, i, f, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_float, ctypes.c_size_t
+    lib.mgn_attn_fwd_ext.argtypes = [vp] * 5 + [i] * 7 + [f, i, vp]
+    lib.mgn_attn_bwd_ext.argtypes = [vp] * 9 + [vp, sz] + [i] * 7 + [f, i, vp]
+
+    def fx(B=1, H=4, Hkv=2, Sq=8, Sk=16, D=64, causal=0, q=A):
+        return lib.mgn_attn_fwd_ext(q, A, A, A, A, B, H, Hkv, Sq, Sk, D, causal, 1.0, 0, None)
+
+    def bx(B=1, H=4, Hkv=2, Sq=8, Sk=16, D=64, causal=0, ws=A, ws_bytes=1 << 30):
+        return lib.mgn_attn_bwd_ext(*([A] * 9), ws, ws_bytes, B, H, Hkv, Sq, Sk, D, causal, 1.0, 0, None)
+
+    assert fx(H=4, Hkv=3) == INVALID
+    assert fx(Hkv=0) == INVALID
+    assert fx(Sk=0) == INVALID
+    assert fx(Sq=16, Sk=8, causal=1) == UNSUPPORTED
+    assert fx(D=48) == UNSUPPORTED
+    assert fx(q=A + 4) == MISALIGNED
+    assert bx(H=4, Hkv=3) == INVALID
+    assert bx(Sq=16, Sk=8, causal=1) == UNSUPPORTED
+    need = lib.mgn_attn_bwd_workspace_bytes(1, 4, 8, 64, 0)       # sized by the query side
+    assert bx(ws_bytes=need - 1) == WORKSPACE
+    import torch
+    if not torch.cuda.is_available():
+        assert fx() in (5, 6) and bx() in (5, 6)
