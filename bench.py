@@ -180,6 +180,32 @@ def quick_measure_ext(mgn, w, mode, dtype, steps, warmup):
             "sum_tflops": 14.0 * unit / ((fwd_ms + bwd_ms) * 1e-3) / 1e12}
 
 
+def measure_deterministic_bwd(mgn, w, steps, warmup):
+    """Strict mode only: the backward without floating-point atomics (fused dK+dV kernel + separate dQ pass)."""
+    q, k, v, d_o = (t.cuda() for t in synth.make_inputs(w, dtype=torch.float32))
+    o = torch.empty_like(q)
+    lse = torch.empty(w.B, w.H, w.S, device="cuda", dtype=torch.float32)
+    dq, dk, dv = (torch.empty_like(q) for _ in range(3))
+    ws = mgn.alloc_workspace(w.B, w.H, w.S, w.D, mgn.MODE_STRICT_F32)
+    mgn.mgn_attn_fwd(q, k, v, o, lse, w.causal, w.scale, mgn.MODE_STRICT_F32)
+    run = lambda: mgn.mgn_attn_bwd_deterministic(q, k, v, o, d_o, lse, dq, dk, dv, ws, w.causal, w.scale,
+                                                 mgn.MODE_STRICT_F32)
+    for _ in range(warmup):
+        run()
+    torch.cuda.synchronize()
+    e = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+    e[0].record()
+    for i in range(steps):
+        run()
+        e[i + 1].record()
+    torch.cuda.synchronize()
+    mgn.mgn_attn_check()
+    ms = statistics.mean(e[i].elapsed_time(e[i + 1]) for i in range(steps))
+    return {"workload": w.name, "bwd_ms": ms, "counted_tflops": flops(w, "bwd") / (ms * 1e-3) / 1e12,
+            "executed_tflops": 1.4 * flops(w, "bwd") / (ms * 1e-3) / 1e12,
+            "note": "no floating-point atomics; 7 matrix products per tile pair instead of 5"}
+
+
 def cpu_info():
     model = "unknown"
     try:
@@ -500,6 +526,8 @@ def main():
                 r["frac_of_peak"] = r["sum_tflops"] / mode_peak
                 ext[name] = r
             line["ext_shapes"] = ext
+            if args.mode == "strict":
+                line["deterministic_bwd"] = measure_deterministic_bwd(mgn, w, K, args.warmup)
         if world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline(w, dtype)
         print(json.dumps(line))

@@ -106,6 +106,21 @@ int mgn_attn_bwd_ext(const void* q, const void* k, const void* v, const void* o,
                      void* stream);
 
 /*
+ * Deterministic backward (the "separate pass" form of the dQ kernel: paper Section 3.3 lists dQ
+ * beside the fused dK+dV kernel, Section 7.3 profiles them separately).  Same arguments, shapes and
+ * results as mgn_attn_bwd_ext, but no floating-point atomics are used: the fused dK+dV kernel runs
+ * without the dQ reductions and a second kernel computes dQ with one CTA per query tile, so dq, dk
+ * and dv are bit-identical from run to run.  It executes seven matrix products per tile pair instead
+ * of five (S and dP are recomputed in the dQ pass).  MGN_MODE_STRICT_F32 only; MGN_MODE_FAST_BF16
+ * returns MGN_ERR_UNSUPPORTED.
+ */
+int mgn_attn_bwd_deterministic(const void* q, const void* k, const void* v, const void* o, const void* d_o,
+                               const float* lse, void* dq, void* dk, void* dv,
+                               void* workspace, size_t workspace_bytes,
+                               int B, int H, int H_kv, int S_q, int S_k, int D, int causal, float scale, int mode,
+                               void* stream);
+
+/*
  * Synchronises `stream`, then reads and clears the device-side status word that
  * kernels set when one of their bounded waits (TMA / tensor-core completion
  * barriers) ran out.  Returns MGN_OK, MGN_ERR_DEVICE_TIMEOUT or MGN_ERR_CUDA.

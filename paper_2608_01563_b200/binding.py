@@ -49,6 +49,8 @@ def lib() -> ctypes.CDLL:
         L.mgn_attn_fwd_ext.restype = i
         L.mgn_attn_bwd_ext.argtypes = [vp] * 9 + [vp, sz, i, i, i, i, i, i, i, f, i, vp]
         L.mgn_attn_bwd_ext.restype = i
+        L.mgn_attn_bwd_deterministic.argtypes = [vp] * 9 + [vp, sz, i, i, i, i, i, i, i, f, i, vp]
+        L.mgn_attn_bwd_deterministic.restype = i
         L.mgn_attn_bwd_workspace_bytes.argtypes = [i, i, i, i, i]
         L.mgn_attn_bwd_workspace_bytes.restype = sz
         L.mgn_attn_check.argtypes = [vp]
@@ -131,6 +133,18 @@ def mgn_attn_bwd_ext(q, k, v, o, d_o, lse, dq, dk, dv, workspace, causal: bool, 
                                 B, H, Hkv, Sq, Sk, D, int(causal), float(scale), int(mode), _stream(stream))
     if st != MGN_OK:
         raise MgnError(st, "mgn_attn_bwd_ext")
+
+
+def mgn_attn_bwd_deterministic(q, k, v, o, d_o, lse, dq, dk, dv, workspace, causal: bool, scale: float,
+                               mode: int, stream: Optional[int] = None) -> None:
+    """Backward without floating-point atomics (strict mode): bit-identical from run to run."""
+    B, H, Hkv, Sq, Sk, D = _ext_dims(q, k)
+    st = lib().mgn_attn_bwd_deterministic(_ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(d_o), _ptr(lse), _ptr(dq),
+                                          _ptr(dk), _ptr(dv), _ptr(workspace),
+                                          workspace.numel() * workspace.element_size(), B, H, Hkv, Sq, Sk, D,
+                                          int(causal), float(scale), int(mode), _stream(stream))
+    if st != MGN_OK:
+        raise MgnError(st, "mgn_attn_bwd_deterministic")
 
 
 def mgn_attn_bwd_noalloc(q, k, v, o, d_o, lse, dq, dk, dv, causal: bool, scale: float, mode: int,

@@ -164,6 +164,41 @@ int mgn_attn_bwd_ext(const void* q, const void* k, const void* v, const void* o,
     return e == cudaSuccess ? MGN_OK : MGN_ERR_CUDA;
 }
 
+int mgn_attn_bwd_deterministic(const void* q, const void* k, const void* v, const void* o, const void* d_o,
+                               const float* lse, void* dq, void* dk, void* dv,
+                               void* workspace, size_t workspace_bytes,
+                               int B, int H, int H_kv, int S_q, int S_k, int D, int causal, float scale, int mode,
+                               void* stream)
+{
+    if (!q || !k || !v || !o || !d_o || !lse || !dq || !dk || !dv) return MGN_ERR_INVALID_ARG;
+    if (int r = check_ext(B, H, H_kv, S_q, S_k, D, causal, scale, mode)) return r;
+    if (mode != MGN_MODE_STRICT_F32) return MGN_ERR_UNSUPPORTED;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(d_o) || !aligned16(lse) ||
+        !aligned16(dq) || !aligned16(dk) || !aligned16(dv))
+        return MGN_ERR_MISALIGNED;
+    const size_t need = mgn_attn_bwd_workspace_bytes(B, H, S_q, D, mode);
+    if (!workspace || workspace_bytes < need) return MGN_ERR_WORKSPACE;
+    if (reinterpret_cast<uintptr_t>(workspace) & 255u) return MGN_ERR_WORKSPACE;
+    unsigned* status = nullptr;
+    if (int r = device_setup(&status)) return r;
+
+    const mgn::Problem p{B, H, H_kv, S_q, S_k, D, causal, scale};
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t rows = static_cast<size_t>(B) * H * S_q;
+    float* delta = static_cast<float*>(workspace);
+    cudaError_t e = mgn::launch_bwd_preprocess(o, d_o, delta, nullptr, rows, D, 0, st);
+    if (e != cudaSuccess) return MGN_ERR_CUDA;
+    MainKernelTimer timer(st);
+    e = mgn::launch_strict_bwd(p, static_cast<const float*>(q), static_cast<const float*>(k),
+                               static_cast<const float*>(v), static_cast<const float*>(d_o), lse, delta, nullptr,
+                               static_cast<float*>(dk), static_cast<float*>(dv), status, st);
+    if (e != cudaSuccess) return MGN_ERR_CUDA;
+    e = mgn::launch_strict_dq(p, static_cast<const float*>(q), static_cast<const float*>(k),
+                              static_cast<const float*>(v), static_cast<const float*>(d_o), lse, delta,
+                              static_cast<float*>(dq), status, st);
+    return e == cudaSuccess ? MGN_OK : MGN_ERR_CUDA;
+}
+
 int mgn_attn_bwd(const void* q, const void* k, const void* v, const void* o, const void* d_o,
                  const float* lse, void* dq, void* dk, void* dv,
                  void* workspace, size_t workspace_bytes,

@@ -25,7 +25,8 @@ bwd_preprocess_kernel(const uint4* __restrict__ o, const uint4* __restrict__ d_o
         if (r < rows) {
             constexpr int ZPL = BF16 ? 2 : 1;      // float4 stores per lane to cover a row of D floats
 #pragma unroll
-            for (int t = 0; t < ZPL; ++t) zero[(r * LANES + lane) * ZPL + t] = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int t = 0; t < ZPL; ++t)
+                if (zero) zero[(r * LANES + lane) * ZPL + t] = make_float4(0.f, 0.f, 0.f, 0.f);
             const uint4 a = __ldg(o + r * LANES + lane);
             const uint4 b = __ldg(d_o + r * LANES + lane);
             if constexpr (BF16) {

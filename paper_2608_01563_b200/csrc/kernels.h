@@ -30,8 +30,14 @@ cudaError_t launch_strict_bwd(const Problem& p, const float* q, const float* k, 
                               const float* d_o, const float* lse, const float* delta,
                               float* dq, float* dk, float* dv, unsigned* status, cudaStream_t st);
 
+// Deterministic strict backward: launch_strict_bwd with dq == nullptr runs the fused dK+dV kernel
+// without the dQ reductions, and this separate pass computes dQ with plain stores.
+cudaError_t launch_strict_dq(const Problem& p, const float* q, const float* k, const float* v,
+                             const float* d_o, const float* lse, const float* delta, float* dq,
+                             unsigned* status, cudaStream_t st);
+
 // delta_i = sum_d dO[i,d] O[i,d]  (f32 or bf16 inputs, f32 output), HBM-bound; also clears the
-// f32 dQ accumulation target `zero` ([rows][D] floats).
+// f32 dQ accumulation target `zero` ([rows][D] floats) unless it is null.
 cudaError_t launch_bwd_preprocess(const void* o, const void* d_o, float* delta, float* zero,
                                   size_t rows, int D, int is_bf16, cudaStream_t st);
 

@@ -62,7 +62,9 @@ __device__ __forceinline__ float f4_get(const float4& v, int u) {
 
 // GEN = false is the square multi-head case (Sk == Sq, one key/value head per query head): the
 // offset, the group loop and the second length fold away at compile time.
-template <int D, int BM, int BN, int THREADS, bool GEN>
+// WITH_DQ = false leaves phase C (the dQ partial and its floating-point reductions) out: the fused
+// dK+dV kernel of the deterministic backward, whose dQ comes from the separate pass in strict_dq.cu.
+template <int D, int BM, int BN, int THREADS, bool GEN, bool WITH_DQ>
 __global__ void __launch_bounds__(THREADS, THREADS == 128 ? 2 : 1)
 strict_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                   const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmdO,
@@ -246,7 +248,7 @@ strict_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         }
 
         // ---- C: dQ partial = dS K : contraction over keys, reduced into global dQ ----------
-        {
+        if constexpr (WITH_DQ) {
             float dq[RM][DV];
 #pragma unroll
             for (int x = 0; x < RM; ++x)
@@ -316,7 +318,7 @@ strict_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         }
 }
 
-template <int D, int BM, int BN, int THREADS, bool GEN>
+template <int D, int BM, int BN, int THREADS, bool GEN, bool WITH_DQ>
 cudaError_t launch_gen(const Problem& p, const float* q, const float* k, const float* v, const float* d_o,
                        const float* lse, const float* delta, float* dq, float* dk, float* dv, unsigned* status,
                        cudaStream_t st)
@@ -327,7 +329,7 @@ cudaError_t launch_gen(const Problem& p, const float* q, const float* k, const f
     if (make_tmap_3d(&tdo, d_o, 4, 0, p.BH(), p.Sq, D, 32, BM)) return cudaErrorInvalidValue;
     if (make_tmap_3d(&tk, k, 4, 0, p.BHkv(), p.Sk, D, 32, BN)) return cudaErrorInvalidValue;
     if (make_tmap_3d(&tv, v, 4, 0, p.BHkv(), p.Sk, D, 32, BN)) return cudaErrorInvalidValue;
-    auto kern = strict_bwd_kernel<D, BM, BN, THREADS, GEN>;
+    auto kern = strict_bwd_kernel<D, BM, BN, THREADS, GEN, WITH_DQ>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM);
     if (e != cudaSuccess) return e;
     const int n_qt = (p.Sq + BM - 1) / BM;
@@ -345,9 +347,11 @@ cudaError_t launch(const Problem& p, const float* q, const float* k, const float
                    const float* lse, const float* delta, float* dq, float* dk, float* dv, unsigned* status,
                    cudaStream_t st)
 {
+    if (dq == nullptr)   // fused dK+dV only (deterministic backward): the general-shape build serves every shape
+        return launch_gen<D, BM, BN, THREADS, true, false>(p, q, k, v, d_o, lse, delta, dq, dk, dv, status, st);
     return (p.Hkv != p.H || p.Sq != p.Sk)
-               ? launch_gen<D, BM, BN, THREADS, true>(p, q, k, v, d_o, lse, delta, dq, dk, dv, status, st)
-               : launch_gen<D, BM, BN, THREADS, false>(p, q, k, v, d_o, lse, delta, dq, dk, dv, status, st);
+               ? launch_gen<D, BM, BN, THREADS, true, true>(p, q, k, v, d_o, lse, delta, dq, dk, dv, status, st)
+               : launch_gen<D, BM, BN, THREADS, false, true>(p, q, k, v, d_o, lse, delta, dq, dk, dv, status, st);
 }
 
 }  // namespace

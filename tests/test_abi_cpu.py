@@ -33,7 +33,8 @@ def test_every_declared_symbol_is_exported(lib):
     syms = declared_symbols()
     assert {"mgn_attn_fwd", "mgn_attn_bwd", "mgn_attn_bwd_workspace_bytes", "mgn_attn_check",
             "mgn_status_string", "mgn_version", "mgn_attn_profile_events", "mgn_attn_bwd_noalloc", "mgn_measure_fp32_ffma_tflops",
-            "mgn_attn_fast_item_order", "mgn_attn_fwd_ext", "mgn_attn_bwd_ext"} <= set(syms)
+            "mgn_attn_fast_item_order", "mgn_attn_fwd_ext", "mgn_attn_bwd_ext",
+            "mgn_attn_bwd_deterministic"} <= set(syms)
     for s in syms:
         assert getattr(lib, s) is not None
 
@@ -146,6 +147,11 @@ def test_extended_shape_argument_validation(lib):
     assert fx(q=A + 4) == MISALIGNED
     assert bx(H=4, Hkv=3) == INVALID
     assert bx(Sq=16, Sk=8, causal=1) == UNSUPPORTED
+    lib.mgn_attn_bwd_deterministic.argtypes = lib.mgn_attn_bwd_ext.argtypes
+    det = lambda mode=0, H=4, Hkv=2: lib.mgn_attn_bwd_deterministic(*([A] * 9), A, 1 << 30, 1, H, Hkv, 8, 16, 64, 0,
+                                                                   1.0, mode, None)
+    assert det(mode=1) == UNSUPPORTED          # strict mode only
+    assert det(H=4, Hkv=3) == INVALID
     need = lib.mgn_attn_bwd_workspace_bytes(1, 4, 8, 64, 0)       # sized by the query side
     assert bx(ws_bytes=need - 1) == WORKSPACE
     import torch
