@@ -206,6 +206,40 @@ def measure_deterministic_bwd(mgn, w, steps, warmup):
             "note": "no floating-point atomics; 7 matrix products per tile pair instead of 5"}
 
 
+def measure_accel_policy(mgn, w, steps, warmup):
+    """The paper's accelerated policy on f32 tensors: f16 tensor-core forward (mgn_attn_fwd_accel, its
+    f32->f16 conversion included) followed by the strict f32 backward."""
+    S32 = mgn.MODE_STRICT_F32
+    q, k, v, d_o = (t.cuda() for t in synth.make_inputs(w, dtype=torch.float32))
+    o = torch.empty_like(q)
+    lse = torch.empty(w.B, w.H, w.S, device="cuda", dtype=torch.float32)
+    dq, dk, dv = (torch.empty_like(q) for _ in range(3))
+    ws = mgn.alloc_workspace(w.B, w.H, w.S, w.D, S32)
+    wsf = torch.empty(mgn.mgn_attn_fwd_accel_workspace_bytes(w.B, w.H, w.H, w.S, w.S, w.D), dtype=torch.uint8,
+                      device="cuda")
+    fwd = lambda: mgn.mgn_attn_fwd_accel(q, k, v, o, lse, wsf, w.causal, w.scale)
+    bwd = lambda: mgn.mgn_attn_bwd(q, k, v, o, d_o, lse, dq, dk, dv, ws, w.causal, w.scale, S32)
+    for _ in range(warmup):
+        fwd()
+        bwd()
+    torch.cuda.synchronize()
+    e = [torch.cuda.Event(enable_timing=True) for _ in range(2 * steps + 1)]
+    e[0].record()
+    for i in range(steps):
+        fwd()
+        e[2 * i + 1].record()
+        bwd()
+        e[2 * i + 2].record()
+    torch.cuda.synchronize()
+    mgn.mgn_attn_check()
+    f_ms = statistics.mean(e[2 * i].elapsed_time(e[2 * i + 1]) for i in range(steps))
+    b_ms = statistics.mean(e[2 * i + 1].elapsed_time(e[2 * i + 2]) for i in range(steps))
+    return {"workload": w.name, "fwd_ms": f_ms, "bwd_ms": b_ms,
+            "fwd_tflops": flops(w, "fwd") / (f_ms * 1e-3) / 1e12,
+            "sum_tflops": flops(w, "sum") / ((f_ms + b_ms) * 1e-3) / 1e12,
+            "note": "f32 tensors; forward: f32->f16 conversion + f16 tensor-core kernel, f32 O; backward: strict f32"}
+
+
 def cpu_info():
     model = "unknown"
     try:
@@ -528,6 +562,8 @@ def main():
             line["ext_shapes"] = ext
             if args.mode == "strict":
                 line["deterministic_bwd"] = measure_deterministic_bwd(mgn, w, K, args.warmup)
+                if w.D in (64, 128):
+                    line["accel_policy"] = measure_accel_policy(mgn, w, K, args.warmup)
         if world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline(w, dtype)
         print(json.dumps(line))

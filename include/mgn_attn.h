@@ -106,6 +106,25 @@ int mgn_attn_bwd_ext(const void* q, const void* k, const void* v, const void* o,
                      void* stream);
 
 /*
+ * Forward of the paper's accelerated ("practical default") arithmetic policy (Section 4.2, table
+ * "Arithmetic permissions"): persistent tensors stay f32; the forward attention inputs are rounded
+ * locally to IEEE f16, multiplied on the tensor cores with f32 accumulation, and O and LSE are stored
+ * as f32; the backward remains f32 -- call mgn_attn_bwd_ext (or mgn_attn_bwd_deterministic) with
+ * MGN_MODE_STRICT_F32 on the same f32 tensors and this forward's o and lse.
+ *   q [B,H,S_q,D], k, v [B,H_kv,S_k,D], o [B,H,S_q,D], lse [B,H,S_q]: all binary32, device pointers.
+ *   D must be 64 or 128.  Shapes, grouping and the causal rule are those of mgn_attn_fwd_ext.
+ *   workspace: device scratch of mgn_attn_fwd_accel_workspace_bytes(...) bytes (f16 copies of q, k
+ *   and v), 256-byte aligned, contents ignored on entry and undefined on exit.
+ * Inputs whose magnitude exceeds the f16 range (65504) become infinities; the softmax probabilities
+ * are rounded to f16 before the second product, so entries below 6e-8 are dropped.
+ * Errors as for mgn_attn_fwd_ext, plus MGN_ERR_WORKSPACE.
+ */
+size_t mgn_attn_fwd_accel_workspace_bytes(int B, int H, int H_kv, int S_q, int S_k, int D);
+int mgn_attn_fwd_accel(const float* q, const float* k, const float* v, float* o, float* lse,
+                       void* workspace, size_t workspace_bytes,
+                       int B, int H, int H_kv, int S_q, int S_k, int D, int causal, float scale, void* stream);
+
+/*
  * Deterministic backward (the "separate pass" form of the dQ kernel: paper Section 3.3 lists dQ
  * beside the fused dK+dV kernel, Section 7.3 profiles them separately).  Same arguments, shapes and
  * results as mgn_attn_bwd_ext, but no floating-point atomics are used: the fused dK+dV kernel runs

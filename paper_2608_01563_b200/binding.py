@@ -49,6 +49,10 @@ def lib() -> ctypes.CDLL:
         L.mgn_attn_fwd_ext.restype = i
         L.mgn_attn_bwd_ext.argtypes = [vp] * 9 + [vp, sz, i, i, i, i, i, i, i, f, i, vp]
         L.mgn_attn_bwd_ext.restype = i
+        L.mgn_attn_fwd_accel.argtypes = [vp] * 5 + [vp, sz, i, i, i, i, i, i, i, f, vp]
+        L.mgn_attn_fwd_accel.restype = i
+        L.mgn_attn_fwd_accel_workspace_bytes.argtypes = [i] * 6
+        L.mgn_attn_fwd_accel_workspace_bytes.restype = sz
         L.mgn_attn_bwd_deterministic.argtypes = [vp] * 9 + [vp, sz, i, i, i, i, i, i, i, f, i, vp]
         L.mgn_attn_bwd_deterministic.restype = i
         L.mgn_attn_bwd_workspace_bytes.argtypes = [i, i, i, i, i]
@@ -133,6 +137,20 @@ def mgn_attn_bwd_ext(q, k, v, o, d_o, lse, dq, dk, dv, workspace, causal: bool, 
                                 B, H, Hkv, Sq, Sk, D, int(causal), float(scale), int(mode), _stream(stream))
     if st != MGN_OK:
         raise MgnError(st, "mgn_attn_bwd_ext")
+
+
+def mgn_attn_fwd_accel_workspace_bytes(B: int, H: int, Hkv: int, Sq: int, Sk: int, D: int) -> int:
+    return int(lib().mgn_attn_fwd_accel_workspace_bytes(B, H, Hkv, Sq, Sk, D))
+
+
+def mgn_attn_fwd_accel(q, k, v, o, lse, workspace, causal: bool, scale: float, stream: Optional[int] = None) -> None:
+    """Forward of the accelerated policy: f32 tensors, f16 tensor-core products, f32 O and LSE."""
+    B, H, Hkv, Sq, Sk, D = _ext_dims(q, k)
+    st = lib().mgn_attn_fwd_accel(_ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse), _ptr(workspace),
+                                  workspace.numel() * workspace.element_size(), B, H, Hkv, Sq, Sk, D,
+                                  int(causal), float(scale), _stream(stream))
+    if st != MGN_OK:
+        raise MgnError(st, "mgn_attn_fwd_accel")
 
 
 def mgn_attn_bwd_deterministic(q, k, v, o, d_o, lse, dq, dk, dv, workspace, causal: bool, scale: float,

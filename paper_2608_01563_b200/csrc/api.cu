@@ -124,6 +124,39 @@ int mgn_attn_fwd(const void* q, const void* k, const void* v, void* o, float* ls
     return mgn_attn_fwd_ext(q, k, v, o, lse, B, H, H, S, S, D, causal, scale, mode, stream);
 }
 
+size_t mgn_attn_fwd_accel_workspace_bytes(int B, int H, int H_kv, int S_q, int S_k, int D)
+{
+    if (check_ext(B, H, H_kv, S_q, S_k, D, 0, 1.0f, MGN_MODE_FAST_BF16) != MGN_OK) return 0;
+    const size_t nq = static_cast<size_t>(B) * H * S_q * D, nk = static_cast<size_t>(B) * H_kv * S_k * D;
+    return align_up(nq * 2, 256) + 2 * align_up(nk * 2, 256);
+}
+
+int mgn_attn_fwd_accel(const float* q, const float* k, const float* v, float* o, float* lse,
+                       void* workspace, size_t workspace_bytes,
+                       int B, int H, int H_kv, int S_q, int S_k, int D, int causal, float scale, void* stream)
+{
+    if (!q || !k || !v || !o || !lse) return MGN_ERR_INVALID_ARG;
+    if (int r = check_ext(B, H, H_kv, S_q, S_k, D, causal, scale, MGN_MODE_FAST_BF16)) return r;   // D in {64,128}
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(lse)) return MGN_ERR_MISALIGNED;
+    const size_t need = mgn_attn_fwd_accel_workspace_bytes(B, H, H_kv, S_q, S_k, D);
+    if (!workspace || workspace_bytes < need) return MGN_ERR_WORKSPACE;
+    if (reinterpret_cast<uintptr_t>(workspace) & 255u) return MGN_ERR_WORKSPACE;
+    unsigned* status = nullptr;
+    if (int r = device_setup(&status)) return r;
+    const mgn::Problem p{B, H, H_kv, S_q, S_k, D, causal, scale};
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t nq = static_cast<size_t>(B) * H * S_q * D, nk = static_cast<size_t>(B) * H_kv * S_k * D;
+    char* w = static_cast<char*>(workspace);
+    void* q16 = w;
+    void* k16 = w + align_up(nq * 2, 256);
+    void* v16 = static_cast<char*>(k16) + align_up(nk * 2, 256);
+    if (mgn::launch_to_f16(q, q16, nq, st) != cudaSuccess || mgn::launch_to_f16(k, k16, nk, st) != cudaSuccess ||
+        mgn::launch_to_f16(v, v16, nk, st) != cudaSuccess)
+        return MGN_ERR_CUDA;
+    MainKernelTimer timer(st);
+    return mgn::launch_fast_fwd_f16(p, q16, k16, v16, o, lse, status, st) == cudaSuccess ? MGN_OK : MGN_ERR_CUDA;
+}
+
 int mgn_attn_bwd_ext(const void* q, const void* k, const void* v, const void* o, const void* d_o,
                      const float* lse, void* dq, void* dk, void* dv,
                      void* workspace, size_t workspace_bytes,

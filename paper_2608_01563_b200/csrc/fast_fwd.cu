@@ -103,11 +103,15 @@ __device__ __forceinline__ int item_index(int c, int k, int G, int n_items, int 
     return it < n_items ? it : -1;
 }
 
-template <int D, bool GEN>
+// F16 = true is the forward of the accelerated policy (paper Section 4.2, table "Arithmetic
+// permissions"): operands are IEEE f16 copies of f32 tensors, P is packed as f16, and O leaves as f32
+// with plain stores (O32); otherwise operands and O are bf16 and O leaves through TMA (tmO).
+template <int D, bool GEN, bool F16>
 __global__ void __launch_bounds__(kThreads, 1)
 fast_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                 const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO,
-                float* __restrict__ LSE, const Dims dm, int n_pairs, int causal, int order, float c2, unsigned* status)
+                float* __restrict__ LSE, float* __restrict__ O32, const Dims dm, int n_pairs, int causal, int order,
+                float c2, unsigned* status)
 {
     using C = Cfg<D>;
     extern __shared__ uint8_t smem_raw[];
@@ -178,8 +182,8 @@ fast_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         // ------------------------------------------------------------------ MMA issuer of tile t
         {
             const int t = warp - 1;
-            constexpr uint32_t idesc_s = umma_idesc_bf16(BM, BN, false, false);
-            constexpr uint32_t idesc_o = umma_idesc_bf16(BM, D, false, true);
+            constexpr uint32_t idesc_s = F16 ? umma_idesc_f16(BM, BN, false, false) : umma_idesc_bf16(BM, BN, false, false);
+            constexpr uint32_t idesc_o = F16 ? umma_idesc_f16(BM, D, false, true) : umma_idesc_bf16(BM, D, false, true);
             // Descriptors are built once; inside the loops only the start-address field moves (the
             // field holds address >> 4 and cannot carry out of its 14 bits within shared memory).
             const uint64_t qd = umma_smem_desc(sQ + t * C::TILE_BYTES, 16, 1024);
@@ -347,8 +351,8 @@ fast_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                             y0 = fmaxf(y0, y[e]); y1 = fmaxf(y1, y[e + 1]); y2 = fmaxf(y2, y[e + 2]); y3 = fmaxf(y3, y[e + 3]);
                             const float p0 = ex2(y[e]), p1 = ex2(y[e + 1]), p2 = ex2(y[e + 2]), p3 = ex2(y[e + 3]);
                             l0 += p0; l1 += p1; l2 += p2; l3 += p3;
-                            pk[16 * c + e / 2] = pack_bf16(p0, p1);
-                            pk[16 * c + e / 2 + 1] = pack_bf16(p2, p3);
+                            pk[16 * c + e / 2] = F16 ? pack_f16(p0, p1) : pack_bf16(p0, p1);
+                            pk[16 * c + e / 2 + 1] = F16 ? pack_f16(p2, p3) : pack_bf16(p2, p3);
                         }
                     }
                     lsum = (l0 + l1) + (l2 + l3);
@@ -394,7 +398,7 @@ fast_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             const uint32_t tO = tmem + lane_base + C::TM_O + t * D + (D / 2) * h;
             const int i = row0[t] + r;
             sts32(my_x, l[t]);
-            if (r == 0 && h == 0) bulk_wait_group_read0();     // the previous store has finished reading the staging tile
+            if (!F16 && r == 0 && h == 0) bulk_wait_group_read0();   // the previous store has finished reading the staging tile
             bar_or(false);
             const float lt = l[t] + lds32f(peer_x);
             mbar_wait(bar(B_OFULL + t), co[t] & 1, status);
@@ -406,35 +410,50 @@ fast_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             tmem_ld_wait();
             tc_fence_before();
             mbar_arrive(bar(B_OEMPTY + t));                    // the next item may overwrite O_t
-#pragma unroll
-            for (int c = 0; c < D / 64; ++c) {
-                uint32_t u[16];
-#pragma unroll
-                for (int e = 0; e < 16; ++e)
-                    u[e] = pack_bf16(__uint_as_float(v[c][2 * e]) * inv, __uint_as_float(v[c][2 * e + 1]) * inv);
-                const int col = (D / 2) * h + 32 * c;          // first output column of this chunk
-                const uint32_t rowaddr = ost + (col >> 6) * C::CHUNK_BYTES + r * 128;
-#pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    const int piece = ((col & 63) >> 3) + q;
-                    sts128(rowaddr + ((piece ^ (r & 7)) << 4), u[4 * q], u[4 * q + 1], u[4 * q + 2], u[4 * q + 3]);
-                }
-            }
             if (h == 0 && i < Sq) LSE[static_cast<size_t>(bh) * Sq + i] = (m_ref[t] + log2f(lt)) * kLn2;
-            fence_proxy_async_smem();
-            bar_or(false);
-            if (r == 0 && h == 0) {
+            if constexpr (F16) {
+                // f32 output: this thread's D/2 contiguous columns of row i, 16-byte stores
+                if (i < Sq) {
+                    float* orow = O32 + (static_cast<size_t>(bh) * Sq + i) * D + (D / 2) * h;
 #pragma unroll
-                for (int ch = 0; ch < C::NCH; ++ch)
-                    tma_store_3d(&tmO, ost + ch * C::CHUNK_BYTES, ch * 64, row0[t], bh);
-                bulk_commit_group();
+                    for (int c = 0; c < D / 64; ++c)
+#pragma unroll
+                        for (int e = 0; e < 8; ++e)
+                            *reinterpret_cast<float4*>(orow + 32 * c + 4 * e) =
+                                make_float4(__uint_as_float(v[c][4 * e]) * inv, __uint_as_float(v[c][4 * e + 1]) * inv,
+                                            __uint_as_float(v[c][4 * e + 2]) * inv, __uint_as_float(v[c][4 * e + 3]) * inv);
+                }
+                bar_or(false);                                 // exchange buffer may be reused
+            } else {
+#pragma unroll
+                for (int c = 0; c < D / 64; ++c) {
+                    uint32_t u[16];
+#pragma unroll
+                    for (int e = 0; e < 16; ++e)
+                        u[e] = pack_bf16(__uint_as_float(v[c][2 * e]) * inv, __uint_as_float(v[c][2 * e + 1]) * inv);
+                    const int col = (D / 2) * h + 32 * c;          // first output column of this chunk
+                    const uint32_t rowaddr = ost + (col >> 6) * C::CHUNK_BYTES + r * 128;
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const int piece = ((col & 63) >> 3) + q;
+                        sts128(rowaddr + ((piece ^ (r & 7)) << 4), u[4 * q], u[4 * q + 1], u[4 * q + 2], u[4 * q + 3]);
+                    }
+                }
+                fence_proxy_async_smem();
+                bar_or(false);
+                if (r == 0 && h == 0) {
+#pragma unroll
+                    for (int ch = 0; ch < C::NCH; ++ch)
+                        tma_store_3d(&tmO, ost + ch * C::CHUNK_BYTES, ch * 64, row0[t], bh);
+                    bulk_commit_group();
+                }
             }
             ++co[t];
         }
         cs[0] += nblk[0];
         cs[1] += nblk[1];
         }   // items
-        if (r == 0 && h == 0) bulk_wait_group_read0();
+        if (!F16 && r == 0 && h == 0) bulk_wait_group_read0();
     }
 
     tc_fence_before();
@@ -442,7 +461,7 @@ fast_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     if (warp == 0) tmem_dealloc(tmem, C::TM_COLS);
 }
 
-template <int D, bool GEN>
+template <int D, bool GEN, bool F16>
 cudaError_t launch_gen(const Problem& p, const void* q, const void* k, const void* v, void* o, float* lse,
                        unsigned* status, cudaStream_t st)
 {
@@ -451,8 +470,9 @@ cudaError_t launch_gen(const Problem& p, const void* q, const void* k, const voi
     if (make_tmap_3d(&tq, q, 2, 1, p.BH(), p.Sq, D, 64, 128)) return cudaErrorInvalidValue;
     if (make_tmap_3d(&tk, k, 2, 1, p.BHkv(), p.Sk, D, 64, 128)) return cudaErrorInvalidValue;
     if (make_tmap_3d(&tv, v, 2, 1, p.BHkv(), p.Sk, D, 64, 128)) return cudaErrorInvalidValue;
-    if (make_tmap_3d(&to, o, 2, 1, p.BH(), p.Sq, D, 64, 128)) return cudaErrorInvalidValue;
-    auto kern = fast_fwd_kernel<D, GEN>;
+    // with f32 output the kernel stores O itself; the map then only has to be a valid one
+    if (make_tmap_3d(&to, F16 ? q : o, 2, 1, p.BH(), p.Sq, D, 64, 128)) return cudaErrorInvalidValue;
+    auto kern = fast_fwd_kernel<D, GEN, F16>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM);
     if (e != cudaSuccess) return e;
     const int n_pairs = (p.Sq + 2 * BM - 1) / (2 * BM);
@@ -466,7 +486,8 @@ cudaError_t launch_gen(const Problem& p, const void* q, const void* k, const voi
     const Dims dm{p.Sq, p.Sk, p.BH(), p.H, p.group(), p.off()};
     // streamed per block and shared between the query tiles of a head: K, V
     const int order = pick_schedule(items, sms, static_cast<double>(p.BHkv()) * p.Sk * D * (2 + 2), dev);
-    kern<<<static_cast<unsigned>(blocks), kThreads, C::SMEM, st>>>(tq, tk, tv, to, lse, dm, n_pairs, p.causal, order,
+    kern<<<static_cast<unsigned>(blocks), kThreads, C::SMEM, st>>>(tq, tk, tv, to, lse, F16 ? static_cast<float*>(o) : nullptr, dm,
+                                                                   n_pairs, p.causal, order,
                                                                    p.scale * kLog2e, status);
     return cudaGetLastError();
 }
@@ -475,11 +496,40 @@ template <int D>
 cudaError_t launch(const Problem& p, const void* q, const void* k, const void* v, void* o, float* lse,
                    unsigned* status, cudaStream_t st)
 {
-    return (p.Hkv != p.H || p.Sq != p.Sk) ? launch_gen<D, true>(p, q, k, v, o, lse, status, st)
-                                          : launch_gen<D, false>(p, q, k, v, o, lse, status, st);
+    return (p.Hkv != p.H || p.Sq != p.Sk) ? launch_gen<D, true, false>(p, q, k, v, o, lse, status, st)
+                                          : launch_gen<D, false, false>(p, q, k, v, o, lse, status, st);
+}
+
+// f32 -> IEEE f16, round to nearest even (HBM-bound, 8 elements per thread and step)
+__global__ void __launch_bounds__(256)
+to_f16_kernel(const float4* __restrict__ in, uint4* __restrict__ out, size_t n8)
+{
+    for (size_t i = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x; i < n8;
+         i += static_cast<size_t>(gridDim.x) * blockDim.x) {
+        const float4 a = in[2 * i], b = in[2 * i + 1];
+        out[i] = make_uint4(pack_f16(a.x, a.y), pack_f16(a.z, a.w), pack_f16(b.x, b.y), pack_f16(b.z, b.w));
+    }
 }
 
 }  // namespace
+
+cudaError_t launch_to_f16(const float* in, void* out, size_t n, cudaStream_t st)
+{
+    const size_t n8 = n / 8;   // callers pass multiples of D >= 32
+    const unsigned blocks = static_cast<unsigned>(n8 / 256 + 1 < 148u * 16u ? n8 / 256 + 1 : 148u * 16u);
+    to_f16_kernel<<<blocks, 256, 0, st>>>(reinterpret_cast<const float4*>(in), static_cast<uint4*>(out), n8);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_fast_fwd_f16(const Problem& p, const void* q16, const void* k16, const void* v16, float* o,
+                                float* lse, unsigned* status, cudaStream_t st)
+{
+    switch (p.D) {
+        case 64:  return launch_gen<64, true, true>(p, q16, k16, v16, o, lse, status, st);
+        case 128: return launch_gen<128, true, true>(p, q16, k16, v16, o, lse, status, st);
+        default:  return cudaErrorNotSupported;
+    }
+}
 
 cudaError_t launch_fast_fwd(const Problem& p, const void* q, const void* k, const void* v, void* o, float* lse,
                             unsigned* status, cudaStream_t st)

@@ -59,6 +59,11 @@ inline int pick_schedule(long long n_items, int sms, double shared_bytes, int de
 // Fast (bf16 tcgen05) kernels.
 cudaError_t launch_fast_fwd(const Problem& p, const void* q, const void* k, const void* v,
                             void* o, float* lse, unsigned* status, cudaStream_t st);
+// Forward of the accelerated policy: q16, k16, v16 are IEEE f16 copies (launch_to_f16) of f32
+// tensors, tensor-core products with f32 accumulation, O and LSE stored as f32.
+cudaError_t launch_to_f16(const float* in, void* out, size_t n, cudaStream_t st);
+cudaError_t launch_fast_fwd_f16(const Problem& p, const void* q16, const void* k16, const void* v16, float* o,
+                                float* lse, unsigned* status, cudaStream_t st);
 cudaError_t launch_fast_bwd(const Problem& p, const void* q, const void* k, const void* v,
                             const void* d_o, const float* lse, const float* delta,
                             float* dq_acc, void* dq, void* dk, void* dv,

@@ -34,7 +34,7 @@ def test_every_declared_symbol_is_exported(lib):
     assert {"mgn_attn_fwd", "mgn_attn_bwd", "mgn_attn_bwd_workspace_bytes", "mgn_attn_check",
             "mgn_status_string", "mgn_version", "mgn_attn_profile_events", "mgn_attn_bwd_noalloc", "mgn_measure_fp32_ffma_tflops",
             "mgn_attn_fast_item_order", "mgn_attn_fwd_ext", "mgn_attn_bwd_ext",
-            "mgn_attn_bwd_deterministic"} <= set(syms)
+            "mgn_attn_bwd_deterministic", "mgn_attn_fwd_accel", "mgn_attn_fwd_accel_workspace_bytes"} <= set(syms)
     for s in syms:
         assert getattr(lib, s) is not None
 
@@ -157,3 +157,24 @@ def test_extended_shape_argument_validation(lib):
     import torch
     if not torch.cuda.is_available():
         assert fx() in (5, 6) and bx() in (5, 6)
+
+
+def test_accel_forward_argument_validation(lib):
+    INVALID, UNSUPPORTED, MISALIGNED, WORKSPACE = 1, 2, 3, 4
+    vp, i, f, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_float, ctypes.c_size_t
+    lib.mgn_attn_fwd_accel.argtypes = [vp] * 5 + [vp, sz] + [i] * 7 + [f, vp]
+    lib.mgn_attn_fwd_accel_workspace_bytes.argtypes = [i] * 6
+    lib.mgn_attn_fwd_accel_workspace_bytes.restype = sz
+    need = lib.mgn_attn_fwd_accel_workspace_bytes(1, 4, 2, 8, 16, 64)
+    assert need >= (4 * 8 + 2 * 2 * 16) * 64 * 2 and need % 256 == 0
+    assert lib.mgn_attn_fwd_accel_workspace_bytes(1, 4, 2, 8, 16, 32) == 0       # D = 32 has no tensor-core path
+
+    def fa(D=64, Hkv=2, ws=A, ws_bytes=1 << 30, q=A):
+        return lib.mgn_attn_fwd_accel(q, A, A, A, A, ws, ws_bytes, 1, 4, Hkv, 8, 16, D, 0, 1.0, None)
+
+    assert fa(D=32) == UNSUPPORTED
+    assert fa(Hkv=3) == INVALID
+    assert fa(q=A + 4) == MISALIGNED
+    assert fa(ws=None) == WORKSPACE
+    assert fa(ws_bytes=need - 1) == WORKSPACE
+    assert fa(ws=A + 16) == WORKSPACE
