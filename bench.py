@@ -180,16 +180,15 @@ def quick_measure_ext(mgn, w, mode, dtype, steps, warmup):
             "sum_tflops": 14.0 * unit / ((fwd_ms + bwd_ms) * 1e-3) / 1e12}
 
 
-def measure_deterministic_bwd(mgn, w, steps, warmup):
-    """Strict mode only: the backward without floating-point atomics (fused dK+dV kernel + separate dQ pass)."""
-    q, k, v, d_o = (t.cuda() for t in synth.make_inputs(w, dtype=torch.float32))
+def measure_deterministic_bwd(mgn, w, mode, dtype, steps, warmup):
+    """The backward without floating-point atomics (fused dK+dV kernel + separate dQ pass)."""
+    q, k, v, d_o = (t.cuda() for t in synth.make_inputs(w, dtype=dtype))
     o = torch.empty_like(q)
     lse = torch.empty(w.B, w.H, w.S, device="cuda", dtype=torch.float32)
     dq, dk, dv = (torch.empty_like(q) for _ in range(3))
-    ws = mgn.alloc_workspace(w.B, w.H, w.S, w.D, mgn.MODE_STRICT_F32)
-    mgn.mgn_attn_fwd(q, k, v, o, lse, w.causal, w.scale, mgn.MODE_STRICT_F32)
-    run = lambda: mgn.mgn_attn_bwd_deterministic(q, k, v, o, d_o, lse, dq, dk, dv, ws, w.causal, w.scale,
-                                                 mgn.MODE_STRICT_F32)
+    ws = mgn.alloc_workspace(w.B, w.H, w.S, w.D, mode)
+    mgn.mgn_attn_fwd(q, k, v, o, lse, w.causal, w.scale, mode)
+    run = lambda: mgn.mgn_attn_bwd_deterministic(q, k, v, o, d_o, lse, dq, dk, dv, ws, w.causal, w.scale, mode)
     for _ in range(warmup):
         run()
     torch.cuda.synchronize()
@@ -568,8 +567,8 @@ def main():
                 r["frac_of_peak"] = r["sum_tflops"] / mode_peak
                 ext[name] = r
             line["ext_shapes"] = ext
+            line["deterministic_bwd"] = measure_deterministic_bwd(mgn, w, mode, dtype, K, args.warmup)
             if args.mode == "strict":
-                line["deterministic_bwd"] = measure_deterministic_bwd(mgn, w, K, args.warmup)
                 if w.D in (64, 128):
                     line["accel_policy"] = measure_accel_policy(mgn, w, K, args.warmup)
         if world == 1 and not args.no_cpu_baseline:

@@ -126,12 +126,12 @@ int mgn_attn_fwd_accel(const float* q, const float* k, const float* v, float* o,
 
 /*
  * Deterministic backward (the "separate pass" form of the dQ kernel: paper Section 3.3 lists dQ
- * beside the fused dK+dV kernel, Section 7.3 profiles them separately).  Same arguments, shapes and
- * results as mgn_attn_bwd_ext, but no floating-point atomics are used: the fused dK+dV kernel runs
- * without the dQ reductions and a second kernel computes dQ with one CTA per query tile, so dq, dk
- * and dv are bit-identical from run to run.  It executes seven matrix products per tile pair instead
- * of five (S and dP are recomputed in the dQ pass).  MGN_MODE_STRICT_F32 only; MGN_MODE_FAST_BF16
- * returns MGN_ERR_UNSUPPORTED.
+ * beside the fused dK+dV kernel, Section 7.3 profiles them separately).  Same arguments, shapes,
+ * modes and results as mgn_attn_bwd_ext, but no floating-point atomics are used: the fused dK+dV
+ * kernel runs without the dQ product and reductions, and a second kernel computes dQ with one CTA per
+ * query tile, so dq, dk and dv are bit-identical from run to run.  It executes seven matrix products
+ * per tile pair instead of five (S and dP are recomputed in the dQ pass).  The workspace holds only
+ * delta, but must still be mgn_attn_bwd_workspace_bytes(B, H, S_q, D, mode) bytes.
  */
 int mgn_attn_bwd_deterministic(const void* q, const void* k, const void* v, const void* o, const void* d_o,
                                const float* lse, void* dq, void* dk, void* dv,

@@ -205,7 +205,6 @@ int mgn_attn_bwd_deterministic(const void* q, const void* k, const void* v, cons
 {
     if (!q || !k || !v || !o || !d_o || !lse || !dq || !dk || !dv) return MGN_ERR_INVALID_ARG;
     if (int r = check_ext(B, H, H_kv, S_q, S_k, D, causal, scale, mode)) return r;
-    if (mode != MGN_MODE_STRICT_F32) return MGN_ERR_UNSUPPORTED;
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(d_o) || !aligned16(lse) ||
         !aligned16(dq) || !aligned16(dk) || !aligned16(dv))
         return MGN_ERR_MISALIGNED;
@@ -219,9 +218,16 @@ int mgn_attn_bwd_deterministic(const void* q, const void* k, const void* v, cons
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const size_t rows = static_cast<size_t>(B) * H * S_q;
     float* delta = static_cast<float*>(workspace);
-    cudaError_t e = mgn::launch_bwd_preprocess(o, d_o, delta, nullptr, rows, D, 0, st);
+    const bool fast = mode == MGN_MODE_FAST_BF16;
+    cudaError_t e = mgn::launch_bwd_preprocess(o, d_o, delta, nullptr, rows, D, fast ? 1 : 0, st);
     if (e != cudaSuccess) return MGN_ERR_CUDA;
     MainKernelTimer timer(st);
+    if (fast) {
+        e = mgn::launch_fast_bwd(p, q, k, v, d_o, lse, delta, nullptr, nullptr, dk, dv, status, st);
+        if (e != cudaSuccess) return MGN_ERR_CUDA;
+        e = mgn::launch_fast_dq(p, q, k, v, d_o, lse, delta, dq, status, st);
+        return e == cudaSuccess ? MGN_OK : MGN_ERR_CUDA;
+    }
     e = mgn::launch_strict_bwd(p, static_cast<const float*>(q), static_cast<const float*>(k),
                                static_cast<const float*>(v), static_cast<const float*>(d_o), lse, delta, nullptr,
                                static_cast<float*>(dk), static_cast<float*>(dv), status, st);

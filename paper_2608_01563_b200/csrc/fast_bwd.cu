@@ -120,7 +120,9 @@ __device__ __forceinline__ int item_index(int c, int k, int G, int n_items, int 
     return it < n_items ? it : -1;
 }
 
-template <int D, bool GEN>
+// WITH_DQ = false leaves the dQ partial product, its drain and the global reductions out: the fused
+// dK+dV kernel of the deterministic backward, whose dQ comes from the separate pass in fast_dq.cu.
+template <int D, bool GEN, bool WITH_DQ>
 __global__ void __launch_bounds__(kThreads, 1)
 fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                 const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmdO,
@@ -274,19 +276,21 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                     const Item<GEN> w = make_item<GEN>(it, dm, causal, order);
                     mbar_wait(bar(B_KV), k & 1, status);
                     mbar_wait(bar(B_DOFULL), g & 1, status);
-                    if (g > 0) mbar_wait(bar(B_DQEMPTY), (g - 1) & 1, status);   // Y: last item's final dQ partial drained
+                    if (WITH_DQ && g > 0) mbar_wait(bar(B_DQEMPTY), (g - 1) & 1, status);   // Y: last item's final dQ partial drained
                     tc_fence_after();
                     mma2();
                     for (int n = 0; n < w.N; ++n, ++g) {
                         const uint64_t qm = mQ + static_cast<uint64_t>(((g & 1) * C::TILE_BYTES) >> 4);
                         mbar_wait(pds_bar(g), (g >> 1) & 1, status);
                         tc_fence_after();
+                        if constexpr (WITH_DQ) {
 #pragma unroll
-                        for (int kk = 0; kk < BLK / 16; ++kk) umma_ss(tYa, mdS + mn_off(kk), mK + mn_off(kk), idesc_dq, kk > 0);
-                        umma_commit(bar(B_DQFULL));
+                            for (int kk = 0; kk < BLK / 16; ++kk) umma_ss(tYa, mdS + mn_off(kk), mK + mn_off(kk), idesc_dq, kk > 0);
+                            umma_commit(bar(B_DQFULL));
+                        }
                         if (n + 1 < w.N) {
                             mbar_wait(bar(B_DOFULL), (g + 1) & 1, status);
-                            mbar_wait(bar(B_DQEMPTY), g & 1, status);            // Y drained
+                            if (WITH_DQ) mbar_wait(bar(B_DQEMPTY), g & 1, status);   // Y drained (else: dP^T(n) was consumed before dS(n) completed)
                             tc_fence_after();
                             mma2();
                         }
@@ -340,7 +344,7 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         const uint32_t tY = tmem + (static_cast<uint32_t>(r & ~31) << 16) + C::TM_Y;
         const uint32_t stage = base + C::OFF_DQ;
         int g = 0;
-        for (int k = 0; k < n_tiers; ++k) {
+        for (int k = 0; WITH_DQ && k < n_tiers; ++k) {
         const int it = item_index(cta, k, G, n_items, order);
         if (it < 0) break;
         const Item<GEN> w = make_item<GEN>(it, dm, causal, order);
@@ -375,7 +379,7 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             }
         }
         }
-        if (r == 0) bulk_wait_group_read0();
+        if (WITH_DQ && r == 0) bulk_wait_group_read0();
     } else {
         // ------------------------------------------------------------------ compute warps
         reg_alloc<128>();
@@ -542,19 +546,22 @@ dq_convert_kernel(const float4* __restrict__ acc, uint2* __restrict__ out, size_
     }
 }
 
-template <int D, bool GEN>
+template <int D, bool GEN, bool WITH_DQ>
 cudaError_t launch_gen(const Problem& p, const void* q, const void* k, const void* v, const void* d_o,
                        const float* lse, const float* delta, float* dq_acc, void* dq, void* dk, void* dv,
                        unsigned* status, cudaStream_t st)
 {
     using C = Cfg<D>;
     CUtensorMap tq, tk, tv, tdo, tdq;
-    if (make_tmap_3d(&tdq, dq_acc, 4, 0, p.BH(), p.Sq, D, 32, BLK)) return cudaErrorInvalidValue;
+    // without the dQ product the map is never used; it only has to be a valid one
+    if (make_tmap_3d(&tdq, WITH_DQ ? static_cast<const void*>(dq_acc) : static_cast<const void*>(delta), 4, 0,
+                     WITH_DQ ? p.BH() : 1, WITH_DQ ? p.Sq : 1, WITH_DQ ? D : 32, 32, WITH_DQ ? BLK : 1))
+        return cudaErrorInvalidValue;
     if (make_tmap_3d(&tq, q, 2, 1, p.BH(), p.Sq, D, 64, BLK)) return cudaErrorInvalidValue;
     if (make_tmap_3d(&tk, k, 2, 1, p.BHkv(), p.Sk, D, 64, BLK)) return cudaErrorInvalidValue;
     if (make_tmap_3d(&tv, v, 2, 1, p.BHkv(), p.Sk, D, 64, BLK)) return cudaErrorInvalidValue;
     if (make_tmap_3d(&tdo, d_o, 2, 1, p.BH(), p.Sq, D, 64, BLK)) return cudaErrorInvalidValue;
-    auto kern = fast_bwd_kernel<D, GEN>;
+    auto kern = fast_bwd_kernel<D, GEN, WITH_DQ>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM);
     if (e != cudaSuccess) return e;
     const int n_kb = (p.Sk + BLK - 1) / BLK;
@@ -573,7 +580,7 @@ cudaError_t launch_gen(const Problem& p, const void* q, const void* k, const voi
                                                                    static_cast<__nv_bfloat16*>(dv), dm, p.causal,
                                                                    order, p.scale, status);
     e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
+    if (e != cudaSuccess || !WITH_DQ) return e;
     const size_t n4 = static_cast<size_t>(p.BH()) * p.Sq * D / 4;
     const unsigned cblocks = static_cast<unsigned>(n4 / 256 + 1 < 148u * 16u ? n4 / 256 + 1 : 148u * 16u);
     dq_convert_kernel<<<cblocks, 256, 0, st>>>(reinterpret_cast<const float4*>(dq_acc), reinterpret_cast<uint2*>(dq), n4,
@@ -586,9 +593,11 @@ cudaError_t launch(const Problem& p, const void* q, const void* k, const void* v
                    const float* lse, const float* delta, float* dq_acc, void* dq, void* dk, void* dv,
                    unsigned* status, cudaStream_t st)
 {
+    if (dq_acc == nullptr)   // fused dK+dV only (deterministic backward): the general-shape build serves every shape
+        return launch_gen<D, true, false>(p, q, k, v, d_o, lse, delta, dq_acc, dq, dk, dv, status, st);
     return (p.Hkv != p.H || p.Sq != p.Sk)
-               ? launch_gen<D, true>(p, q, k, v, d_o, lse, delta, dq_acc, dq, dk, dv, status, st)
-               : launch_gen<D, false>(p, q, k, v, d_o, lse, delta, dq_acc, dq, dk, dv, status, st);
+               ? launch_gen<D, true, true>(p, q, k, v, d_o, lse, delta, dq_acc, dq, dk, dv, status, st)
+               : launch_gen<D, false, true>(p, q, k, v, d_o, lse, delta, dq_acc, dq, dk, dv, status, st);
 }
 
 }  // namespace

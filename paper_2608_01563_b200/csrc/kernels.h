@@ -69,4 +69,9 @@ cudaError_t launch_fast_bwd(const Problem& p, const void* q, const void* k, cons
                             float* dq_acc, void* dq, void* dk, void* dv,
                             unsigned* status, cudaStream_t st);
 
+// Deterministic fast backward: launch_fast_bwd with dq_acc == nullptr runs the fused dK+dV kernel
+// without the dQ product and reductions (dq is not touched), and this separate pass computes dQ.
+cudaError_t launch_fast_dq(const Problem& p, const void* q, const void* k, const void* v, const void* d_o,
+                           const float* lse, const float* delta, void* dq, unsigned* status, cudaStream_t st);
+
 }  // namespace mgn

@@ -150,7 +150,7 @@ def test_extended_shape_argument_validation(lib):
     lib.mgn_attn_bwd_deterministic.argtypes = lib.mgn_attn_bwd_ext.argtypes
     det = lambda mode=0, H=4, Hkv=2: lib.mgn_attn_bwd_deterministic(*([A] * 9), A, 1 << 30, 1, H, Hkv, 8, 16, 64, 0,
                                                                    1.0, mode, None)
-    assert det(mode=1) == UNSUPPORTED          # strict mode only
+    assert det(mode=7) == INVALID
     assert det(H=4, Hkv=3) == INVALID
     need = lib.mgn_attn_bwd_workspace_bytes(1, 4, 8, 64, 0)       # sized by the query side
     assert bx(ws_bytes=need - 1) == WORKSPACE
