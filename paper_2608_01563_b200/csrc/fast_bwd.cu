@@ -325,8 +325,8 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
                         const bool ok = i + e < Sq;
-                        l2[e] = ok ? LSE[row0 + i + e] * kLog2e : INFINITY;
-                        dl[e] = ok ? DELTA[row0 + i + e] : 0.f;
+                        l2[e] = ok ? -LSE[row0 + i + e] * kLog2e : -INFINITY;   // negated: added in the exponent
+                        dl[e] = ok ? -DELTA[row0 + i + e] : 0.f;                  // negated: added to dP
                     }
                     sts128(buf + lane * 16, __float_as_uint(l2[0]), __float_as_uint(l2[1]), __float_as_uint(l2[2]),
                            __float_as_uint(l2[3]));
@@ -391,6 +391,7 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         uint32_t pk[32];                                                     // P^T of the current pair, packed bf16
 
         // P^T = exp2(S^T c - lse) of pair n: bf16 into X (A operand of dV) and into pk (for dS)
+        const uint64_t c2x2 = f2_pack(c2, c2);
         auto exp_phase = [&](const Item<GEN>& w, int n, int g) {
             // key lane r (key j0 + r) is visible to query column c (query i0 + c) iff r <= c + dlt
             const int dlt = w.i0(n) + coff - w.j0;
@@ -407,11 +408,17 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                 float p[32];
 #pragma unroll
                 for (int e4 = 0; e4 < 8; ++e4) {
+                    // s c - lse in the log2 domain, two columns per instruction (the buffer holds -lse)
                     const float4 l4 = lds128(statL + (half * 64 + 32 * c + 4 * e4) * 4);
-                    p[4 * e4 + 0] = ex2(fmaf(__uint_as_float(v[4 * e4 + 0]), c2, -l4.x));
-                    p[4 * e4 + 1] = ex2(fmaf(__uint_as_float(v[4 * e4 + 1]), c2, -l4.y));
-                    p[4 * e4 + 2] = ex2(fmaf(__uint_as_float(v[4 * e4 + 2]), c2, -l4.z));
-                    p[4 * e4 + 3] = ex2(fmaf(__uint_as_float(v[4 * e4 + 3]), c2, -l4.w));
+                    float y0, y1, y2, y3;
+                    f2_unpack(f2_fma(f2_pack(__uint_as_float(v[4 * e4 + 0]), __uint_as_float(v[4 * e4 + 1])), c2x2,
+                                     f2_pack(l4.x, l4.y)), y0, y1);
+                    f2_unpack(f2_fma(f2_pack(__uint_as_float(v[4 * e4 + 2]), __uint_as_float(v[4 * e4 + 3])), c2x2,
+                                     f2_pack(l4.z, l4.w)), y2, y3);
+                    p[4 * e4 + 0] = ex2(y0);
+                    p[4 * e4 + 1] = ex2(y1);
+                    p[4 * e4 + 2] = ex2(y2);
+                    p[4 * e4 + 3] = ex2(y3);
                 }
                 if (diag) {   // keep key j <= query i, i.e. lane r <= column
 #pragma unroll
@@ -454,10 +461,14 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                 for (int e4 = 0; e4 < 8; ++e4) {
                     const float4 d4 = lds128(statD + (half * 64 + 32 * c + 4 * e4) * 4);
                     const uint32_t k0 = pk[16 * c + 2 * e4], k1 = pk[16 * c + 2 * e4 + 1];
-                    const float a0 = __uint_as_float(k0 << 16) * (__uint_as_float(v[4 * e4 + 0]) - d4.x);
-                    const float a1 = __uint_as_float(k0 & 0xffff0000u) * (__uint_as_float(v[4 * e4 + 1]) - d4.y);
-                    const float a2 = __uint_as_float(k1 << 16) * (__uint_as_float(v[4 * e4 + 2]) - d4.z);
-                    const float a3 = __uint_as_float(k1 & 0xffff0000u) * (__uint_as_float(v[4 * e4 + 3]) - d4.w);
+                    // P (dP - delta), two columns per instruction (the buffer holds -delta)
+                    float a0, a1, a2, a3;
+                    f2_unpack(f2_mul(f2_pack(__uint_as_float(k0 << 16), __uint_as_float(k0 & 0xffff0000u)),
+                                     f2_add(f2_pack(__uint_as_float(v[4 * e4 + 0]), __uint_as_float(v[4 * e4 + 1])),
+                                            f2_pack(d4.x, d4.y))), a0, a1);
+                    f2_unpack(f2_mul(f2_pack(__uint_as_float(k1 << 16), __uint_as_float(k1 & 0xffff0000u)),
+                                     f2_add(f2_pack(__uint_as_float(v[4 * e4 + 2]), __uint_as_float(v[4 * e4 + 3])),
+                                            f2_pack(d4.z, d4.w))), a2, a3);
                     u[2 * e4] = pack_bf16(a0, a1);
                     u[2 * e4 + 1] = pack_bf16(a2, a3);
                 }
