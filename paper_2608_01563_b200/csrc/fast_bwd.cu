@@ -2,14 +2,14 @@
 // accumulation in tensor memory (paper Section 3.3 "dQ, and fused dK+dV kernels"; Section 7.3
 // FlashGradKV / FlashGradQ; Section 4.2 for the reduced-input arithmetic contract).
 //
-// Single pass, persistent: one CTA per SM walks over work items (one 128-key block of one head
-// each, heaviest first, dealt out in snake order).  Per item it keeps the K, V tiles resident in
+// Single pass, persistent: one CTA per SM walks over work items (one 128-key block of one
+// key/value head each; two item orders, see below).  Per item it keeps the K, V tiles resident in
 // shared memory, holds the dK and dV accumulators of that block in tensor memory, and walks over
-// the 128-row query blocks (from the diagonal down when causal).  Every barrier keeps counting
-// across items (g = running pair count, k = running item count), so the producer and the issuers
-// start the next item (loads, first S^T and dP^T) while the compute warps write out dK/dV.  All score-shaped tiles are computed TRANSPOSED
-// (lanes = keys, columns = queries) so that P^T can feed dV = P^T dO straight from tensor
-// memory.  Per (key block, query block) pair:
+// (query head of the group, 128-row query block) pairs -- from the first block that sees the key block
+// when causal.  Every barrier keeps counting across items (g = running pair count, k = running item
+// count), so the producer and the issuers start the next item (loads, first S^T and dP^T) while the
+// compute warps write out dK/dV.  All score-shaped tiles are computed TRANSPOSED (lanes = keys,
+// columns = queries) so that P^T can feed dV = P^T dO straight from tensor memory.  Per pair:
 //   MMA1  S^T  = K Q^T            -> X            MMA2  dP^T = V dO^T -> Y
 //   compute (256 threads, one key lane x 64 query columns each):
 //         P^T = exp2(S^T c - LSE) -> bf16 into X;  dS^T = P^T (dP^T - delta) -> bf16 into shared
@@ -27,11 +27,14 @@
 // is in tensor memory (before dS(n) exists), so the next scores are ready when the compute warps
 // come back for them; issuer B runs MMA6(n), MMA2(n+1), MMA5(n) once dS(n) is in shared memory
 // (the dQ partial first so its drain starts early, dP^T of the next pair as soon as Y has been
-// drained, dK last: nothing waits for it).  The compute warps then never wait for the tensor core
-// in steady state: exp(n+1) and dS(n+1) run back to back.
+// drained, then dK).  Y holds dP^T and then the dQ partial, and all 512 tensor-memory columns are
+// taken at D = 128, so each pair runs the serial cycle  dS -> MMA6 -> drain -> MMA2 -> dS.
+// Item epilogue: dK (scaled) and dV leave through bf16 registers, the idle dS buffer and coalesced
+// 16-byte stores.
 // Tensor memory: X [0,128)  Y [128,256)  dK [256,256+D)  dV [256+D,256+2D).
-// Warp roles (512 threads): warp 0 TMA producer, warps 1-2 MMA issuers, warps 4-11 compute,
-// warps 12-15 dQ drain; register budgets are rebalanced with setmaxnreg (104 / 128 / 128 / 152).
+// Warp roles (512 threads): warp 0 TMA producer, warps 1-2 MMA issuers, warp 3 row statistics
+// (LSE, delta staged two pairs ahead), warps 4-11 compute, warps 12-15 dQ drain; register budgets
+// are rebalanced with setmaxnreg (104 / 128 / 128 / 152).
 #include <cuda_bf16.h>
 
 #include "kernels.h"

@@ -3,11 +3,11 @@
 // forward"; Section 4.2: the validated reduced-input path with f32 accumulation).
 //
 // Persistent kernel: one CTA per SM walks over work items (two 128-row query tiles of one head
-// each, heaviest first, dealt out in snake order so that every CTA gets the same amount of
-// work) and, per item, over 128-key blocks.  All barriers keep counting across items, so the
-// producer prefetches the next item's Q/K/V and the issuers compute its first scores while the
-// softmax warps are still writing the previous item's output: the per-item fill and drain
-// (about 10 us against 2 us per key block) is hidden instead of paid by every CTA.
+// each; two item orders, see make_item) and, per item, over 128-key blocks of that head's
+// key/value head.  All barriers keep counting across items, so the producer prefetches the next
+// item's Q/K/V and the issuers compute its first scores while the softmax warps are still writing
+// the previous item's output: most of the per-item fill and drain is hidden instead of paid by
+// every CTA.
 // Warp roles (384 threads):
 //   warp 0      TMA producer: Q tiles once, then K and V blocks through a 2-stage ring
 //   warps 1, 2  MMA issuers, one per query tile: S_t = Q_t K^T (operands in shared memory) and
