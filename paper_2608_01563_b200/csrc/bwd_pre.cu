@@ -10,6 +10,27 @@
 namespace mgn {
 namespace {
 
+// L2 eviction hints: the accumulator that the next kernel reduces into should stay in L2, the
+// streamed inputs should not push it out.
+__device__ __forceinline__ uint64_t l2_policy_keep() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ uint64_t l2_policy_stream() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ void st_hint(float4* a, float4 v, uint64_t pol) {
+    asm volatile("st.global.L2::cache_hint.v4.f32 [%0], {%1,%2,%3,%4}, %5;" ::"l"(a), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w), "l"(pol) : "memory");
+}
+__device__ __forceinline__ uint4 ld_hint(const uint4* a, uint64_t pol) {
+    uint4 v;
+    asm volatile("ld.global.nc.L2::cache_hint.v4.u32 {%0,%1,%2,%3}, [%4], %5;" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(a), "l"(pol));
+    return v;
+}
+
 template <int LANES, bool BF16>
 __global__ void __launch_bounds__(256)
 bwd_preprocess_kernel(const uint4* __restrict__ o, const uint4* __restrict__ d_o, float* __restrict__ delta,
@@ -18,6 +39,7 @@ bwd_preprocess_kernel(const uint4* __restrict__ o, const uint4* __restrict__ d_o
     constexpr int ROWS_PER_BLOCK = 256 / LANES;
     const int lane = threadIdx.x % LANES;
     const int sub = threadIdx.x / LANES;
+    const uint64_t keep = l2_policy_keep(), stream = l2_policy_stream();
     for (size_t r0 = static_cast<size_t>(blockIdx.x) * ROWS_PER_BLOCK; r0 < rows;
          r0 += static_cast<size_t>(gridDim.x) * ROWS_PER_BLOCK) {
         const size_t r = r0 + sub;
@@ -26,9 +48,9 @@ bwd_preprocess_kernel(const uint4* __restrict__ o, const uint4* __restrict__ d_o
             constexpr int ZPL = BF16 ? 2 : 1;      // float4 stores per lane to cover a row of D floats
 #pragma unroll
             for (int t = 0; t < ZPL; ++t)
-                if (zero) zero[(r * LANES + lane) * ZPL + t] = make_float4(0.f, 0.f, 0.f, 0.f);
-            const uint4 a = __ldg(o + r * LANES + lane);
-            const uint4 b = __ldg(d_o + r * LANES + lane);
+                if (zero) st_hint(&zero[(r * LANES + lane) * ZPL + t], make_float4(0.f, 0.f, 0.f, 0.f), keep);
+            const uint4 a = ld_hint(o + r * LANES + lane, stream);
+            const uint4 b = ld_hint(d_o + r * LANES + lane, stream);
             if constexpr (BF16) {
                 const __nv_bfloat162* pa = reinterpret_cast<const __nv_bfloat162*>(&a);
                 const __nv_bfloat162* pb = reinterpret_cast<const __nv_bfloat162*>(&b);
