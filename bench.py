@@ -78,7 +78,7 @@ def whole_job_tflops(w, world, steps, total_ms):
 class ClockSampler:
     QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
-             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap,timestamp")
 
     def __init__(self, gpu_index):
         self.gpu_index = gpu_index
@@ -96,7 +96,17 @@ class ClockSampler:
         except Exception:
             self.proc = None
 
-    def stop(self):
+    @staticmethod
+    def _epoch(stamp):
+        """nvidia-smi's 'YYYY/MM/DD HH:MM:SS.mmm' (local time) as seconds since the epoch."""
+        try:
+            head, _, ms = stamp.partition(".")
+            return time.mktime(time.strptime(head, "%Y/%m/%d %H:%M:%S")) + float("0." + (ms or "0"))
+        except ValueError:
+            return None
+
+    def stop(self, t_begin=None, t_end=None):
+        """Statistics over the samples taken between the two wall-clock times (all samples if none given)."""
         out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
         if self.proc is None:
             return out
@@ -111,6 +121,10 @@ class ClockSampler:
             parts = [p.strip() for p in line.split(",")]
             if len(parts) < 9:
                 continue
+            if t_begin is not None and len(parts) >= 10:
+                t = self._epoch(parts[9])
+                if t is not None and not (t_begin <= t <= t_end):
+                    continue
             try:
                 sm.append(float(parts[1])); mx.append(float(parts[2])); power.append(float(parts[3]))
             except ValueError:
@@ -415,6 +429,7 @@ def main():
         sampler.start()
         time.sleep(0.3)
     barrier()
+    t_load0 = time.time()
     e_step0.record()
     for i in range(K):
         a, b = pairs["fwd_main"][i]
@@ -425,9 +440,19 @@ def main():
         mgn.mgn_attn_profile_events(a.cuda_event, b.cuda_event)
         mgn.mgn_attn_bwd(qd, kd, vd, o, dod, lse, dq, dk, dv, ws, w.causal, w.scale, mode)
     e_step1.record()
-    barrier()
     mgn.mgn_attn_profile_events(None, None)
-    clocks = sampler.stop() if rank == 0 else None
+    # The timed region lasts tens of milliseconds, about one sampling period: the same step loop keeps
+    # running (untimed) for a little longer so that the clock record holds samples taken under this load.
+    barrier()
+    t_cont = time.time()
+    while time.time() - t_cont < 0.4:
+        for _ in range(10):
+            step()
+        torch.cuda.synchronize()
+    t_load1 = time.time()
+    clocks = sampler.stop(t_load0, t_load1) if rank == 0 else None
+    if clocks is not None:
+        clocks["window"] = "samples between the start of the timed region and the end of a 0.4 s continuation of the same step loop"
     mgn.mgn_attn_check()
 
     total_ms = e_step0.elapsed_time(e_step1)
