@@ -38,6 +38,7 @@
 #include <cuda_bf16.h>
 
 #include "kernels.h"
+#include "fast_items.cuh"
 #include "umma.cuh"
 
 namespace mgn {
@@ -81,11 +82,6 @@ enum { B_KV = 0, B_QFULL = 1, B_QEMPTY = 3, B_DOFULL = 5, B_DOEMPTY = 6, B_SFULL
 //     remaining block, so that two consecutive items always weigh the same; CTA c takes the item
 //     pairs c, c+G, c+2G, ...  The CTAs running at one time share a few heads, whose dQ accumulator,
 //     Q and dO stay in L2.  Balanced only when there are many item pairs per CTA.
-// Shapes: q, d_o, dq [BH = B*H, Sq, D]; k, v, dk, dv [BHkv = B*H/G, Sk, D]; query head h reads
-// key/value head h / G; causal: key j is visible to query i iff j <= i + off, off = Sk - Sq >= 0.
-struct Dims {
-    int Sq, Sk, BH, H, G, off;
-};
 // An item is one key block of one key/value head; its pairs run over the query heads of the group
 // and, for each, over the query blocks that see the key block.
 // GEN = false is the square multi-head case (Sk == Sq, G == 1): the head mapping, the offset and the
@@ -116,11 +112,6 @@ __device__ __forceinline__ Item<GEN> make_item(int it, const Dims& dm, int causa
     w.nq = nqb - w.qb0;                                   // query blocks visited per head (>= 1)
     w.N = G * w.nq;
     return w;
-}
-// k-th item of CTA c out of G, -1 past the end (then also for every larger k).
-__device__ __forceinline__ int item_index(int c, int k, int G, int n_items, int order) {
-    const int it = order == 0 ? k * G + ((k & 1) ? (G - 1 - c) : c) : 2 * (c + G * (k >> 1)) + (k & 1);
-    return it < n_items ? it : -1;
 }
 
 // WITH_DQ = false leaves the dQ partial product, its drain and the global reductions out: the fused

@@ -17,6 +17,7 @@
 #include <cuda_bf16.h>
 
 #include "kernels.h"
+#include "fast_items.cuh"
 #include "umma.cuh"
 
 namespace mgn {
@@ -44,9 +45,6 @@ struct Cfg {
 enum { B_Q = 0, B_KFULL = 1, B_KEMPTY = 3, B_VFULL = 5, B_VEMPTY = 7, B_SPFULL = 9, B_DSFULL = 10, B_DQFULL = 11,
        B_COUNT = 12 };
 
-struct Dims {
-    int Sq, Sk, BH, H, G, off;
-};
 
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1)

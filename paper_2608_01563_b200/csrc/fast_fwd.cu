@@ -26,6 +26,7 @@
 // any reference point works for a softmax as long as nothing overflows.  The two threads of a
 // row agree on that through a barrier with an OR-reduction per block.
 #include "kernels.h"
+#include "fast_items.cuh"
 #include "umma.cuh"
 
 namespace mgn {
@@ -64,11 +65,6 @@ enum { B_Q = 0, B_KFULL = 1, B_KEMPTY = 3, B_VFULL = 5, B_VEMPTY = 7, B_SFULL = 
 // every head.  Order 1 (head-major): the tile pairs of a head are consecutive, heaviest and lightest
 // remaining in turn, and CTA c takes the item pairs c, c+G, ... -- the CTAs running at one time
 // share the K, V of a few heads, which then stay in L2.  The launcher chooses (pick_schedule).
-// Shapes: q, o [BH = B*H, Sq, D]; k, v [B*H/G, Sk, D]; query head h reads key/value head h / G;
-// causal: key j is visible to query i iff j <= i + off, off = Sk - Sq >= 0.
-struct Dims {
-    int Sq, Sk, BH, H, G, off;
-};
 struct Item {
     int pair, bh, bhk, row0[2], nblk[2], n_max;
 };
@@ -96,11 +92,6 @@ __device__ __forceinline__ Item make_item(int it, const Dims& dm, int n_pairs, i
     }
     w.n_max = max(w.nblk[0], w.nblk[1]);
     return w;
-}
-// k-th item of CTA c out of G: tiers of G items, odd tiers dealt backwards (snake), -1 past the end.
-__device__ __forceinline__ int item_index(int c, int k, int G, int n_items, int order) {
-    const int it = order == 0 ? k * G + ((k & 1) ? (G - 1 - c) : c) : 2 * (c + G * (k >> 1)) + (k & 1);
-    return it < n_items ? it : -1;
 }
 
 // F16 = true is the forward of the accelerated policy (paper Section 4.2, table "Arithmetic

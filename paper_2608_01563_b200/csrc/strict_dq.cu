@@ -11,7 +11,7 @@
 //   C. dQ += dS K (contraction over the keys of the tile), accumulated in registers over all tiles.
 // Thread layout, tile layout in shared memory and the two phases are those of strict_bwd.cu.
 #include "kernels.h"
-#include "ptx.cuh"
+#include "strict_tiles.cuh"
 
 namespace mgn {
 namespace {
@@ -32,25 +32,6 @@ struct DqCfg {
     static constexpr int SMEM = 2 * KV_BYTES + 2 * Q_BYTES + P_BYTES + 64 + 1024;
 };
 
-// d columns owned by column group tc: D=32 -> {2tc, 2tc+1}; else {4tc + 64e + 0..3}.
-template <int D, int R>
-__device__ __forceinline__ void load_row_cols(uint32_t tile, int r, int r7, int tc, float (&out)[D / 16]) {
-    if constexpr (D == 32) {
-        const float2 t = lds64(tile + r * 128 + (((tc >> 1) ^ r7) << 4) + (tc & 1) * 8);
-        out[0] = t.x; out[1] = t.y;
-    } else {
-#pragma unroll
-        for (int e = 0; e < D / 64; ++e) {
-            const int piece = tc + 16 * e;
-            const float4 t = lds128(tile + (piece >> 3) * (R * 128) + r * 128 + (((piece & 7) ^ r7) << 4));
-            out[4 * e + 0] = t.x; out[4 * e + 1] = t.y; out[4 * e + 2] = t.z; out[4 * e + 3] = t.w;
-        }
-    }
-}
-
-__device__ __forceinline__ float f4_get(const float4& v, int u) {
-    return u == 0 ? v.x : u == 1 ? v.y : u == 2 ? v.z : v.w;
-}
 
 template <int D, int BM, int BN, int THREADS>
 __global__ void __launch_bounds__(THREADS, THREADS == 128 ? 2 : 1)
