@@ -85,6 +85,27 @@ size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 size_t ws_delta_bytes(size_t rows) { return align_up(rows * sizeof(float), 256); }
 
 }  // namespace
+extern "C" size_t mgn_attn_bwd_workspace_bytes(int B, int H, int S, int D, int mode);
+namespace {
+
+// Argument checks shared by the backward entry points, in the documented order, then the device set-up.
+int check_bwd_call(const void* q, const void* k, const void* v, const void* o, const void* d_o, const float* lse,
+                   const void* dq, const void* dk, const void* dv, const void* workspace, size_t workspace_bytes,
+                   int B, int H, int H_kv, int S_q, int S_k, int D, int causal, float scale, int mode,
+                   unsigned** status)
+{
+    if (!q || !k || !v || !o || !d_o || !lse || !dq || !dk || !dv) return MGN_ERR_INVALID_ARG;
+    if (int r = check_ext(B, H, H_kv, S_q, S_k, D, causal, scale, mode)) return r;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(d_o) || !aligned16(lse) ||
+        !aligned16(dq) || !aligned16(dk) || !aligned16(dv))
+        return MGN_ERR_MISALIGNED;
+    const size_t need = mgn_attn_bwd_workspace_bytes(B, H, S_q, D, mode);
+    if (!workspace || workspace_bytes < need) return MGN_ERR_WORKSPACE;
+    if (reinterpret_cast<uintptr_t>(workspace) & 255u) return MGN_ERR_WORKSPACE;
+    return device_setup(status);
+}
+
+}  // namespace
 
 extern "C" {
 
@@ -163,16 +184,10 @@ int mgn_attn_bwd_ext(const void* q, const void* k, const void* v, const void* o,
                      int B, int H, int H_kv, int S_q, int S_k, int D, int causal, float scale, int mode,
                      void* stream)
 {
-    if (!q || !k || !v || !o || !d_o || !lse || !dq || !dk || !dv) return MGN_ERR_INVALID_ARG;
-    if (int r = check_ext(B, H, H_kv, S_q, S_k, D, causal, scale, mode)) return r;
-    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(d_o) || !aligned16(lse) ||
-        !aligned16(dq) || !aligned16(dk) || !aligned16(dv))
-        return MGN_ERR_MISALIGNED;
-    const size_t need = mgn_attn_bwd_workspace_bytes(B, H, S_q, D, mode);
-    if (!workspace || workspace_bytes < need) return MGN_ERR_WORKSPACE;
-    if (reinterpret_cast<uintptr_t>(workspace) & 255u) return MGN_ERR_WORKSPACE;
     unsigned* status = nullptr;
-    if (int r = device_setup(&status)) return r;
+    if (int r = check_bwd_call(q, k, v, o, d_o, lse, dq, dk, dv, workspace, workspace_bytes, B, H, H_kv, S_q, S_k, D,
+                               causal, scale, mode, &status))
+        return r;
 
     const mgn::Problem p{B, H, H_kv, S_q, S_k, D, causal, scale};
     cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -203,16 +218,10 @@ int mgn_attn_bwd_deterministic(const void* q, const void* k, const void* v, cons
                                int B, int H, int H_kv, int S_q, int S_k, int D, int causal, float scale, int mode,
                                void* stream)
 {
-    if (!q || !k || !v || !o || !d_o || !lse || !dq || !dk || !dv) return MGN_ERR_INVALID_ARG;
-    if (int r = check_ext(B, H, H_kv, S_q, S_k, D, causal, scale, mode)) return r;
-    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(d_o) || !aligned16(lse) ||
-        !aligned16(dq) || !aligned16(dk) || !aligned16(dv))
-        return MGN_ERR_MISALIGNED;
-    const size_t need = mgn_attn_bwd_workspace_bytes(B, H, S_q, D, mode);
-    if (!workspace || workspace_bytes < need) return MGN_ERR_WORKSPACE;
-    if (reinterpret_cast<uintptr_t>(workspace) & 255u) return MGN_ERR_WORKSPACE;
     unsigned* status = nullptr;
-    if (int r = device_setup(&status)) return r;
+    if (int r = check_bwd_call(q, k, v, o, d_o, lse, dq, dk, dv, workspace, workspace_bytes, B, H, H_kv, S_q, S_k, D,
+                               causal, scale, mode, &status))
+        return r;
 
     const mgn::Problem p{B, H, H_kv, S_q, S_k, D, causal, scale};
     cudaStream_t st = static_cast<cudaStream_t>(stream);
