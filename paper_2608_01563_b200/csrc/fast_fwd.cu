@@ -3,7 +3,7 @@
 // forward"; Section 4.2: the validated reduced-input path with f32 accumulation).
 //
 // Persistent kernel: one CTA per SM walks over work items (two 128-row query tiles of one head
-// each; two item orders, see make_item) and, per item, over 128-key blocks of that head's
+// each -- one tile when there would be fewer items than SMs; two item orders, see make_item) and, per item, over 128-key blocks of that head's
 // key/value head.  All barriers keep counting across items, so the producer prefetches the next
 // item's Q/K/V and the issuers compute its first scores while the softmax warps are still writing
 // the previous item's output: most of the per-item fill and drain is hidden instead of paid by
@@ -70,7 +70,7 @@ struct Item {
 };
 // GEN = false is the square multi-head case (Sk == Sq, G == 1): offsets and the head mapping fold away.
 template <bool GEN>
-__device__ __forceinline__ Item make_item(int it, const Dims& dm, int n_pairs, int causal, int order) {
+__device__ __forceinline__ Item make_item(int it, const Dims& dm, int n_pairs, int tpi, int causal, int order) {
     const int BH = dm.BH;
     const int Sk = GEN ? dm.Sk : dm.Sq, off = GEN ? dm.off : 0;
     Item w;
@@ -86,8 +86,8 @@ __device__ __forceinline__ Item make_item(int it, const Dims& dm, int n_pairs, i
     const int n_kb = (Sk + BN - 1) / BN;
 #pragma unroll
     for (int t = 0; t < 2; ++t) {
-        w.row0[t] = w.pair * 2 * BM + t * BM;
-        if (w.row0[t] >= dm.Sq) w.nblk[t] = 0;
+        w.row0[t] = (w.pair * tpi + t) * BM;          // tpi = tiles per item: 2, or 1 when items would be too few
+        if (t >= tpi || w.row0[t] >= dm.Sq) w.nblk[t] = 0;
         else w.nblk[t] = causal ? min(n_kb, (min(w.row0[t] + BM, dm.Sq) - 1 + off) / BN + 1) : n_kb;
     }
     w.n_max = max(w.nblk[0], w.nblk[1]);
@@ -101,7 +101,7 @@ template <int D, bool GEN, bool F16>
 __global__ void __launch_bounds__(kThreads, 1)
 fast_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                 const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO,
-                float* __restrict__ LSE, float* __restrict__ O32, const Dims dm, int n_pairs, int causal, int order,
+                float* __restrict__ LSE, float* __restrict__ O32, const Dims dm, int n_pairs, int tpi, int causal, int order,
                 float c2, unsigned* status)
 {
     using C = Cfg<D>;
@@ -145,7 +145,7 @@ fast_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             for (int k = 0; k < n_tiers; ++k) {
                 const int it = item_index(cta, k, G, n_items, order);
                 if (it < 0) break;
-                const Item w = make_item<GEN>(it, dm, n_pairs, causal, order);
+                const Item w = make_item<GEN>(it, dm, n_pairs, tpi, causal, order);
                 mbar_wait(bar(B_QEMPTY), (k & 1) ^ 1, status);   // both issuers are done with the previous Q tiles
                 const int nq = (w.nblk[1] > 0) ? 2 : 1;
                 mbar_arrive_expect_tx(bar(B_Q), nq * C::TILE_BYTES);
@@ -203,7 +203,7 @@ fast_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             for (int k = 0; k < n_tiers; ++k) {
                 const int it = item_index(cta, k, G, n_items, order);
                 if (it < 0) break;
-                const Item w = make_item<GEN>(it, dm, n_pairs, causal, order);
+                const Item w = make_item<GEN>(it, dm, n_pairs, tpi, causal, order);
                 const int nb = w.nblk[t];
                 mbar_wait(bar(B_Q), k & 1, status);
                 mbar_wait(bar(B_KFULL + (g & 1)), (g >> 1) & 1, status);
@@ -265,7 +265,7 @@ fast_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         for (int k = 0; k < n_tiers; ++k) {
         const int it = item_index(cta, k, G, n_items, order);
         if (it < 0) break;
-        const Item w = make_item<GEN>(it, dm, n_pairs, causal, order);
+        const Item w = make_item<GEN>(it, dm, n_pairs, tpi, causal, order);
         const int bh = w.bh, n_max = w.n_max;
         const int row0[2] = {w.row0[0], w.row0[1]}, nblk[2] = {w.nblk[0], w.nblk[1]};
         float m_ref[2] = {-INFINITY, -INFINITY}, l[2] = {0.f, 0.f};
@@ -466,19 +466,23 @@ cudaError_t launch_gen(const Problem& p, const void* q, const void* k, const voi
     auto kern = fast_fwd_kernel<D, GEN, F16>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM);
     if (e != cudaSuccess) return e;
-    const int n_pairs = (p.Sq + 2 * BM - 1) / (2 * BM);
-    const long long items = static_cast<long long>(n_pairs) * p.BH();
-    if (items > 0x7fffffffLL) return cudaErrorInvalidValue;
     int dev = 0, sms = 0;
     if (cudaGetDevice(&dev) != cudaSuccess ||
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
         return cudaErrorInvalidValue;
+    // An item is two query tiles of a head (their softmax and products interleave); with fewer such
+    // items than SMs an item is one tile instead, so that twice as many SMs have work.
+    const int n_tiles = (p.Sq + BM - 1) / BM;
+    const int tpi = (static_cast<long long>((n_tiles + 1) / 2) * p.BH() < sms && n_tiles > 1) ? 1 : 2;
+    const int n_pairs = (n_tiles + tpi - 1) / tpi;
+    const long long items = static_cast<long long>(n_pairs) * p.BH();
+    if (items > 0x7fffffffLL) return cudaErrorInvalidValue;
     const long long blocks = items < sms ? items : sms;       // persistent: one CTA per SM
     const Dims dm{p.Sq, p.Sk, p.BH(), p.H, p.group(), p.off()};
     // streamed per block and shared between the query tiles of a head: K, V
     const int order = pick_schedule(items, sms, static_cast<double>(p.BHkv()) * p.Sk * D * (2 + 2), dev);
     kern<<<static_cast<unsigned>(blocks), kThreads, C::SMEM, st>>>(tq, tk, tv, to, lse, F16 ? static_cast<float*>(o) : nullptr, dm,
-                                                                   n_pairs, p.causal, order,
+                                                                   n_pairs, tpi, p.causal, order,
                                                                    p.scale * kLog2e, status);
     return cudaGetLastError();
 }
