@@ -138,3 +138,25 @@ def test_softmax_rows_and_shape_errors():
         orc.attn_fwd_ext(rand(1, 2, 9, 4), rand(1, 2, 4, 4), rand(1, 2, 4, 4), True, 1.0)   # causal, S_q > S_k
     with pytest.raises(AssertionError):
         orc.attn_fwd_ext(rand(1, 3, 4, 4), rand(1, 2, 4, 4), rand(1, 2, 4, 4), False, 1.0)  # H % H_kv != 0
+
+
+def test_hand_worked_grouped_head_example():
+    """tests/golden/hand_case_grouped_heads.json: exact fractions derived by hand (see its citation)."""
+    import json
+    import os
+    fx = json.load(open(os.path.join(os.path.dirname(__file__), "golden", "hand_case_grouped_heads.json")))
+    q = np.array(fx["Q"]).reshape(1, 2, 1, 1)
+    k = np.array(fx["K"]).reshape(1, 1, 2, 1)
+    v = np.array(fx["V"]).reshape(1, 1, 2, 1)
+    d_o = np.array(fx["dO"]).reshape(1, 2, 1, 1)
+    assert abs(fx["ln2"] - math.log(2)) < 1e-15 and abs(fx["ln3"] - math.log(3)) < 1e-15
+    o, lse, dq, dk, dv = orc.attn_bwd_ext(q, k, v, d_o, False, fx["scale"])
+    np.testing.assert_allclose(o.reshape(2), np.array(fx["O"]).reshape(2), atol=1e-14)
+    np.testing.assert_allclose(lse.reshape(2), np.array(fx["LSE"]), atol=1e-14)
+    np.testing.assert_allclose(dq.reshape(2), np.array(fx["dQ"]).reshape(2), atol=1e-14)
+    np.testing.assert_allclose(dk.reshape(2), np.array(fx["dK"]).reshape(2), atol=1e-14)
+    np.testing.assert_allclose(dv.reshape(2), np.array(fx["dV"]).reshape(2), atol=1e-14)
+    # the causal mask of a single query over two keys is bottom-right aligned: the query sees both keys
+    oc, lsec, dqc, dkc, dvc = orc.attn_bwd_ext(q, k, v, d_o, True, fx["scale"])
+    for a, b in ((o, oc), (lse, lsec), (dq, dqc), (dk, dkc), (dv, dvc)):
+        np.testing.assert_allclose(b, a, atol=1e-15)
