@@ -301,6 +301,6 @@ const char* mgn_status_string(int status)
     }
 }
 
-int mgn_version(void) { return 100; }
+int mgn_version(void) { return 200; }   // 0.2.0: extended shapes, deterministic backward, accelerated forward
 
 }  // extern "C"
