@@ -171,6 +171,19 @@ int mgn_attn_profile_events(void* before_main, void* after_main);
 int mgn_attn_fast_item_order(int order);
 
 /*
+ * Which tile shapes the strict-mode kernels run a problem with (host-only query; library plumbing,
+ * the paper has no counterpart).  The strict kernels cover the score matrix with tiles of
+ * fwd_bm x fwd_bn (forward) and bwd_bm x bwd_bn (backward) query rows x keys, and execute whole
+ * tiles; for short sequences whose lengths are far from tile multiples (197 tokens of a vision
+ * transformer, Section 4.1 workload table) a second shape with less padding is chosen.  Writes the
+ * four sizes through host pointers out[0..3] = {fwd_bm, fwd_bn, bwd_bm, bwd_bn}.  Arguments as in
+ * mgn_attn_fwd_ext.  Touches no device.  Returns MGN_OK, MGN_ERR_INVALID_ARG (out null, a size
+ * <= 0, H % H_kv != 0, causal not 0/1) or MGN_ERR_UNSUPPORTED (D not in {32, 64, 128}; causal with
+ * S_q > S_k).
+ */
+int mgn_attn_strict_tiles(int B, int H, int H_kv, int S_q, int S_k, int D, int causal, int* out);
+
+/*
  * Backward for callers that cannot allocate device memory.  (The paper has no counterpart:
  * this is a convenience of this library.)
  *

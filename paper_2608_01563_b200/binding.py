@@ -69,6 +69,8 @@ def lib() -> ctypes.CDLL:
         L.mgn_attn_profile_events.restype = i
         L.mgn_attn_fast_item_order.argtypes = [i]
         L.mgn_attn_fast_item_order.restype = i
+        L.mgn_attn_strict_tiles.argtypes = [i] * 7 + [ctypes.POINTER(ctypes.c_int)]
+        L.mgn_attn_strict_tiles.restype = i
         L.mgn_status_string.argtypes = [i]
         L.mgn_status_string.restype = ctypes.c_char_p
         L.mgn_version.argtypes = []
@@ -196,6 +198,15 @@ def mgn_attn_fast_item_order(order: int) -> None:
     st = lib().mgn_attn_fast_item_order(int(order))
     if st != MGN_OK:
         raise MgnError(st, "mgn_attn_fast_item_order")
+
+
+def mgn_attn_strict_tiles(B: int, H: int, H_kv: int, S_q: int, S_k: int, D: int, causal: bool):
+    """(fwd_bm, fwd_bn, bwd_bm, bwd_bn): tile shapes the strict kernels run this problem with."""
+    out = (ctypes.c_int * 4)()
+    st = lib().mgn_attn_strict_tiles(B, H, H_kv, S_q, S_k, D, int(bool(causal)), out)
+    if st != MGN_OK:
+        raise MgnError(st, "mgn_attn_strict_tiles")
+    return tuple(out)
 
 
 def mgn_measure_fp32_ffma_tflops(stream: Optional[int] = None) -> float:

@@ -286,6 +286,17 @@ int mgn_attn_fast_item_order(int order)
     return MGN_OK;
 }
 
+int mgn_attn_strict_tiles(int B, int H, int H_kv, int S_q, int S_k, int D, int causal, int* out)
+{
+    if (out == nullptr || B <= 0 || H <= 0 || H_kv <= 0 || S_q <= 0 || S_k <= 0 || D <= 0) return MGN_ERR_INVALID_ARG;
+    if (H % H_kv != 0 || (causal != 0 && causal != 1)) return MGN_ERR_INVALID_ARG;
+    if ((D != 32 && D != 64 && D != 128) || (causal && S_q > S_k)) return MGN_ERR_UNSUPPORTED;
+    const mgn::Problem p{B, H, H_kv, S_q, S_k, D, causal, 1.0f};
+    mgn::strict_fwd_tiles(p, &out[0], &out[1]);
+    mgn::strict_bwd_tiles(p, &out[2], &out[3]);
+    return MGN_OK;
+}
+
 const char* mgn_status_string(int status)
 {
     switch (status) {

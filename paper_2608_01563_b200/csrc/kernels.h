@@ -18,6 +18,37 @@ struct Problem {
     int off() const { return Sk - Sq; }
 };
 
+// Tile pairs x tile area that a (BM-row query tile, BN-key tile) decomposition executes: the padded
+// work that picks between tile shapes for short or ragged sequences.
+inline double tiled_work(const Problem& p, int BM, int BN) {
+    const int n_qt = (p.Sq + BM - 1) / BM, n_kt = (p.Sk + BN - 1) / BN;
+    long long pairs = 0;
+    for (int qt = 0; qt < n_qt; ++qt) {
+        const int i_last = (qt * BM + BM < p.Sq ? qt * BM + BM : p.Sq) - 1;
+        const int vis = p.causal ? (i_last + p.off()) / BN + 1 : n_kt;
+        pairs += vis < n_kt ? vis : n_kt;
+    }
+    return static_cast<double>(pairs) * BM * BN;
+}
+// Tile shapes of the strict kernels (query rows x keys per CTA step).  Short sequences (both lengths
+// <= 512) at D = 64 whose padded work under the default tiles exceeds that under the alternative by
+// more than a seventh run with the alternative: 197 tokens execute 200 x 224 (forward) and
+// 200 x 256 (backward) instead of 256 x 256.
+inline bool prefer_alt_tiles(const Problem& p, int BM, int BN, int BM_alt, int BN_alt) {
+    if (p.Sq > 512 || p.Sk > 512) return false;
+    return tiled_work(p, BM_alt, BN_alt) * 8.0 < tiled_work(p, BM, BN) * 7.0;
+}
+inline void strict_fwd_tiles(const Problem& p, int* BM, int* BN) {
+    *BM = p.D == 128 ? 128 : 64;
+    *BN = p.D == 128 ? 64 : 128;
+    if (p.D == 64 && prefer_alt_tiles(p, 64, 128, 40, 112)) { *BM = 40; *BN = 112; }
+}
+inline void strict_bwd_tiles(const Problem& p, int* BM, int* BN) {
+    *BM = 64;
+    *BN = 64;
+    if (p.D == 64 && prefer_alt_tiles(p, 64, 64, 40, 64)) *BM = 40;
+}
+
 // Tensor maps (host side).  rank-3 view (D, S, BH) of a dense [BH,S,D] tensor with
 // a (box_d, box_rows, 1) box and the 128-byte swizzle.  Returns 0 on success.
 int make_tmap_3d(CUtensorMap* out, const void* base, int elem_bytes, int is_bf16,

@@ -341,9 +341,14 @@ cudaError_t launch_strict_bwd(const Problem& p, const float* q, const float* k, 
                               const float* d_o, const float* lse, const float* delta,
                               float* dq, float* dk, float* dv, unsigned* status, cudaStream_t st)
 {
+    int BM, BN;
+    strict_bwd_tiles(p, &BM, &BN);
     switch (p.D) {
         case 32:  return launch<32, 64, 64, 128>(p, q, k, v, d_o, lse, delta, dq, dk, dv, status, st);
-        case 64:  return launch<64, 64, 64, 128>(p, q, k, v, d_o, lse, delta, dq, dk, dv, status, st);
+        case 64:
+            if (BM == 40)   // short ragged sequences
+                return launch<64, 40, 64, 128>(p, q, k, v, d_o, lse, delta, dq, dk, dv, status, st);
+            return launch<64, 64, 64, 128>(p, q, k, v, d_o, lse, delta, dq, dk, dv, status, st);
         case 128: return launch<128, 64, 64, 256>(p, q, k, v, d_o, lse, delta, dq, dk, dv, status, st);
         default:  return cudaErrorInvalidValue;
     }

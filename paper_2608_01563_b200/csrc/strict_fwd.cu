@@ -32,7 +32,8 @@ struct FwdCfg {
     static constexpr int RN = BN / 16;    // key columns per thread
     static constexpr int DV = D / 16;     // output columns per thread
     static constexpr int NCH = D / 32;    // 128-byte chunks per row
-    static constexpr int PSTR = BN;       // row stride of P (floats); 16-byte pieces XOR-swizzled by row
+    // row stride of P (floats); 16-byte pieces XOR-swizzled by row within groups of eight pieces
+    static constexpr int PSTR = (BN + 31) / 32 * 32;
     static constexpr int Q_BYTES = BM * D * 4;
     static constexpr int KV_BYTES = BN * D * 4;
     static constexpr int P_BYTES = BM * PSTR * 4;
@@ -303,9 +304,13 @@ cudaError_t launch(const Problem& p, const float* q, const float* k, const float
 cudaError_t launch_strict_fwd(const Problem& p, const float* q, const float* k, const float* v,
                               float* o, float* lse, unsigned* status, cudaStream_t st)
 {
+    int BM, BN;
+    strict_fwd_tiles(p, &BM, &BN);
     switch (p.D) {
         case 32:  return launch<32, 64, 128, 128>(p, q, k, v, o, lse, status, st);
-        case 64:  return launch<64, 64, 128, 128>(p, q, k, v, o, lse, status, st);
+        case 64:
+            if (BM == 40) return launch<64, 40, 112, 128>(p, q, k, v, o, lse, status, st);   // short ragged sequences
+            return launch<64, 64, 128, 128>(p, q, k, v, o, lse, status, st);
         case 128: return launch<128, 128, 64, 256>(p, q, k, v, o, lse, status, st);
         default:  return cudaErrorInvalidValue;
     }

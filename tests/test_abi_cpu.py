@@ -34,7 +34,8 @@ def test_every_declared_symbol_is_exported(lib):
     assert {"mgn_attn_fwd", "mgn_attn_bwd", "mgn_attn_bwd_workspace_bytes", "mgn_attn_check",
             "mgn_status_string", "mgn_version", "mgn_attn_profile_events", "mgn_attn_bwd_noalloc", "mgn_measure_fp32_ffma_tflops",
             "mgn_attn_fast_item_order", "mgn_attn_fwd_ext", "mgn_attn_bwd_ext",
-            "mgn_attn_bwd_deterministic", "mgn_attn_fwd_accel", "mgn_attn_fwd_accel_workspace_bytes"} <= set(syms)
+            "mgn_attn_bwd_deterministic", "mgn_attn_fwd_accel", "mgn_attn_fwd_accel_workspace_bytes",
+            "mgn_attn_strict_tiles"} <= set(syms)
     for s in syms:
         assert getattr(lib, s) is not None
 
@@ -178,3 +179,37 @@ def test_accel_forward_argument_validation(lib):
     assert fa(ws=None) == WORKSPACE
     assert fa(ws_bytes=need - 1) == WORKSPACE
     assert fa(ws=A + 16) == WORKSPACE
+
+
+def test_strict_tile_shapes_follow_the_padded_work():
+    """Host-only query: short ragged lengths at D = 64 get the low-padding tiles, everything else the defaults."""
+    from paper_2608_01563_b200 import binding
+    tiles = binding.mgn_attn_strict_tiles
+    assert tiles(32, 12, 12, 197, 197, 64, False) == (40, 112, 40, 64)     # 200 x 224 and 200 x 256 instead of 256 x 256
+    assert tiles(1, 4, 4, 197, 197, 64, True) == (40, 112, 40, 64)
+    assert tiles(8, 12, 12, 1024, 1024, 64, True) == (64, 128, 64, 64)     # long sequences keep the defaults
+    assert tiles(1, 2, 2, 128, 128, 64, False) == (64, 128, 64, 64)        # an exact fit stays
+    assert tiles(1, 2, 2, 256, 256, 64, True) == (64, 128, 64, 64)
+    assert tiles(1, 2, 2, 197, 197, 128, False) == (128, 64, 64, 64)       # other head sizes have one shape
+    assert tiles(1, 2, 2, 64, 64, 32, False) == (64, 128, 64, 64)
+    assert tiles(2, 8, 2, 150, 400, 64, True) == (40, 112, 40, 64)         # 150 rows: 160 executed instead of 192
+    assert tiles(2, 8, 8, 50, 16, 64, False) == (64, 128, 64, 64)          # one tile either way
+    # the chosen shape never executes more padded work than the default
+    def work(Sq, Sk, bm, bn, causal):
+        n_qt, n_kt = -(-Sq // bm), -(-Sk // bn)
+        pairs = 0
+        for qt in range(n_qt):
+            i_last = min(qt * bm + bm, Sq) - 1
+            pairs += min((i_last + Sk - Sq) // bn + 1, n_kt) if causal else n_kt
+        return pairs * bm * bn
+    for Sq, Sk, causal in [(197, 197, False), (41, 300, True), (300, 300, True), (77, 77, False), (500, 512, True),
+                           (50, 16, False), (1, 300, True), (129, 129, False), (513, 513, False)]:
+        fbm, fbn, bbm, bbn = tiles(1, 2, 2, Sq, Sk, 64, causal)
+        assert work(Sq, Sk, fbm, fbn, causal) <= work(Sq, Sk, 64, 128, causal)
+        assert work(Sq, Sk, bbm, bbn, causal) <= work(Sq, Sk, 64, 64, causal)
+    with pytest.raises(binding.MgnError):
+        tiles(1, 3, 2, 8, 8, 64, False)
+    with pytest.raises(binding.MgnError):
+        tiles(1, 2, 2, 16, 8, 64, True)
+    with pytest.raises(binding.MgnError):
+        tiles(1, 2, 2, 8, 8, 48, False)
