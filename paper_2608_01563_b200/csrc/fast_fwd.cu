@@ -22,9 +22,10 @@
 // Tensor memory (512 columns): S_0 [0,128), S_1 [128,256), O_0 [256,256+D), O_1 [256+D,256+2D).
 // P_t (bf16) overwrites S_t: keys 0-63 at S_t[0,32), keys 64-127 at S_t[64,96) (each half in the
 // columns its own threads have already read).  The softmax reference point of a row only moves
-// (and O is rescaled in tensor memory) when a score outgrows it by more than 2^8, which is exact:
-// any reference point works for a softmax as long as nothing overflows.  The two threads of a
-// row agree on that through a barrier with an OR-reduction per block.
+// (and O is rescaled in tensor memory) when a row outgrows it so far that a thread's partial sum of
+// exponentials passes 2^12, which is exact: any reference point works for a softmax as long as
+// nothing overflows.  The two threads of a row agree on that through a barrier with an
+// OR-reduction per block.
 #include "kernels.h"
 #include "fast_items.cuh"
 #include "umma.cuh"
@@ -38,7 +39,9 @@ constexpr int BN = 128;      // keys per block
 constexpr int kStages = 2;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
-constexpr float kRescaleThreshold = 8.0f;
+// A thread's partial row sum (64 columns) above this moves the reference points: every p stays
+// below it, far inside the range of bf16 and of IEEE f16 (65504), and the sums inside that of f32.
+constexpr float kGrowthLimit = 4096.0f;
 
 template <int D>
 struct Cfg {
@@ -315,15 +318,17 @@ fast_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                 }
 
                 // One pass: y = s*c2 - m_ref, p = exp2(y), partial row sum, bf16 pack (kept in
-                // registers), and the largest y.  If any row outgrew its reference point by more than
-                // the threshold, move the reference points, rescale O and l, and redo the pass (S is
-                // still intact: P is written over it only afterwards).
+                // registers); two columns per fma / add instruction.  A row that outgrew its reference
+                // point shows in its partial sum (every p <= the sum): if any partial sum passes the
+                // limit, the rows find their current maxima in a second look at S (still intact: P is
+                // written over it only afterwards), move their reference points, rescale O and l, and
+                // the pass is redone.  The common case pays no per-element maximum.
                 uint32_t pk[32];
                 float lsum = 0.f;
                 for (int attempt = 0; attempt < 2; ++attempt) {
-                    float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
-                    float y0 = -INFINITY, y1 = -INFINITY, y2 = -INFINITY, y3 = -INFINITY;
+                    uint64_t la = f2_pack(0.f, 0.f), lb = la;
                     const float neg_m = -m_ref[t];
+                    const uint64_t c2x2 = f2_pack(c2, c2), nm2 = f2_pack(neg_m, neg_m);
 #pragma unroll
                     for (int c = 0; c < 2; ++c) {
                         uint32_t v[32];
@@ -331,7 +336,8 @@ fast_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                         tmem_ld_wait();
                         float y[32];
 #pragma unroll
-                        for (int e = 0; e < 32; ++e) y[e] = fmaf(__uint_as_float(v[e]), c2, neg_m);
+                        for (int e = 0; e < 32; e += 2)
+                            f2_unpack(f2_fma(f2_pack(__uint_as_float(v[e]), __uint_as_float(v[e + 1])), c2x2, nm2), y[e], y[e + 1]);
                         if (masked) {
 #pragma unroll
                             for (int e = 0; e < 32; ++e)
@@ -339,19 +345,34 @@ fast_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                         }
 #pragma unroll
                         for (int e = 0; e < 32; e += 4) {
-                            y0 = fmaxf(y0, y[e]); y1 = fmaxf(y1, y[e + 1]); y2 = fmaxf(y2, y[e + 2]); y3 = fmaxf(y3, y[e + 3]);
                             const float p0 = ex2(y[e]), p1 = ex2(y[e + 1]), p2 = ex2(y[e + 2]), p3 = ex2(y[e + 3]);
-                            l0 += p0; l1 += p1; l2 += p2; l3 += p3;
+                            la = f2_add(la, f2_pack(p0, p1));
+                            lb = f2_add(lb, f2_pack(p2, p3));
                             pk[16 * c + e / 2] = F16 ? pack_f16(p0, p1) : pack_bf16(p0, p1);
                             pk[16 * c + e / 2 + 1] = F16 ? pack_f16(p2, p3) : pack_bf16(p2, p3);
                         }
                     }
-                    lsum = (l0 + l1) + (l2 + l3);
-                    const float ymax = fmaxf(fmaxf(y0, y1), fmaxf(y2, y3));
+                    {
+                        float a0, a1, a2, a3;
+                        f2_unpack(la, a0, a1);
+                        f2_unpack(lb, a2, a3);
+                        lsum = (a0 + a1) + (a2 + a3);
+                    }
                     if (attempt == 1) break;
-                    sts32(my_x, ymax);
-                    if (!bar_or(ymax > kRescaleThreshold)) break;
+                    if (!bar_or(!(lsum <= kGrowthLimit))) break;      // also true for an overflowed (inf / nan) sum
                     // some row grew: every row moves its reference point to its current maximum
+                    float ymax = -INFINITY;
+#pragma unroll
+                    for (int c = 0; c < 2; ++c) {
+                        uint32_t v[32];
+                        tmem_ld32(tS + 32 * c, v);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int e = 0; e < 32; ++e)
+                            if (!masked || 32 * c + e <= jmax) ymax = fmaxf(ymax, fmaf(__uint_as_float(v[e]), c2, neg_m));
+                    }
+                    sts32(my_x, ymax);
+                    bar_or(false);
                     const float ym = fmaxf(ymax, lds32f(peer_x));
                     const float m_new = fmaxf(m_ref[t], m_ref[t] + ym);
                     const float alpha = ex2(m_ref[t] - m_new);
