@@ -95,3 +95,21 @@ def test_argument_errors():
     with pytest.raises(mgn.MgnError) as e:
         mgn.mgn_attn_fwd_accel(q, q, q, torch.empty_like(q), lse, ws[:16], False, 1.0)
     assert e.value.status == 4
+
+
+def test_stepwise_growth_keeps_f16_probabilities_in_range():
+    """Key block b scaled by b + 1: every 128-key block moves the softmax reference point, and every
+    probability that the kernel packs to f16 must stay below the f16 maximum (the growth limit of the
+    pass is 2^12).  Compared with the oracle on f16-rounded inputs (the scores are large here, so input
+    rounding would dominate a comparison on the original inputs)."""
+    B, H, S, D = 1, 2, 640, 128
+    q, k, v, d_o = synth.random_inputs(1002, B, H, S, D)
+    k = k * (torch.arange(S) // 128 + 1).view(1, 1, S, 1).float()
+    q16, k16, v16 = (t.half().float() for t in (q, k, v))
+    for causal in (False, True):
+        got = _run(q16, k16, v16, d_o, causal, 0.5)
+        ref = hp.run_oracle_ext(q16, k16, v16, d_o, causal, 0.5)
+        assert np.isfinite(got["O"]).all() and np.isfinite(got["LSE"]).all()
+        r = hp.rel_l2(got["O"], ref["O"])
+        assert r <= GATE_ROUNDED, f"O: rel-L2 {r:.3e}"
+        assert (np.abs(got["LSE"] - ref["LSE"]) <= 2e-3 + 1e-5 * np.abs(ref["LSE"])).all()

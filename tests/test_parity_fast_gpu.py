@@ -78,6 +78,24 @@ def test_forward_large_max_growth_triggers_rescale():
         hp.check_fast(hp.select(res, B, H), ref, names=("O",))
 
 
+@pytest.mark.parametrize("causal", [False, True])
+def test_forward_stepwise_growth_moves_the_reference_point_in_every_block(causal):
+    """Key block b is scaled by b + 1, so the row maxima jump by far more than the growth limit from
+    each 128-key block to the next: every block takes the redo path (find the maxima, rescale O and
+    l, repeat the pass).  O and the saved log-sum-exp must still match."""
+    B, H, S, D = 1, 2, 1152, 128
+    q, k, v, d_o = synth.random_inputs(13, B, H, S, D, dtype=torch.float32)
+    step = (torch.arange(S) // 128 + 1).view(1, 1, S, 1).float()
+    k = (k * step).to(BF)
+    q, v, d_o = q.to(BF), v.to(BF), d_o.to(BF)
+    res = hp.run_cuda(q, k, v, d_o, causal, 0.5, MODE, run_bwd=False)
+    ref = hp.run_oracle(q, k, v, d_o, causal, 0.5)
+    got = hp.select(res, B, H)
+    hp.check_fast(got, ref, names=("O",), label="stepwise growth ")
+    err = np.abs(got["LSE"] - ref["LSE"])
+    assert (err <= 2e-2 + 1e-3 * np.abs(ref["LSE"])).all(), f"LSE off by up to {err.max()}"
+
+
 @pytest.mark.parametrize("scale", [0.0, -0.2])
 def test_forward_unusual_scales(scale):
     B, H, S, D = 1, 2, 300, 64
