@@ -355,7 +355,7 @@ def main():
     ap.add_argument("--mode", default="strict", choices=["strict", "fast"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
-    ap.add_argument("--no-fast", action="store_true", help="skip the extra fast-mode measurement")
+    ap.add_argument("--no-fast", action="store_true", help="skip the extra measurements (other mode, other shapes, other workloads)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -592,6 +592,22 @@ def main():
                 r["frac_of_peak"] = r["sum_tflops"] / mode_peak
                 ext[name] = r
             line["ext_shapes"] = ext
+            # the other configured workloads in this run's arithmetic mode (few steps each): the ragged
+            # vision-transformer shape (strict) and the decoder sweep, device-resident like `value`
+            names = (["vit_b_ragged"] if args.mode == "strict" else []) + \
+                    [n for n in synth.WORKLOADS if n.startswith("decoder_sweep_S")]
+            table = {}
+            for name in names:
+                wt = synth.WORKLOADS[name]
+                steps_t = max(2, min(K, 5 if wt.S <= 2048 else 2))
+                f_ms, b_ms = quick_measure(mgn, wt, mode, dtype, steps_t, 2)
+                tfl = flops(wt, "sum") / ((f_ms + b_ms) * 1e-3) / 1e12
+                table[name] = {"B": wt.B, "H": wt.H, "S": wt.S, "D": wt.D, "causal": bool(wt.causal), "steps": steps_t,
+                               "fwd_ms": f_ms, "bwd_ms": b_ms,
+                               "fwd_tflops": flops(wt, "fwd") / (f_ms * 1e-3) / 1e12,
+                               "bwd_tflops": flops(wt, "bwd") / (b_ms * 1e-3) / 1e12,
+                               "sum_tflops": tfl, "frac_of_peak": tfl / mode_peak}
+            line["other_workloads"] = table
             line["deterministic_bwd"] = measure_deterministic_bwd(mgn, w, mode, dtype, K, args.warmup)
             if args.mode == "strict":
                 if w.D in (64, 128):
