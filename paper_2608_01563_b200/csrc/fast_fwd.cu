@@ -23,7 +23,7 @@
 // P_t (bf16) overwrites S_t: keys 0-63 at S_t[0,32), keys 64-127 at S_t[64,96) (each half in the
 // columns its own threads have already read).  The softmax reference point of a row only moves
 // (and O is rescaled in tensor memory) when a row outgrows it so far that a thread's partial sum of
-// exponentials passes 2^12, which is exact: any reference point works for a softmax as long as
+// exponentials passes a limit (2^60; 2^12 with f16 probabilities), which is exact: any reference point works for a softmax as long as
 // nothing overflows.  The two threads of a row agree on that through a barrier with an
 // OR-reduction per block.
 #include "kernels.h"
@@ -39,9 +39,14 @@ constexpr int BN = 128;      // keys per block
 constexpr int kStages = 2;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
-// A thread's partial row sum (64 columns) above this moves the reference points: every p stays
-// below it, far inside the range of bf16 and of IEEE f16 (65504), and the sums inside that of f32.
-constexpr float kGrowthLimit = 4096.0f;
+// A thread's partial row sum (64 columns) above this limit moves the reference points.  Every p stays
+// below the limit and the sums of a row below 2^13 times it, so nothing overflows.  With f16
+// probabilities the limit is 2^12 (f16 ends at 65504).  With bf16 it is 2^60: bf16 and f32 share the
+// exponent range, a softmax is exact for any reference point, and a low limit is expensive -- one row
+// in 128 passing it makes the whole tile repeat the pass, which heavy-tailed scores (1 % of the
+// inputs scaled by 8 in the decoder sweep) did in most key blocks: forward +50-60 % there.
+constexpr float kGrowthLimitF16 = 4096.0f;
+constexpr float kGrowthLimitBf16 = 1152921504606846976.0f;   // 2^60
 
 template <int D>
 struct Cfg {
@@ -359,7 +364,7 @@ fast_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                         lsum = (a0 + a1) + (a2 + a3);
                     }
                     if (attempt == 1) break;
-                    if (!bar_or(!(lsum <= kGrowthLimit))) break;      // also true for an overflowed (inf / nan) sum
+                    if (!bar_or(!(lsum <= (F16 ? kGrowthLimitF16 : kGrowthLimitBf16)))) break;      // also true for an overflowed (inf / nan) sum
                     // some row grew: every row moves its reference point to its current maximum
                     float ymax = -INFINITY;
 #pragma unroll

@@ -80,18 +80,38 @@ def test_forward_large_max_growth_triggers_rescale():
 
 @pytest.mark.parametrize("causal", [False, True])
 def test_forward_stepwise_growth_moves_the_reference_point_in_every_block(causal):
-    """Key block b is scaled by b + 1, so the row maxima jump by far more than the growth limit from
-    each 128-key block to the next: every block takes the redo path (find the maxima, rescale O and
-    l, repeat the pass).  O and the saved log-sum-exp must still match."""
+    """Every query has 4 and key block b has 25 b in component 0, so with scale 0.5 the scores of a
+    row jump by 50 (72 in the log2 domain) from each 128-key block to the next: more than the growth
+    limit of the pass (2^60), so every block takes the redo path (find the maxima, rescale O and l,
+    repeat the pass).  O and the saved log-sum-exp must still match."""
     B, H, S, D = 1, 2, 1152, 128
     q, k, v, d_o = synth.random_inputs(13, B, H, S, D, dtype=torch.float32)
-    step = (torch.arange(S) // 128 + 1).view(1, 1, S, 1).float()
-    k = (k * step).to(BF)
-    q, v, d_o = q.to(BF), v.to(BF), d_o.to(BF)
+    q[..., 0] = 4.0
+    k[..., 0] = (25.0 * (torch.arange(S) // 128)).view(1, 1, S)
+    q, k, v, d_o = q.to(BF), k.to(BF), v.to(BF), d_o.to(BF)
     res = hp.run_cuda(q, k, v, d_o, causal, 0.5, MODE, run_bwd=False)
     ref = hp.run_oracle(q, k, v, d_o, causal, 0.5)
     got = hp.select(res, B, H)
     hp.check_fast(got, ref, names=("O",), label="stepwise growth ")
+    err = np.abs(got["LSE"] - ref["LSE"])
+    assert (err <= 2e-2 + 1e-3 * np.abs(ref["LSE"])).all(), f"LSE off by up to {err.max()}"
+
+
+def test_forward_heavy_tailed_scores_below_the_growth_limit():
+    """1 % of Q and K scaled by 8 (the decoder sweep's distribution) at a length of several blocks:
+    the reference point of a row stays where the first block put it although later scores are far
+    larger (p up to about 2^40); O and LSE must match."""
+    B, H, S, D = 1, 2, 1024, 128
+    q, k, v, d_o = synth.random_inputs(14, B, H, S, D, dtype=torch.float32)
+    g = torch.Generator().manual_seed(15)
+    q = torch.where(torch.rand(q.shape, generator=g) < 0.01, 8.0 * q, q)
+    k = torch.where(torch.rand(k.shape, generator=g) < 0.01, 8.0 * k, k)
+    k[:, :, :128] *= 0.05                       # the first block sets a low reference point
+    q, k, v, d_o = q.to(BF), k.to(BF), v.to(BF), d_o.to(BF)
+    res = hp.run_cuda(q, k, v, d_o, False, 0.5, MODE, run_bwd=False)
+    ref = hp.run_oracle(q, k, v, d_o, False, 0.5)
+    got = hp.select(res, B, H)
+    hp.check_fast(got, ref, names=("O",), label="heavy tails ")
     err = np.abs(got["LSE"] - ref["LSE"])
     assert (err <= 2e-2 + 1e-3 * np.abs(ref["LSE"])).all(), f"LSE off by up to {err.max()}"
 
