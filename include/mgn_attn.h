@@ -54,6 +54,10 @@ enum { MGN_MODE_STRICT_F32 = 0, MGN_MODE_FAST_BF16 = 1 };
  * q,k,v: in.  o: out [B,H,S,D] (mode's element type).  lse: out [B,H,S] f32.
  * Strict mode computes in f32 FFMA; fast mode multiplies bf16 operands on the
  * tensor cores with f32 accumulation and f32 softmax statistics.
+ * Range (fast mode): a row's running softmax reference may stay up to 2^60 below the
+ * largest score seen so far, so the unnormalised sums reach 2^60 * S_k * max|v|; they
+ * are f32.  Finite results need max|v| * S_k below about 2^60 (1e18), far beyond
+ * any activation; inside that range o and lse do not depend on the lag.
  */
 int mgn_attn_fwd(const void* q, const void* k, const void* v, void* o, float* lse,
                  int B, int H, int S, int D, int causal, float scale, int mode, void* stream);
