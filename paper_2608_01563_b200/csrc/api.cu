@@ -312,6 +312,6 @@ const char* mgn_status_string(int status)
     }
 }
 
-int mgn_version(void) { return 200; }   // 0.2.0: extended shapes, deterministic backward, accelerated forward
+int mgn_version(void) { return 210; }   // 0.2.1: tile-shape query, low-padding strict tiles, leaner fast forward (0.2.0: extended shapes, deterministic backward, accelerated forward)
 
 }  // extern "C"
