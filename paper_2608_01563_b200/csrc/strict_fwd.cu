@@ -135,7 +135,12 @@ strict_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         {
             const uint32_t qa = sQ + tr * 128, ka = sK + tc * 128;
             const int xq = tr & 7, xk = tc & 7;
-#pragma unroll
+            // Loop bodies of about 2000 FFMAs (eight contraction steps here, eight groups of keys in the
+            // second product) run best at D = 64: larger ones miss the instruction cache, smaller ones
+            // leave the operand loads less room to be hoisted (measured; other head sizes keep the
+            // forms they were tuned with).
+            constexpr int kUnrollQK = (D == 64) ? 8 : D / 4;
+#pragma unroll kUnrollQK
             for (int pc = 0; pc < D / 4; ++pc) {
                 const uint32_t oq = (pc >> 3) * (BM * 128) + (((pc & 7) ^ xq) << 4);
                 const uint32_t ok = (pc >> 3) * (BN * 128) + (((pc & 7) ^ xk) << 4);
@@ -204,7 +209,8 @@ strict_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         // ---- O += P V : contraction along keys ----------------------------------------------
         {
             const uint32_t pa = sP + tr * PSTR * 4;
-#pragma unroll 2
+            constexpr int kUnrollPV = (D == 64) ? 8 : 2;
+#pragma unroll kUnrollPV
             for (int j8 = 0; j8 < BN / 8; ++j8) {
                 float4 p[2][RM];
 #pragma unroll
