@@ -97,19 +97,20 @@ def test_forward_stepwise_growth_moves_the_reference_point_in_every_block(causal
     assert (err <= 2e-2 + 1e-3 * np.abs(ref["LSE"])).all(), f"LSE off by up to {err.max()}"
 
 
-def test_forward_heavy_tailed_scores_below_the_growth_limit():
+@pytest.mark.parametrize("D,causal", [(128, False), (128, True), (64, True)])
+def test_forward_heavy_tailed_scores_below_the_growth_limit(D, causal):
     """1 % of Q and K scaled by 8 (the decoder sweep's distribution) at a length of several blocks:
     the reference point of a row stays where the first block put it although later scores are far
     larger (p up to about 2^40); O and LSE must match."""
-    B, H, S, D = 1, 2, 1024, 128
+    B, H, S = 1, 2, 1024
     q, k, v, d_o = synth.random_inputs(14, B, H, S, D, dtype=torch.float32)
     g = torch.Generator().manual_seed(15)
     q = torch.where(torch.rand(q.shape, generator=g) < 0.01, 8.0 * q, q)
     k = torch.where(torch.rand(k.shape, generator=g) < 0.01, 8.0 * k, k)
     k[:, :, :128] *= 0.05                       # the first block sets a low reference point
     q, k, v, d_o = q.to(BF), k.to(BF), v.to(BF), d_o.to(BF)
-    res = hp.run_cuda(q, k, v, d_o, False, 0.5, MODE, run_bwd=False)
-    ref = hp.run_oracle(q, k, v, d_o, False, 0.5)
+    res = hp.run_cuda(q, k, v, d_o, causal, 0.5, MODE, run_bwd=False)
+    ref = hp.run_oracle(q, k, v, d_o, causal, 0.5)
     got = hp.select(res, B, H)
     hp.check_fast(got, ref, names=("O",), label="heavy tails ")
     err = np.abs(got["LSE"] - ref["LSE"])
