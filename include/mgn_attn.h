@@ -23,6 +23,21 @@
  *   - Errors are reported by return code only (mgn_status); nothing is printed and
  *     nothing aborts.  Argument errors are detected before any launch, in the
  *     order INVALID_ARG, UNSUPPORTED, MISALIGNED, WORKSPACE, ARCH.
+ *   - Device status word.  Every wait inside a kernel is bounded; a wait that runs out
+ *     sets one status word PER DEVICE (not per stream, not per call).  While that word is
+ *     non-zero every later attention kernel of this library on that device -- forward,
+ *     backward, dQ pass, on any stream -- returns at once WITHOUT WRITING ITS OUTPUTS (o, lse,
+ *     dq, dk, dv of such calls are unwritten or partial), and the entry points still return
+ *     MGN_OK (they only enqueue).  Only mgn_attn_check() reads and clears the word.  A
+ *     caller that must know that its results are valid calls mgn_attn_check(stream)
+ *     after the calls it cares about; MGN_OK from it means that no kernel of this library
+ *     that has completed on the device so far gave up.  Because the word is shared, a time-out
+ *     cannot be attributed to one call, and a check on one stream also clears a flag raised
+ *     by another stream's kernel.
+ *   - Threads.  Distinct host threads may call the attention entry points concurrently on
+ *     distinct streams.  mgn_attn_profile_events() and mgn_attn_fast_item_order() change
+ *     process-wide settings that those calls read without synchronisation: use them only
+ *     while no other thread is inside the library.
  */
 #ifndef MGN_ATTN_H
 #define MGN_ATTN_H
@@ -147,6 +162,9 @@ int mgn_attn_bwd_deterministic(const void* q, const void* k, const void* v, cons
  * Synchronises `stream`, then reads and clears the device-side status word that
  * kernels set when one of their bounded waits (TMA / tensor-core completion
  * barriers) ran out.  Returns MGN_OK, MGN_ERR_DEVICE_TIMEOUT or MGN_ERR_CUDA.
+ * The word belongs to the current device, not to `stream`: see "Device status word"
+ * above.  After a MGN_ERR_DEVICE_TIMEOUT the outputs of every call since the last
+ * MGN_OK check are to be treated as unwritten; the next call runs normally again.
  * (Library plumbing; the paper has no counterpart.)
  */
 int mgn_attn_check(void* stream);
@@ -228,6 +246,18 @@ size_t mgn_attn_bwd_noalloc_max_workspace_bytes(void);
  * counterpart.  Returns MGN_OK, MGN_ERR_INVALID_ARG or MGN_ERR_CUDA.
  */
 int mgn_measure_fp32_ffma_tflops(float* scratch, double* tflops, void* stream);
+
+/*
+ * Self-test of the bounded waits (library plumbing; the paper has no counterpart; present only in
+ * builds with MGN_BUILD_SELFTEST, which the in-tree build sets).  Enqueues a one-CTA kernel that
+ * waits, with a limit of 1024 polls, on a barrier that nothing arrives on: the wait gives up, the
+ * kernel sets the device status word and returns -- the path a product kernel would take if a
+ * copy or a tensor-core completion never came.  Afterwards the device is in the state described
+ * under "Device status word": kernels of this library skip their work until mgn_attn_check() has
+ * returned MGN_ERR_DEVICE_TIMEOUT once.  `gave_up` is an optional DEVICE pointer that receives 1
+ * if the wait ran out (0 if it did not).  Returns MGN_OK, MGN_ERR_ARCH or MGN_ERR_CUDA.
+ */
+int mgn_selftest_wait_timeout(unsigned* gave_up, void* stream);
 
 /* Static string naming a status code. */
 const char* mgn_status_string(int status);

@@ -71,6 +71,8 @@ def lib() -> ctypes.CDLL:
         L.mgn_attn_fast_item_order.restype = i
         L.mgn_attn_strict_tiles.argtypes = [i] * 7 + [ctypes.POINTER(ctypes.c_int)]
         L.mgn_attn_strict_tiles.restype = i
+        L.mgn_selftest_wait_timeout.argtypes = [vp, vp]
+        L.mgn_selftest_wait_timeout.restype = i
         L.mgn_status_string.argtypes = [i]
         L.mgn_status_string.restype = ctypes.c_char_p
         L.mgn_version.argtypes = []
@@ -216,6 +218,12 @@ def mgn_measure_fp32_ffma_tflops(stream: Optional[int] = None) -> float:
     if st != MGN_OK:
         raise MgnError(st, "mgn_measure_fp32_ffma_tflops")
     return float(out.value)
+
+
+def mgn_selftest_wait_timeout(gave_up: Optional[torch.Tensor] = None, stream: Optional[int] = None) -> None:
+    st = lib().mgn_selftest_wait_timeout(_ptr(gave_up), _stream(stream))
+    if st != MGN_OK:
+        raise MgnError(st, "mgn_selftest_wait_timeout")
 
 
 def mgn_status_string(status: int) -> str:

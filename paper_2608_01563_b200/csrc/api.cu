@@ -79,6 +79,12 @@ int device_setup(unsigned** status)
     return MGN_OK;
 }
 
+}  // namespace
+namespace mgn {
+int device_status_word(unsigned** status) { return device_setup(status); }
+}
+namespace {
+
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 // Workspace layout: [delta: BH*S f32][fast mode only: dQ accumulator BH*S*D f32], 256-byte granules.

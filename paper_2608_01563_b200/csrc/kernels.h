@@ -49,6 +49,10 @@ inline void strict_bwd_tiles(const Problem& p, int* BM, int* BN) {
     if (p.D == 64 && prefer_alt_tiles(p, 64, 64, 40, 64)) *BM = 40;
 }
 
+// Per-device set-up shared by every entry point: checks the architecture of the current device and
+// returns the device address of its status word.  Returns an mgn_status code.
+int device_status_word(unsigned** status);
+
 // Tensor maps (host side).  rank-3 view (D, S, BH) of a dense [BH,S,D] tensor with
 // a (box_d, box_rows, 1) box and the 128-byte swizzle.  Returns 0 on success.
 int make_tmap_3d(CUtensorMap* out, const void* base, int elem_bytes, int is_bf16,

@@ -35,22 +35,25 @@ extern "C" int mgn_measure_fp32_ffma_tflops(float* scratch, double* tflops, void
     int dev = 0, sms = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return MGN_ERR_CUDA;
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return MGN_ERR_CUDA;
-    cudaEvent_t e0, e1;
-    if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess) return MGN_ERR_CUDA;
+    cudaEvent_t e0 = nullptr, e1 = nullptr;
+    if (cudaEventCreate(&e0) != cudaSuccess) return MGN_ERR_CUDA;
+    if (cudaEventCreate(&e1) != cudaSuccess) { cudaEventDestroy(e0); return MGN_ERR_CUDA; }
     const int threads = 512, grid = sms * 4, iters = 4096;
     double best = 0.0;
-    for (int rep = 0; rep < 4; ++rep) {     // first repetition warms up
-        cudaEventRecord(e0, st);
+    bool ok = true;
+    for (int rep = 0; ok && rep < 4; ++rep) {     // first repetition warms up
+        ok = cudaEventRecord(e0, st) == cudaSuccess;
         ffma_loop_kernel<<<grid, threads, 0, st>>>(scratch, 1.0001f, 0.5f, iters);
-        cudaEventRecord(e1, st);
-        if (cudaEventSynchronize(e1) != cudaSuccess) { cudaEventDestroy(e0); cudaEventDestroy(e1); return MGN_ERR_CUDA; }
+        ok = ok && cudaGetLastError() == cudaSuccess;          // a failed launch must not pass as 0 TFLOP/s
+        ok = ok && cudaEventRecord(e1, st) == cudaSuccess && cudaEventSynchronize(e1) == cudaSuccess;
         float ms = 0.f;
-        cudaEventElapsedTime(&ms, e0, e1);
+        ok = ok && cudaEventElapsedTime(&ms, e0, e1) == cudaSuccess;
         const double fl = 2.0 * 16 * 8 * iters * static_cast<double>(grid) * threads;
-        if (rep > 0 && ms > 0.f && fl / ms / 1e9 > best) best = fl / ms / 1e9;
+        if (ok && rep > 0 && ms > 0.f && fl / ms / 1e9 > best) best = fl / ms / 1e9;
     }
     cudaEventDestroy(e0);
     cudaEventDestroy(e1);
+    if (!ok || best <= 0.0) { cudaGetLastError(); return MGN_ERR_CUDA; }
     *tflops = best;
-    return cudaGetLastError() == cudaSuccess ? MGN_OK : MGN_ERR_CUDA;
+    return MGN_OK;
 }

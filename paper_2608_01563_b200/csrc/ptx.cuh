@@ -42,15 +42,18 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok;
 }
-// Bounded wait.  Returns false (after flagging the status word) if it gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, unsigned* status) {
-    for (uint32_t it = 0; it < kMaxPolls; ++it) {
+// Bounded wait of at most `max_polls` polls.  Returns false (after flagging the status word) if it gave up.
+__device__ __forceinline__ bool mbar_wait_polls(uint32_t bar, uint32_t parity, unsigned* status, uint32_t max_polls) {
+    for (uint32_t it = 0; it < max_polls; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
         // once any wait on the device has given up, every other wait gives up quickly too
         if ((it & 0xfffu) == 0xfffu && status && *reinterpret_cast<volatile unsigned*>(status) != 0) return false;
     }
     if (status) atomicMax(status, kStatusTimeout);
     return false;
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, unsigned* status) {
+    return mbar_wait_polls(bar, parity, status, kMaxPolls);
 }
 
 // TMA: rank-3 tiled load global -> shared (this CTA), completion on an mbarrier.
@@ -90,6 +93,42 @@ __device__ __forceinline__ float lg2(float x) {
     float y;
     asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
+}
+// Packed pairs of f32 (one 64-bit register): one instruction for two lanes of arithmetic.  The FMA
+// pipe does not get faster, but loops that are bound by instruction issue do.
+__device__ __forceinline__ uint64_t f2_pack(float lo, float hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void f2_unpack(uint64_t v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t f2_fma(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+__device__ __forceinline__ uint64_t f2_mul(uint64_t a, uint64_t b) {
+    uint64_t r;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ uint64_t f2_add(uint64_t a, uint64_t b) {
+    uint64_t r;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+
+struct U64x2 { uint64_t lo, hi; };
+// 128-bit shared load as two packed pairs: {x, y} and {z, w} of a float4.
+__device__ __forceinline__ U64x2 lds128_pairs(uint32_t addr) {
+    U64x2 v;
+    asm volatile("ld.shared.v2.b64 {%0,%1}, [%2];" : "=l"(v.lo), "=l"(v.hi) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ void sts128f(uint32_t addr, float a, float b, float c, float d) {
+    asm volatile("st.shared.v4.f32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
 }
 // 128-bit floating-point reduction into global memory (no return value).
 __device__ __forceinline__ void red_add_v4(float* addr, float a, float b, float c, float d) {

@@ -59,6 +59,7 @@ strict_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     constexpr int RM = C::RM, RN = C::RN, JN = C::JN, DV = C::DV, NCH = C::NCH, PSTR = C::PSTR, TR = C::TR;
 
     extern __shared__ uint8_t smem_raw[];
+    if (*reinterpret_cast<volatile unsigned*>(status) != 0) return;   // an earlier wait on this device gave up
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t sK = base;
     const uint32_t sV = sK + C::KV_BYTES;
@@ -105,11 +106,12 @@ strict_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         }
     }
 
-    float dk[JN][DV], dv[JN][DV];
+    // dK, dV accumulators as packed pairs of adjacent key rows: [a][e] = {key 2a, key 2a+1} of column e
+    uint64_t dk[JN / 2][DV], dv[JN / 2][DV];
 #pragma unroll
-    for (int a = 0; a < JN; ++a)
+    for (int a = 0; a < JN / 2; ++a)
 #pragma unroll
-        for (int e = 0; e < DV; ++e) { dk[a][e] = 0.f; dv[a][e] = 0.f; }
+        for (int e = 0; e < DV; ++e) { dk[a][e] = f2_pack(0.f, 0.f); dv[a][e] = f2_pack(0.f, 0.f); }
 
     mbar_wait(barKV, 0, status);
 
@@ -204,21 +206,24 @@ strict_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
 #pragma unroll
             for (int iu = 0; iu < 8; ++iu) {
                 const int i = i8 + iu;
+                // Two adjacent keys per packed FMA: the pairs of P and dS come as they are stored
+                // (row-major, keys contiguous), dO and Q values are duplicated into both lanes.
                 float dov[DV], qv[DV];
                 load_row_cols<D, BM>(sdO, i, iu, tc, dov);
                 load_row_cols<D, BM>(sQ, i, iu, tc, qv);
+                uint64_t do2[DV], q2[DV];
+#pragma unroll
+                for (int e = 0; e < DV; ++e) { do2[e] = f2_pack(dov[e], dov[e]); q2[e] = f2_pack(qv[e], qv[e]); }
 #pragma unroll
                 for (int g = 0; g < JN / 4; ++g) {
-                    const float4 p4 = lds128(sP + (i * PSTR + 4 * tr + 4 * TR * g) * 4);
-                    const float4 d4 = lds128(sdS + (i * PSTR + 4 * tr + 4 * TR * g) * 4);
+                    const U64x2 p4 = lds128_pairs(sP + (i * PSTR + 4 * tr + 4 * TR * g) * 4);
+                    const U64x2 d4 = lds128_pairs(sdS + (i * PSTR + 4 * tr + 4 * TR * g) * 4);
 #pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        const float pj = f4_get(p4, u), dj = f4_get(d4, u);
-#pragma unroll
-                        for (int e = 0; e < DV; ++e) {
-                            dv[4 * g + u][e] = fmaf(pj, dov[e], dv[4 * g + u][e]);
-                            dk[4 * g + u][e] = fmaf(dj, qv[e], dk[4 * g + u][e]);
-                        }
+                    for (int e = 0; e < DV; ++e) {
+                        dv[2 * g][e] = f2_fma(p4.lo, do2[e], dv[2 * g][e]);
+                        dv[2 * g + 1][e] = f2_fma(p4.hi, do2[e], dv[2 * g + 1][e]);
+                        dk[2 * g][e] = f2_fma(d4.lo, q2[e], dk[2 * g][e]);
+                        dk[2 * g + 1][e] = f2_fma(d4.hi, q2[e], dk[2 * g + 1][e]);
                     }
                 }
             }
@@ -286,20 +291,27 @@ strict_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
             const int j = j0 + 4 * tr + 4 * TR * g + u;
+            float kx[DV], vx[DV];
+#pragma unroll
+            for (int e = 0; e < DV; ++e) {
+                float lo, hi;
+                f2_unpack(dk[2 * g + (u >> 1)][e], lo, hi);
+                kx[e] = ((u & 1) ? hi : lo) * scale;
+                f2_unpack(dv[2 * g + (u >> 1)][e], lo, hi);
+                vx[e] = (u & 1) ? hi : lo;
+            }
             if (j < Sk) {
                 const size_t off = (static_cast<size_t>(bhk) * Sk + j) * D;
-                const int a = 4 * g + u;
                 if constexpr (DV == 2) {
-                    *reinterpret_cast<float2*>(dK + off + 2 * tc) = make_float2(dk[a][0] * scale, dk[a][1] * scale);
-                    *reinterpret_cast<float2*>(dV + off + 2 * tc) = make_float2(dv[a][0], dv[a][1]);
+                    *reinterpret_cast<float2*>(dK + off + 2 * tc) = make_float2(kx[0], kx[1]);
+                    *reinterpret_cast<float2*>(dV + off + 2 * tc) = make_float2(vx[0], vx[1]);
                 } else {
 #pragma unroll
                     for (int e = 0; e < DV / 4; ++e) {
                         *reinterpret_cast<float4*>(dK + off + 4 * tc + 64 * e) =
-                            make_float4(dk[a][4 * e] * scale, dk[a][4 * e + 1] * scale, dk[a][4 * e + 2] * scale,
-                                        dk[a][4 * e + 3] * scale);
+                            make_float4(kx[4 * e], kx[4 * e + 1], kx[4 * e + 2], kx[4 * e + 3]);
                         *reinterpret_cast<float4*>(dV + off + 4 * tc + 64 * e) =
-                            make_float4(dv[a][4 * e], dv[a][4 * e + 1], dv[a][4 * e + 2], dv[a][4 * e + 3]);
+                            make_float4(vx[4 * e], vx[4 * e + 1], vx[4 * e + 2], vx[4 * e + 3]);
                     }
                 }
             }

@@ -44,6 +44,7 @@ strict_dq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     constexpr int RM = C::RM, RN = C::RN, DV = C::DV, NCH = C::NCH, PSTR = C::PSTR, TR = C::TR;
 
     extern __shared__ uint8_t smem_raw[];
+    if (*reinterpret_cast<volatile unsigned*>(status) != 0) return;   // an earlier wait on this device gave up
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t sQ = base;
     const uint32_t sdO = sQ + C::Q_BYTES;

@@ -32,11 +32,17 @@ struct FwdCfg {
     static constexpr int RN = BN / 16;    // key columns per thread
     static constexpr int DV = D / 16;     // output columns per thread
     static constexpr int NCH = D / 32;    // 128-byte chunks per row
-    // row stride of P (floats); 16-byte pieces XOR-swizzled by row within groups of eight pieces
-    static constexpr int PSTR = (BN + 31) / 32 * 32;
+    // P is stored key-major as pairs of query rows: for key column j, row group tr owns 32 bytes =
+    // four (row 2q, row 2q+1) pairs of its own rows (pairs past RM are zero); 16-byte piece
+    // c = 2 tr + h sits at piece position c ^ (j & 7).  A packed two-lane FMA then takes a pair as
+    // one operand, and both the stores (one column per lane) and the loads (one row group per half
+    // warp) are conflict free.
+    static constexpr int RP = (RM + 1) / 2;   // row pairs per thread
+    static constexpr int PROW = TR * 32;      // bytes per key column
     static constexpr int Q_BYTES = BM * D * 4;
     static constexpr int KV_BYTES = BN * D * 4;
-    static constexpr int P_BYTES = BM * PSTR * 4;
+    static constexpr int P_BYTES = BN * PROW;
+    static_assert(RM <= 8, "a row group's pairs fill two 16-byte pieces");
     static constexpr int PAYLOAD = Q_BYTES + 2 * KV_BYTES + P_BYTES + 64;
     // Two 128-thread CTAs per SM must fit 2 x (SMEM + 1 KB reserved) into 228 KB, which leaves less
     // than the 1023 bytes a worst-case 1024-byte alignment of the tile base could need; the kernel
@@ -63,9 +69,10 @@ strict_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     const int Sk = GEN ? Sk_ : Sq;
     const int G = GEN ? G_ : 1;
     using C = FwdCfg<D, BM, BN, THREADS>;
-    constexpr int RM = C::RM, RN = C::RN, DV = C::DV, NCH = C::NCH, PSTR = C::PSTR, TR = C::TR;
+    constexpr int RM = C::RM, RN = C::RN, DV = C::DV, NCH = C::NCH, TR = C::TR, RP = C::RP, PROW = C::PROW;
 
     extern __shared__ uint8_t smem_raw[];
+    if (*reinterpret_cast<volatile unsigned*>(status) != 0) return;   // an earlier wait on this device gave up
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t sQ = base;
     const uint32_t sK = sQ + C::Q_BYTES;
@@ -109,15 +116,18 @@ strict_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         for (int ch = 0; ch < NCH; ++ch) tma_load_3d(sV + ch * BN * 128, &tmV, barV, ch * 32, 0, bhk);
     }
 
-    float o[RM][DV];
+    // O accumulators as packed pairs: o[q][e] = {row 2q, row 2q+1} of output column e
+    uint64_t o[RP][DV];
     float m[RM], l[RM];
 #pragma unroll
     for (int x = 0; x < RM; ++x) {
         m[x] = -INFINITY;
         l[x] = 0.f;
-#pragma unroll
-        for (int e = 0; e < DV; ++e) o[x][e] = 0.f;
     }
+#pragma unroll
+    for (int q = 0; q < RP; ++q)
+#pragma unroll
+        for (int e = 0; e < DV; ++e) o[q][e] = f2_pack(0.f, 0.f);
 
     mbar_wait(barQ, 0, status);
 
@@ -169,6 +179,7 @@ strict_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
 
         // ---- scale into the log2 domain, mask, online softmax ------------------------------
         const bool need_mask = (causal && (j0 + BN - 1 > i0 + off)) || (j0 + BN > Sk);
+        float alpha[2 * RP];
 #pragma unroll
         for (int x = 0; x < RM; ++x) {
             const int i = i0 + tr + TR * x;
@@ -188,59 +199,73 @@ strict_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
             mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 8));
             const float m_new = fmaxf(m[x], mx);    // finite from the first tile on (key 0 is never masked)
-            const float alpha = ex2(m[x] - m_new);
+            alpha[x] = ex2(m[x] - m_new);
             m[x] = m_new;
             float psum = 0.f;
-            // P[i][j] lives at row i, 16-byte piece (j/4) ^ (i & 7); i & 7 == tr & 7 for all of a thread's rows
-            const uint32_t prow = sP + (tr + TR * x) * PSTR * 4 + (tc & 3) * 4;
 #pragma unroll
             for (int y = 0; y < RN; ++y) {
                 const float p = ex2(s[x][y] - m_new);
                 psum += p;
-                sts32(prow + ((((tc >> 2) + 4 * y) ^ (tr & 7)) << 4), p);
+                s[x][y] = p;
             }
-            l[x] = fmaf(l[x], alpha, psum);
+            l[x] = fmaf(l[x], alpha[x], psum);
+        }
+        if constexpr (RM & 1) alpha[RM] = 1.f;
+        // P: this thread's rows of key column j = tc + 16 y as row pairs, two 16-byte stores per column
 #pragma unroll
-            for (int e = 0; e < DV; ++e) o[x][e] *= alpha;
+        for (int y = 0; y < RN; ++y) {
+            const uint32_t col = sP + (tc + 16 * y) * PROW;
+            const int jx = tc & 7;                      // (tc + 16 y) & 7
+            auto pv = [&](int x) { return x < RM ? s[x < RM ? x : 0][y] : 0.f; };
+            sts128f(col + (((2 * tr) ^ jx) << 4), pv(0), pv(1), pv(2), pv(3));
+            if constexpr (RM > 4) sts128f(col + (((2 * tr + 1) ^ jx) << 4), pv(4), pv(5), pv(6), pv(7));
+        }
+#pragma unroll
+        for (int q = 0; q < RP; ++q) {
+            const uint64_t a2 = f2_pack(alpha[2 * q], alpha[2 * q + 1]);
+#pragma unroll
+            for (int e = 0; e < DV; ++e) o[q][e] = f2_mul(o[q][e], a2);
         }
         __syncthreads();   // P visible
         mbar_wait(barV, ph, status);
 
-        // ---- O += P V : contraction along keys ----------------------------------------------
+        // ---- O += P V : contraction along keys, two query rows per packed FMA ------------------
+        // Per key: V's columns of this thread are loaded once and duplicated into both lanes, the
+        // row pairs of P come as they are stored; DV * RP packed FMAs follow.
         {
-            const uint32_t pa = sP + tr * PSTR * 4;
-            constexpr int kUnrollPV = (D == 64) ? 8 : 2;
+            const uint32_t pa = sP + ((2 * tr) << 4);
+            constexpr int kUnrollPV = (D == 32) ? 8 : 32;
 #pragma unroll kUnrollPV
-            for (int j8 = 0; j8 < BN / 8; ++j8) {
-                float4 p[2][RM];
+            for (int j = 0; j < BN; ++j) {
+                const int u = j & 7;
+                float vv[DV];
+                if constexpr (DV == 2) {
+                    const float2 t = lds64(sV + j * 128 + ((((tc >> 1)) ^ u) << 4) + (tc & 1) * 8);
+                    vv[0] = t.x; vv[1] = t.y;
+                } else {
 #pragma unroll
-                for (int hlf = 0; hlf < 2; ++hlf)
-#pragma unroll
-                    for (int x = 0; x < RM; ++x)
-                        p[hlf][x] = lds128(pa + x * TR * PSTR * 4 + (((2 * j8 + hlf) ^ (tr & 7)) << 4));
-#pragma unroll
-                for (int u = 0; u < 8; ++u) {
-                    const int j = j8 * 8 + u;
-                    float vv[DV];
-                    if constexpr (DV == 2) {
-                        const float2 t = lds64(sV + j * 128 + ((((tc >> 1)) ^ u) << 4) + (tc & 1) * 8);
-                        vv[0] = t.x; vv[1] = t.y;
-                    } else {
-#pragma unroll
-                        for (int e = 0; e < DV / 4; ++e) {
-                            const int piece = tc + 16 * e;
-                            const float4 t = lds128(sV + (piece >> 3) * (BN * 128) + j * 128 + (((piece & 7) ^ u) << 4));
-                            vv[4 * e + 0] = t.x; vv[4 * e + 1] = t.y; vv[4 * e + 2] = t.z; vv[4 * e + 3] = t.w;
-                        }
-                    }
-#pragma unroll
-                    for (int x = 0; x < RM; ++x) {
-                        const float4 pp = p[u >> 2][x];
-                        const float pv = (u & 3) == 0 ? pp.x : (u & 3) == 1 ? pp.y : (u & 3) == 2 ? pp.z : pp.w;
-#pragma unroll
-                        for (int e = 0; e < DV; ++e) o[x][e] = fmaf(pv, vv[e], o[x][e]);
+                    for (int e = 0; e < DV / 4; ++e) {
+                        const int piece = tc + 16 * e;
+                        const float4 t = lds128(sV + (piece >> 3) * (BN * 128) + j * 128 + (((piece & 7) ^ u) << 4));
+                        vv[4 * e + 0] = t.x; vv[4 * e + 1] = t.y; vv[4 * e + 2] = t.z; vv[4 * e + 3] = t.w;
                     }
                 }
+                uint64_t vd[DV];
+#pragma unroll
+                for (int e = 0; e < DV; ++e) vd[e] = f2_pack(vv[e], vv[e]);
+                // pieces 2 tr and 2 tr + 1 of column j: positions (2 tr) ^ u and that with bit 0 flipped
+                const uint32_t pj = (pa + j * PROW) ^ static_cast<uint32_t>(u << 4);
+                const U64x2 p01 = lds128_pairs(pj);
+                uint64_t pp[4] = {p01.lo, p01.hi, 0ull, 0ull};
+                if constexpr (RP > 2) {
+                    const U64x2 p23 = lds128_pairs(pj ^ 16u);
+                    pp[2] = p23.lo;
+                    pp[3] = p23.hi;
+                }
+#pragma unroll
+                for (int q = 0; q < RP; ++q)
+#pragma unroll
+                    for (int e = 0; e < DV; ++e) o[q][e] = f2_fma(pp[q], vd[e], o[q][e]);
             }
         }
         __syncthreads();   // every warp is done with this V tile and with P
@@ -260,16 +285,23 @@ strict_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         lt += __shfl_xor_sync(0xffffffffu, lt, 4);
         lt += __shfl_xor_sync(0xffffffffu, lt, 8);
         const int i = i0 + tr + TR * x;
+        float ox[DV];
+#pragma unroll
+        for (int e = 0; e < DV; ++e) {
+            float lo, hi;
+            f2_unpack(o[x >> 1][e], lo, hi);
+            ox[e] = (x & 1) ? hi : lo;
+        }
         if (i < Sq) {
             const float inv = 1.0f / lt;
             float* orow = O + (static_cast<size_t>(bh) * Sq + i) * D;
             if constexpr (DV == 2) {
-                *reinterpret_cast<float2*>(orow + 2 * tc) = make_float2(o[x][0] * inv, o[x][1] * inv);
+                *reinterpret_cast<float2*>(orow + 2 * tc) = make_float2(ox[0] * inv, ox[1] * inv);
             } else {
 #pragma unroll
                 for (int e = 0; e < DV / 4; ++e)
                     *reinterpret_cast<float4*>(orow + 4 * tc + 64 * e) =
-                        make_float4(o[x][4 * e] * inv, o[x][4 * e + 1] * inv, o[x][4 * e + 2] * inv, o[x][4 * e + 3] * inv);
+                        make_float4(ox[4 * e] * inv, ox[4 * e + 1] * inv, ox[4 * e + 2] * inv, ox[4 * e + 3] * inv);
             }
             if (tc == 0) LSE[static_cast<size_t>(bh) * Sq + i] = (m[x] + log2f(lt)) * kLn2;
         }

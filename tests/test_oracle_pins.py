@@ -82,6 +82,8 @@ def test_matches_dense_matrix_form(S, D, causal):
     np.testing.assert_allclose(lse2[0, 0], lse[0, 0], rtol=0, atol=0)
     np.testing.assert_allclose(lse[0, 0], ref["LSE"], **tol)
     np.testing.assert_allclose(P, ref["P"], **tol)
+    visible = np.tril(np.ones((S, S), dtype=bool)) if causal else np.ones((S, S), dtype=bool)
+    np.testing.assert_allclose(dP, np.where(visible, dO @ V.T, 0.0), **tol)   # dP on its own (masked entries are 0)
     np.testing.assert_allclose(dS, ref["dS"], **tol)
     np.testing.assert_allclose(dq[0, 0], ref["dQ"], **tol)
     np.testing.assert_allclose(dk[0, 0], ref["dK"], **tol)

@@ -136,8 +136,8 @@ def _workload_parity(name, heads):
     return rep
 
 
-def test_long_context_head_subset():
-    _workload_parity("long_context", [0, 13, 31])
+def test_long_context_all_heads():
+    _workload_parity("long_context", None)
 
 
 @pytest.mark.parametrize("name,heads", [

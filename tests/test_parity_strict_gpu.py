@@ -39,6 +39,7 @@ def test_vit_b_shaped_ragged_all_heads():
 @pytest.mark.parametrize("name,heads", [
     ("decoder_sweep_S512", [0, 37, 90, 127]),
     ("decoder_sweep_S1024", [0, 127]),
+    ("decoder_sweep_S2048", [64]),
 ])
 def test_decoder_sweep_outliers_head_subset(name, heads):
     # Scores reach +-64 here and |dQ|,|dK| reach tens: the absolute bound is applied

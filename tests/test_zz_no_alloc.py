@@ -1,7 +1,8 @@
 """mgn_attn_bwd_noalloc: the backward entry point for callers that cannot allocate device memory
 (plug-ins that are only handed tensors, serving loops where cudaMalloc would stall the GPU).
-It must give what mgn_attn_bwd gives, call after call, although every call reuses the same
-built-in scratch array and finds the previous call's leftovers in it.
+It must give what mgn_attn_bwd gives -- and what the f64 oracle gives, within the tolerances of
+the other parity tests -- call after call, although every call reuses the same built-in scratch
+array and finds the previous call's leftovers in it.
 
 Collected last on purpose (file name), so a run that stops at the first failure has already
 run every other test."""
@@ -56,6 +57,15 @@ def test_noalloc_backward_matches_workspace_backward_twice_in_a_row(mode, dtype,
                 assert hp.max_abs(g64, w64) <= hp.STRICT_MAX_ABS
         # dK and dV do not depend on accumulation order: identical bits
         assert torch.equal(got[1], want[1]) and torch.equal(got[2], want[2])
+
+        # and against the f64 oracle directly, at the tolerances of the other parity tests
+        host = [t.cpu() for t in (q, k, v, d_o)]
+        ref = hp.run_oracle(*host, causal, scale)
+        mine = hp.select({"dQ": got[0].cpu(), "dK": got[1].cpu(), "dV": got[2].cpu()}, B, H)
+        if mode == mgn.MODE_STRICT_F32:
+            hp.check_strict(mine, ref, names=("dQ", "dK", "dV"), label=f"noalloc call {call} ")
+        else:
+            hp.check_fast(mine, ref, names=("dQ", "dK", "dV"), label=f"noalloc call {call} ")
 
 
 def test_noalloc_rejects_sizes_beyond_its_scratch():
