@@ -29,9 +29,15 @@ sys.path.insert(0, ROOT)
 from paper_2608_01563_b200 import inputs as synth  # noqa: E402
 
 METRIC = "attention fwd+bwd TFLOP/s per B200 (strict f32, bf16) and % of matching peak"
-# dram__bytes_read.sum + dram__bytes_write.sum of the backward main kernel, one launch, from the ncu
-# captures summarised under profiles/ (same workload and launch configuration as the bench)
-NCU_TRAFFIC_BYTES = {("strict", "gpt2_small"): 146.9e6 + 45.5e6, ("fast", "long_context"): 440.2e6 + 214.6e6}
+# dram__bytes_read.sum + dram__bytes_write.sum of the backward main kernel, one launch, as recorded in the
+# ncu summary named beside it (same workload and launch configuration as the bench; re-taken when that
+# kernel changes -- the record carries the file so that a stale figure can be told)
+NCU_TRAFFIC = {
+    ("strict", "gpt2_small"): (146.9e6 + 45.5e6, "profiles/strict_fwd_bwd_gpt2_small.md",
+                               "strict_bwd_kernel<64,64,64,128,false,true>"),
+    ("fast", "long_context"): (440.2e6 + 214.6e6, "profiles/fast_fwd_bwd_long_context.md",
+                               "fast_bwd_kernel<128,false,true>"),
+}
 SM_COUNT = 148
 FP32_LANES_PER_SM = 128
 
@@ -165,6 +171,69 @@ def quick_measure(mgn, w, mode, dtype, steps, warmup):
     return fwd_ms, bwd_ms
 
 
+def fast_mode_summary(mgn, peaks, gpu_index, steps, warmup):
+    """The fast (bf16 tensor-core) mode on its own target workloads, with a clock record of its own:
+    long_context timed like the headline (whole calls and the backward main kernel through the
+    profile-event hook), then the decoder sweep on its own heavy-tailed inputs.  Compact on purpose:
+    it is the last key of the JSON line."""
+    wf = synth.WORKLOADS["long_context"]
+    mode, dt = mgn.MODE_FAST_BF16, torch.bfloat16
+    q, k, v, d_o = (t.cuda() for t in synth.make_inputs(wf, dtype=dt))
+    o = torch.empty_like(q)
+    lse = torch.empty(wf.B, wf.H, wf.S, device="cuda", dtype=torch.float32)
+    dq, dk, dv = (torch.empty_like(q) for _ in range(3))
+    ws = mgn.alloc_workspace(wf.B, wf.H, wf.S, wf.D, mode)
+    fwd = lambda: mgn.mgn_attn_fwd(q, k, v, o, lse, wf.causal, wf.scale, mode)
+    bwd = lambda: mgn.mgn_attn_bwd(q, k, v, o, d_o, lse, dq, dk, dv, ws, wf.causal, wf.scale, mode)
+    for _ in range(warmup):
+        fwd(); bwd()
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    e = [ev() for _ in range(2 * steps + 1)]
+    main = [(ev(), ev()) for _ in range(steps)]
+    for a, b in main:
+        a.record(); b.record()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(gpu_index)
+    sampler.start()
+    time.sleep(0.2)
+    t0 = time.time()
+    e[0].record()
+    for i in range(steps):
+        fwd()
+        e[2 * i + 1].record()
+        mgn.mgn_attn_profile_events(main[i][0].cuda_event, main[i][1].cuda_event)
+        bwd()
+        mgn.mgn_attn_profile_events(None, None)
+        e[2 * i + 2].record()
+    torch.cuda.synchronize()
+    t_cont = time.time()
+    while time.time() - t_cont < 0.4:       # keep the same load up until the sampler has seen it
+        for _ in range(10):
+            fwd(); bwd()
+        torch.cuda.synchronize()
+    clocks = sampler.stop(t0, time.time())
+    mgn.mgn_attn_check()
+    f_ms = statistics.median(e[2 * i].elapsed_time(e[2 * i + 1]) for i in range(steps))
+    b_ms = statistics.median(e[2 * i + 1].elapsed_time(e[2 * i + 2]) for i in range(steps))
+    bm_ms = statistics.median(a.elapsed_time(b) for a, b in main)
+    tfl = flops(wf, "sum") / ((f_ms + b_ms) * 1e-3) / 1e12
+    out = {"workload": wf.name, "fwd_ms": round(f_ms, 4), "bwd_ms": round(b_ms, 4), "bwd_main_ms": round(bm_ms, 4),
+           "sum_tflops": round(tfl, 1), "frac_burst": round(tfl / peaks["bf16_tflops"], 3),
+           "frac_sustained": round(tfl / peaks["bf16_tflops_sustained"], 3),
+           "clocks": {"sm_mhz": clocks.get("sm_mhz"), "reasons": clocks.get("reasons")}}
+    del q, k, v, d_o, o, lse, dq, dk, dv, ws
+    sweep = {}
+    for name in [n for n in synth.WORKLOADS if n.startswith("decoder_sweep_S")]:
+        wt = synth.WORKLOADS[name]
+        steps_t = max(2, min(steps, 5 if wt.S <= 2048 else 2))
+        fm, bm = quick_measure(mgn, wt, mode, dt, steps_t, 3)
+        t = flops(wt, "sum") / ((fm + bm) * 1e-3) / 1e12
+        sweep[f"S{wt.S}"] = {"fwd_ms": round(fm, 4), "bwd_ms": round(bm, 4), "sum_tflops": round(t, 1),
+                             "frac_burst": round(t / peaks["bf16_tflops"], 3)}
+    out["decoder_sweep"] = sweep
+    return out
+
+
 def quick_measure_ext(mgn, w, mode, dtype, steps, warmup):
     """Device-resident timing of one cross-attention / grouped-head workload (CUDA events)."""
     q, k, v, d_o = (t.cuda() for t in synth.make_inputs_ext(w, dtype=dtype))
@@ -266,6 +335,7 @@ def cpu_info():
 
 
 _oracle_inputs = {}
+_oracle_outputs = {}
 
 
 def time_oracle(w, dtype, heads, repeats=1):
@@ -274,6 +344,7 @@ def time_oracle(w, dtype, heads, repeats=1):
     key = (w.name, w.sweep, dtype, heads)
     if key not in _oracle_inputs:
         _oracle_inputs.clear()
+        _oracle_outputs.clear()
         _oracle_inputs[key] = [t.double().numpy() for t in synth.make_inputs(w, dtype=dtype, heads=heads)]
     a = _oracle_inputs[key]
     best_f = best_b = float("inf")
@@ -281,10 +352,29 @@ def time_oracle(w, dtype, heads, repeats=1):
         t0 = time.perf_counter()
         orc.attn_fwd(a[0], a[1], a[2], w.causal, w.scale)
         t1 = time.perf_counter()
-        orc.attn_bwd(a[0], a[1], a[2], a[3], w.causal, w.scale)
+        _oracle_outputs[key] = orc.attn_bwd(a[0], a[1], a[2], a[3], w.causal, w.scale)
         t2 = time.perf_counter()
         best_f, best_b = min(best_f, t1 - t0), min(best_b, t2 - t1)
     return best_f, best_b, orc.max_threads()
+
+
+def parity_figures(w, dtype, heads, gpu_outputs):
+    """Per-tensor error of the timed workload's CUDA outputs against the oracle's outputs on the head
+    subset the cpu_baseline leg has just computed: rel-L2, the literal max-abs and the max-abs relative to
+    max(1, max|ref|) (the strict gate's form on the heavy-tailed decoder sweep)."""
+    import numpy as np
+    ref = _oracle_outputs.get((w.name, w.sweep, dtype, heads))
+    if ref is None:
+        return None
+    out = {"heads": f"first {heads} of {w.BH}"}
+    for name, got, want in zip(("O", "LSE", "dQ", "dK", "dV"), gpu_outputs, ref):
+        g = got.reshape(1, w.BH, *got.shape[2:])[:, :heads].double().cpu().numpy()
+        err = np.abs(g - want)
+        den = float(np.linalg.norm(want.ravel()))
+        out[name] = {"rel_l2": float(np.linalg.norm((g - want).ravel())) / (den if den > 0 else 1.0),
+                     "max_abs": float(err.max()),
+                     "max_abs_normalised": float(err.max()) / max(1.0, float(np.abs(want).max()))}
+    return out
 
 
 def cpu_baseline(w, dtype, budget_s=15.0):
@@ -311,7 +401,7 @@ def cpu_baseline(w, dtype, budget_s=15.0):
     return {"value": fl / (tf + tb) / 1e12, "unit": "TFLOP/s", "cores": threads, "kind": "oracle",
             "sample": (f"first {heads} of {w.BH} heads of {w.name}, mean of {passes} passes "
                        f"(f64, fwd {tf:.2f} s + bwd {tb:.2f} s per pass)"),
-            "cpu_model": cpu_info()}
+            "cpu_model": cpu_info(), "heads": heads}
 
 
 def run_reference(args, w, dtype):
@@ -554,8 +644,10 @@ def main():
             "fwd_ms": fwd_call_ms, "bwd_ms": bwd_call_ms,
             "roofline": {"kernel": "bwd_main (fused dK/dV/dQ)", "bound": bound, "achieved": bwd_main_tflops,
                          "peak": peak, "unit": "TFLOP/s", "frac": bwd_main_tflops / peak,
-                         "traffic": NCU_TRAFFIC_BYTES.get((args.mode, w.name)),
-                         "traffic_unit": "bytes per launch (ncu dram read+write, see profiles/)",
+                         "traffic": NCU_TRAFFIC.get((args.mode, w.name), (None,))[0],
+                         "traffic_unit": "bytes per launch (ncu dram read+write)",
+                         "traffic_source": list(NCU_TRAFFIC.get((args.mode, w.name), (None, None, None))[1:]),
+                         "algorithmic_bytes": w.BH * w.S * (8 * w.D * qd.element_size() + 8),
                          "ms_per_launch": bwd_main_ms, "peak_source": peak_note,
                          "fwd_kernel": {"achieved": fwd_main_tflops, "frac": fwd_main_tflops / peak,
                                         "ms_per_launch": fwd_main_ms}},
@@ -571,18 +663,6 @@ def main():
             measured = mgn.mgn_measure_fp32_ffma_tflops()
             line["fp32_ffma_measured_tflops"] = measured
             line["frac_of_measured_ffma_peak"] = value / world / measured if measured > 0 else None
-        if world == 1 and args.mode == "strict" and args.workload is None and not args.no_fast:
-            # the other arithmetic mode of the same library on its own target workload, for the record
-            wf = synth.WORKLOADS["long_context"]
-            f_ms, b_ms = quick_measure(mgn, wf, mgn.MODE_FAST_BF16, torch.bfloat16, K, args.warmup)
-            tf = lambda which, ms: flops(wf, which) / (ms * 1e-3) / 1e12
-            line["fast_mode"] = {
-                "workload": wf.name, "dtype": "bf16", "fwd_ms": f_ms, "bwd_ms": b_ms,
-                "fwd_tflops": tf("fwd", f_ms), "bwd_tflops": tf("bwd", b_ms),
-                "sum_tflops": flops(wf, "sum") / ((f_ms + b_ms) * 1e-3) / 1e12,
-                "peak_tflops": peaks["bf16_tflops"], "peak_note": f"{peak_src} dense bf16 burst",
-                "frac_of_peak": flops(wf, "sum") / ((f_ms + b_ms) * 1e-3) / 1e12 / peaks["bf16_tflops"],
-            }
         if world == 1 and args.workload is None and not args.no_fast:
             # cross-attention and grouped key/value heads (mgn_attn_*_ext), in this run's arithmetic mode
             mode_peak = peak if args.mode == "strict" else peaks["bf16_tflops"]
@@ -614,6 +694,12 @@ def main():
                     line["accel_policy"] = measure_accel_policy(mgn, w, K, args.warmup)
         if world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline(w, dtype)
+            # error of the timed workload's outputs against the oracle outputs that leg has just produced
+            line["parity"] = parity_figures(w, dtype, line["cpu_baseline"].pop("heads"), (o, lse, dq, dk, dv))
+        if world == 1 and args.mode == "strict" and args.workload is None and not args.no_fast:
+            # The other arithmetic mode of the same library on its own target workloads.  Last key of
+            # the line, and compact, so that a reader who keeps only the end of the line still has it.
+            line["fast_mode"] = fast_mode_summary(mgn, peaks, gpu_index, K, args.warmup)
         print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()

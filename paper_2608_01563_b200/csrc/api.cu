@@ -87,8 +87,10 @@ namespace {
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
-// Workspace layout: [delta: BH*S f32][fast mode only: dQ accumulator BH*S*D f32], 256-byte granules.
+// Workspace layout: [delta: BH*S f32][fast mode only: 256 bytes holding the work-item counter of the
+// persistent kernel][fast mode only: dQ accumulator BH*S*D f32], 256-byte granules.
 size_t ws_delta_bytes(size_t rows) { return align_up(rows * sizeof(float), 256); }
+constexpr size_t kSchedBytes = 256;
 
 }  // namespace
 extern "C" size_t mgn_attn_bwd_workspace_bytes(int B, int H, int S, int D, int mode);
@@ -120,7 +122,7 @@ size_t mgn_attn_bwd_workspace_bytes(int B, int H, int S, int D, int mode)
     if (check_common(B, H, S, D, 0, 1.0f, mode) != MGN_OK) return 0;
     const size_t rows = static_cast<size_t>(B) * H * S;
     size_t bytes = ws_delta_bytes(rows);
-    if (mode == MGN_MODE_FAST_BF16) bytes += align_up(rows * D * sizeof(float), 256);
+    if (mode == MGN_MODE_FAST_BF16) bytes += kSchedBytes + align_up(rows * D * sizeof(float), 256);
     return bytes;
 }
 
@@ -203,9 +205,10 @@ int mgn_attn_bwd_ext(const void* q, const void* k, const void* v, const void* o,
 
     // delta, and the dQ accumulation target cleared in the same pass (dQ is accumulated by
     // floating-point reductions: in place in strict mode, in an f32 workspace tensor in fast mode)
-    float* dq_acc = fast ? reinterpret_cast<float*>(static_cast<char*>(workspace) + ws_delta_bytes(rows))
+    unsigned* sched = fast ? reinterpret_cast<unsigned*>(static_cast<char*>(workspace) + ws_delta_bytes(rows)) : nullptr;
+    float* dq_acc = fast ? reinterpret_cast<float*>(static_cast<char*>(workspace) + ws_delta_bytes(rows) + kSchedBytes)
                          : static_cast<float*>(dq);
-    cudaError_t e = mgn::launch_bwd_preprocess(o, d_o, delta, dq_acc, rows, D, fast ? 1 : 0, st);
+    cudaError_t e = mgn::launch_bwd_preprocess(o, d_o, delta, dq_acc, sched, rows, D, fast ? 1 : 0, st);
     if (e != cudaSuccess) return MGN_ERR_CUDA;
     MainKernelTimer timer(st);
     if (!fast)
@@ -214,7 +217,7 @@ int mgn_attn_bwd_ext(const void* q, const void* k, const void* v, const void* o,
                                    static_cast<float*>(dq), static_cast<float*>(dk), static_cast<float*>(dv), status,
                                    st);
     else
-        e = mgn::launch_fast_bwd(p, q, k, v, d_o, lse, delta, dq_acc, dq, dk, dv, status, st);
+        e = mgn::launch_fast_bwd(p, q, k, v, d_o, lse, delta, dq_acc, dq, dk, dv, sched, status, st);
     return e == cudaSuccess ? MGN_OK : MGN_ERR_CUDA;
 }
 
@@ -234,11 +237,12 @@ int mgn_attn_bwd_deterministic(const void* q, const void* k, const void* v, cons
     const size_t rows = static_cast<size_t>(B) * H * S_q;
     float* delta = static_cast<float*>(workspace);
     const bool fast = mode == MGN_MODE_FAST_BF16;
-    cudaError_t e = mgn::launch_bwd_preprocess(o, d_o, delta, nullptr, rows, D, fast ? 1 : 0, st);
+    unsigned* sched = fast ? reinterpret_cast<unsigned*>(static_cast<char*>(workspace) + ws_delta_bytes(rows)) : nullptr;
+    cudaError_t e = mgn::launch_bwd_preprocess(o, d_o, delta, nullptr, sched, rows, D, fast ? 1 : 0, st);
     if (e != cudaSuccess) return MGN_ERR_CUDA;
     MainKernelTimer timer(st);
     if (fast) {
-        e = mgn::launch_fast_bwd(p, q, k, v, d_o, lse, delta, nullptr, nullptr, dk, dv, status, st);
+        e = mgn::launch_fast_bwd(p, q, k, v, d_o, lse, delta, nullptr, nullptr, dk, dv, sched, status, st);
         if (e != cudaSuccess) return MGN_ERR_CUDA;
         e = mgn::launch_fast_dq(p, q, k, v, d_o, lse, delta, dq, status, st);
         return e == cudaSuccess ? MGN_OK : MGN_ERR_CUDA;

@@ -6,6 +6,7 @@
 #include <cuda_bf16.h>
 
 #include "kernels.h"
+#include "ptx.cuh"
 
 namespace mgn {
 namespace {
@@ -34,8 +35,10 @@ __device__ __forceinline__ uint4 ld_hint(const uint4* a, uint64_t pol) {
 template <int LANES, bool BF16>
 __global__ void __launch_bounds__(256)
 bwd_preprocess_kernel(const uint4* __restrict__ o, const uint4* __restrict__ d_o, float* __restrict__ delta,
-                      float4* __restrict__ zero, size_t rows)
+                      float4* __restrict__ zero, unsigned* __restrict__ counter, size_t rows)
 {
+    pdl_launch_dependents();   // the backward main kernel may set itself up while this one streams
+    if (counter && blockIdx.x == 0 && threadIdx.x == 0) *counter = 0u;
     constexpr int ROWS_PER_BLOCK = 256 / LANES;
     const int lane = threadIdx.x % LANES;
     const int sub = threadIdx.x / LANES;
@@ -74,33 +77,33 @@ bwd_preprocess_kernel(const uint4* __restrict__ o, const uint4* __restrict__ d_o
 }
 
 template <int LANES, bool BF16>
-cudaError_t run(const void* o, const void* d_o, float* delta, float* zero, size_t rows, cudaStream_t st)
+cudaError_t run(const void* o, const void* d_o, float* delta, float* zero, unsigned* counter, size_t rows, cudaStream_t st)
 {
     constexpr int ROWS_PER_BLOCK = 256 / LANES;
     size_t blocks = (rows + ROWS_PER_BLOCK - 1) / ROWS_PER_BLOCK;
     const size_t cap = 148u * 8u * 4u;
     if (blocks > cap) blocks = cap;
     bwd_preprocess_kernel<LANES, BF16><<<static_cast<unsigned>(blocks), 256, 0, st>>>(
-        static_cast<const uint4*>(o), static_cast<const uint4*>(d_o), delta, reinterpret_cast<float4*>(zero), rows);
+        static_cast<const uint4*>(o), static_cast<const uint4*>(d_o), delta, reinterpret_cast<float4*>(zero), counter, rows);
     return cudaGetLastError();
 }
 
 }  // namespace
 
-cudaError_t launch_bwd_preprocess(const void* o, const void* d_o, float* delta, float* zero, size_t rows, int D,
-                                  int is_bf16, cudaStream_t st)
+cudaError_t launch_bwd_preprocess(const void* o, const void* d_o, float* delta, float* zero, unsigned* counter,
+                                  size_t rows, int D, int is_bf16, cudaStream_t st)
 {
     if (is_bf16) {
         switch (D) {
-            case 32:  return run<4, true>(o, d_o, delta, zero, rows, st);
-            case 64:  return run<8, true>(o, d_o, delta, zero, rows, st);
-            case 128: return run<16, true>(o, d_o, delta, zero, rows, st);
+            case 32:  return run<4, true>(o, d_o, delta, zero, counter, rows, st);
+            case 64:  return run<8, true>(o, d_o, delta, zero, counter, rows, st);
+            case 128: return run<16, true>(o, d_o, delta, zero, counter, rows, st);
         }
     } else {
         switch (D) {
-            case 32:  return run<8, false>(o, d_o, delta, zero, rows, st);
-            case 64:  return run<16, false>(o, d_o, delta, zero, rows, st);
-            case 128: return run<32, false>(o, d_o, delta, zero, rows, st);
+            case 32:  return run<8, false>(o, d_o, delta, zero, counter, rows, st);
+            case 64:  return run<16, false>(o, d_o, delta, zero, counter, rows, st);
+            case 128: return run<32, false>(o, d_o, delta, zero, counter, rows, st);
         }
     }
     return cudaErrorInvalidValue;

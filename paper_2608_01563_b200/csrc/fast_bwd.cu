@@ -62,7 +62,7 @@ struct Cfg {
     static constexpr int OFF_DQ = OFF_DS + DS_BYTES;           // dQ staging: 2 boxes of 128 rows x 32 f32
     static constexpr int OFF_STAT = OFF_DQ + 2 * CHUNK_BYTES;  // [2 stages][lse2 | delta][128] f32
     static constexpr int OFF_BAR = OFF_STAT + 2 * 2 * BLK * 4;
-    static constexpr int PAYLOAD = OFF_BAR + 176;   // 21 barriers + the tensor-memory slot
+    static constexpr int PAYLOAD = OFF_BAR + 224;   // 25 barriers, the tensor-memory slot, four work-item slots
     // Aligning the tile base to 1024 bytes can cost up to 1023 bytes; only 864 are left under the
     // 227 KB per-block limit at D = 128.  The kernel checks the slack it actually got.
     static constexpr int SMEM = (PAYLOAD + 1024 <= 232448) ? PAYLOAD + 1024 : 232448;
@@ -72,16 +72,42 @@ struct Cfg {
 
 enum { B_KV = 0, B_QFULL = 1, B_QEMPTY = 3, B_DOFULL = 5, B_DOEMPTY = 6, B_SFULL = 7, B_DPFULL = 8,
        B_PDSFULL = 9, B_DQFULL = 10, B_DQEMPTY = 11, B_DVFULL = 12, B_DSEMPTY = 13, B_PFULL = 14, B_STATFULL = 15 /* two: one per buffer */,
-       B_KVEMPTY = 17, B_DKVEMPTY = 18, B_PDSFULL1 = 19 /* dS of odd pairs; B_PDSFULL: even pairs */, B_DKFULL = 20, B_COUNT = 21 };
+       B_KVEMPTY = 17, B_DKVEMPTY = 18, B_PDSFULL1 = 19 /* dS of odd pairs; B_PDSFULL: even pairs */, B_DKFULL = 20,
+       B_ITEM = 21 /* four: work-item slot k & 3 has been filled */, B_COUNT = 25 };
 
-// Work items are (key block, head).  Two orders, chosen by the launcher (pick_schedule):
-//   order 0, block-major: items sorted heaviest first (key block 0 of every head, then block 1, ...),
-//     dealt to the CTAs in tiers of G, odd tiers backwards (snake).  Balanced for any item count,
-//     but the CTAs running at one time touch every head.
-//   order 1, head-major: all blocks of a head are consecutive, alternating heaviest / lightest
-//     remaining block, so that two consecutive items always weigh the same; CTA c takes the item
-//     pairs c, c+G, c+2G, ...  The CTAs running at one time share a few heads, whose dQ accumulator,
-//     Q and dO stay in L2.  Balanced only when there are many item pairs per CTA.
+// Work items are (key block, head), handed out at run time: the producer thread of a CTA takes the
+// next position of one global list with an atomic add on a counter in the workspace (cleared by the
+// preprocess kernel) and publishes it to the other roles through a four-slot ring in shared memory.
+// The list keeps both the load balance of a heaviest-first order and the L2 locality of a
+// head-by-head order: heads are taken in groups of Hg whose tensors fit L2 (the f32 dQ accumulator,
+// Q, dO, K, V of a group); a group's heavy half (its first key blocks, which see the most query
+// blocks under a causal mask) is interleaved with the light half of the group before it, so that
+// every stretch of the list holds the same mix of weights, the list starts with heavy items only and
+// ends with the lightest ones.  Hg = all heads gives a plain heaviest-first list, Hg = 1 a
+// head-by-head one.  Positions whose head does not exist (last group) are skipped.
+__device__ __forceinline__ int pos_to_item(unsigned pos, int nb, int BHkv, int Hg) {
+    const int nh = nb / 2, nl = nb - nh, ng = (BHkv + Hg - 1) / Hg;
+    const unsigned first = static_cast<unsigned>(Hg) * nh, per = static_cast<unsigned>(Hg) * nb;
+    int g, kb, c;
+    if (pos < first) {                       // phase 0: heavy half of group 0
+        g = 0; kb = static_cast<int>(pos) / Hg; c = static_cast<int>(pos) % Hg;
+    } else {
+        const unsigned q = pos - first;
+        const int ph = 1 + static_cast<int>(q / per), rem = static_cast<int>(q % per);
+        if (ph >= ng) {                      // last phase: light half of the last group
+            if (ph > ng || rem >= Hg * nl) return -1;
+            g = ng - 1; kb = nh + rem / Hg; c = rem % Hg;
+        } else if (rem < nh * 2 * Hg) {      // rows of Hg heavy items of group ph, then Hg light items of group ph - 1
+            const int r = rem / (2 * Hg);
+            c = rem % (2 * Hg);
+            if (c < Hg) { g = ph; kb = r; } else { g = ph - 1; kb = nh + r; c -= Hg; }
+        } else {                             // odd number of blocks: the lightest block of group ph - 1
+            g = ph - 1; kb = nb - 1; c = rem - nh * 2 * Hg;
+        }
+    }
+    const int head = g * Hg + c;
+    return head < BHkv ? kb * BHkv + head : -2;   // -2: no such head, take the next position
+}
 // An item is one key block of one key/value head; its pairs run over the query heads of the group
 // and, for each, over the query blocks that see the key block.
 // GEN = false is the square multi-head case (Sk == Sq, G == 1): the head mapping, the offset and the
@@ -93,19 +119,14 @@ struct Item {
     __device__ __forceinline__ int i0(int n) const { return (qb0 + (GEN ? n % nq : n)) * BLK; }   // first query row of pair n
 };
 template <bool GEN>
-__device__ __forceinline__ Item<GEN> make_item(int it, const Dims& dm, int causal, int order) {
+__device__ __forceinline__ Item<GEN> make_item(int it, const Dims& dm, int causal) {
     Item<GEN> w;
     const int Sk = GEN ? dm.Sk : dm.Sq, G = GEN ? dm.G : 1, off = GEN ? dm.off : 0;
-    const int nb = (Sk + BLK - 1) / BLK, nqb = (dm.Sq + BLK - 1) / BLK;
+    const int nqb = (dm.Sq + BLK - 1) / BLK;
     const int Hkv = dm.H / G, BHkv = dm.BH / G;
-    if (order == 0) {
-        w.kb = it / BHkv;
-        w.bhk = it % BHkv;
-    } else {
-        w.bhk = it / nb;
-        const int j = it % nb;
-        w.kb = (j & 1) ? nb - 1 - (j >> 1) : (j >> 1);
-    }
+    w.kb = it / BHkv;                                     // pos_to_item's encoding
+    w.bhk = it % BHkv;
+    (void)Sk;
     w.bhq0 = GEN ? (w.bhk / Hkv) * dm.H + (w.bhk % Hkv) * G : w.bhk;
     w.j0 = w.kb * BLK;
     w.qb0 = causal ? max(w.j0 - off, 0) / BLK : 0;       // first query block with a row that sees key j0
@@ -123,7 +144,7 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                 const __grid_constant__ CUtensorMap tmdQ,
                 const float* __restrict__ LSE, const float* __restrict__ DELTA,
                 __nv_bfloat16* __restrict__ dK, __nv_bfloat16* __restrict__ dV,
-                const Dims dm, int causal, int order, float scale, unsigned* status)
+                const Dims dm, int causal, int Hg, unsigned* __restrict__ sched, float scale, unsigned* status)
 {
     using C = Cfg<D>;
     extern __shared__ uint8_t smem_raw[];
@@ -143,9 +164,30 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     }
 
     const int Sq = dm.Sq, Sk = GEN ? dm.Sk : dm.Sq, coff = GEN ? dm.off : 0;
-    const int n_items = ((Sk + BLK - 1) / BLK) * (dm.BH / (GEN ? dm.G : 1));
-    const int G = static_cast<int>(gridDim.x), cta = static_cast<int>(blockIdx.x);
-    const int n_tiers = 2 * ((n_items + 2 * G - 1) / (2 * G));   // upper bound on items per CTA in either order
+    const int n_kb = (Sk + BLK - 1) / BLK, BHkv = dm.BH / (GEN ? dm.G : 1);
+    const unsigned n_pos = static_cast<unsigned>((BHkv + Hg - 1) / Hg) * Hg * n_kb;   // list positions, skipped ones included
+    const uint32_t item_slot = tmem_slot + 16;
+    // Work item k of this CTA (-1: none left).  The producer thread takes it from the global list and
+    // publishes it; every other role reads it from slot k & 3.  A slot is rewritten four items later:
+    // the producer loads item k only after both issuers have finished item k - 2, and by then every
+    // role has read the slots up to k - 2.
+    auto take_item = [&](int k) -> int {
+        int it = -1;
+        for (;;) {
+            const unsigned pos = atomicAdd(sched, 1u);
+            if (pos >= n_pos) break;
+            it = pos_to_item(pos, n_kb, BHkv, Hg);
+            if (it != -2) break;
+        }
+        if (it == -2) it = -1;
+        asm volatile("st.shared.u32 [%0], %1;" ::"r"(item_slot + 4u * (k & 3)), "r"(it) : "memory");
+        mbar_arrive(bar(B_ITEM + (k & 3)));
+        return it;
+    };
+    auto read_item = [&](int k) -> int {
+        if (!mbar_wait(bar(B_ITEM + (k & 3)), (k >> 2) & 1, status)) return -1;
+        return static_cast<int>(lds32u(item_slot + 4u * (k & 3)));
+    };
     const float c2 = scale * kLog2e;
 
     if (tid == 0) {
@@ -165,6 +207,10 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = lds32u(tmem_slot);
+    // Launched as a programmatic dependent of the preprocess kernel: everything above overlapped its
+    // tail; delta, the cleared accumulator and the work-item counter are read only after this wait.
+    pdl_launch_dependents();
+    pdl_wait();
 
     if (warp < 4) {
         reg_dealloc<104>();
@@ -172,10 +218,10 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         // ------------------------------------------------------------------ TMA producer
         {
             int g = 0;                                          // pairs loaded so far (all items)
-            for (int k = 0; k < n_tiers; ++k) {
-                const int it = item_index(cta, k, G, n_items, order);
+            for (int k = 0;; ++k) {
+                const int it = take_item(k);
                 if (it < 0) break;
-                const Item<GEN> w = make_item<GEN>(it, dm, causal, order);
+                const Item<GEN> w = make_item<GEN>(it, dm, causal);
                 mbar_wait(bar(B_KVEMPTY), (k & 1) ^ 1, status);  // both issuers are done with the previous K, V
                 mbar_arrive_expect_tx(bar(B_KV), 2 * C::TILE_BYTES);
 #pragma unroll
@@ -221,10 +267,10 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                     umma_commit(bar(B_SFULL));
                 };
                 int g = 0;
-                for (int k = 0; k < n_tiers; ++k) {
-                    const int it = item_index(cta, k, G, n_items, order);
+                for (int k = 0;; ++k) {
+                    const int it = read_item(k);
                     if (it < 0) break;
-                    const Item<GEN> w = make_item<GEN>(it, dm, causal, order);
+                    const Item<GEN> w = make_item<GEN>(it, dm, causal);
                     mbar_wait(bar(B_KV), k & 1, status);
                     mbar_wait(bar(B_QFULL + (g & 1)), (g >> 1) & 1, status);
                     tc_fence_after();
@@ -264,10 +310,10 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                     umma_commit(bar(B_DOEMPTY));     // with issuer A's arrival after dV: both readers of dO are done
                 };
                 int g = 0;
-                for (int k = 0; k < n_tiers; ++k) {
-                    const int it = item_index(cta, k, G, n_items, order);
+                for (int k = 0;; ++k) {
+                    const int it = read_item(k);
                     if (it < 0) break;
-                    const Item<GEN> w = make_item<GEN>(it, dm, causal, order);
+                    const Item<GEN> w = make_item<GEN>(it, dm, causal);
                     mbar_wait(bar(B_KV), k & 1, status);
                     mbar_wait(bar(B_DOFULL), g & 1, status);
                     if (WITH_DQ && g > 0) mbar_wait(bar(B_DQEMPTY), (g - 1) & 1, status);   // Y: last item's final dQ partial drained
@@ -306,10 +352,10 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         // ahead of the compute warps (across item boundaries), so that they find them there
         // without global loads of their own.  Buffer g&1 may be rewritten once dS(g-2) is complete.
             int g = 0;
-            for (int k = 0; k < n_tiers; ++k) {
-                const int it = item_index(cta, k, G, n_items, order);
+            for (int k = 0;; ++k) {
+                const int it = read_item(k);
                 if (it < 0) break;
-                const Item<GEN> w = make_item<GEN>(it, dm, causal, order);
+                const Item<GEN> w = make_item<GEN>(it, dm, causal);
                 for (int n = 0; n < w.N; ++n, ++g) {
                     if (g >= 2) mbar_wait(pds_bar(g), ((g - 2) >> 1) & 1, status);
                     const uint32_t buf = sStat + (g & 1) * (2 * BLK * 4);
@@ -338,10 +384,10 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         const uint32_t tY = tmem + (static_cast<uint32_t>(r & ~31) << 16) + C::TM_Y;
         const uint32_t stage = base + C::OFF_DQ;
         int g = 0;
-        for (int k = 0; WITH_DQ && k < n_tiers; ++k) {
-        const int it = item_index(cta, k, G, n_items, order);
+        for (int k = 0; WITH_DQ; ++k) {
+        const int it = read_item(k);
         if (it < 0) break;
-        const Item<GEN> w = make_item<GEN>(it, dm, causal, order);
+        const Item<GEN> w = make_item<GEN>(it, dm, causal);
         for (int n = 0; n < w.N; ++n, ++g) {
             const int i0 = w.i0(n), bh = w.bh(n);
             mbar_wait(bar(B_DQFULL), g & 1, status);
@@ -433,10 +479,10 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         };
 
         int g = 0;
-        for (int k = 0; k < n_tiers; ++k) {
-        const int it = item_index(cta, k, G, n_items, order);
+        for (int k = 0;; ++k) {
+        const int it = read_item(k);
         if (it < 0) break;
-        const Item<GEN> w = make_item<GEN>(it, dm, causal, order);
+        const Item<GEN> w = make_item<GEN>(it, dm, causal);
         exp_phase(w, 0, g);
 
         for (int n = 0; n < w.N; ++n, ++g) {
@@ -541,6 +587,7 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
 __global__ void __launch_bounds__(256)
 dq_convert_kernel(const float4* __restrict__ acc, uint2* __restrict__ out, size_t n4, float scale)
 {
+    pdl_wait();   // programmatic dependent of the main kernel: resident early, reads after it has completed
     for (size_t i = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x; i < n4;
          i += static_cast<size_t>(gridDim.x) * blockDim.x) {
         const float4 a = acc[i];
@@ -554,7 +601,7 @@ dq_convert_kernel(const float4* __restrict__ acc, uint2* __restrict__ out, size_
 template <int D, bool GEN, bool WITH_DQ>
 cudaError_t launch_gen(const Problem& p, const void* q, const void* k, const void* v, const void* d_o,
                        const float* lse, const float* delta, float* dq_acc, void* dq, void* dk, void* dv,
-                       unsigned* status, cudaStream_t st)
+                       unsigned* sched, unsigned* status, cudaStream_t st)
 {
     using C = Cfg<D>;
     CUtensorMap tq, tk, tv, tdo, tdq;
@@ -577,43 +624,53 @@ cudaError_t launch_gen(const Problem& p, const void* q, const void* k, const voi
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
         return cudaErrorInvalidValue;
     const long long blocks = items < sms ? items : sms;       // persistent: one CTA per SM
-    // streamed per pair and shared between the key blocks of a head: dQ accumulator (f32), Q, dO
-    const int order = pick_schedule(items, sms, static_cast<double>(p.BH()) * p.Sq * D * (4 + 2 + 2), dev);
+    // Heads per group of the work-item list: what the items of a group share -- the f32 dQ accumulator,
+    // Q and dO of its query heads, K and V -- should stay in L2 while two groups are in flight
+    // (measured: half of L2 per group is the best size from 1024 to 8192 tokens).
+    int l2 = 0;
+    if (cudaDeviceGetAttribute(&l2, cudaDevAttrL2CacheSize, dev) != cudaSuccess || l2 <= 0) l2 = 64 << 20;
+    const double per_head = static_cast<double>(p.group()) * p.Sq * D * (4 + 2 + 2) + static_cast<double>(p.Sk) * D * 4;
+    long long hg = static_cast<long long>(0.5 * l2 / per_head);
+    hg = hg < 1 ? 1 : hg > p.BHkv() ? p.BHkv() : hg;
+    const long long n_groups = (p.BHkv() + hg - 1) / hg;
+    hg = (p.BHkv() + n_groups - 1) / n_groups;       // equal groups: a short last group unbalances the end of the list
+    if (g_forced_item_order == 0) hg = p.BHkv();      // one group: plain heaviest-first list
+    if (g_forced_item_order == 1) hg = 1;             // head by head
+    const int Hg = static_cast<int>(hg);
     const Dims dm{p.Sq, p.Sk, p.BH(), p.H, p.group(), p.off()};
-    kern<<<static_cast<unsigned>(blocks), kThreads, C::SMEM, st>>>(tq, tk, tv, tdo, tdq, lse, delta,
-                                                                   static_cast<__nv_bfloat16*>(dk),
-                                                                   static_cast<__nv_bfloat16*>(dv), dm, p.causal,
-                                                                   order, p.scale, status);
+    e = launch_pdl(kern, static_cast<unsigned>(blocks), kThreads, C::SMEM, st, tq, tk, tv, tdo, tdq, lse, delta,
+                   static_cast<__nv_bfloat16*>(dk), static_cast<__nv_bfloat16*>(dv), dm, p.causal, Hg, sched, p.scale,
+                   status);
+    if (e != cudaSuccess) return e;
     e = cudaGetLastError();
     if (e != cudaSuccess || !WITH_DQ) return e;
     const size_t n4 = static_cast<size_t>(p.BH()) * p.Sq * D / 4;
     const unsigned cblocks = static_cast<unsigned>(n4 / 256 + 1 < 148u * 16u ? n4 / 256 + 1 : 148u * 16u);
-    dq_convert_kernel<<<cblocks, 256, 0, st>>>(reinterpret_cast<const float4*>(dq_acc), reinterpret_cast<uint2*>(dq), n4,
-                                               p.scale);
-    return cudaGetLastError();
+    return launch_pdl(dq_convert_kernel, cblocks, 256, 0, st, reinterpret_cast<const float4*>(dq_acc),
+                      reinterpret_cast<uint2*>(dq), n4, p.scale);
 }
 
 template <int D>
 cudaError_t launch(const Problem& p, const void* q, const void* k, const void* v, const void* d_o,
                    const float* lse, const float* delta, float* dq_acc, void* dq, void* dk, void* dv,
-                   unsigned* status, cudaStream_t st)
+                   unsigned* sched, unsigned* status, cudaStream_t st)
 {
     if (dq_acc == nullptr)   // fused dK+dV only (deterministic backward): the general-shape build serves every shape
-        return launch_gen<D, true, false>(p, q, k, v, d_o, lse, delta, dq_acc, dq, dk, dv, status, st);
+        return launch_gen<D, true, false>(p, q, k, v, d_o, lse, delta, dq_acc, dq, dk, dv, sched, status, st);
     return (p.Hkv != p.H || p.Sq != p.Sk)
-               ? launch_gen<D, true, true>(p, q, k, v, d_o, lse, delta, dq_acc, dq, dk, dv, status, st)
-               : launch_gen<D, false, true>(p, q, k, v, d_o, lse, delta, dq_acc, dq, dk, dv, status, st);
+               ? launch_gen<D, true, true>(p, q, k, v, d_o, lse, delta, dq_acc, dq, dk, dv, sched, status, st)
+               : launch_gen<D, false, true>(p, q, k, v, d_o, lse, delta, dq_acc, dq, dk, dv, sched, status, st);
 }
 
 }  // namespace
 
 cudaError_t launch_fast_bwd(const Problem& p, const void* q, const void* k, const void* v, const void* d_o,
                             const float* lse, const float* delta, float* dq_acc, void* dq, void* dk, void* dv,
-                            unsigned* status, cudaStream_t st)
+                            unsigned* sched, unsigned* status, cudaStream_t st)
 {
     switch (p.D) {
-        case 64:  return launch<64>(p, q, k, v, d_o, lse, delta, dq_acc, dq, dk, dv, status, st);
-        case 128: return launch<128>(p, q, k, v, d_o, lse, delta, dq_acc, dq, dk, dv, status, st);
+        case 64:  return launch<64>(p, q, k, v, d_o, lse, delta, dq_acc, dq, dk, dv, sched, status, st);
+        case 128: return launch<128>(p, q, k, v, d_o, lse, delta, dq_acc, dq, dk, dv, sched, status, st);
         default:  return cudaErrorNotSupported;
     }
 }

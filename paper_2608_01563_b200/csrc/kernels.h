@@ -53,6 +53,24 @@ inline void strict_bwd_tiles(const Problem& p, int* BM, int* BN) {
 // returns the device address of its status word.  Returns an mgn_status code.
 int device_status_word(unsigned** status);
 
+// Launches `kern` as a programmatic dependent of the previous kernel on the stream (the kernel must
+// call pdl_wait() before it reads that kernel's results).
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kern)(KArgs...), unsigned grid, unsigned block, size_t smem, cudaStream_t st,
+                              Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(block);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
+}
+
 // Tensor maps (host side).  rank-3 view (D, S, BH) of a dense [BH,S,D] tensor with
 // a (box_d, box_rows, 1) box and the 128-byte swizzle.  Returns 0 on success.
 int make_tmap_3d(CUtensorMap* out, const void* base, int elem_bytes, int is_bf16,
@@ -73,7 +91,8 @@ cudaError_t launch_strict_dq(const Problem& p, const float* q, const float* k, c
 
 // delta_i = sum_d dO[i,d] O[i,d]  (f32 or bf16 inputs, f32 output), HBM-bound; also clears the
 // f32 dQ accumulation target `zero` ([rows][D] floats) unless it is null.
-cudaError_t launch_bwd_preprocess(const void* o, const void* d_o, float* delta, float* zero,
+// `counter` (one unsigned, may be null) is cleared too: the work-item counter of the fast backward.
+cudaError_t launch_bwd_preprocess(const void* o, const void* d_o, float* delta, float* zero, unsigned* counter,
                                   size_t rows, int D, int is_bf16, cudaStream_t st);
 
 // Work-item order of the persistent fast kernels (see the kernels for the two orders).  Head-major
@@ -102,7 +121,7 @@ cudaError_t launch_fast_fwd_f16(const Problem& p, const void* q16, const void* k
 cudaError_t launch_fast_bwd(const Problem& p, const void* q, const void* k, const void* v,
                             const void* d_o, const float* lse, const float* delta,
                             float* dq_acc, void* dq, void* dk, void* dv,
-                            unsigned* status, cudaStream_t st);
+                            unsigned* sched, unsigned* status, cudaStream_t st);
 
 // Deterministic fast backward: launch_fast_bwd with dq_acc == nullptr runs the fused dK+dV kernel
 // without the dQ product and reductions (dq is not touched), and this separate pass computes dQ.

@@ -56,6 +56,13 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, unsigne
     return mbar_wait_polls(bar, parity, status, kMaxPolls);
 }
 
+// Programmatic dependent launch.  A kernel launched with launch_pdl() may become resident while the
+// kernel before it on the stream is still running; pdl_wait() blocks until that kernel has completed
+// and its writes are visible, and must precede every read of its results.  pdl_launch_dependents()
+// lets the next such kernel on the stream start launching once every CTA has called it or exited.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // TMA: rank-3 tiled load global -> shared (this CTA), completion on an mbarrier.
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar,
                                             int c0, int c1, int c2) {
