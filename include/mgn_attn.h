@@ -13,8 +13,8 @@
  *   - q, k, v, o, d_o, dq, dk, dv are dense row-major [B,H,S,D], D innermost, no
  *     padding.  Element type: MGN_MODE_STRICT_F32 -> IEEE binary32,
  *     MGN_MODE_FAST_BF16 -> bfloat16.  lse is [B,H,S] binary32 in both modes.
- *   - Every tensor pointer must be 16-byte aligned.  D must be 32, 64 or 128 in strict
- *     mode and 64 or 128 in fast mode.
+ *   - Every tensor pointer must be 16-byte aligned.  D must be 32, 64 or 128 (in fast mode
+ *     D = 32 runs as a zero-padded 64-wide problem: correct, at the cost of D = 64).
  *   - The caller owns every buffer.  The library allocates no device memory.
  *   - Calls only enqueue work on `stream` (a cudaStream_t passed as void*; NULL is
  *     the legacy default stream) and return without synchronising.  Inputs must

@@ -159,7 +159,7 @@ def mgn_attn_fwd_accel(q, k, v, o, lse, workspace, causal: bool, scale: float, s
 
 def mgn_attn_bwd_deterministic(q, k, v, o, d_o, lse, dq, dk, dv, workspace, causal: bool, scale: float,
                                mode: int, stream: Optional[int] = None) -> None:
-    """Backward without floating-point atomics (strict mode): bit-identical from run to run."""
+    """Backward without floating-point atomics (both modes): bit-identical from run to run."""
     B, H, Hkv, Sq, Sk, D = _ext_dims(q, k)
     st = lib().mgn_attn_bwd_deterministic(_ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(d_o), _ptr(lse), _ptr(dq),
                                           _ptr(dk), _ptr(dv), _ptr(workspace),

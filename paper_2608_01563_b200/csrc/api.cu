@@ -40,7 +40,6 @@ int check_common(int B, int H, int S, int D, int causal, float scale, int mode)
     if (D != 32 && D != 64 && D != 128) return MGN_ERR_UNSUPPORTED;
     const long long bh = static_cast<long long>(B) * H;
     if (bh > 0x7fffffffLL) return MGN_ERR_UNSUPPORTED;
-    if (mode == MGN_MODE_FAST_BF16 && D == 32) return MGN_ERR_UNSUPPORTED;   // tensor-core path: D in {64,128}
     if (S > (1 << 24)) return MGN_ERR_UNSUPPORTED;
     // grid and byte-offset plan: tiles*BH must fit an int, element counts must fit 2^40
     if (bh * ((S + 63) / 64) > 0x7fffffffLL) return MGN_ERR_UNSUPPORTED;
@@ -155,7 +154,7 @@ int mgn_attn_fwd(const void* q, const void* k, const void* v, void* o, float* ls
 
 size_t mgn_attn_fwd_accel_workspace_bytes(int B, int H, int H_kv, int S_q, int S_k, int D)
 {
-    if (check_ext(B, H, H_kv, S_q, S_k, D, 0, 1.0f, MGN_MODE_FAST_BF16) != MGN_OK) return 0;
+    if (D == 32 || check_ext(B, H, H_kv, S_q, S_k, D, 0, 1.0f, MGN_MODE_FAST_BF16) != MGN_OK) return 0;   // f16 forward: D in {64,128}
     const size_t nq = static_cast<size_t>(B) * H * S_q * D, nk = static_cast<size_t>(B) * H_kv * S_k * D;
     return align_up(nq * 2, 256) + 2 * align_up(nk * 2, 256);
 }
@@ -165,7 +164,8 @@ int mgn_attn_fwd_accel(const float* q, const float* k, const float* v, float* o,
                        int B, int H, int H_kv, int S_q, int S_k, int D, int causal, float scale, void* stream)
 {
     if (!q || !k || !v || !o || !lse) return MGN_ERR_INVALID_ARG;
-    if (int r = check_ext(B, H, H_kv, S_q, S_k, D, causal, scale, MGN_MODE_FAST_BF16)) return r;   // D in {64,128}
+    if (int r = check_ext(B, H, H_kv, S_q, S_k, D, causal, scale, MGN_MODE_FAST_BF16)) return r;
+    if (D == 32) return MGN_ERR_UNSUPPORTED;   // the f16 forward stores f32 rows itself: D in {64,128}
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(lse)) return MGN_ERR_MISALIGNED;
     const size_t need = mgn_attn_fwd_accel_workspace_bytes(B, H, H_kv, S_q, S_k, D);
     if (!workspace || workspace_bytes < need) return MGN_ERR_WORKSPACE;

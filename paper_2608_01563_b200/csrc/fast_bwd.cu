@@ -144,8 +144,10 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                 const __grid_constant__ CUtensorMap tmdQ,
                 const float* __restrict__ LSE, const float* __restrict__ DELTA,
                 __nv_bfloat16* __restrict__ dK, __nv_bfloat16* __restrict__ dV,
-                const Dims dm, int causal, int Hg, unsigned* __restrict__ sched, float scale, unsigned* status)
+                const Dims dm, int causal, int Hg, unsigned* __restrict__ sched, float scale, int Dg, unsigned* status)
 {
+    // Dg: head size in global memory.  Dg = 32 runs the D = 64 build on operand tiles whose columns
+    // 32-63 are zero-filled by the tensor maps; only the first 32 columns of dQ, dK, dV are written.
     using C = Cfg<D>;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -413,7 +415,7 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                 named_bar_sync(4, 128);
                 if (r == 0) {
                     tma_reduce_add_3d(&tmdQ, stage, 64 * round, i0, bh);
-                    tma_reduce_add_3d(&tmdQ, stage + C::CHUNK_BYTES, 64 * round + 32, i0, bh);
+                    if (64 * round + 32 < Dg) tma_reduce_add_3d(&tmdQ, stage + C::CHUNK_BYTES, 64 * round + 32, i0, bh);
                     bulk_commit_group();
                 }
             }
@@ -553,7 +555,8 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                 for (int q = 0; q < PCS; ++q)
                     sts128(stage + r * (HC * 2) + (swz(q, r) << 4), u[4 * q], u[4 * q + 1], u[4 * q + 2], u[4 * q + 3]);
                 named_bar_sync(2 + half, 128);
-                out += (static_cast<size_t>(w.bhk) * Sk + w.j0) * D + half * HC;
+                out += (static_cast<size_t>(w.bhk) * Sk + w.j0) * Dg + half * HC;
+                const bool cols_exist = half * HC < Dg;
                 float4 val[PCS];
 #pragma unroll
                 for (int i = 0; i < PCS; ++i) {
@@ -563,7 +566,8 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
 #pragma unroll
                 for (int i = 0; i < PCS; ++i) {
                     const int idx = i * 128 + r, row = idx / PCS, piece = idx % PCS;
-                    if (w.j0 + row < Sk) *reinterpret_cast<float4*>(out + static_cast<size_t>(row) * D + piece * 8) = val[i];
+                    if (cols_exist && w.j0 + row < Sk)
+                        *reinterpret_cast<float4*>(out + static_cast<size_t>(row) * Dg + piece * 8) = val[i];
                 }
                 named_bar_sync(2 + half, 128);             // the slab has been read: the buffer may be rewritten
             };
@@ -607,12 +611,12 @@ cudaError_t launch_gen(const Problem& p, const void* q, const void* k, const voi
     CUtensorMap tq, tk, tv, tdo, tdq;
     // without the dQ product the map is never used; it only has to be a valid one
     if (make_tmap_3d(&tdq, WITH_DQ ? static_cast<const void*>(dq_acc) : static_cast<const void*>(delta), 4, 0,
-                     WITH_DQ ? p.BH() : 1, WITH_DQ ? p.Sq : 1, WITH_DQ ? D : 32, 32, WITH_DQ ? BLK : 1))
+                     WITH_DQ ? p.BH() : 1, WITH_DQ ? p.Sq : 1, WITH_DQ ? p.D : 32, 32, WITH_DQ ? BLK : 1))
         return cudaErrorInvalidValue;
-    if (make_tmap_3d(&tq, q, 2, 1, p.BH(), p.Sq, D, 64, BLK)) return cudaErrorInvalidValue;
-    if (make_tmap_3d(&tk, k, 2, 1, p.BHkv(), p.Sk, D, 64, BLK)) return cudaErrorInvalidValue;
-    if (make_tmap_3d(&tv, v, 2, 1, p.BHkv(), p.Sk, D, 64, BLK)) return cudaErrorInvalidValue;
-    if (make_tmap_3d(&tdo, d_o, 2, 1, p.BH(), p.Sq, D, 64, BLK)) return cudaErrorInvalidValue;
+    if (make_tmap_3d(&tq, q, 2, 1, p.BH(), p.Sq, p.D, 64, BLK)) return cudaErrorInvalidValue;
+    if (make_tmap_3d(&tk, k, 2, 1, p.BHkv(), p.Sk, p.D, 64, BLK)) return cudaErrorInvalidValue;
+    if (make_tmap_3d(&tv, v, 2, 1, p.BHkv(), p.Sk, p.D, 64, BLK)) return cudaErrorInvalidValue;
+    if (make_tmap_3d(&tdo, d_o, 2, 1, p.BH(), p.Sq, p.D, 64, BLK)) return cudaErrorInvalidValue;
     auto kern = fast_bwd_kernel<D, GEN, WITH_DQ>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM);
     if (e != cudaSuccess) return e;
@@ -640,11 +644,11 @@ cudaError_t launch_gen(const Problem& p, const void* q, const void* k, const voi
     const Dims dm{p.Sq, p.Sk, p.BH(), p.H, p.group(), p.off()};
     e = launch_pdl(kern, static_cast<unsigned>(blocks), kThreads, C::SMEM, st, tq, tk, tv, tdo, tdq, lse, delta,
                    static_cast<__nv_bfloat16*>(dk), static_cast<__nv_bfloat16*>(dv), dm, p.causal, Hg, sched, p.scale,
-                   status);
+                   p.D, status);
     if (e != cudaSuccess) return e;
     e = cudaGetLastError();
     if (e != cudaSuccess || !WITH_DQ) return e;
-    const size_t n4 = static_cast<size_t>(p.BH()) * p.Sq * D / 4;
+    const size_t n4 = static_cast<size_t>(p.BH()) * p.Sq * p.D / 4;
     const unsigned cblocks = static_cast<unsigned>(n4 / 256 + 1 < 148u * 16u ? n4 / 256 + 1 : 148u * 16u);
     return launch_pdl(dq_convert_kernel, cblocks, 256, 0, st, reinterpret_cast<const float4*>(dq_acc),
                       reinterpret_cast<uint2*>(dq), n4, p.scale);
@@ -669,6 +673,7 @@ cudaError_t launch_fast_bwd(const Problem& p, const void* q, const void* k, cons
                             unsigned* sched, unsigned* status, cudaStream_t st)
 {
     switch (p.D) {
+        case 32:  // the 64-wide build on zero-filled 32-element rows (see fast_fwd.cu)
         case 64:  return launch<64>(p, q, k, v, d_o, lse, delta, dq_acc, dq, dk, dv, sched, status, st);
         case 128: return launch<128>(p, q, k, v, d_o, lse, delta, dq_acc, dq, dk, dv, sched, status, st);
         default:  return cudaErrorNotSupported;

@@ -238,11 +238,11 @@ cudaError_t launch(const Problem& p, const void* q, const void* k, const void* v
 {
     using C = Cfg<D>;
     CUtensorMap tq, tk, tv, tdo, tdq;
-    if (make_tmap_3d(&tq, q, 2, 1, p.BH(), p.Sq, D, 64, BLK)) return cudaErrorInvalidValue;
-    if (make_tmap_3d(&tdo, d_o, 2, 1, p.BH(), p.Sq, D, 64, BLK)) return cudaErrorInvalidValue;
-    if (make_tmap_3d(&tk, k, 2, 1, p.BHkv(), p.Sk, D, 64, BLK)) return cudaErrorInvalidValue;
-    if (make_tmap_3d(&tv, v, 2, 1, p.BHkv(), p.Sk, D, 64, BLK)) return cudaErrorInvalidValue;
-    if (make_tmap_3d(&tdq, dq, 2, 1, p.BH(), p.Sq, D, 64, BLK)) return cudaErrorInvalidValue;
+    if (make_tmap_3d(&tq, q, 2, 1, p.BH(), p.Sq, p.D, 64, BLK)) return cudaErrorInvalidValue;
+    if (make_tmap_3d(&tdo, d_o, 2, 1, p.BH(), p.Sq, p.D, 64, BLK)) return cudaErrorInvalidValue;
+    if (make_tmap_3d(&tk, k, 2, 1, p.BHkv(), p.Sk, p.D, 64, BLK)) return cudaErrorInvalidValue;
+    if (make_tmap_3d(&tv, v, 2, 1, p.BHkv(), p.Sk, p.D, 64, BLK)) return cudaErrorInvalidValue;
+    if (make_tmap_3d(&tdq, dq, 2, 1, p.BH(), p.Sq, p.D, 64, BLK)) return cudaErrorInvalidValue;
     auto kern = fast_dq_kernel<D>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM);
     if (e != cudaSuccess) return e;
@@ -261,6 +261,7 @@ cudaError_t launch_fast_dq(const Problem& p, const void* q, const void* k, const
                            const float* lse, const float* delta, void* dq, unsigned* status, cudaStream_t st)
 {
     switch (p.D) {
+        case 32:  // the 64-wide build on zero-filled 32-element rows (see fast_fwd.cu)
         case 64:  return launch<64>(p, q, k, v, d_o, lse, delta, dq, status, st);
         case 128: return launch<128>(p, q, k, v, d_o, lse, delta, dq, status, st);
         default:  return cudaErrorNotSupported;

@@ -484,11 +484,11 @@ cudaError_t launch_gen(const Problem& p, const void* q, const void* k, const voi
 {
     using C = Cfg<D>;
     CUtensorMap tq, tk, tv, to;
-    if (make_tmap_3d(&tq, q, 2, 1, p.BH(), p.Sq, D, 64, 128)) return cudaErrorInvalidValue;
-    if (make_tmap_3d(&tk, k, 2, 1, p.BHkv(), p.Sk, D, 64, 128)) return cudaErrorInvalidValue;
-    if (make_tmap_3d(&tv, v, 2, 1, p.BHkv(), p.Sk, D, 64, 128)) return cudaErrorInvalidValue;
+    if (make_tmap_3d(&tq, q, 2, 1, p.BH(), p.Sq, p.D, 64, 128)) return cudaErrorInvalidValue;
+    if (make_tmap_3d(&tk, k, 2, 1, p.BHkv(), p.Sk, p.D, 64, 128)) return cudaErrorInvalidValue;
+    if (make_tmap_3d(&tv, v, 2, 1, p.BHkv(), p.Sk, p.D, 64, 128)) return cudaErrorInvalidValue;
     // with f32 output the kernel stores O itself; the map then only has to be a valid one
-    if (make_tmap_3d(&to, F16 ? q : o, 2, 1, p.BH(), p.Sq, D, 64, 128)) return cudaErrorInvalidValue;
+    if (make_tmap_3d(&to, F16 ? q : o, 2, 1, p.BH(), p.Sq, p.D, 64, 128)) return cudaErrorInvalidValue;
     auto kern = fast_fwd_kernel<D, GEN, F16>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM);
     if (e != cudaSuccess) return e;
@@ -556,6 +556,10 @@ cudaError_t launch_fast_fwd(const Problem& p, const void* q, const void* k, cons
                             unsigned* status, cudaStream_t st)
 {
     switch (p.D) {
+        // Head size 32 runs the 64-wide build: the tensor maps describe 32-element rows and a
+        // 64-element box, so columns 32-63 of every operand tile are zero-filled on load (they add
+        // nothing to the scores and give zero output columns) and clipped on store.
+        case 32:
         case 64:  return launch<64>(p, q, k, v, o, lse, status, st);
         case 128: return launch<128>(p, q, k, v, o, lse, status, st);
         default:  return cudaErrorNotSupported;

@@ -168,7 +168,7 @@ def test_accel_forward_argument_validation(lib):
     lib.mgn_attn_fwd_accel_workspace_bytes.restype = sz
     need = lib.mgn_attn_fwd_accel_workspace_bytes(1, 4, 2, 8, 16, 64)
     assert need >= (4 * 8 + 2 * 2 * 16) * 64 * 2 and need % 256 == 0
-    assert lib.mgn_attn_fwd_accel_workspace_bytes(1, 4, 2, 8, 16, 32) == 0       # D = 32 has no tensor-core path
+    assert lib.mgn_attn_fwd_accel_workspace_bytes(1, 4, 2, 8, 16, 32) == 0       # the f16 forward takes D in {64,128} only
 
     def fa(D=64, Hkv=2, ws=A, ws_bytes=1 << 30, q=A):
         return lib.mgn_attn_fwd_accel(q, A, A, A, A, ws, ws_bytes, 1, 4, Hkv, 8, 16, D, 0, 1.0, None)

@@ -18,7 +18,7 @@ MODE = mgn.MODE_FAST_BF16
 BF = torch.bfloat16
 
 
-@pytest.mark.parametrize("D", [64, 128])
+@pytest.mark.parametrize("D", [32, 64, 128])
 @pytest.mark.parametrize("causal", [False, True])
 @pytest.mark.parametrize("S", [1, 2, 63, 64, 65, 127, 128, 129, 197, 256, 257, 300, 520])
 def test_forward_edge_shapes(S, D, causal):
@@ -30,7 +30,7 @@ def test_forward_edge_shapes(S, D, causal):
     hp.check_fast(hp.select(res, B, H), ref, names=("O",), label=f"S={S} D={D} causal={causal} ")
 
 
-@pytest.mark.parametrize("D", [64, 128])
+@pytest.mark.parametrize("D", [32, 64, 128])
 @pytest.mark.parametrize("causal", [False, True])
 @pytest.mark.parametrize("S", [1, 2, 63, 64, 65, 127, 128, 129, 197, 256, 257, 300, 520])
 def test_forward_backward_edge_shapes(S, D, causal):
@@ -159,9 +159,26 @@ def test_decoder_sweep_longest_sequence_two_heads():
     hp.check_invariants(q, k, v, d_o, res, rtol=2e-2, max_heads=16)
 
 
-def test_d32_is_reported_unsupported_in_fast_mode():
-    q = torch.zeros(1, 1, 8, 32, device="cuda", dtype=BF)
-    lse = torch.zeros(1, 1, 8, device="cuda")
-    with pytest.raises(mgn.MgnError) as e:
-        mgn.mgn_attn_fwd(q, q, q, torch.empty_like(q), lse, False, 1.0, MODE)
-    assert e.value.status == 2
+@pytest.mark.parametrize("order", [0, 1])
+def test_head_size_32_several_items_per_cta(order):
+    """Head size 32 (run as a zero-padded 64-wide problem) at a size with several work items per
+    CTA, under both extremes of the work-item list, and through the deterministic backward."""
+    B, H, S, D, causal = 2, 80, 700, 32, True
+    scale = 1.0 / math.sqrt(D)
+    q, k, v, d_o = synth.random_inputs(91 + order, B, H, S, D, dtype=BF)
+    heads = [0, 77, B * H - 1]
+    mgn.mgn_attn_fast_item_order(order)
+    try:
+        res = hp.run_cuda(q, k, v, d_o, causal, scale, MODE)
+    finally:
+        mgn.mgn_attn_fast_item_order(-1)
+    ref = hp.run_oracle(q, k, v, d_o, causal, scale, heads)
+    hp.check_fast(hp.select(res, B, H, heads), ref, label=f"D=32 order={order} ")
+    hp.check_invariants(q, k, v, d_o, res, rtol=2e-2)
+    qd, kd, vd, dod = (t.cuda() for t in (q, k, v, d_o))
+    dq, dk, dv = (torch.full_like(qd, float("nan")) for _ in range(3))
+    ws = mgn.alloc_workspace(B, H, S, D, MODE)
+    mgn.mgn_attn_bwd_deterministic(qd, kd, vd, res["O"].cuda(), dod, res["LSE"].cuda(), dq, dk, dv, ws, causal, scale, MODE)
+    mgn.mgn_attn_check()
+    det = hp.select({"dQ": dq.cpu(), "dK": dk.cpu(), "dV": dv.cpu()}, B, H, heads)
+    hp.check_fast(det, ref, names=("dQ", "dK", "dV"), label="D=32 deterministic ")
