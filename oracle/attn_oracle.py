@@ -19,6 +19,7 @@ import numpy as np
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "attn_ref.c")
 _SRC_EXT = os.path.join(_HERE, "attn_ref_ext.c")      # separate query/key lengths, grouped K/V heads
+_SRC_PROJ = os.path.join(_HERE, "proj_ref.c")         # output projection of the concatenated heads
 _LIB = os.path.join(_HERE, "libmgn_oracle.so")
 _lib = None
 
@@ -27,11 +28,11 @@ _dp = ctypes.POINTER(ctypes.c_double)
 
 def build(force: bool = False) -> str:
     """Compile the oracle with gcc (-O2, OpenMP, no fast-math). Returns the .so path."""
-    newest = max(os.path.getmtime(_SRC), os.path.getmtime(_SRC_EXT))
+    newest = max(os.path.getmtime(_SRC), os.path.getmtime(_SRC_EXT), os.path.getmtime(_SRC_PROJ))
     if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < newest:
         tmp = _LIB + f".tmp{os.getpid()}"
         subprocess.check_call(
-            ["gcc", "-O2", "-std=c11", "-fopenmp", "-fPIC", "-shared", "-o", tmp, _SRC, _SRC_EXT, "-lm"]
+            ["gcc", "-O2", "-std=c11", "-fopenmp", "-fPIC", "-shared", "-o", tmp, _SRC, _SRC_EXT, _SRC_PROJ, "-lm"]
         )
         os.replace(tmp, _LIB)
     return _LIB
@@ -54,6 +55,12 @@ def _load():
         lib.ref_attn_fwd_ext.restype = i
         lib.ref_attn_bwd_ext.argtypes = [_dp] * 9 + [i] * 7 + [d, i]
         lib.ref_attn_bwd_ext.restype = i
+        lib.ref_out_proj_fwd.argtypes = [_dp] * 3 + [i] * 5
+        lib.ref_out_proj_fwd.restype = None
+        lib.ref_out_proj_bwd_data.argtypes = [_dp] * 5 + [i] * 5
+        lib.ref_out_proj_bwd_data.restype = None
+        lib.ref_out_proj_bwd_weight.argtypes = [_dp] * 3 + [i] * 5
+        lib.ref_out_proj_bwd_weight.restype = None
         lib.ref_max_threads.argtypes = []
         lib.ref_max_threads.restype = i
         _lib = lib
@@ -152,3 +159,28 @@ def attn_bwd_ext(q, k, v, d_o, causal: bool, scale: float, nthreads: int = 0):
     if rc != 0:
         raise ValueError("shapes outside the definition (H % Hkv != 0, or causal with Sq > Sk)")
     return o, lse, dq, dk, dv
+
+
+def out_proj_fwd(o, w):
+    """Output projection of the concatenated heads: o [B,H,S,D], w [H*D,E] -> Y [B,S,E], float64."""
+    o, w = _c(o), _c(w)
+    B, H, S, D = o.shape
+    assert w.shape[0] == H * D
+    E = w.shape[1]
+    y = np.empty((B, S, E), dtype=np.float64)
+    _load().ref_out_proj_fwd(_p(o), _p(w), _p(y), B, H, S, D, E)
+    return y
+
+
+def out_proj_bwd(d_y, w, o):
+    """Backward of out_proj_fwd: returns (dO [B,H,S,D], delta [B,H,S] = rowsum(dO o O), dW [H*D,E])."""
+    d_y, w, o = _c(d_y), _c(w), _c(o)
+    B, H, S, D = o.shape
+    E = w.shape[1]
+    assert w.shape[0] == H * D and d_y.shape == (B, S, E)
+    d_o = np.empty_like(o)
+    delta = np.empty((B, H, S), dtype=np.float64)
+    d_w = np.empty_like(w)
+    _load().ref_out_proj_bwd_data(_p(d_y), _p(w), _p(o), _p(d_o), _p(delta), B, H, S, D, E)
+    _load().ref_out_proj_bwd_weight(_p(o), _p(d_y), _p(d_w), B, H, S, D, E)
+    return d_o, delta, d_w
