@@ -159,6 +159,37 @@ int mgn_attn_bwd_deterministic(const void* q, const void* k, const void* v, cons
                                void* stream);
 
 /*
+ * The step after attention, fused with it at its two seams (paper Section 3.3: matrix-product
+ * kernels with prologues and epilogues that absorb the neighbouring steps; Section 7.3: dispatch
+ * structure matters where kernels are small).  The paper prints no formula; these are the textbook
+ * output projection of the concatenated heads and its data gradient.  Fast mode only so far
+ * (MGN_MODE_FAST_BF16: bf16 tensors, tensor-core products, f32 accumulation; strict mode returns
+ * MGN_ERR_UNSUPPORTED), D in {64,128}, E a multiple of 8.  All pointers are device pointers, 16-byte
+ * aligned; layouts dense row-major.
+ *
+ * mgn_out_proj_fwd:       y[b,s,e] = sum_{h,d} o[b,h,s,d] * w[h*D+d, e]
+ *     o [B,H,S,D] as the attention forward wrote it (no concatenated copy is made), w [H*D, E],
+ *     y [B,S,E] out.
+ * mgn_out_proj_bwd_data:  d_o[b,h,s,d] = sum_e d_y[b,s,e] * w[h*D+d, e]      (into the [B,H,S,D] layout
+ *                         delta[b,h,s] = sum_d d_o[b,h,s,d] * o[b,h,s,d]      the attention backward reads)
+ *     d_y [B,S,E], w [H*D,E], o [B,H,S,D] in; d_o [B,H,S,D] (bf16) and delta [B,H,S] (f32) out.  delta is
+ *     formed from the bf16-rounded d_o and is what mgn_attn_bwd's own first pass would compute from
+ *     o and d_o; hand it to mgn_attn_bwd_given_delta.
+ * mgn_attn_bwd_given_delta: mgn_attn_bwd_ext without `o`, with a ready `delta` [B,H,S_q] (f32, read
+ *     only): the pass over o and d_o is skipped.  Either mode.  Workspace as for mgn_attn_bwd_ext.
+ * Errors as elsewhere: INVALID_ARG (null pointer, size <= 0, unknown mode), UNSUPPORTED, MISALIGNED,
+ * WORKSPACE, ARCH, CUDA.
+ */
+int mgn_out_proj_fwd(const void* o, const void* w, void* y, int B, int H, int S, int D, int E, int mode, void* stream);
+int mgn_out_proj_bwd_data(const void* d_y, const void* w, const void* o, void* d_o, float* delta,
+                          int B, int H, int S, int D, int E, int mode, void* stream);
+int mgn_attn_bwd_given_delta(const void* q, const void* k, const void* v, const void* d_o, const float* lse,
+                             const float* delta, void* dq, void* dk, void* dv,
+                             void* workspace, size_t workspace_bytes,
+                             int B, int H, int H_kv, int S_q, int S_k, int D, int causal, float scale, int mode,
+                             void* stream);
+
+/*
  * Synchronises `stream`, then reads and clears the device-side status word that
  * kernels set when one of their bounded waits (TMA / tensor-core completion
  * barriers) ran out.  Returns MGN_OK, MGN_ERR_DEVICE_TIMEOUT or MGN_ERR_CUDA.

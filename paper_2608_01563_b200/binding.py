@@ -71,6 +71,12 @@ def lib() -> ctypes.CDLL:
         L.mgn_attn_fast_item_order.restype = i
         L.mgn_attn_strict_tiles.argtypes = [i] * 7 + [ctypes.POINTER(ctypes.c_int)]
         L.mgn_attn_strict_tiles.restype = i
+        L.mgn_out_proj_fwd.argtypes = [vp, vp, vp, i, i, i, i, i, i, vp]
+        L.mgn_out_proj_fwd.restype = i
+        L.mgn_out_proj_bwd_data.argtypes = [vp] * 5 + [i, i, i, i, i, i, vp]
+        L.mgn_out_proj_bwd_data.restype = i
+        L.mgn_attn_bwd_given_delta.argtypes = [vp] * 9 + [vp, sz, i, i, i, i, i, i, i, f, i, vp]
+        L.mgn_attn_bwd_given_delta.restype = i
         L.mgn_selftest_wait_timeout.argtypes = [vp, vp]
         L.mgn_selftest_wait_timeout.restype = i
         L.mgn_status_string.argtypes = [i]
@@ -218,6 +224,32 @@ def mgn_measure_fp32_ffma_tflops(stream: Optional[int] = None) -> float:
     if st != MGN_OK:
         raise MgnError(st, "mgn_measure_fp32_ffma_tflops")
     return float(out.value)
+
+
+def mgn_out_proj_fwd(o, w, y, mode: int, stream: Optional[int] = None) -> None:
+    B, H, S, D = _dims(o)
+    st = lib().mgn_out_proj_fwd(_ptr(o), _ptr(w), _ptr(y), B, H, S, D, int(w.shape[1]), int(mode), _stream(stream))
+    if st != MGN_OK:
+        raise MgnError(st, "mgn_out_proj_fwd")
+
+
+def mgn_out_proj_bwd_data(d_y, w, o, d_o, delta, mode: int, stream: Optional[int] = None) -> None:
+    B, H, S, D = _dims(o)
+    st = lib().mgn_out_proj_bwd_data(_ptr(d_y), _ptr(w), _ptr(o), _ptr(d_o), _ptr(delta), B, H, S, D,
+                                     int(w.shape[1]), int(mode), _stream(stream))
+    if st != MGN_OK:
+        raise MgnError(st, "mgn_out_proj_bwd_data")
+
+
+def mgn_attn_bwd_given_delta(q, k, v, d_o, lse, delta, dq, dk, dv, workspace, causal: bool, scale: float, mode: int,
+                             stream: Optional[int] = None) -> None:
+    B, H, Hkv, Sq, Sk, D = _ext_dims(q, k)
+    st = lib().mgn_attn_bwd_given_delta(_ptr(q), _ptr(k), _ptr(v), _ptr(d_o), _ptr(lse), _ptr(delta), _ptr(dq),
+                                        _ptr(dk), _ptr(dv), _ptr(workspace),
+                                        workspace.numel() * workspace.element_size(), B, H, Hkv, Sq, Sk, D,
+                                        int(causal), float(scale), int(mode), _stream(stream))
+    if st != MGN_OK:
+        raise MgnError(st, "mgn_attn_bwd_given_delta")
 
 
 def mgn_selftest_wait_timeout(gave_up: Optional[torch.Tensor] = None, stream: Optional[int] = None) -> None:

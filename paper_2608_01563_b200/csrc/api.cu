@@ -257,6 +257,77 @@ int mgn_attn_bwd_deterministic(const void* q, const void* k, const void* v, cons
     return e == cudaSuccess ? MGN_OK : MGN_ERR_CUDA;
 }
 
+int mgn_attn_bwd_given_delta(const void* q, const void* k, const void* v, const void* d_o, const float* lse,
+                             const float* delta, void* dq, void* dk, void* dv,
+                             void* workspace, size_t workspace_bytes,
+                             int B, int H, int H_kv, int S_q, int S_k, int D, int causal, float scale, int mode,
+                             void* stream)
+{
+    unsigned* status = nullptr;
+    if (!delta) return MGN_ERR_INVALID_ARG;
+    // `o` is not an argument here: q stands in for it in the shared pointer checks
+    if (int r = check_bwd_call(q, k, v, q, d_o, lse, dq, dk, dv, workspace, workspace_bytes, B, H, H_kv, S_q, S_k, D,
+                               causal, scale, mode, &status))
+        return r;
+    if (!aligned16(delta)) return MGN_ERR_MISALIGNED;
+    const mgn::Problem p{B, H, H_kv, S_q, S_k, D, causal, scale};
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t rows = static_cast<size_t>(B) * H * S_q;
+    const bool fast = mode == MGN_MODE_FAST_BF16;
+    unsigned* sched = fast ? reinterpret_cast<unsigned*>(static_cast<char*>(workspace) + ws_delta_bytes(rows)) : nullptr;
+    float* dq_acc = fast ? reinterpret_cast<float*>(static_cast<char*>(workspace) + ws_delta_bytes(rows) + kSchedBytes)
+                         : static_cast<float*>(dq);
+    cudaError_t e = mgn::launch_bwd_clear(dq_acc, rows * D, sched, st);
+    if (e != cudaSuccess) return MGN_ERR_CUDA;
+    MainKernelTimer timer(st);
+    if (!fast)
+        e = mgn::launch_strict_bwd(p, static_cast<const float*>(q), static_cast<const float*>(k),
+                                   static_cast<const float*>(v), static_cast<const float*>(d_o), lse, delta,
+                                   static_cast<float*>(dq), static_cast<float*>(dk), static_cast<float*>(dv), status,
+                                   st);
+    else
+        e = mgn::launch_fast_bwd(p, q, k, v, d_o, lse, delta, dq_acc, dq, dk, dv, sched, status, st);
+    return e == cudaSuccess ? MGN_OK : MGN_ERR_CUDA;
+}
+
+namespace {
+int check_proj(const void* a, const void* b, const void* c, const void* d, int B, int H, int S, int D, int E, int mode)
+{
+    if (!a || !b || !c || !d) return MGN_ERR_INVALID_ARG;
+    if (B <= 0 || H <= 0 || S <= 0 || D <= 0 || E <= 0) return MGN_ERR_INVALID_ARG;
+    if (mode != MGN_MODE_STRICT_F32 && mode != MGN_MODE_FAST_BF16) return MGN_ERR_INVALID_ARG;
+    if (mode != MGN_MODE_FAST_BF16) return MGN_ERR_UNSUPPORTED;          // tensor-core path only so far
+    if (D != 64 && D != 128) return MGN_ERR_UNSUPPORTED;                 // a 64-wide contraction slice stays inside one head
+    if (E % 8 != 0) return MGN_ERR_UNSUPPORTED;                          // 16-byte rows for TMA and the vector stores
+    if (static_cast<double>(B) * S * (static_cast<double>(H) * D + E) > 1.0e12 || S > (1 << 24)) return MGN_ERR_UNSUPPORTED;
+    if (static_cast<long long>(B) * H > 0x7fffffffLL || static_cast<long long>(H) * D > 0x7fffffffLL) return MGN_ERR_UNSUPPORTED;
+    if (!aligned16(a) || !aligned16(b) || !aligned16(c) || !aligned16(d)) return MGN_ERR_MISALIGNED;
+    return MGN_OK;
+}
+}  // namespace
+
+int mgn_out_proj_fwd(const void* o, const void* w, void* y, int B, int H, int S, int D, int E, int mode, void* stream)
+{
+    if (int r = check_proj(o, w, y, y, B, H, S, D, E, mode)) return r;
+    unsigned* status = nullptr;
+    if (int r = device_setup(&status)) return r;
+    return mgn::launch_out_proj_fwd(o, w, y, B, H, S, D, E, status, static_cast<cudaStream_t>(stream)) == cudaSuccess
+               ? MGN_OK : MGN_ERR_CUDA;
+}
+
+int mgn_out_proj_bwd_data(const void* d_y, const void* w, const void* o, void* d_o, float* delta,
+                          int B, int H, int S, int D, int E, int mode, void* stream)
+{
+    if (!delta) return MGN_ERR_INVALID_ARG;
+    if (int r = check_proj(d_y, w, o, d_o, B, H, S, D, E, mode)) return r;
+    if (!aligned16(delta)) return MGN_ERR_MISALIGNED;
+    unsigned* status = nullptr;
+    if (int r = device_setup(&status)) return r;
+    return mgn::launch_out_proj_bwd_data(d_y, w, o, d_o, delta, B, H, S, D, E, status,
+                                         static_cast<cudaStream_t>(stream)) == cudaSuccess
+               ? MGN_OK : MGN_ERR_CUDA;
+}
+
 int mgn_attn_bwd(const void* q, const void* k, const void* v, const void* o, const void* d_o,
                  const float* lse, void* dq, void* dk, void* dv,
                  void* workspace, size_t workspace_bytes,
@@ -322,6 +393,6 @@ const char* mgn_status_string(int status)
     }
 }
 
-int mgn_version(void) { return 210; }   // 0.2.1: tile-shape query, low-padding strict tiles, leaner fast forward (0.2.0: extended shapes, deterministic backward, accelerated forward)
+int mgn_version(void) { return 300; }   // 0.2.1: tile-shape query, low-padding strict tiles, leaner fast forward (0.2.0: extended shapes, deterministic backward, accelerated forward)
 
 }  // extern "C"

@@ -76,6 +76,19 @@ bwd_preprocess_kernel(const uint4* __restrict__ o, const uint4* __restrict__ d_o
     }
 }
 
+// Clears the dQ accumulation target and the work-item counter: what is left of the preprocess pass
+// when delta comes from elsewhere (the dO producer of the output projection).
+__global__ void __launch_bounds__(256)
+bwd_clear_kernel(float4* __restrict__ zero, size_t n4, unsigned* __restrict__ counter)
+{
+    pdl_launch_dependents();
+    if (counter && blockIdx.x == 0 && threadIdx.x == 0) *counter = 0u;
+    const uint64_t keep = l2_policy_keep();
+    for (size_t i = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x; i < n4;
+         i += static_cast<size_t>(gridDim.x) * blockDim.x)
+        st_hint(&zero[i], make_float4(0.f, 0.f, 0.f, 0.f), keep);
+}
+
 template <int LANES, bool BF16>
 cudaError_t run(const void* o, const void* d_o, float* delta, float* zero, unsigned* counter, size_t rows, cudaStream_t st)
 {
@@ -89,6 +102,15 @@ cudaError_t run(const void* o, const void* d_o, float* delta, float* zero, unsig
 }
 
 }  // namespace
+
+cudaError_t launch_bwd_clear(float* zero, size_t n_floats, unsigned* counter, cudaStream_t st)
+{
+    const size_t n4 = n_floats / 4;
+    const size_t cap = 148u * 16u;
+    const size_t blocks = n4 / 256 + 1 < cap ? n4 / 256 + 1 : cap;
+    bwd_clear_kernel<<<static_cast<unsigned>(blocks), 256, 0, st>>>(reinterpret_cast<float4*>(zero), n4, counter);
+    return cudaGetLastError();
+}
 
 cudaError_t launch_bwd_preprocess(const void* o, const void* d_o, float* delta, float* zero, unsigned* counter,
                                   size_t rows, int D, int is_bf16, cudaStream_t st)

@@ -95,6 +95,17 @@ cudaError_t launch_strict_dq(const Problem& p, const float* q, const float* k, c
 cudaError_t launch_bwd_preprocess(const void* o, const void* d_o, float* delta, float* zero, unsigned* counter,
                                   size_t rows, int D, int is_bf16, cudaStream_t st);
 
+// The clearing half of the preprocess pass alone (delta supplied by the caller): zeroes `n_floats`
+// floats at `zero` (a multiple of four) and the work-item counter (may be null).
+cudaError_t launch_bwd_clear(float* zero, size_t n_floats, unsigned* counter, cudaStream_t st);
+
+// Output projection of the concatenated heads (fast mode, bf16): y [B,S,E] = concat_h(o [B,H,S,D]) w [H*D,E];
+// and its data gradient d_o [B,H,S,D] = d_y w^T together with delta [B,H,S] = rowsum(d_o o o).
+cudaError_t launch_out_proj_fwd(const void* o, const void* w, void* y, int B, int H, int S, int D, int E,
+                                unsigned* status, cudaStream_t st);
+cudaError_t launch_out_proj_bwd_data(const void* d_y, const void* w, const void* o, void* d_o, float* delta, int B,
+                                     int H, int S, int D, int E, unsigned* status, cudaStream_t st);
+
 // Work-item order of the persistent fast kernels (see the kernels for the two orders).  Head-major
 // order (1) is chosen when the data that the items of one head share (`shared_bytes`, over all
 // heads) would not stay in L2 under block-major order, and there are enough item pairs per CTA

@@ -35,7 +35,8 @@ def test_every_declared_symbol_is_exported(lib):
             "mgn_status_string", "mgn_version", "mgn_attn_profile_events", "mgn_attn_bwd_noalloc", "mgn_measure_fp32_ffma_tflops",
             "mgn_attn_fast_item_order", "mgn_attn_fwd_ext", "mgn_attn_bwd_ext",
             "mgn_attn_bwd_deterministic", "mgn_attn_fwd_accel", "mgn_attn_fwd_accel_workspace_bytes",
-            "mgn_attn_strict_tiles", "mgn_selftest_wait_timeout"} <= set(syms)
+            "mgn_attn_strict_tiles", "mgn_selftest_wait_timeout", "mgn_out_proj_fwd", "mgn_out_proj_bwd_data",
+            "mgn_attn_bwd_given_delta"} <= set(syms)
     for s in syms:
         assert getattr(lib, s) is not None
 
