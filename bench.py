@@ -234,6 +234,62 @@ def fast_mode_summary(mgn, peaks, gpu_index, steps, warmup):
     return out
 
 
+def measure_proj_fusion(mgn, steps, warmup):
+    """The output projection at attention's two seams on the long_context shape (E = H*D): this
+    library's fused kernels against the unfused sequence (torch's library GEMM plus the layout copy it
+    needs, and the attention backward with its own delta pass).  Device-resident, CUDA events."""
+    wl = synth.WORKLOADS["long_context"]
+    B, H, S, D = wl.B, wl.H, wl.S, wl.D
+    E = H * D
+    mode, dt = mgn.MODE_FAST_BF16, torch.bfloat16
+    q, k, v, _ = (t.cuda() for t in synth.make_inputs(wl, dtype=dt))
+    g = torch.Generator(device="cuda").manual_seed(7)
+    w = (torch.randn(H * D, E, device="cuda", generator=g) / (H * D) ** 0.5).to(dt)
+    d_y = torch.randn(B, S, E, device="cuda", generator=g).to(dt)
+    o = torch.empty_like(q); lse = torch.empty(B, H, S, device="cuda")
+    mgn.mgn_attn_fwd(q, k, v, o, lse, wl.causal, wl.scale, mode)
+    y = torch.empty(B, S, E, device="cuda", dtype=dt)
+    d_o = torch.empty_like(q); delta = torch.empty(B, H, S, device="cuda")
+    dq, dk, dv = (torch.empty_like(q) for _ in range(3))
+    ws = mgn.alloc_workspace(B, H, S, D, mode)
+
+    def timed(fn):
+        for _ in range(warmup):
+            fn()
+        torch.cuda.synchronize()
+        e = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+        e[0].record()
+        for i in range(steps):
+            fn()
+            e[i + 1].record()
+        torch.cuda.synchronize()
+        return statistics.median(e[i].elapsed_time(e[i + 1]) for i in range(steps))
+
+    def unfused_fwd():
+        torch.matmul(o.transpose(1, 2).reshape(B, S, H * D), w, out=y)
+
+    def unfused_bwd():
+        d_o.copy_(torch.matmul(d_y, w.t()).view(B, S, H, D).transpose(1, 2))
+        mgn.mgn_attn_bwd(q, k, v, o, d_o, lse, dq, dk, dv, ws, wl.causal, wl.scale, mode)
+
+    def fused_bwd():
+        mgn.mgn_out_proj_bwd_data(d_y, w, o, d_o, delta, mode)
+        mgn.mgn_attn_bwd_given_delta(q, k, v, d_o, lse, delta, dq, dk, dv, ws, wl.causal, wl.scale, mode)
+
+    gemm_flops = 2.0 * B * S * H * D * E
+    f_fused = timed(lambda: mgn.mgn_out_proj_fwd(o, w, y, mode))
+    f_unf = timed(unfused_fwd)
+    p_fused = timed(lambda: mgn.mgn_out_proj_bwd_data(d_y, w, o, d_o, delta, mode))
+    b_fused = timed(fused_bwd)
+    b_unf = timed(unfused_bwd)
+    mgn.mgn_attn_check()
+    return {"shape": {"B": B, "H": H, "S": S, "D": D, "E": E},
+            "out_proj_fwd_ms": {"fused": round(f_fused, 4), "library_gemm_plus_layout_copy": round(f_unf, 4)},
+            "out_proj_fwd_tflops": round(gemm_flops / (f_fused * 1e-3) / 1e12, 1),
+            "do_producer_ms": round(p_fused, 4), "do_producer_tflops": round(gemm_flops / (p_fused * 1e-3) / 1e12, 1),
+            "proj_bwd_plus_attn_bwd_ms": {"fused": round(b_fused, 4), "library_gemm_plus_layout_copy_plus_attn_bwd": round(b_unf, 4)}}
+
+
 def quick_measure_ext(mgn, w, mode, dtype, steps, warmup):
     """Device-resident timing of one cross-attention / grouped-head workload (CUDA events)."""
     q, k, v, d_o = (t.cuda() for t in synth.make_inputs_ext(w, dtype=dtype))
@@ -689,6 +745,7 @@ def main():
                                "sum_tflops": tfl, "frac_of_peak": tfl / mode_peak}
             line["other_workloads"] = table
             line["deterministic_bwd"] = measure_deterministic_bwd(mgn, w, mode, dtype, K, args.warmup)
+            line["proj_fusion"] = measure_proj_fusion(mgn, K, args.warmup)
             if args.mode == "strict":
                 if w.D in (64, 128):
                     line["accel_policy"] = measure_accel_policy(mgn, w, K, args.warmup)
