@@ -208,7 +208,8 @@ int mgn_attn_bwd_ext(const void* q, const void* k, const void* v, const void* o,
     unsigned* sched = fast ? reinterpret_cast<unsigned*>(static_cast<char*>(workspace) + ws_delta_bytes(rows)) : nullptr;
     float* dq_acc = fast ? reinterpret_cast<float*>(static_cast<char*>(workspace) + ws_delta_bytes(rows) + kSchedBytes)
                          : static_cast<float*>(dq);
-    cudaError_t e = mgn::launch_bwd_preprocess(o, d_o, delta, dq_acc, sched, rows, D, fast ? 1 : 0, st);
+    const bool no_acc = fast && mgn::fast_bwd_writes_dq_directly(p);     // single key block: nothing accumulates
+    cudaError_t e = mgn::launch_bwd_preprocess(o, d_o, delta, no_acc ? nullptr : dq_acc, sched, rows, D, fast ? 1 : 0, st);
     if (e != cudaSuccess) return MGN_ERR_CUDA;
     MainKernelTimer timer(st);
     if (!fast)
@@ -277,7 +278,8 @@ int mgn_attn_bwd_given_delta(const void* q, const void* k, const void* v, const 
     unsigned* sched = fast ? reinterpret_cast<unsigned*>(static_cast<char*>(workspace) + ws_delta_bytes(rows)) : nullptr;
     float* dq_acc = fast ? reinterpret_cast<float*>(static_cast<char*>(workspace) + ws_delta_bytes(rows) + kSchedBytes)
                          : static_cast<float*>(dq);
-    cudaError_t e = mgn::launch_bwd_clear(dq_acc, rows * D, sched, st);
+    const bool no_acc = fast && mgn::fast_bwd_writes_dq_directly(p);
+    cudaError_t e = mgn::launch_bwd_clear(no_acc ? nullptr : dq_acc, rows * D, sched, st);
     if (e != cudaSuccess) return MGN_ERR_CUDA;
     MainKernelTimer timer(st);
     if (!fast)

@@ -83,6 +83,7 @@ bwd_clear_kernel(float4* __restrict__ zero, size_t n4, unsigned* __restrict__ co
 {
     pdl_launch_dependents();
     if (counter && blockIdx.x == 0 && threadIdx.x == 0) *counter = 0u;
+    if (!zero) return;
     const uint64_t keep = l2_policy_keep();
     for (size_t i = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x; i < n4;
          i += static_cast<size_t>(gridDim.x) * blockDim.x)

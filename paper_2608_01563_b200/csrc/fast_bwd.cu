@@ -144,8 +144,12 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                 const __grid_constant__ CUtensorMap tmdQ,
                 const float* __restrict__ LSE, const float* __restrict__ DELTA,
                 __nv_bfloat16* __restrict__ dK, __nv_bfloat16* __restrict__ dV,
-                const Dims dm, int causal, int Hg, unsigned* __restrict__ sched, float scale, int Dg, unsigned* status)
+                const Dims dm, int causal, int Hg, unsigned* __restrict__ sched, float scale, int Dg,
+                __nv_bfloat16* __restrict__ dQ_direct, unsigned* status)
 {
+    // dQ_direct (non-null only when the problem has a single key block): every (query head, query block)
+    // tile then receives exactly one partial, which is the final dQ -- it is scaled, rounded and stored
+    // from registers, and no f32 accumulator, clearing pass or conversion pass is needed.
     // Dg: head size in global memory.  Dg = 32 runs the D = 64 build on operand tiles whose columns
     // 32-63 are zero-filled by the tensor maps; only the first 32 columns of dQ, dK, dV are written.
     using C = Cfg<D>;
@@ -400,6 +404,23 @@ fast_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             tmem_ld_wait();
             tc_fence_before();
             mbar_arrive(bar(B_DQEMPTY));                   // Y may be overwritten by dP^T of the next pair
+            if (dQ_direct != nullptr) {
+                if (i0 + r < Sq) {
+                    __nv_bfloat16* row = dQ_direct + (static_cast<size_t>(bh) * Sq + i0 + r) * Dg;
+#pragma unroll
+                    for (int c = 0; c < D / 32; ++c)
+                        if (32 * c < Dg) {
+                            uint32_t u[16];
+#pragma unroll
+                            for (int e = 0; e < 16; ++e)
+                                u[e] = pack_bf16(__uint_as_float(v[c][2 * e]) * scale, __uint_as_float(v[c][2 * e + 1]) * scale);
+#pragma unroll
+                            for (int q = 0; q < 4; ++q)
+                                *reinterpret_cast<uint4*>(row + 32 * c + 8 * q) = make_uint4(u[4 * q], u[4 * q + 1], u[4 * q + 2], u[4 * q + 3]);
+                        }
+                }
+                continue;
+            }
 #pragma unroll
             for (int round = 0; round < D / 64; ++round) {
                 // the previous reduction must have finished reading the staging area
@@ -635,6 +656,10 @@ cudaError_t launch_gen(const Problem& p, const void* q, const void* k, const voi
     if (cudaDeviceGetAttribute(&l2, cudaDevAttrL2CacheSize, dev) != cudaSuccess || l2 <= 0) l2 = 64 << 20;
     const double per_head = static_cast<double>(p.group()) * p.Sq * D * (4 + 2 + 2) + static_cast<double>(p.Sk) * D * 4;
     long long hg = static_cast<long long>(0.5 * l2 / per_head);
+    // ... but a group must hold enough items to keep every CTA busy through its phase of the list
+    // (measured: 96 long items per group cost a grouped-head decoder shape 10 %)
+    const long long hg_min = (3LL * sms / 2 + n_kb - 1) / n_kb;
+    if (hg < hg_min) hg = hg_min;
     hg = hg < 1 ? 1 : hg > p.BHkv() ? p.BHkv() : hg;
     const long long n_groups = (p.BHkv() + hg - 1) / hg;
     hg = (p.BHkv() + n_groups - 1) / n_groups;       // equal groups: a short last group unbalances the end of the list
@@ -642,10 +667,11 @@ cudaError_t launch_gen(const Problem& p, const void* q, const void* k, const voi
     if (g_forced_item_order == 1) hg = 1;             // head by head
     const int Hg = static_cast<int>(hg);
     const Dims dm{p.Sq, p.Sk, p.BH(), p.H, p.group(), p.off()};
+    const bool direct = WITH_DQ && fast_bwd_writes_dq_directly(p);
     e = launch_pdl(kern, static_cast<unsigned>(blocks), kThreads, C::SMEM, st, tq, tk, tv, tdo, tdq, lse, delta,
                    static_cast<__nv_bfloat16*>(dk), static_cast<__nv_bfloat16*>(dv), dm, p.causal, Hg, sched, p.scale,
-                   p.D, status);
-    if (e != cudaSuccess) return e;
+                   p.D, direct ? static_cast<__nv_bfloat16*>(dq) : nullptr, status);
+    if (e != cudaSuccess || direct) return e;
     e = cudaGetLastError();
     if (e != cudaSuccess || !WITH_DQ) return e;
     const size_t n4 = static_cast<size_t>(p.BH()) * p.Sq * p.D / 4;

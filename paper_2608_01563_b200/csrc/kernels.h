@@ -129,6 +129,9 @@ cudaError_t launch_fast_fwd(const Problem& p, const void* q, const void* k, cons
 cudaError_t launch_to_f16(const float* in, void* out, size_t n, cudaStream_t st);
 cudaError_t launch_fast_fwd_f16(const Problem& p, const void* q16, const void* k16, const void* v16, float* o,
                                 float* lse, unsigned* status, cudaStream_t st);
+// With a single 128-key block every dQ tile receives one partial: the fused kernel then stores dq itself
+// and neither clears nor converts the f32 accumulator (which the caller need not clear either).
+inline bool fast_bwd_writes_dq_directly(const Problem& p) { return p.Sk <= 128; }
 cudaError_t launch_fast_bwd(const Problem& p, const void* q, const void* k, const void* v,
                             const void* d_o, const float* lse, const float* delta,
                             float* dq_acc, void* dq, void* dk, void* dv,
