@@ -142,9 +142,13 @@ strict_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             for (int y = 0; y < RN; ++y) { s[x][y] = 0.f; dp[x][y] = 0.f; }
         {
             const int xq = tr & 7, xk = tc & 7;
-            // Fully unrolled for the 8-row micro-tile; the 5-row one (40-row query tiles) runs 8 % faster
-            // with two steps per iteration (measured), the rolled loop being kinder to the instruction cache.
-            constexpr int kUnrollA = (RM == 5) ? 2 : D / 4;
+            // Unroll factors are set by the instruction cache: with the packed FMAs of phase B the top
+            // stall of this kernel became instruction fetch (0.94 stalled warps per issue), and a fully
+            // unrolled phase A alone is 70 KB of code.  Measured at D = 64 with 64-row tiles: 16 / 8 / 4 / 2 / 1
+            // steps per iteration -> 0.808 / 0.760 / 0.731 / 0.724 / 0.723 ms on the GPT-2-small shape; at
+            // D = 128 four steps are best (2.13 against 2.16 ms unrolled, 2.23 with two); the 5-row
+            // micro-tile of the 40-row tiles prefers eight (0.300 against 0.310 ms with two).
+            constexpr int kUnrollA = (RM == 5) ? 8 : (D == 128) ? 4 : 2;
 #pragma unroll kUnrollA
             for (int pc = 0; pc < D / 4; ++pc) {
                 const uint32_t oq = (pc >> 3) * (BM * 128) + tr * 128 + (((pc & 7) ^ xq) << 4);
@@ -200,7 +204,7 @@ strict_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             // this thread's key rows: j = 4*tr + 64*g + u, g < JN/4, u < 4
             // two groups of eight query rows per iteration (and four groups of keys in phase C) run 1 % faster
             // with the 64-row tiles; the 40-row tiles lose 11 % that way and keep the rolled forms (measured)
-            constexpr int kUnrollB = (RM == 5) ? 1 : 2;
+                        constexpr int kUnrollB = (RM == 5) ? 1 : 2;
 #pragma unroll kUnrollB
             for (int i8 = 0; i8 < BM; i8 += 8)
 #pragma unroll
@@ -246,7 +250,7 @@ strict_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             for (int x = 0; x < RM; ++x)
 #pragma unroll
                 for (int e = 0; e < DV; ++e) dq[x][e] = 0.f;
-            constexpr int kUnrollC = (RM == 5) ? 2 : 4;
+                        constexpr int kUnrollC = (RM == 5 || D <= 64) ? 2 : 4;
 #pragma unroll kUnrollC
             for (int j8 = 0; j8 < BN / 8; ++j8) {
                 float4 d4[2][RM];

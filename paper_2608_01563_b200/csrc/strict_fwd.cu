@@ -145,11 +145,12 @@ strict_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         {
             const uint32_t qa = sQ + tr * 128, ka = sK + tc * 128;
             const int xq = tr & 7, xk = tc & 7;
-            // Loop bodies of about 2000 FFMAs (eight contraction steps here, eight groups of keys in the
-            // second product) run best at D = 64: larger ones miss the instruction cache, smaller ones
-            // leave the operand loads less room to be hoisted (measured; other head sizes keep the
-            // forms they were tuned with).
-            constexpr int kUnrollQK = (D == 64) ? 8 : D / 4;
+            // Unroll factors are set by the instruction cache (instruction fetch is this kernel's top stall,
+            // 0.87 stalled warps per issue with the loops of both products unrolled far): measured on the
+            // GPT-2-small shape, 8 contraction steps x 32 keys per iteration -> 0.363 ms, 4 x 32 -> 0.326,
+            // 4 x 16 -> 0.328, 1 x 16 -> 0.324; at D = 128, 32 x 32 -> 0.844 ms, 16 x 16 -> 0.828; the 5-row
+            // micro-tile of the 40-row tiles keeps 8 x 32 (0.135 against 0.137-0.139 ms).
+            constexpr int kUnrollQK = (RM == 5) ? 8 : (D == 128) ? 16 : 4;
 #pragma unroll kUnrollQK
             for (int pc = 0; pc < D / 4; ++pc) {
                 const uint32_t oq = (pc >> 3) * (BM * 128) + (((pc & 7) ^ xq) << 4);
@@ -234,7 +235,7 @@ strict_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         // row pairs of P come as they are stored; DV * RP packed FMAs follow.
         {
             const uint32_t pa = sP + ((2 * tr) << 4);
-            constexpr int kUnrollPV = (D == 32) ? 8 : 32;
+                        constexpr int kUnrollPV = (D == 32) ? 8 : (D == 128) ? 16 : 32;
 #pragma unroll kUnrollPV
             for (int j = 0; j < BN; ++j) {
                 const int u = j & 7;
