@@ -613,13 +613,21 @@ __global__ void __launch_bounds__(256)
 dq_convert_kernel(const float4* __restrict__ acc, uint2* __restrict__ out, size_t n4, float scale)
 {
     pdl_wait();   // programmatic dependent of the main kernel: resident early, reads after it has completed
-    for (size_t i = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x; i < n4;
-         i += static_cast<size_t>(gridDim.x) * blockDim.x) {
-        const float4 a = acc[i];
-        uint2 o;
-        o.x = pack_bf16(a.x * scale, a.y * scale);
-        o.y = pack_bf16(a.z * scale, a.w * scale);
-        out[i] = o;
+    constexpr int UNR = 4;     // loads in flight per thread (one at a time ran at half the DRAM rate)
+    const size_t step = static_cast<size_t>(gridDim.x) * blockDim.x;
+    for (size_t i0 = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x; i0 < n4; i0 += UNR * step) {
+        float4 a[UNR];
+#pragma unroll
+        for (int u = 0; u < UNR; ++u)
+            if (i0 + u * step < n4) a[u] = acc[i0 + u * step];
+#pragma unroll
+        for (int u = 0; u < UNR; ++u)
+            if (i0 + u * step < n4) {
+                uint2 o;
+                o.x = pack_bf16(a[u].x * scale, a[u].y * scale);
+                o.y = pack_bf16(a[u].z * scale, a[u].w * scale);
+                out[i0 + u * step] = o;
+            }
     }
 }
 
