@@ -61,6 +61,8 @@ def _load():
         lib.ref_out_proj_bwd_data.restype = None
         lib.ref_out_proj_bwd_weight.argtypes = [_dp] * 3 + [i] * 5
         lib.ref_out_proj_bwd_weight.restype = None
+        lib.ref_qkv_rope.argtypes = [_dp] * 7 + [i] * 6
+        lib.ref_qkv_rope.restype = None
         lib.ref_max_threads.argtypes = []
         lib.ref_max_threads.restype = i
         _lib = lib
@@ -184,3 +186,14 @@ def out_proj_bwd(d_y, w, o):
     _load().ref_out_proj_bwd_data(_p(d_y), _p(w), _p(o), _p(d_o), _p(delta), B, H, S, D, E)
     _load().ref_out_proj_bwd_weight(_p(o), _p(d_y), _p(d_w), B, H, S, D, E)
     return d_o, delta, d_w
+
+
+def qkv_rope(x, w, cos_t, sin_t, H: int, Hkv: int, D: int):
+    """Fused query/key/value projection with rotary embedding (rotate-half pairing, caller's angle table):
+    x [B,S,E], w [(H+2Hkv)*D, E], cos_t, sin_t [S, D/2] -> (Q [B,H,S,D], K, V [B,Hkv,S,D]), float64."""
+    x, w, cos_t, sin_t = _c(x), _c(w), _c(cos_t), _c(sin_t)
+    B, S, E = x.shape
+    assert w.shape == ((H + 2 * Hkv) * D, E) and cos_t.shape == (S, D // 2) and sin_t.shape == (S, D // 2) and D <= 1024
+    q = np.empty((B, H, S, D)); k = np.empty((B, Hkv, S, D)); v = np.empty((B, Hkv, S, D))
+    _load().ref_qkv_rope(_p(x), _p(w), _p(cos_t), _p(sin_t), _p(q), _p(k), _p(v), B, S, E, H, Hkv, D)
+    return q, k, v

@@ -82,3 +82,49 @@ void ref_out_proj_bwd_weight(const double *O, const double *dY, double *dW, int 
             }
     }
 }
+
+/*
+ * The step before attention: the fused query/key/value projection with rotary position embedding.
+ * (Same sections of the paper: a matrix product whose epilogue absorbs the step that follows it.  The
+ * paper prints no formula; this is the textbook definition, with the "rotate-half" pairing of
+ * columns d and d + D/2 and the angle table supplied by the caller, so no convention about the
+ * frequency base is baked in.)
+ *
+ *   X [B,S,E]   W [(H + 2 Hkv) D, E]  (rows: all query heads, then all key heads, then all value heads)
+ *   y[b,s,n]  = sum_e X[b,s,e] * W[n,e]
+ *   for query and key heads, with c = cos_t[s, d], sn = sin_t[s, d], d < D/2:
+ *       out[d]       = y[d] * c - y[d + D/2] * sn
+ *       out[d + D/2] = y[d + D/2] * c + y[d] * sn
+ *   value heads are copied.  Q [B,H,S,D], K, V [B,Hkv,S,D].
+ */
+void ref_qkv_rope(const double *X, const double *W, const double *cos_t, const double *sin_t,
+                  double *Q, double *K, double *V, int B, int S, int E, int H, int Hkv, int D)
+{
+    const int heads = H + 2 * Hkv, half = D / 2;
+    const long rows = (long)B * S;
+#pragma omp parallel for schedule(static)
+    for (long r = 0; r < rows; ++r) {
+        const int b = (int)(r / S), s = (int)(r % S);
+        const double *x = X + (size_t)r * E;
+        for (int hh = 0; hh < heads; ++hh) {
+            double y[1024];                                   /* D <= 1024 */
+            for (int d = 0; d < D; ++d) {
+                const double *w = W + ((size_t)hh * D + d) * E;
+                double acc = 0.0;
+                for (int e = 0; e < E; ++e) acc += x[e] * w[e];
+                y[d] = acc;
+            }
+            double *out;
+            int rope = 1;
+            if (hh < H) out = Q + (((size_t)b * H + hh) * S + s) * D;
+            else if (hh < H + Hkv) out = K + (((size_t)b * Hkv + (hh - H)) * S + s) * D;
+            else { out = V + (((size_t)b * Hkv + (hh - H - Hkv)) * S + s) * D; rope = 0; }
+            if (!rope) { for (int d = 0; d < D; ++d) out[d] = y[d]; continue; }
+            for (int d = 0; d < half; ++d) {
+                const double c = cos_t[(size_t)s * half + d], sn = sin_t[(size_t)s * half + d];
+                out[d] = y[d] * c - y[d + half] * sn;
+                out[d + half] = y[d + half] * c + y[d] * sn;
+            }
+        }
+    }
+}

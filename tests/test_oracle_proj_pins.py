@@ -86,3 +86,59 @@ def test_delta_is_the_row_statistic_of_the_attention_backward():
     d_o, delta, _ = orc.out_proj_bwd(d_y, w, o)
     P, dP, _ = orc.head_matrices(q, k, v, d_o[0, 0], True, 0.5)
     np.testing.assert_allclose(delta[0, 0], (P * dP).sum(axis=1), rtol=1e-12, atol=1e-13)
+
+
+# --------------------------------------------------------------------------- QKV projection + rotary embedding
+def _angles(S, D, base=10000.0):
+    inv = base ** (-np.arange(D // 2) * 2.0 / D)
+    ang = np.arange(S)[:, None] * inv[None, :]
+    return np.cos(ang), np.sin(ang)
+
+
+def test_qkv_rope_hand_worked_example():
+    # B=1, S=2, E=1, H=1, Hkv=1, D=2: y = x * w; position 0 is not rotated, position 1 by angle a
+    x = np.array([[[2.0], [3.0]]])
+    w = np.array([[1.0], [2.0], [-1.0], [0.5], [4.0], [5.0]])          # q: (1,2)  k: (-1,0.5)  v: (4,5)
+    a = 0.3
+    cos_t, sin_t = np.array([[1.0], [math_cos := np.cos(a)]]), np.array([[0.0], [math_sin := np.sin(a)]])
+    q, k, v = orc.qkv_rope(x, w, cos_t, sin_t, 1, 1, 2)
+    np.testing.assert_allclose(q[0, 0, 0], [2.0, 4.0], atol=1e-15)                    # x=2, no rotation
+    np.testing.assert_allclose(q[0, 0, 1], [3 * math_cos - 6 * math_sin, 6 * math_cos + 3 * math_sin], atol=1e-15)
+    np.testing.assert_allclose(k[0, 0, 1], [-3 * math_cos - 1.5 * math_sin, 1.5 * math_cos - 3 * math_sin], atol=1e-15)
+    np.testing.assert_allclose(v[0, 0], [[8.0, 10.0], [12.0, 15.0]], atol=1e-15)      # values are not rotated
+
+
+@pytest.mark.parametrize("B,S,E,H,Hkv,D", [(2, 5, 7, 3, 1, 4), (1, 9, 6, 2, 2, 8)])
+def test_qkv_rope_matches_torch_float64(B, S, E, H, Hkv, D):
+    g = torch.Generator().manual_seed(S + E)
+    x = torch.randn(B, S, E, generator=g, dtype=torch.float64)
+    w = torch.randn((H + 2 * Hkv) * D, E, generator=g, dtype=torch.float64)
+    cos_t, sin_t = _angles(S, D)
+    y = (x @ w.t()).view(B, S, H + 2 * Hkv, D).permute(0, 2, 1, 3)                     # [B, heads, S, D]
+    c = torch.from_numpy(np.concatenate([cos_t, cos_t], axis=1))                        # rotate-half, written the usual way
+    s_ = torch.from_numpy(np.concatenate([sin_t, sin_t], axis=1))
+    rot = torch.cat([-y[..., D // 2:], y[..., :D // 2]], dim=-1)
+    yr = y * c + rot * s_
+    q, k, v = orc.qkv_rope(x.numpy(), w.numpy(), cos_t, sin_t, H, Hkv, D)
+    tol = dict(rtol=1e-12, atol=1e-12)
+    np.testing.assert_allclose(q, yr[:, :H].numpy(), **tol)
+    np.testing.assert_allclose(k, yr[:, H:H + Hkv].numpy(), **tol)
+    np.testing.assert_allclose(v, y[:, H + Hkv:].numpy(), **tol)
+
+
+def test_qkv_rope_invariants():
+    """A rotation keeps the norm of every (d, d + D/2) pair; q.k of rotated vectors depends only on the
+    position difference; zero angles leave the plain projection."""
+    B, S, E, H, Hkv, D = 1, 6, 5, 1, 1, 4
+    x, w = rnd(20, B, S, E), rnd(21, (H + 2 * Hkv) * D, E)
+    cos_t, sin_t = _angles(S, D)
+    q, k, v = orc.qkv_rope(x, w, cos_t, sin_t, H, Hkv, D)
+    q0, k0, v0 = orc.qkv_rope(x, w, np.ones_like(cos_t), np.zeros_like(sin_t), H, Hkv, D)
+    np.testing.assert_allclose(v, v0, rtol=0, atol=0)
+    np.testing.assert_allclose(q0[0, 0], x[0] @ w[:D].T, rtol=1e-13, atol=1e-13)
+    pair_norm = lambda t: t[..., :D // 2] ** 2 + t[..., D // 2:] ** 2
+    np.testing.assert_allclose(pair_norm(q), pair_norm(q0), rtol=1e-12, atol=1e-12)
+    # the same unrotated vectors placed at positions (1, 3) and (2, 4) give the same rotated dot product
+    xs = np.zeros((1, 6, E)); xs[0, 1] = xs[0, 2] = x[0, 0]; xs[0, 3] = xs[0, 4] = x[0, 5]
+    q, k, _ = orc.qkv_rope(xs, w, cos_t, sin_t, H, Hkv, D)
+    np.testing.assert_allclose(q[0, 0, 3] @ k[0, 0, 1], q[0, 0, 4] @ k[0, 0, 2], rtol=1e-12, atol=1e-12)
