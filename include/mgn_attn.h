@@ -175,6 +175,14 @@ int mgn_attn_bwd_deterministic(const void* q, const void* k, const void* v, cons
  *     d_y [B,S,E], w [H*D,E], o [B,H,S,D] in; d_o [B,H,S,D] (bf16) and delta [B,H,S] (f32) out.  delta is
  *     formed from the bf16-rounded d_o and is what mgn_attn_bwd's own first pass would compute from
  *     o and d_o; hand it to mgn_attn_bwd_given_delta.
+ * mgn_out_proj_bwd_weight: d_w[h*D+d, e] = sum_{b,s} o[b,h,s,d] * d_y[b,s,e]
+ *     o [B,H,S,D] read head-major again, d_y [B,S,E] in; d_w [H*D,E] (bf16) out.
+ * mgn_qkv_rope_fwd:  the step before attention.  y[b,s,n] = sum_e x[b,s,e] * w[n,e] with
+ *     w [(H + 2 H_kv) D, E]: rows of all query heads, then all key heads, then all value heads; query and
+ *     key heads are rotated pairwise, columns d and d + D/2 ("rotate-half"), by the caller's angle tables
+ *     cos_t, sin_t [S, D/2] (f32, device): out[d] = y[d] c - y[d+D/2] s, out[d+D/2] = y[d+D/2] c + y[d] s;
+ *     value heads are copied.  q [B,H,S,D], k, v [B,H_kv,S,D] (bf16) out, in the layout the attention
+ *     entry points read.  The rotation is done in f32 on the accumulators, before the one rounding to bf16.
  * mgn_attn_bwd_given_delta: mgn_attn_bwd_ext without `o`, with a ready `delta` [B,H,S_q] (f32, read
  *     only): the pass over o and d_o is skipped.  Either mode.  Workspace as for mgn_attn_bwd_ext.
  * Errors as elsewhere: INVALID_ARG (null pointer, size <= 0, unknown mode), UNSUPPORTED, MISALIGNED,
@@ -183,6 +191,10 @@ int mgn_attn_bwd_deterministic(const void* q, const void* k, const void* v, cons
 int mgn_out_proj_fwd(const void* o, const void* w, void* y, int B, int H, int S, int D, int E, int mode, void* stream);
 int mgn_out_proj_bwd_data(const void* d_y, const void* w, const void* o, void* d_o, float* delta,
                           int B, int H, int S, int D, int E, int mode, void* stream);
+int mgn_out_proj_bwd_weight(const void* o, const void* d_y, void* d_w, int B, int H, int S, int D, int E, int mode,
+                            void* stream);
+int mgn_qkv_rope_fwd(const void* x, const void* w, const float* cos_t, const float* sin_t, void* q, void* k, void* v,
+                     int B, int S, int E, int H, int H_kv, int D, int mode, void* stream);
 int mgn_attn_bwd_given_delta(const void* q, const void* k, const void* v, const void* d_o, const float* lse,
                              const float* delta, void* dq, void* dk, void* dv,
                              void* workspace, size_t workspace_bytes,

@@ -75,6 +75,10 @@ def lib() -> ctypes.CDLL:
         L.mgn_out_proj_fwd.restype = i
         L.mgn_out_proj_bwd_data.argtypes = [vp] * 5 + [i, i, i, i, i, i, vp]
         L.mgn_out_proj_bwd_data.restype = i
+        L.mgn_out_proj_bwd_weight.argtypes = [vp, vp, vp, i, i, i, i, i, i, vp]
+        L.mgn_out_proj_bwd_weight.restype = i
+        L.mgn_qkv_rope_fwd.argtypes = [vp] * 7 + [i] * 7 + [vp]
+        L.mgn_qkv_rope_fwd.restype = i
         L.mgn_attn_bwd_given_delta.argtypes = [vp] * 9 + [vp, sz, i, i, i, i, i, i, i, f, i, vp]
         L.mgn_attn_bwd_given_delta.restype = i
         L.mgn_selftest_wait_timeout.argtypes = [vp, vp]
@@ -239,6 +243,21 @@ def mgn_out_proj_bwd_data(d_y, w, o, d_o, delta, mode: int, stream: Optional[int
                                      int(w.shape[1]), int(mode), _stream(stream))
     if st != MGN_OK:
         raise MgnError(st, "mgn_out_proj_bwd_data")
+
+
+def mgn_out_proj_bwd_weight(o, d_y, d_w, mode: int, stream: Optional[int] = None) -> None:
+    B, H, S, D = _dims(o)
+    st = lib().mgn_out_proj_bwd_weight(_ptr(o), _ptr(d_y), _ptr(d_w), B, H, S, D, int(d_w.shape[1]), int(mode), _stream(stream))
+    if st != MGN_OK:
+        raise MgnError(st, "mgn_out_proj_bwd_weight")
+
+
+def mgn_qkv_rope_fwd(x, w, cos_t, sin_t, q, k, v, mode: int, stream: Optional[int] = None) -> None:
+    B, H, S, D = _dims(q)
+    st = lib().mgn_qkv_rope_fwd(_ptr(x), _ptr(w), _ptr(cos_t), _ptr(sin_t), _ptr(q), _ptr(k), _ptr(v), B, S,
+                                int(x.shape[2]), H, int(k.shape[1]), D, int(mode), _stream(stream))
+    if st != MGN_OK:
+        raise MgnError(st, "mgn_qkv_rope_fwd")
 
 
 def mgn_attn_bwd_given_delta(q, k, v, d_o, lse, delta, dq, dk, dv, workspace, causal: bool, scale: float, mode: int,

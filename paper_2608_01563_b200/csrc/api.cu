@@ -330,6 +330,31 @@ int mgn_out_proj_bwd_data(const void* d_y, const void* w, const void* o, void* d
                ? MGN_OK : MGN_ERR_CUDA;
 }
 
+int mgn_out_proj_bwd_weight(const void* o, const void* d_y, void* d_w, int B, int H, int S, int D, int E, int mode,
+                            void* stream)
+{
+    if (int r = check_proj(o, d_y, d_w, d_w, B, H, S, D, E, mode)) return r;
+    unsigned* status = nullptr;
+    if (int r = device_setup(&status)) return r;
+    return mgn::launch_out_proj_bwd_weight(o, d_y, d_w, B, H, S, D, E, status, static_cast<cudaStream_t>(stream)) ==
+                   cudaSuccess
+               ? MGN_OK : MGN_ERR_CUDA;
+}
+
+int mgn_qkv_rope_fwd(const void* x, const void* w, const float* cos_t, const float* sin_t, void* q, void* k, void* v,
+                     int B, int S, int E, int H, int H_kv, int D, int mode, void* stream)
+{
+    if (!cos_t || !sin_t || !k || !v || H_kv <= 0) return MGN_ERR_INVALID_ARG;
+    if (int r = check_proj(x, w, q, k, B, H, S, D, E, mode)) return r;
+    if (static_cast<long long>(H + 2LL * H_kv) * D > 0x7fffffffLL) return MGN_ERR_UNSUPPORTED;
+    if (!aligned16(v) || !aligned16(cos_t) || !aligned16(sin_t)) return MGN_ERR_MISALIGNED;
+    unsigned* status = nullptr;
+    if (int r = device_setup(&status)) return r;
+    return mgn::launch_qkv_rope(x, w, cos_t, sin_t, q, k, v, B, S, E, H, H_kv, D, status,
+                                static_cast<cudaStream_t>(stream)) == cudaSuccess
+               ? MGN_OK : MGN_ERR_CUDA;
+}
+
 int mgn_attn_bwd(const void* q, const void* k, const void* v, const void* o, const void* d_o,
                  const float* lse, void* dq, void* dk, void* dv,
                  void* workspace, size_t workspace_bytes,
@@ -395,6 +420,6 @@ const char* mgn_status_string(int status)
     }
 }
 
-int mgn_version(void) { return 300; }   // 0.2.1: tile-shape query, low-padding strict tiles, leaner fast forward (0.2.0: extended shapes, deterministic backward, accelerated forward)
+int mgn_version(void) { return 310; }   // 0.2.1: tile-shape query, low-padding strict tiles, leaner fast forward (0.2.0: extended shapes, deterministic backward, accelerated forward)
 
 }  // extern "C"

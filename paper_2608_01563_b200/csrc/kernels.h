@@ -105,6 +105,13 @@ cudaError_t launch_out_proj_fwd(const void* o, const void* w, void* y, int B, in
                                 unsigned* status, cudaStream_t st);
 cudaError_t launch_out_proj_bwd_data(const void* d_y, const void* w, const void* o, void* d_o, float* delta, int B,
                                      int H, int S, int D, int E, unsigned* status, cudaStream_t st);
+// d_w [H*D,E] = concat_h(o)^T d_y, contracting over all B*S positions.
+cudaError_t launch_out_proj_bwd_weight(const void* o, const void* d_y, void* d_w, int B, int H, int S, int D, int E,
+                                       unsigned* status, cudaStream_t st);
+// (q | k | v) = x [B,S,E] w^T, w [(H+2Hkv)*D, E] (query heads, key heads, value heads), rotary embedding
+// (rotate-half pairing, angle tables cos_t, sin_t [S, D/2] f32) applied to q and k; q [B,H,S,D], k, v [B,Hkv,S,D].
+cudaError_t launch_qkv_rope(const void* x, const void* w, const float* cos_t, const float* sin_t, void* q, void* k,
+                            void* v, int B, int S, int E, int H, int Hkv, int D, unsigned* status, cudaStream_t st);
 
 // Work-item order of the persistent fast kernels (see the kernels for the two orders).  Head-major
 // order (1) is chosen when the data that the items of one head share (`shared_bytes`, over all

@@ -1,20 +1,21 @@
-// Output projection around attention, fast mode (bf16 operands, tcgen05 products, f32 accumulation).
+// The projections either side of attention, fast mode (bf16 operands, tcgen05 products, f32 accumulation).
 //
 // The paper gives its matrix-product kernels prologues and epilogues that absorb the steps around
 // them (Section 3.3, kernel archetypes) and finds that dispatch structure matters where kernels are
-// small (Section 7.3).  The step after attention is the projection of the concatenated heads,
-//     Y[b,s,:] = sum_h O[b,h,s,:] W[h*D:(h+1)*D, :],
-// and two fusions fall out of writing that product here instead of calling a library GEMM:
-//   FWD  reads O where attention left it ([B,H,S,D], heads separate): the operand tiles are fetched by
-//        TMA from the head-major tensor, so no transposed / concatenated copy of O is ever made;
-//   DO   the backward product dO = dY W^T writes dO straight into the [B,H,S,D] layout the attention
-//        backward reads, and its epilogue also emits delta = rowsum(dO o O) -- the attention
-//        backward's preprocess pass -- while the dO tile is still in registers.
-// One CTA computes a 128 x 256 output tile: rows are 128 positions s of one batch element, columns
-// are 256 output features (FWD) or 256 (head, d) columns = 256 / D whole heads (DO).  Warp 0 streams
-// 64-wide contraction slices of both operands through a four-stage TMA ring, one lane of warp 1
-// issues the products into a 256-column tensor-memory accumulator, warps 2-5 (one thread per row)
-// read it out.
+// small (Section 7.3).  Four products are written here instead of calling a library GEMM, because each
+// absorbs a layout change or a pass that would otherwise be a kernel of its own:
+//   QKV  (Q | K | V) = X W^T with the rotary embedding applied to Q and K in the epilogue, written
+//        straight into the [B,H,S,D] / [B,Hkv,S,D] layouts the attention kernels read;
+//   FWD  Y = O_concat W_o reads O where attention left it ([B,H,S,D], heads separate): the operand tiles
+//        are fetched by TMA from the head-major tensor, no concatenated copy of O is made;
+//   DO   dO = dY W_o^T writes dO into the [B,H,S,D] layout the attention backward reads, and its
+//        epilogue also emits delta = rowsum(dO o O) -- the attention backward's preprocess pass -- while
+//        the dO tile is still in registers;
+//   DW   dW_o = O_concat^T dY contracts over the positions, again reading O head-major (both operands
+//        are fed to the tensor core with the non-contracted index contiguous).
+// One CTA computes a 128 x 256 output tile.  Warp 0 streams 64-wide contraction slices of both
+// operands through a four-stage TMA ring, one lane of warp 1 issues the products into a 256-column
+// tensor-memory accumulator, warps 2-5 (one thread per accumulator row) read it out.
 #include <cuda_bf16.h>
 
 #include "kernels.h"
@@ -31,14 +32,106 @@ constexpr int OFF_A = 0, OFF_B = kStages * A_BYTES, OFF_BAR = OFF_B + kStages * 
 constexpr int PAYLOAD = OFF_BAR + 128;
 constexpr int SMEM = PAYLOAD + 1024;
 enum { B_FULL = 0, B_EMPTY = kStages, B_ACC = 2 * kStages, B_COUNT = 2 * kStages + 1 };
+enum { V_FWD = 0, V_DO = 1, V_DW = 2, V_QKV = 3 };
 
-// DO = false: Y = O_concat W       A = O  (rank-3 map D x S x B*H),  B = W as MN-major operand (rows = k)
-// DO = true : dO = dY W^T, delta   A = dY (rank-3 map E x S x B),    B = W as K-major operand (rows = n)
-template <bool DO>
+struct ProjArgs {
+    __nv_bfloat16* out;          // FWD: y   DO: d_o   DW: d_w   QKV: q
+    __nv_bfloat16* out_k;        // QKV: k
+    __nv_bfloat16* out_v;        // QKV: v
+    const __nv_bfloat16* o;      // DO: attention output, for delta
+    float* delta;                // DO
+    const float* cos_t;          // QKV: [S, D/2]
+    const float* sin_t;
+    int B, H, Hkv, S, D, E;
+};
+
+__device__ __forceinline__ void store_row32(__nv_bfloat16* dst, const uint32_t (&u)[16], int pieces) {
+#pragma unroll
+    for (int p4 = 0; p4 < 4; ++p4)
+        if (p4 < pieces) reinterpret_cast<uint4*>(dst)[p4] = make_uint4(u[4 * p4], u[4 * p4 + 1], u[4 * p4 + 2], u[4 * p4 + 3]);
+}
+
+// Epilogue of the plain products: row `row` of the output (global row index), 32 columns starting at n.
+template <int V>
+__device__ __forceinline__ void epilogue_plain(const ProjArgs& a, const uint32_t (&v)[32], int b, int row, int n, float& dl)
+{
+    uint32_t u[16];
+#pragma unroll
+    for (int e = 0; e < 16; ++e) u[e] = pack_bf16(__uint_as_float(v[2 * e]), __uint_as_float(v[2 * e + 1]));
+    if constexpr (V == V_DO) {
+        const int h = n / a.D, d = n % a.D;
+        const size_t off = ((static_cast<size_t>(b) * a.H + h) * a.S + row) * a.D + d;
+        store_row32(a.out + off, u, 4);
+        const uint4* orow = reinterpret_cast<const uint4*>(a.o + off);
+#pragma unroll
+        for (int p4 = 0; p4 < 4; ++p4) {
+            const uint4 ov = orow[p4];
+            const uint32_t ow[4] = {ov.x, ov.y, ov.z, ov.w};
+#pragma unroll
+            for (int t = 0; t < 4; ++t) {
+                // delta from the bf16 values the attention backward will read
+                const uint32_t dv = u[4 * p4 + t];
+                dl = fmaf(__uint_as_float(dv << 16), __uint_as_float(ow[t] << 16), dl);
+                dl = fmaf(__uint_as_float(dv & 0xffff0000u), __uint_as_float(ow[t] & 0xffff0000u), dl);
+            }
+        }
+        if (d + 32 == a.D) {                  // last chunk of this head
+            a.delta[(static_cast<size_t>(b) * a.H + h) * a.S + row] = dl;
+            dl = 0.f;
+        }
+    } else {
+        // FWD: y[b, row, n..]   DW: d_w[row, n..]   (E is a multiple of 8: whole 16-byte pieces)
+        const size_t r = V == V_FWD ? static_cast<size_t>(b) * a.S + row : static_cast<size_t>(row);
+        store_row32(a.out + r * a.E + n, u, (a.E - n) / 8);
+    }
+}
+
+// Epilogue of the QKV product: one head (D accumulator columns of this thread's row) at a time --
+// rotate the (d, d + D/2) pairs of query and key heads by the caller's angles, round, store.
+template <int D>
+__device__ __forceinline__ void epilogue_qkv_head(const ProjArgs& a, uint32_t tacc_head, int b, int s, int hh, bool row_ok)
+{
+    constexpr int NC = D / 32, HALF = D / 2;
+    uint32_t v[NC][32];
+#pragma unroll
+    for (int c = 0; c < NC; ++c) tmem_ld32(tacc_head + 32 * c, v[c]);      // whole warp, whatever the row
+    tmem_ld_wait();
+    if (!row_ok || hh >= a.H + 2 * a.Hkv) return;
+    __nv_bfloat16* dst;
+    if (hh < a.H) dst = a.out + ((static_cast<size_t>(b) * a.H + hh) * a.S + s) * D;
+    else if (hh < a.H + a.Hkv) dst = a.out_k + ((static_cast<size_t>(b) * a.Hkv + (hh - a.H)) * a.S + s) * D;
+    else dst = a.out_v + ((static_cast<size_t>(b) * a.Hkv + (hh - a.H - a.Hkv)) * a.S + s) * D;
+    if (hh < a.H + a.Hkv) {
+        const float* ct = a.cos_t + static_cast<size_t>(s) * HALF;
+        const float* st = a.sin_t + static_cast<size_t>(s) * HALF;
+#pragma unroll
+        for (int c = 0; c < NC / 2; ++c)
+#pragma unroll
+            for (int e4 = 0; e4 < 8; ++e4) {
+                const float4 c4 = *reinterpret_cast<const float4*>(ct + 32 * c + 4 * e4);
+                const float4 s4 = *reinterpret_cast<const float4*>(st + 32 * c + 4 * e4);
+                const float cc[4] = {c4.x, c4.y, c4.z, c4.w}, ss[4] = {s4.x, s4.y, s4.z, s4.w};
+#pragma unroll
+                for (int t = 0; t < 4; ++t) {
+                    const float lo = __uint_as_float(v[c][4 * e4 + t]), hi = __uint_as_float(v[c + NC / 2][4 * e4 + t]);
+                    v[c][4 * e4 + t] = __float_as_uint(lo * cc[t] - hi * ss[t]);
+                    v[c + NC / 2][4 * e4 + t] = __float_as_uint(hi * cc[t] + lo * ss[t]);
+                }
+            }
+    }
+#pragma unroll
+    for (int c = 0; c < NC; ++c) {
+        uint32_t u[16];
+#pragma unroll
+        for (int e = 0; e < 16; ++e) u[e] = pack_bf16(__uint_as_float(v[c][2 * e]), __uint_as_float(v[c][2 * e + 1]));
+        store_row32(dst + 32 * c, u, 4);
+    }
+}
+
+template <int V>
 __global__ void __launch_bounds__(kThreads, 1)
-proj_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-            __nv_bfloat16* __restrict__ out, const __nv_bfloat16* __restrict__ O, float* __restrict__ delta,
-            int H, int S, int D, int E, unsigned* status)
+proj_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const ProjArgs a,
+            unsigned* status)
 {
     extern __shared__ uint8_t smem_raw[];
     if (*reinterpret_cast<volatile unsigned*>(status) != 0) return;   // an earlier wait on this device gave up
@@ -47,9 +140,13 @@ proj_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     const uint32_t tmem_slot = bars + B_COUNT * 8;
     auto bar = [&](int i) { return bars + 8u * i; };
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int n0 = static_cast<int>(blockIdx.x) * TN, s0 = static_cast<int>(blockIdx.y) * TM, b = static_cast<int>(blockIdx.z);
-    const int K = DO ? E : H * D, N = DO ? H * D : E;
-    const int n_kt = (K + TK - 1) / TK;
+    // tile: TN output columns from n0; TM rows from r0 (positions s of batch element b, or for DW rows (h,d) of d_w)
+    const int n0 = static_cast<int>(blockIdx.x) * TN, r0 = static_cast<int>(blockIdx.y) * TM, b = static_cast<int>(blockIdx.z);
+    const int HD = a.H * a.D;
+    const int n_sc = (a.S + TK - 1) / TK;                              // DW: 64-position slices per batch element
+    const int N = V == V_DO ? HD : V == V_QKV ? (a.H + 2 * a.Hkv) * a.D : a.E;
+    const int n_kt = V == V_FWD ? HD / TK : V == V_DW ? a.B * n_sc : (a.E + TK - 1) / TK;
+    const int rows = V == V_DW ? HD : a.S;
 
     if (tid == 0) {
         for (int i = 0; i < B_COUNT; ++i) mbar_init(bar(i), 1);
@@ -68,79 +165,69 @@ proj_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             const int st = kt % kStages, k0 = kt * TK;
             if (kt >= kStages) mbar_wait(bar(B_EMPTY + st), ((kt / kStages) - 1) & 1, status);
             mbar_arrive_expect_tx(bar(B_FULL + st), A_BYTES + B_BYTES);
-            if constexpr (DO) {
-                tma_load_3d(sA + st * A_BYTES, &tmA, bar(B_FULL + st), k0, s0, b);
-                tma_load_3d(sB + st * B_BYTES, &tmB, bar(B_FULL + st), k0, n0, 0);          // 256 rows n x 64 k
-            } else {
-                tma_load_3d(sA + st * A_BYTES, &tmA, bar(B_FULL + st), k0 % D, s0, b * H + k0 / D);
+            const uint32_t dA = sA + st * A_BYTES, dB = sB + st * B_BYTES, full = bar(B_FULL + st);
+            if constexpr (V == V_DO || V == V_QKV) {
+                tma_load_3d(dA, &tmA, full, k0, r0, b);                                  // 128 positions x 64 e
+                tma_load_3d(dB, &tmB, full, k0, n0, 0);                                  // 256 rows n x 64 e
+            } else if constexpr (V == V_FWD) {
+                tma_load_3d(dA, &tmA, full, k0 % a.D, r0, b * a.H + k0 / a.D);           // 128 positions x 64 d of one head
 #pragma unroll
-                for (int c = 0; c < TN / 64; ++c)                                             // four blocks of 64 k rows x 64 n
-                    tma_load_3d(sB + st * B_BYTES + c * (TK * 128), &tmB, bar(B_FULL + st), n0 + 64 * c, k0, 0);
+                for (int c = 0; c < TN / 64; ++c)                                         // four blocks of 64 k rows x 64 n
+                    tma_load_3d(dB + c * (TK * 128), &tmB, full, n0 + 64 * c, k0, 0);
+            } else {
+                const int bb = kt / n_sc, s0 = (kt % n_sc) * TK;
+#pragma unroll
+                for (int c = 0; c < TM / 64; ++c) {                                       // two blocks of 64 positions x 64 rows m
+                    const int m = r0 + 64 * c;
+                    tma_load_3d(dA + c * (TK * 128), &tmA, full, m % a.D, s0, bb * a.H + m / a.D);
+                }
+#pragma unroll
+                for (int c = 0; c < TN / 64; ++c)                                         // four blocks of 64 positions x 64 e
+                    tma_load_3d(dB + c * (TK * 128), &tmB, full, n0 + 64 * c, s0, bb);
             }
         }
     } else if (warp == 1 && lane == 0) {
         // ---------------------------------------------------------------- MMA issuer
-        constexpr uint32_t idesc = umma_idesc_bf16(TM, TN, false, !DO);
-        const uint64_t dA = umma_smem_desc(sA, 16, 1024);
-        const uint64_t dB = DO ? umma_smem_desc(sB, 16, 1024) : umma_smem_desc(sB, TK * 128, 1024);
+        constexpr bool A_MN = V == V_DW, B_MN = V == V_FWD || V == V_DW;
+        constexpr uint32_t idesc = umma_idesc_bf16(TM, TN, A_MN, B_MN);
+        const uint64_t dA = A_MN ? umma_smem_desc(sA, TK * 128, 1024) : umma_smem_desc(sA, 16, 1024);
+        const uint64_t dB = B_MN ? umma_smem_desc(sB, TK * 128, 1024) : umma_smem_desc(sB, 16, 1024);
         for (int kt = 0; kt < n_kt; ++kt) {
             const int st = kt % kStages;
             mbar_wait(bar(B_FULL + st), (kt / kStages) & 1, status);
             tc_fence_after();
 #pragma unroll
             for (int kk = 0; kk < TK / 16; ++kk) {
-                const uint64_t a = dA + static_cast<uint64_t>((st * A_BYTES + kk * 32) >> 4);
-                const uint64_t bb = dB + static_cast<uint64_t>((st * B_BYTES + (DO ? kk * 32 : kk * 2048)) >> 4);
-                umma_ss(tmem, a, bb, idesc, (kt > 0 || kk > 0) ? 1u : 0u);
+                const uint64_t da = dA + static_cast<uint64_t>((st * A_BYTES + (A_MN ? kk * 2048 : kk * 32)) >> 4);
+                const uint64_t db = dB + static_cast<uint64_t>((st * B_BYTES + (B_MN ? kk * 2048 : kk * 32)) >> 4);
+                umma_ss(tmem, da, db, idesc, (kt > 0 || kk > 0) ? 1u : 0u);
             }
             umma_commit(bar(B_EMPTY + st));
         }
         umma_commit(bar(B_ACC));
     } else if (warp >= 2) {
         // ---------------------------------------------------------------- epilogue: one thread per row
-        const int q4 = warp & 3, r = 32 * q4 + lane, s = s0 + r;
+        const int q4 = warp & 3, r = 32 * q4 + lane, row = r0 + r;
         const uint32_t tacc = tmem + (static_cast<uint32_t>(32 * q4) << 16);
         mbar_wait(bar(B_ACC), 0, status);
         tc_fence_after();
-        float dl = 0.f;
+        if constexpr (V == V_QKV) {
+            if (a.D == 128) {
 #pragma unroll 1
-        for (int c = 0; c < TN / 32; ++c) {
-            uint32_t v[32];
-            tmem_ld32(tacc + 32 * c, v);          // whole warp, whatever the row
-            tmem_ld_wait();
-            const int n = n0 + 32 * c;
-            if (s >= S || n >= N) continue;
-            uint32_t u[16];
-#pragma unroll
-            for (int e = 0; e < 16; ++e) u[e] = pack_bf16(__uint_as_float(v[2 * e]), __uint_as_float(v[2 * e + 1]));
-            if constexpr (DO) {
-                const int h = n / D, d = n % D;
-                const size_t row = ((static_cast<size_t>(b) * H + h) * S + s) * D + d;
-                const uint4* orow = reinterpret_cast<const uint4*>(O + row);
-                uint4* drow = reinterpret_cast<uint4*>(out + row);
-#pragma unroll
-                for (int p4 = 0; p4 < 4; ++p4) {
-                    drow[p4] = make_uint4(u[4 * p4], u[4 * p4 + 1], u[4 * p4 + 2], u[4 * p4 + 3]);
-                    const uint4 ov = orow[p4];
-                    const uint32_t ow[4] = {ov.x, ov.y, ov.z, ov.w};
-#pragma unroll
-                    for (int t = 0; t < 4; ++t) {
-                        // delta from the bf16 values the attention backward will read
-                        const uint32_t dv = u[4 * p4 + t];
-                        dl = fmaf(__uint_as_float(dv << 16), __uint_as_float(ow[t] << 16), dl);
-                        dl = fmaf(__uint_as_float(dv & 0xffff0000u), __uint_as_float(ow[t] & 0xffff0000u), dl);
-                    }
-                }
-                if (d + 32 == D) {                // last chunk of this head
-                    delta[(static_cast<size_t>(b) * H + h) * S + s] = dl;
-                    dl = 0.f;
-                }
+                for (int hh = 0; hh < TN / 128; ++hh) epilogue_qkv_head<128>(a, tacc + 128 * hh, b, row, n0 / 128 + hh, row < rows);
             } else {
-                uint4* yrow = reinterpret_cast<uint4*>(out + (static_cast<size_t>(b) * S + s) * E + n);
-                const int valid = (E - n) / 8;    // 16-byte pieces inside the row (E is a multiple of 8)
-#pragma unroll
-                for (int p4 = 0; p4 < 4; ++p4)
-                    if (p4 < valid) yrow[p4] = make_uint4(u[4 * p4], u[4 * p4 + 1], u[4 * p4 + 2], u[4 * p4 + 3]);
+#pragma unroll 1
+                for (int hh = 0; hh < TN / 64; ++hh) epilogue_qkv_head<64>(a, tacc + 64 * hh, b, row, n0 / 64 + hh, row < rows);
+            }
+        } else {
+            float dl = 0.f;
+#pragma unroll 1
+            for (int c = 0; c < TN / 32; ++c) {
+                uint32_t v[32];
+                tmem_ld32(tacc + 32 * c, v);          // whole warp, whatever the row
+                tmem_ld_wait();
+                const int n = n0 + 32 * c;
+                if (row < rows && n < N) epilogue_plain<V>(a, v, b, row, n, dl);
             }
         }
     }
@@ -149,17 +236,16 @@ proj_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     if (warp == 0) tmem_dealloc(tmem, TN);
 }
 
-template <bool DO>
-cudaError_t launch(const CUtensorMap& ta, const CUtensorMap& tb, void* out, const void* o, float* delta, int B, int H,
-                   int S, int D, int E, unsigned* status, cudaStream_t st)
+template <int V>
+cudaError_t launch(const CUtensorMap& ta, const CUtensorMap& tb, const ProjArgs& a, unsigned* status, cudaStream_t st)
 {
-    auto kern = proj_kernel<DO>;
+    auto kern = proj_kernel<V>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
     if (e != cudaSuccess) return e;
-    const int N = DO ? H * D : E;
-    const dim3 grid((N + TN - 1) / TN, (S + TM - 1) / TM, B);
-    kern<<<grid, kThreads, SMEM, st>>>(ta, tb, static_cast<__nv_bfloat16*>(out), static_cast<const __nv_bfloat16*>(o),
-                                       delta, H, S, D, E, status);
+    const int N = V == V_DO ? a.H * a.D : V == V_QKV ? (a.H + 2 * a.Hkv) * a.D : a.E;
+    const int rows = V == V_DW ? a.H * a.D : a.S;
+    const dim3 grid((N + TN - 1) / TN, (rows + TM - 1) / TM, V == V_DW ? 1 : a.B);
+    kern<<<grid, kThreads, SMEM, st>>>(ta, tb, a, status);
     return cudaGetLastError();
 }
 
@@ -171,7 +257,8 @@ cudaError_t launch_out_proj_fwd(const void* o, const void* w, void* y, int B, in
     CUtensorMap ta, tb;
     if (make_tmap_3d(&ta, o, 2, 1, B * H, S, D, 64, TM)) return cudaErrorInvalidValue;
     if (make_tmap_3d(&tb, w, 2, 1, 1, H * D, E, 64, TK)) return cudaErrorInvalidValue;
-    return launch<false>(ta, tb, y, nullptr, nullptr, B, H, S, D, E, status, st);
+    ProjArgs a{static_cast<__nv_bfloat16*>(y), nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, B, H, H, S, D, E};
+    return launch<V_FWD>(ta, tb, a, status, st);
 }
 
 cudaError_t launch_out_proj_bwd_data(const void* d_y, const void* w, const void* o, void* d_o, float* delta, int B,
@@ -180,7 +267,30 @@ cudaError_t launch_out_proj_bwd_data(const void* d_y, const void* w, const void*
     CUtensorMap ta, tb;
     if (make_tmap_3d(&ta, d_y, 2, 1, B, S, E, 64, TM)) return cudaErrorInvalidValue;
     if (make_tmap_3d(&tb, w, 2, 1, 1, H * D, E, 64, TN)) return cudaErrorInvalidValue;
-    return launch<true>(ta, tb, d_o, o, delta, B, H, S, D, E, status, st);
+    ProjArgs a{static_cast<__nv_bfloat16*>(d_o), nullptr, nullptr, static_cast<const __nv_bfloat16*>(o), delta, nullptr,
+               nullptr, B, H, H, S, D, E};
+    return launch<V_DO>(ta, tb, a, status, st);
+}
+
+cudaError_t launch_out_proj_bwd_weight(const void* o, const void* d_y, void* d_w, int B, int H, int S, int D, int E,
+                                       unsigned* status, cudaStream_t st)
+{
+    CUtensorMap ta, tb;
+    if (make_tmap_3d(&ta, o, 2, 1, B * H, S, D, 64, TK)) return cudaErrorInvalidValue;
+    if (make_tmap_3d(&tb, d_y, 2, 1, B, S, E, 64, TK)) return cudaErrorInvalidValue;
+    ProjArgs a{static_cast<__nv_bfloat16*>(d_w), nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, B, H, H, S, D, E};
+    return launch<V_DW>(ta, tb, a, status, st);
+}
+
+cudaError_t launch_qkv_rope(const void* x, const void* w, const float* cos_t, const float* sin_t, void* q, void* k,
+                            void* v, int B, int S, int E, int H, int Hkv, int D, unsigned* status, cudaStream_t st)
+{
+    CUtensorMap ta, tb;
+    if (make_tmap_3d(&ta, x, 2, 1, B, S, E, 64, TM)) return cudaErrorInvalidValue;
+    if (make_tmap_3d(&tb, w, 2, 1, 1, (H + 2 * Hkv) * D, E, 64, TN)) return cudaErrorInvalidValue;
+    ProjArgs a{static_cast<__nv_bfloat16*>(q), static_cast<__nv_bfloat16*>(k), static_cast<__nv_bfloat16*>(v), nullptr,
+               nullptr, cos_t, sin_t, B, H, Hkv, S, D, E};
+    return launch<V_QKV>(ta, tb, a, status, st);
 }
 
 }  // namespace mgn

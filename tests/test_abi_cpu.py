@@ -36,7 +36,7 @@ def test_every_declared_symbol_is_exported(lib):
             "mgn_attn_fast_item_order", "mgn_attn_fwd_ext", "mgn_attn_bwd_ext",
             "mgn_attn_bwd_deterministic", "mgn_attn_fwd_accel", "mgn_attn_fwd_accel_workspace_bytes",
             "mgn_attn_strict_tiles", "mgn_selftest_wait_timeout", "mgn_out_proj_fwd", "mgn_out_proj_bwd_data",
-            "mgn_attn_bwd_given_delta"} <= set(syms)
+            "mgn_attn_bwd_given_delta", "mgn_out_proj_bwd_weight", "mgn_qkv_rope_fwd"} <= set(syms)
     for s in syms:
         assert getattr(lib, s) is not None
 

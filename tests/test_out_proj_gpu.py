@@ -118,3 +118,38 @@ def test_projection_then_attention_backward_end_to_end():
     for name, got, ref in (("dQ", dq, dq_r), ("dK", dk, dk_r), ("dV", dv, dv_r)):
         err = hp.rel_l2(got.double().cpu().numpy(), ref)
         assert err <= hp.FAST_REL_L2, f"{name}: {err:.3e}"
+
+
+@pytest.mark.parametrize("B,H,S,D,E", SHAPES)
+def test_weight_gradient_contracts_over_all_positions(B, H, S, D, E):
+    o, w, d_y = _draw(40 + S, B, H, S, D, E)
+    d_w = hp.Guarded((H * D, E), BF)
+    mgn.mgn_out_proj_bwd_weight(o.cuda(), d_y.cuda(), d_w.view, MODE)
+    mgn.mgn_attn_check()
+    got = d_w.check("dW").double().numpy()
+    _, _, ref = orc.out_proj_bwd(d_y.double().numpy(), w.double().numpy(), o.double().numpy())
+    assert hp.rel_l2(got, ref) <= hp.FAST_REL_L2, hp.rel_l2(got, ref)
+
+
+@pytest.mark.parametrize("B,S,E,H,Hkv,D", [
+    (1, 128, 64, 2, 2, 128),       # one tile
+    (2, 197, 200, 3, 1, 64),       # ragged rows, E not a slice multiple, (H + 2 Hkv) D not a tile multiple
+    (1, 300, 512, 5, 5, 128),      # odd head count: a column tile that mixes key and value heads
+    (3, 1, 8, 4, 2, 64),           # a single position
+    (2, 520, 1024, 8, 2, 128),     # grouped key/value heads, several row tiles and contraction slices
+])
+def test_qkv_projection_with_rotary_embedding(B, S, E, H, Hkv, D):
+    g = torch.Generator().manual_seed(50 + S)
+    x = torch.randn(B, S, E, generator=g).to(BF)
+    w = (torch.randn((H + 2 * Hkv) * D, E, generator=g) / math.sqrt(E)).to(BF)
+    inv = 10000.0 ** (-torch.arange(D // 2, dtype=torch.float64) * 2.0 / D)
+    ang = torch.arange(S, dtype=torch.float64)[:, None] * inv[None, :]
+    cos_t, sin_t = torch.cos(ang).float().contiguous(), torch.sin(ang).float().contiguous()
+    q = hp.Guarded((B, H, S, D), BF)
+    k, v = (hp.Guarded((B, Hkv, S, D), BF) for _ in range(2))
+    mgn.mgn_qkv_rope_fwd(x.cuda(), w.cuda(), cos_t.cuda(), sin_t.cuda(), q.view, k.view, v.view, MODE)
+    mgn.mgn_attn_check()
+    rq, rk, rv = orc.qkv_rope(x.double().numpy(), w.double().numpy(), cos_t.double().numpy(), sin_t.double().numpy(), H, Hkv, D)
+    for name, got, ref in (("Q", q, rq), ("K", k, rk), ("V", v, rv)):
+        err = hp.rel_l2(got.check(name).double().numpy(), ref)
+        assert err <= hp.FAST_REL_L2, f"{name}: {err:.3e}"
