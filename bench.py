@@ -276,7 +276,32 @@ def measure_proj_fusion(mgn, steps, warmup):
         mgn.mgn_out_proj_bwd_data(d_y, w, o, d_o, delta, mode)
         mgn.mgn_attn_bwd_given_delta(q, k, v, d_o, lse, delta, dq, dk, dv, ws, wl.causal, wl.scale, mode)
 
+    # weight gradient and the fused QKV projection with rotary embedding (query/key/value heads = H each)
+    d_w = torch.empty_like(w)
+    x = torch.randn(B, S, E, device="cuda", generator=g).to(dt)
+    w_qkv = (torch.randn(3 * H * D, E, device="cuda", generator=g) / E ** 0.5).to(dt)
+    inv = 10000.0 ** (-torch.arange(D // 2, device="cuda", dtype=torch.float32) * 2.0 / D)
+    ang = torch.arange(S, device="cuda", dtype=torch.float32)[:, None] * inv[None, :]
+    cos_t, sin_t = torch.cos(ang).contiguous(), torch.sin(ang).contiguous()
+    q2, k2, v2 = (torch.empty_like(q) for _ in range(3))
+
+    def unfused_dw():
+        torch.matmul(o.transpose(1, 2).reshape(B * S, H * D).t(), d_y.view(B * S, E), out=d_w)
+
+    def unfused_qkv():
+        yq = torch.matmul(x, w_qkv.t()).view(B, S, 3 * H, D).transpose(1, 2)          # [B, 3H, S, D] view
+        c = torch.cat([cos_t, cos_t], dim=1).to(dt)
+        s_ = torch.cat([sin_t, sin_t], dim=1).to(dt)
+        qk = yq[:, :2 * H]
+        rot = torch.cat([-qk[..., D // 2:], qk[..., :D // 2]], dim=-1)
+        qk = qk * c + rot * s_
+        q2.copy_(qk[:, :H]); k2.copy_(qk[:, H:]); v2.copy_(yq[:, 2 * H:])
+
     gemm_flops = 2.0 * B * S * H * D * E
+    w_fused = timed(lambda: mgn.mgn_out_proj_bwd_weight(o, d_y, d_w, mode))
+    w_unf = timed(unfused_dw)
+    qkv_fused = timed(lambda: mgn.mgn_qkv_rope_fwd(x, w_qkv, cos_t, sin_t, q2, k2, v2, mode))
+    qkv_unf = timed(unfused_qkv)
     f_fused = timed(lambda: mgn.mgn_out_proj_fwd(o, w, y, mode))
     f_unf = timed(unfused_fwd)
     p_fused = timed(lambda: mgn.mgn_out_proj_bwd_data(d_y, w, o, d_o, delta, mode))
@@ -286,6 +311,9 @@ def measure_proj_fusion(mgn, steps, warmup):
     return {"shape": {"B": B, "H": H, "S": S, "D": D, "E": E},
             "out_proj_fwd_ms": {"fused": round(f_fused, 4), "library_gemm_plus_layout_copy": round(f_unf, 4)},
             "out_proj_fwd_tflops": round(gemm_flops / (f_fused * 1e-3) / 1e12, 1),
+            "weight_grad_ms": {"fused": round(w_fused, 4), "library_gemm_plus_layout_copy": round(w_unf, 4)},
+            "qkv_rope_ms": {"fused": round(qkv_fused, 4), "library_gemm_plus_eager_rotation_and_copies": round(qkv_unf, 4)},
+            "qkv_rope_tflops": round(3 * gemm_flops / (qkv_fused * 1e-3) / 1e12, 1),
             "do_producer_ms": round(p_fused, 4), "do_producer_tflops": round(gemm_flops / (p_fused * 1e-3) / 1e12, 1),
             "proj_bwd_plus_attn_bwd_ms": {"fused": round(b_fused, 4), "library_gemm_plus_layout_copy_plus_attn_bwd": round(b_unf, 4)}}
 
