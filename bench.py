@@ -33,9 +33,9 @@ METRIC = "attention fwd+bwd TFLOP/s per B200 (strict f32, bf16) and % of matchin
 # ncu summary named beside it (same workload and launch configuration as the bench; re-taken when that
 # kernel changes -- the record carries the file so that a stale figure can be told)
 NCU_TRAFFIC = {
-    ("strict", "gpt2_small"): (146.9e6 + 45.5e6, "profiles/strict_fwd_bwd_gpt2_small.md",
+    ("strict", "gpt2_small"): (140.9e6 + 41.3e6, "profiles/strict_fwd_bwd_gpt2_small.md",
                                "strict_bwd_kernel<64,64,64,128,false,true>"),
-    ("fast", "long_context"): (440.2e6 + 214.6e6, "profiles/fast_fwd_bwd_long_context.md",
+    ("fast", "long_context"): (203.3e6 + 88.7e6, "profiles/fast_fwd_bwd_long_context.md",
                                "fast_bwd_kernel<128,false,true>"),
 }
 SM_COUNT = 148
