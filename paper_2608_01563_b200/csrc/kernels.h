@@ -39,7 +39,7 @@ inline bool prefer_alt_tiles(const Problem& p, int BM, int BN, int BM_alt, int B
     return tiled_work(p, BM_alt, BN_alt) * 8.0 < tiled_work(p, BM, BN) * 7.0;
 }
 inline void strict_fwd_tiles(const Problem& p, int* BM, int* BN) {
-    *BM = p.D == 128 ? 128 : 64;
+    *BM = 64;
     *BN = p.D == 128 ? 64 : 128;
     if (p.D == 64 && prefer_alt_tiles(p, 64, 128, 40, 112)) { *BM = 40; *BN = 112; }
 }

@@ -148,9 +148,11 @@ strict_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             // Unroll factors are set by the instruction cache (instruction fetch is this kernel's top stall,
             // 0.87 stalled warps per issue with the loops of both products unrolled far): measured on the
             // GPT-2-small shape, 8 contraction steps x 32 keys per iteration -> 0.363 ms, 4 x 32 -> 0.326,
-            // 4 x 16 -> 0.328, 1 x 16 -> 0.324; at D = 128, 32 x 32 -> 0.844 ms, 16 x 16 -> 0.828; the 5-row
-            // micro-tile of the 40-row tiles keeps 8 x 32 (0.135 against 0.137-0.139 ms).
-            constexpr int kUnrollQK = (RM == 5) ? 8 : (D == 128) ? 16 : 4;
+            // 4 x 16 -> 0.328, 1 x 16 -> 0.324; the 5-row micro-tile of the 40-row tiles keeps 8 x 32 (0.135 against
+            // 0.137-0.139 ms).  D = 128 (decoder sweep, S = 1024): one 256-thread CTA per SM with 128 x 64 tiles ran
+            // 0.844 ms at 32 x 32 and 0.828 at 16 x 16; two 128-thread CTAs per SM with 64 x 64 tiles run 0.776 at
+            // 16 x 16, 0.754 at 4 x 16 and 0.739 at 8 x 16, which is what D = 128 now uses.
+                        constexpr int kUnrollQK = (RM == 5 || D == 128) ? 8 : 4;
 #pragma unroll kUnrollQK
             for (int pc = 0; pc < D / 4; ++pc) {
                 const uint32_t oq = (pc >> 3) * (BM * 128) + (((pc & 7) ^ xq) << 4);
@@ -235,7 +237,7 @@ strict_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         // row pairs of P come as they are stored; DV * RP packed FMAs follow.
         {
             const uint32_t pa = sP + ((2 * tr) << 4);
-                        constexpr int kUnrollPV = (D == 32) ? 8 : (D == 128) ? 16 : 32;
+                                    constexpr int kUnrollPV = (D == 32) ? 8 : (D == 128) ? 16 : 32;
 #pragma unroll kUnrollPV
             for (int j = 0; j < BN; ++j) {
                 const int u = j & 7;
@@ -350,7 +352,7 @@ cudaError_t launch_strict_fwd(const Problem& p, const float* q, const float* k, 
         case 64:
             if (BM == 40) return launch<64, 40, 112, 128>(p, q, k, v, o, lse, status, st);   // short ragged sequences
             return launch<64, 64, 128, 128>(p, q, k, v, o, lse, status, st);
-        case 128: return launch<128, 128, 64, 256>(p, q, k, v, o, lse, status, st);
+        case 128: return launch<128, 64, 64, 128>(p, q, k, v, o, lse, status, st);
         default:  return cudaErrorInvalidValue;
     }
 }
