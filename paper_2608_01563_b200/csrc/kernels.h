@@ -44,7 +44,7 @@ inline void strict_fwd_tiles(const Problem& p, int* BM, int* BN) {
     if (p.D == 64 && prefer_alt_tiles(p, 64, 128, 40, 112)) { *BM = 40; *BN = 112; }
 }
 inline void strict_bwd_tiles(const Problem& p, int* BM, int* BN) {
-    *BM = 64;
+    *BM = p.D == 128 ? 32 : 64;
     *BN = 64;
     if (p.D == 64 && prefer_alt_tiles(p, 64, 64, 40, 64)) *BM = 40;
 }

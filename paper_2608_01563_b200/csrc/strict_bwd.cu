@@ -32,11 +32,16 @@ struct BwdCfg {
     static constexpr int JN = BN / TR;   // key rows per thread (phase B), groups of 4 contiguous
     static constexpr int DV = D / 16;    // d columns per thread (phases B, C)
     static constexpr int NCH = D / 32;
-    static constexpr int PSTR = BN + 4;
+    static constexpr int PSTR = (D == 128 && THREADS == 128) ? BN : BN + 4;   // no room for the pad beside 128-wide tiles with two CTAs per SM
     static constexpr int KV_BYTES = BN * D * 4;
     static constexpr int Q_BYTES = BM * D * 4;
     static constexpr int P_BYTES = BM * PSTR * 4;
-    static constexpr int SMEM = 2 * KV_BYTES + 2 * Q_BYTES + 2 * P_BYTES + 64 + 1024;
+    static constexpr int PAYLOAD = 2 * KV_BYTES + 2 * Q_BYTES + 2 * P_BYTES + 64;
+    // Two 128-thread CTAs per SM must fit 2 x (SMEM + 1 KB reserved) into 228 KB; where that leaves less than
+    // the 1023 bytes a worst-case alignment of the tile base could need, the kernel checks the slack it got.
+    static constexpr int SLACK = (THREADS == 128 && PAYLOAD + 1024 > 115712) ? 115712 - PAYLOAD : 1024;
+    static constexpr int SMEM = PAYLOAD + SLACK;
+    static_assert(SLACK >= 0, "shared memory budget");
     static_assert(JN % 4 == 0, "key rows per thread come in float4 groups");
 };
 
@@ -68,6 +73,10 @@ strict_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     const uint32_t sP = sdO + C::Q_BYTES;
     const uint32_t sdS = sP + C::P_BYTES;
     const uint32_t barKV = sdS + C::P_BYTES, barQ = barKV + 8;
+    if (base + C::PAYLOAD > smem_u32(smem_raw) + C::SMEM) {      // alignment slack ran out
+        if (threadIdx.x == 0) atomicMax(status, kStatusSmemLayout);
+        return;
+    }
 
     const int tid = threadIdx.x;
     const int tr = 2 * (tid >> 5) + ((tid & 31) >> 4);   // 0..15
@@ -146,9 +155,11 @@ strict_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             // stall of this kernel became instruction fetch (0.94 stalled warps per issue), and a fully
             // unrolled phase A alone is 70 KB of code.  Measured at D = 64 with 64-row tiles: 16 / 8 / 4 / 2 / 1
             // steps per iteration -> 0.808 / 0.760 / 0.731 / 0.724 / 0.723 ms on the GPT-2-small shape; at
-            // D = 128 four steps are best (2.13 against 2.16 ms unrolled, 2.23 with two); the 5-row
-            // micro-tile of the 40-row tiles prefers eight (0.300 against 0.310 ms with two).
-            constexpr int kUnrollA = (RM == 5) ? 8 : (D == 128) ? 4 : 2;
+            // D = 128 (one 256-thread CTA per SM, 64-row tiles) four steps were best (2.13 against 2.16 ms unrolled,
+            // 2.23 with two); the 5-row micro-tile of the 40-row tiles prefers eight (0.300 against 0.310 ms with
+            // two).  D = 128 now runs two 128-thread CTAs per SM with 32-row query tiles (1.94 ms; 1.92 with
+            // eight steps here, one row group in phase B and two key groups in phase C per iteration).
+            constexpr int kUnrollA = (D == 128) ? (GEN ? 4 : 8) : (RM == 5) ? 8 : 2;   // (the general-shape build at D = 128 spills one register with eight)
 #pragma unroll kUnrollA
             for (int pc = 0; pc < D / 4; ++pc) {
                 const uint32_t oq = (pc >> 3) * (BM * 128) + tr * 128 + (((pc & 7) ^ xq) << 4);
@@ -204,7 +215,7 @@ strict_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             // this thread's key rows: j = 4*tr + 64*g + u, g < JN/4, u < 4
             // two groups of eight query rows per iteration (and four groups of keys in phase C) run 1 % faster
             // with the 64-row tiles; the 40-row tiles lose 11 % that way and keep the rolled forms (measured)
-                        constexpr int kUnrollB = (RM == 5) ? 1 : 2;
+                        constexpr int kUnrollB = (RM == 5 || D == 128) ? 1 : 2;
 #pragma unroll kUnrollB
             for (int i8 = 0; i8 < BM; i8 += 8)
 #pragma unroll
@@ -250,7 +261,7 @@ strict_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             for (int x = 0; x < RM; ++x)
 #pragma unroll
                 for (int e = 0; e < DV; ++e) dq[x][e] = 0.f;
-                        constexpr int kUnrollC = (RM == 5 || D <= 64) ? 2 : 4;
+                        constexpr int kUnrollC = 2;
 #pragma unroll kUnrollC
             for (int j8 = 0; j8 < BN / 8; ++j8) {
                 float4 d4[2][RM];
@@ -372,7 +383,7 @@ cudaError_t launch_strict_bwd(const Problem& p, const float* q, const float* k, 
             if (BM == 40)   // short ragged sequences
                 return launch<64, 40, 64, 128>(p, q, k, v, d_o, lse, delta, dq, dk, dv, status, st);
             return launch<64, 64, 64, 128>(p, q, k, v, d_o, lse, delta, dq, dk, dv, status, st);
-        case 128: return launch<128, 64, 64, 256>(p, q, k, v, d_o, lse, delta, dq, dk, dv, status, st);
+        case 128: return launch<128, 32, 64, 128>(p, q, k, v, d_o, lse, delta, dq, dk, dv, status, st);
         default:  return cudaErrorInvalidValue;
     }
 }

@@ -191,7 +191,7 @@ def test_strict_tile_shapes_follow_the_padded_work():
     assert tiles(8, 12, 12, 1024, 1024, 64, True) == (64, 128, 64, 64)     # long sequences keep the defaults
     assert tiles(1, 2, 2, 128, 128, 64, False) == (64, 128, 64, 64)        # an exact fit stays
     assert tiles(1, 2, 2, 256, 256, 64, True) == (64, 128, 64, 64)
-    assert tiles(1, 2, 2, 197, 197, 128, False) == (64, 64, 64, 64)        # other head sizes have one shape
+    assert tiles(1, 2, 2, 197, 197, 128, False) == (64, 64, 32, 64)        # other head sizes have one shape
     assert tiles(1, 2, 2, 64, 64, 32, False) == (64, 128, 64, 64)
     assert tiles(2, 8, 2, 150, 400, 64, True) == (40, 112, 40, 64)         # 150 rows: 160 executed instead of 192
     assert tiles(2, 8, 8, 50, 16, 64, False) == (64, 128, 64, 64)          # one tile either way
