@@ -20,8 +20,9 @@
  *     the legacy default stream) and return without synchronising.  Inputs must
  *     stay valid, and outputs untouched, until the stream has passed the call.
  *   - Outputs need not be initialised.  Outputs must not alias inputs or each other.
- *   - Errors are reported by return code only (mgn_status); nothing is printed and
- *     nothing aborts.  Argument errors are detected before any launch, in the
+ *   - Errors are reported by return code only (mgn_status); nothing aborts, and nothing is
+ *     printed unless the environment variable MGN_LOG is set (then a launch path that
+ *     gives up says on stderr where and with which CUDA error).  Argument errors are detected before any launch, in the
  *     order INVALID_ARG, UNSUPPORTED, MISALIGNED, WORKSPACE, ARCH.
  *   - Device status word.  Every wait inside a kernel is bounded; a wait that runs out
  *     sets one status word PER DEVICE (not per stream, not per call).  While that word is

@@ -265,12 +265,10 @@ int mgn_attn_bwd_given_delta(const void* q, const void* k, const void* v, const 
                              void* stream)
 {
     unsigned* status = nullptr;
-    if (!delta) return MGN_ERR_INVALID_ARG;
-    // `o` is not an argument here: q stands in for it in the shared pointer checks
-    if (int r = check_bwd_call(q, k, v, q, d_o, lse, dq, dk, dv, workspace, workspace_bytes, B, H, H_kv, S_q, S_k, D,
+    // `o` is not an argument here: delta takes its place in the shared null / alignment checks
+    if (int r = check_bwd_call(q, k, v, delta, d_o, lse, dq, dk, dv, workspace, workspace_bytes, B, H, H_kv, S_q, S_k, D,
                                causal, scale, mode, &status))
         return r;
-    if (!aligned16(delta)) return MGN_ERR_MISALIGNED;
     const mgn::Problem p{B, H, H_kv, S_q, S_k, D, causal, scale};
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const size_t rows = static_cast<size_t>(B) * H * S_q;

@@ -484,14 +484,14 @@ cudaError_t launch_gen(const Problem& p, const void* q, const void* k, const voi
 {
     using C = Cfg<D>;
     CUtensorMap tq, tk, tv, to;
-    if (make_tmap_3d(&tq, q, 2, 1, p.BH(), p.Sq, p.D, 64, 128)) return cudaErrorInvalidValue;
-    if (make_tmap_3d(&tk, k, 2, 1, p.BHkv(), p.Sk, p.D, 64, 128)) return cudaErrorInvalidValue;
-    if (make_tmap_3d(&tv, v, 2, 1, p.BHkv(), p.Sk, p.D, 64, 128)) return cudaErrorInvalidValue;
+    if (make_tmap_3d(&tq, q, 2, 1, p.BH(), p.Sq, p.D, 64, 128)) return MGN_FAIL(cudaErrorInvalidValue, "tensor map q");
+    if (make_tmap_3d(&tk, k, 2, 1, p.BHkv(), p.Sk, p.D, 64, 128)) return MGN_FAIL(cudaErrorInvalidValue, "tensor map k");
+    if (make_tmap_3d(&tv, v, 2, 1, p.BHkv(), p.Sk, p.D, 64, 128)) return MGN_FAIL(cudaErrorInvalidValue, "tensor map v");
     // with f32 output the kernel stores O itself; the map then only has to be a valid one
-    if (make_tmap_3d(&to, F16 ? q : o, 2, 1, p.BH(), p.Sq, p.D, 64, 128)) return cudaErrorInvalidValue;
+    if (make_tmap_3d(&to, F16 ? q : o, 2, 1, p.BH(), p.Sq, p.D, 64, 128)) return MGN_FAIL(cudaErrorInvalidValue, "tensor map o");
     auto kern = fast_fwd_kernel<D, GEN, F16>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM);
-    if (e != cudaSuccess) return e;
+    if (e != cudaSuccess) return MGN_FAIL(e, "cudaFuncSetAttribute");
     int dev = 0, sms = 0;
     if (cudaGetDevice(&dev) != cudaSuccess ||
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
@@ -510,7 +510,7 @@ cudaError_t launch_gen(const Problem& p, const void* q, const void* k, const voi
     kern<<<static_cast<unsigned>(blocks), kThreads, C::SMEM, st>>>(tq, tk, tv, to, lse, F16 ? static_cast<float*>(o) : nullptr, dm,
                                                                    n_pairs, tpi, p.causal, order,
                                                                    p.scale * kLog2e, status);
-    return cudaGetLastError();
+    return MGN_FAIL(cudaGetLastError(), "forward launch");
 }
 
 template <int D>

@@ -4,7 +4,17 @@
 #include <cuda_runtime.h>
 #include <stddef.h>
 
+#include <stdio.h>
+#include <stdlib.h>
+
 namespace mgn {
+
+// Diagnostics, off unless the environment variable MGN_LOG is set: where a launch path gave up.
+inline cudaError_t log_fail(cudaError_t e, const char* what, int line) {
+    if (e != cudaSuccess && getenv("MGN_LOG")) fprintf(stderr, "mgn_attn: %s failed at line %d: %s\n", what, line, cudaGetErrorString(e));
+    return e;
+}
+#define MGN_FAIL(e, what) ::mgn::log_fail((e), (what), __LINE__)
 
 // q, o, d_o, dq: [B,H,Sq,D]; k, v, dk, dv: [B,Hkv,Sk,D]; query head h reads key/value head
 // h / (H/Hkv).  With a causal mask key j is visible to query i iff j <= i + (Sk - Sq)

@@ -69,10 +69,19 @@ int make_tmap_3d(CUtensorMap* out, const void* base, int elem_bytes, int is_bf16
                                    static_cast<cuuint64_t>(S) * D * elem_bytes};
     const cuuint32_t box[3] = {static_cast<cuuint32_t>(box_d), static_cast<cuuint32_t>(box_rows), 1u};
     const cuuint32_t estr[3] = {1u, 1u, 1u};
-    const CUresult r = enc(out, is_bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3,
-                           const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                           CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    auto encode = [&] {
+        return enc(out, is_bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3,
+                   const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                   CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    };
+    CUresult r = encode();
+    if (r != CUDA_SUCCESS) {
+        // The encoder is a driver call and wants a current context: a host thread whose first CUDA work is
+        // this library call has none bound yet (the runtime binds it lazily, and nothing before this point
+        // needs it).  Bind it -- cudaFree(nullptr) allocates and frees nothing -- and try once more.
+        cudaFree(nullptr);
+        r = encode();
+    }
     if (r != CUDA_SUCCESS) return 2;
     {
         std::lock_guard<std::mutex> lock(g_cache_mu);

@@ -214,3 +214,67 @@ def test_strict_tile_shapes_follow_the_padded_work():
         tiles(1, 2, 2, 16, 8, 64, True)
     with pytest.raises(binding.MgnError):
         tiles(1, 2, 2, 8, 8, 48, False)
+
+
+def test_projection_entry_points_validate_before_any_launch(lib):
+    """mgn_out_proj_*, mgn_qkv_rope_fwd and mgn_attn_bwd_given_delta name argument errors in the documented
+    order (INVALID_ARG, UNSUPPORTED, MISALIGNED, WORKSPACE) without touching a device."""
+    import ctypes
+    vp, i, f, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_float, ctypes.c_size_t
+    INVALID, UNSUPPORTED, MISALIGNED, WORKSPACE = 1, 2, 3, 4
+    lib.mgn_out_proj_fwd.argtypes = [vp, vp, vp, i, i, i, i, i, i, vp]
+    lib.mgn_out_proj_bwd_data.argtypes = [vp] * 5 + [i] * 6 + [vp]
+    lib.mgn_out_proj_bwd_weight.argtypes = [vp, vp, vp, i, i, i, i, i, i, vp]
+    lib.mgn_qkv_rope_fwd.argtypes = [vp] * 7 + [i] * 7 + [vp]
+    lib.mgn_attn_bwd_given_delta.argtypes = [vp] * 9 + [vp, sz] + [i] * 7 + [f, i, vp]
+
+    def pf(o=A, w=A, y=A, B=1, H=2, S=8, D=64, E=64, mode=1):
+        return lib.mgn_out_proj_fwd(o, w, y, B, H, S, D, E, mode, None)
+
+    assert pf(o=None) == INVALID and pf(y=None) == INVALID
+    assert pf(S=0) == INVALID and pf(E=-8) == INVALID and pf(mode=3) == INVALID
+    assert pf(mode=0) == UNSUPPORTED                       # strict-mode projections are not built
+    assert pf(D=32) == UNSUPPORTED and pf(D=48) == UNSUPPORTED
+    assert pf(E=60) == UNSUPPORTED                         # rows of E elements must be whole 16-byte pieces
+    assert pf(w=A + 2) == MISALIGNED
+    assert pf(w=A + 2, E=60) == UNSUPPORTED and pf(w=A + 2, E=60, H=0) == INVALID
+
+    def pd(ptrs=None, delta=A, D=64, E=64, mode=1):
+        p = [A] * 4 if ptrs is None else ptrs
+        return lib.mgn_out_proj_bwd_data(*p, delta, 1, 2, 8, D, E, mode, None)
+
+    for idx in range(4):
+        p = [A] * 4
+        p[idx] = None
+        assert pd(ptrs=p) == INVALID
+    assert pd(delta=None) == INVALID and pd(delta=A + 4) == MISALIGNED and pd(D=100) == UNSUPPORTED
+
+    assert lib.mgn_out_proj_bwd_weight(A, A, None, 1, 2, 8, 64, 64, 1, None) == INVALID
+    assert lib.mgn_out_proj_bwd_weight(A, A, A, 1, 2, 8, 64, 12, 1, None) == UNSUPPORTED
+
+    def qk(ptrs=None, Hkv=1, D=128, E=64, mode=1):
+        p = [A] * 7 if ptrs is None else ptrs
+        return lib.mgn_qkv_rope_fwd(*p, 1, 8, E, 2, Hkv, D, mode, None)
+
+    for idx in range(7):
+        p = [A] * 7
+        p[idx] = None
+        assert qk(ptrs=p) == INVALID
+    assert qk(Hkv=0) == INVALID and qk(D=32) == UNSUPPORTED and qk(mode=0) == UNSUPPORTED
+    p = [A] * 7
+    p[3] = A + 8                                            # the sine table
+    assert qk(ptrs=p) == MISALIGNED
+
+    def gd(ptrs=None, ws=A, ws_bytes=1 << 30, Sq=8, Sk=16, D=64, causal=0, mode=0, H=4, Hkv=2):
+        p = [A] * 9 if ptrs is None else ptrs
+        return lib.mgn_attn_bwd_given_delta(*p, ws, ws_bytes, 1, H, Hkv, Sq, Sk, D, causal, 1.0, mode, None)
+
+    for idx in range(9):                                    # q, k, v, d_o, lse, delta, dq, dk, dv
+        p = [A] * 9
+        p[idx] = None
+        assert gd(ptrs=p) == INVALID
+    assert gd(Hkv=3) == INVALID and gd(Sq=32, Sk=16, causal=1) == UNSUPPORTED and gd(D=48) == UNSUPPORTED
+    p = [A] * 9
+    p[5] = A + 4                                            # delta
+    assert gd(ptrs=p) == MISALIGNED
+    assert gd(ws=None) == WORKSPACE and gd(ws_bytes=8) == WORKSPACE

@@ -55,3 +55,61 @@ def test_fast_and_strict_agree_with_each_other():
 def test_check_reports_ok_after_clean_runs():
     mgn.mgn_attn_check()
     assert mgn.mgn_status_string(0) == "MGN_OK"
+
+
+@pytest.mark.parametrize("mode,dtype", [(mgn.MODE_STRICT_F32, torch.float32), (mgn.MODE_FAST_BF16, torch.bfloat16)])
+def test_two_host_threads_on_two_streams(mode, dtype):
+    """The header allows distinct host threads on distinct streams (the tensor-map cache and the
+    per-device set-up are shared state behind a mutex; every call has its own workspace).  Two threads
+    run different problems twenty times each; every result must equal what the same call gives alone."""
+    import threading
+    shapes = [(2, 4, 300, 64, True), (1, 6, 200, 128, False)]
+    work = []
+    for n, (B, H, S, D, causal) in enumerate(shapes):
+        q, k, v, d_o = (t.cuda() for t in synth.random_inputs(60 + n, B, H, S, D, dtype=dtype))
+        work.append(dict(q=q, k=k, v=v, d_o=d_o, causal=causal, scale=D ** -0.5, S=S,
+                         ws=mgn.alloc_workspace(B, H, S, D, mode), stream=torch.cuda.Stream()))
+
+    def run(w, outs):
+        B, H, S, D = w["q"].shape
+        o = torch.empty_like(w["q"]); lse = torch.empty(B, H, S, device="cuda")
+        dq, dk, dv = (torch.empty_like(w["q"]) for _ in range(3))
+        st = w["stream"].cuda_stream
+        mgn.mgn_attn_fwd(w["q"], w["k"], w["v"], o, lse, w["causal"], w["scale"], mode, stream=st)
+        mgn.mgn_attn_bwd(w["q"], w["k"], w["v"], o, w["d_o"], lse, dq, dk, dv, w["ws"], w["causal"], w["scale"], mode, stream=st)
+        outs.append((o, lse, dq, dk, dv))
+
+    torch.cuda.synchronize()
+    alone = []
+    for w in work:
+        outs = []
+        run(w, outs)
+        w["stream"].synchronize()
+        alone.append(outs[0])
+
+    results = [[], []]
+    errors = []
+
+    def loop(idx):
+        try:
+            for _ in range(20):
+                run(work[idx], results[idx])
+            work[idx]["stream"].synchronize()
+        except Exception as exc:                     # surfaces in the main thread below
+            errors.append(exc)
+
+    threads = [threading.Thread(target=loop, args=(idx,)) for idx in range(2)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    assert not errors, errors
+    mgn.mgn_attn_check()
+    for idx in range(2):
+        ref = alone[idx]
+        for got in results[idx]:
+            for name, g, r in zip(("O", "LSE", "dQ", "dK", "dV"), got, ref):
+                if name == "dQ":                     # accumulated with floating-point reductions: order varies
+                    assert hp.rel_l2(g.double().cpu().numpy(), r.double().cpu().numpy()) <= (1e-6 if mode == mgn.MODE_STRICT_F32 else 2e-2)
+                else:
+                    assert torch.equal(g, r), (name, idx, float((g.float() - r.float()).abs().max()), int((g != r).sum()))
