@@ -13,7 +13,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "build")
 LIB = os.path.join(HERE, "libmgn_attn.so")
-SOURCES = ["api.cu", "tmap.cu", "bwd_pre.cu", "strict_fwd.cu", "strict_bwd.cu", "strict_dq.cu", "fast_fwd.cu", "fast_bwd.cu", "fast_dq.cu", "noalloc.cu", "peaks.cu", "selftest.cu", "proj.cu"]
+SOURCES = ["api.cu", "tmap.cu", "bwd_pre.cu", "strict_fwd.cu", "strict_bwd.cu", "strict_dq.cu", "fast_fwd.cu", "fast_fwd_small.cu", "fast_bwd.cu", "fast_dq.cu", "noalloc.cu", "peaks.cu", "selftest.cu", "proj.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",
     "-Xcompiler", "-fPIC", "-Xptxas", "-v",

@@ -555,6 +555,7 @@ cudaError_t launch_fast_fwd_f16(const Problem& p, const void* q16, const void* k
 cudaError_t launch_fast_fwd(const Problem& p, const void* q, const void* k, const void* v, void* o, float* lse,
                             unsigned* status, cudaStream_t st)
 {
+    if (fast_fwd_is_small(p)) return launch_fast_fwd_small(p, q, k, v, o, lse, status, st);
     switch (p.D) {
         // Head size 32 runs the 64-wide build: the tensor maps describe 32-element rows and a
         // 64-element box, so columns 32-63 of every operand tile are zero-filled on load (they add

@@ -141,6 +141,11 @@ inline int pick_schedule(long long n_items, int sms, double shared_bytes, int de
 // Fast (bf16 tcgen05) kernels.
 cudaError_t launch_fast_fwd(const Problem& p, const void* q, const void* k, const void* v,
                             void* o, float* lse, unsigned* status, cudaStream_t st);
+// The latency path of the forward: at most two 128-key blocks per head (Sk <= 256), one small CTA per
+// 128-row query tile, several per SM.  launch_fast_fwd hands such problems to it.
+inline bool fast_fwd_is_small(const Problem& p) { return p.Sk <= 256; }
+cudaError_t launch_fast_fwd_small(const Problem& p, const void* q, const void* k, const void* v, void* o, float* lse,
+                                  unsigned* status, cudaStream_t st);
 // Forward of the accelerated policy: q16, k16, v16 are IEEE f16 copies (launch_to_f16) of f32
 // tensors, tensor-core products with f32 accumulation, O and LSE stored as f32.
 cudaError_t launch_to_f16(const float* in, void* out, size_t n, cudaStream_t st);
