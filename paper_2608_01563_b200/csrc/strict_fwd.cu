@@ -16,6 +16,8 @@
 #include "kernels.h"
 #include "ptx.cuh"
 
+#include <type_traits>
+
 namespace mgn {
 namespace {
 
@@ -39,6 +41,9 @@ struct FwdCfg {
     // warp) are conflict free.
     static constexpr int RP = (RM + 1) / 2;   // row pairs per thread
     static constexpr int PROW = TR * 32;      // bytes per key column
+    // Half-tile form of the two products (first BN/2 keys only): needs the half to be whole column groups
+    // and a whole number of the P V loop's unrolled key groups (32 keys at most).
+    static constexpr bool HALF_OK = (BN % 64 == 0);
     static constexpr int Q_BYTES = BM * D * 4;
     static constexpr int KV_BYTES = BN * D * 4;
     static constexpr int P_BYTES = BN * PROW;
@@ -140,9 +145,16 @@ strict_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
 #pragma unroll
             for (int y = 0; y < RN; ++y) s[x][y] = 0.f;
 
+        // Keys of this tile that some row of the query tile can see.  When they fill at most the first half of
+        // the tile (the last tile of every other query tile under a causal mask with BN = 2 BM; a ragged
+        // tail), both products run over that half only; the scores of the other half stay 0 and are masked.
+        const int k_vis = min(Sk, causal ? i_last + off + 1 : Sk) - j0;
+        const bool half_tile = C::HALF_OK && k_vis <= BN / 2;
+
         mbar_wait(barK, ph, status);
         // ---- S = Q K^T : contraction along d, float4 pieces --------------------------------
-        {
+        auto qk = [&](auto yn_tag) {
+            constexpr int YN = decltype(yn_tag)::value;
             const uint32_t qa = sQ + tr * 128, ka = sK + tc * 128;
             const int xq = tr & 7, xk = tc & 7;
             // Unroll factors are set by the instruction cache (instruction fetch is this kernel's top stall,
@@ -152,19 +164,19 @@ strict_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             // 0.137-0.139 ms).  D = 128 (decoder sweep, S = 1024): one 256-thread CTA per SM with 128 x 64 tiles ran
             // 0.844 ms at 32 x 32 and 0.828 at 16 x 16; two 128-thread CTAs per SM with 64 x 64 tiles run 0.776 at
             // 16 x 16, 0.754 at 4 x 16 and 0.739 at 8 x 16, which is what D = 128 now uses.
-                        constexpr int kUnrollQK = (RM == 5 || D == 128) ? 8 : 4;
+            constexpr int kUnrollQK = (RM == 5 || D == 128) ? 8 : 4;
 #pragma unroll kUnrollQK
             for (int pc = 0; pc < D / 4; ++pc) {
                 const uint32_t oq = (pc >> 3) * (BM * 128) + (((pc & 7) ^ xq) << 4);
                 const uint32_t ok = (pc >> 3) * (BN * 128) + (((pc & 7) ^ xk) << 4);
-                float4 b[RN];
+                float4 b[YN];
 #pragma unroll
-                for (int y = 0; y < RN; ++y) b[y] = lds128(ka + ok + y * 16 * 128);
+                for (int y = 0; y < YN; ++y) b[y] = lds128(ka + ok + y * 16 * 128);
 #pragma unroll
                 for (int x = 0; x < RM; ++x) {
                     const float4 a = lds128(qa + oq + x * TR * 128);
 #pragma unroll
-                    for (int y = 0; y < RN; ++y) {
+                    for (int y = 0; y < YN; ++y) {
                         s[x][y] = fmaf(a.x, b[y].x, s[x][y]);
                         s[x][y] = fmaf(a.y, b[y].y, s[x][y]);
                         s[x][y] = fmaf(a.z, b[y].z, s[x][y]);
@@ -172,6 +184,12 @@ strict_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                     }
                 }
             }
+        };
+        if constexpr (C::HALF_OK) {
+            if (half_tile) qk(std::integral_constant<int, RN / 2>{});
+            else qk(std::integral_constant<int, RN>{});
+        } else {
+            qk(std::integral_constant<int, RN>{});
         }
         __syncthreads();   // every warp is done with this K tile (and with P of the previous tile)
         if (tid == 0 && kt + 1 < n_kt) {
@@ -237,9 +255,9 @@ strict_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         // row pairs of P come as they are stored; DV * RP packed FMAs follow.
         {
             const uint32_t pa = sP + ((2 * tr) << 4);
-                                    constexpr int kUnrollPV = (D == 32) ? 8 : (D == 128) ? 16 : 32;
-#pragma unroll kUnrollPV
-            for (int j = 0; j < BN; ++j) {
+            constexpr int kUnrollPV = (D == 32) ? 8 : (D == 128) ? 16 : 32;
+            static_assert(!C::HALF_OK || (BN / 2) % kUnrollPV == 0, "half a tile is whole unrolled groups");
+            auto pv_key = [&](int j) {
                 const int u = j & 7;
                 float vv[DV];
                 if constexpr (DV == 2) {
@@ -269,6 +287,15 @@ strict_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 for (int q = 0; q < RP; ++q)
 #pragma unroll
                     for (int e = 0; e < DV; ++e) o[q][e] = f2_fma(pp[q], vd[e], o[q][e]);
+            };
+            if constexpr (C::HALF_OK) {          // run-time key count, a whole number of unrolled groups
+                const int jn = half_tile ? BN / 2 : BN;
+                for (int jb = 0; jb < jn; jb += kUnrollPV)
+#pragma unroll
+                    for (int jj = 0; jj < kUnrollPV; ++jj) pv_key(jb + jj);
+            } else {
+#pragma unroll kUnrollPV
+                for (int j = 0; j < BN; ++j) pv_key(j);
             }
         }
         __syncthreads();   // every warp is done with this V tile and with P

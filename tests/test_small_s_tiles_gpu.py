@@ -51,3 +51,29 @@ def test_square_entry_point_uses_them_too():
     got = hp.select(hp.run_cuda(q, k, v, d_o, True, w.scale, mgn.MODE_STRICT_F32), 2, 3)
     ref = hp.run_oracle(q, k, v, d_o, True, w.scale)
     hp.check_strict(got, ref, literal_max_abs=False, label="small-S tiles square causal ")
+
+
+# Shapes whose last key tile holds visible keys in its first half only: the forward then runs both
+# products of that tile over half of it.  Each keeps the default tiles (checked), so the path taken
+# is the half-tile one of the 64 x 128 (D <= 64) and 64 x 64 (D = 128) builds.
+HALF_TILE_CASES = [
+    # B, H, Hkv, Sq, Sk, D, causal
+    (1, 3, 3, 1024, 1024, 64, True),     # every other query tile ends on a half-visible key tile
+    (2, 4, 2, 700, 1070, 64, False),     # ragged tail: 46 keys in the ninth key tile
+    (1, 4, 4, 600, 650, 64, True),       # bottom-right offset 50: half tiles from the offset and the tail
+    (2, 2, 2, 640, 640, 32, True),       # head size 32 (eight-key unrolled groups)
+    (1, 4, 1, 600, 592, 128, False),     # D = 128: 16 keys in the tenth 64-key tile
+    (1, 2, 2, 540, 550, 128, True),      # D = 128, offset 10
+]
+
+
+@pytest.mark.parametrize("B,H,Hkv,Sq,Sk,D,causal", HALF_TILE_CASES)
+def test_half_visible_key_tiles_match_the_oracle(B, H, Hkv, Sq, Sk, D, causal):
+    fbm, fbn, _, _ = mgn.mgn_attn_strict_tiles(B, H, Hkv, Sq, Sk, D, causal)
+    assert (fbm, fbn) == ((64, 64) if D == 128 else (64, 128))
+    scale = 1.0 / math.sqrt(D)
+    q, k, v, d_o = _inputs(950, B, H, Hkv, Sq, Sk, D)
+    got = hp.run_cuda_ext(q, k, v, d_o, causal, scale, mgn.MODE_STRICT_F32, run_bwd=False)
+    ref = hp.run_oracle_ext(q, k, v, d_o, causal, scale)
+    hp.check_strict(got, ref, names=("O", "LSE"), literal_max_abs=False,
+                    label=f"half key tiles {B,H,Hkv,Sq,Sk,D,causal} ")
