@@ -2,30 +2,26 @@
 // accumulation in tensor memory, f32 softmax statistics (paper Section 3.3 "tiled attention
 // forward"; Section 4.2: the validated reduced-input path with f32 accumulation).
 //
-// Persistent kernel: one CTA per SM walks over work items (two 128-row query tiles of one head
-// each -- one tile when there would be fewer items than SMs; two item orders, see make_item) and, per item, over 128-key blocks of that head's
-// key/value head.  All barriers keep counting across items, so the producer prefetches the next
-// item's Q/K/V and the issuers compute its first scores while the softmax warps are still writing
-// the previous item's output: most of the per-item fill and drain is hidden instead of paid by
-// every CTA.
-// Warp roles (384 threads):
-//   warp 0      TMA producer: Q tiles once, then K and V blocks through a 2-stage ring
-//   warps 1, 2  MMA issuers, one per query tile: S_t = Q_t K^T (operands in shared memory) and
-//               O_t += P_t V (P_t read from tensor memory, V as an MN-major shared-memory
-//               operand).  One lane each; with two issuers the tensor core keeps working on one
-//               tile while the other issuer sits in a barrier wait (a wait costs a few hundred
-//               clocks even when it succeeds at once, and the issue queue is shallow)
-//   warps 4-11  softmax: all 256 threads work on ONE query tile at a time, two threads per row
-//               (64 key columns each), alternating between the two tiles.  A lone warp per
-//               scheduler cannot keep the exp2 unit busy; two can, so a tile's softmax takes half
-//               as long and the tensor core's S/PV products of the other tile hide it.
-// Tensor memory (512 columns): S_0 [0,128), S_1 [128,256), O_0 [256,256+D), O_1 [256+D,256+2D).
-// P_t (bf16) overwrites S_t: keys 0-63 at S_t[0,32), keys 64-127 at S_t[64,96) (each half in the
-// columns its own threads have already read).  The softmax reference point of a row only moves
-// (and O is rescaled in tensor memory) when a row outgrows it so far that a thread's partial sum of
-// exponentials passes a limit (2^60; 2^12 with f16 probabilities), which is exact: any reference point works for a softmax as long as
-// nothing overflows.  The two threads of a row agree on that through a barrier with an
-// OR-reduction per block.
+// Persistent kernel: one CTA per SM walks over work items (one 128-row query tile of one head; two
+// item orders, see make_item) and, per item, over 128-key blocks of that head's key/value head.
+// The score tile is double-buffered in tensor memory and P has columns of its own, so the product
+// S(n+2) = Q K(n+2)^T is issued as soon as the softmax warps have READ S(n): the scores of the next
+// block are always waiting when a softmax pass ends, and neither product sits on the path between
+// two passes.  All barriers and the block counter keep counting across items, so the first scores of
+// the next item are computed, and its Q tile loaded, while the current item finishes, and the
+// output of an item is written by a warpgroup of its own while the softmax warps start the next one.
+// Warp roles (512 threads):
+//   warps 0, 2    TMA producers: the Q tile of each item (two stages) and the K blocks; the V blocks (2-stage rings)
+//   warps 1, 3    MMA issuers (one lane each): S(g) = Q K(g)^T (operands in shared memory), up to two blocks
+//                 ahead; O += P(g) V(g) (P read from tensor memory, V as an MN-major shared-memory operand)
+//   warps 4-11    softmax: two threads per row (64 key columns each), one block after the other
+//   warps 12-15   epilogue: O / l -> bf16 -> shared memory -> TMA store (f32 build: plain stores), LSE
+// Tensor memory (512 columns): S(even blocks) [0,128), S(odd) [128,256), P(even) [256,320),
+// P(odd) [320,384), O [384,384+D).  The softmax reference point of a row only moves (and O is rescaled
+// in tensor memory) when a row outgrows it so far that a thread's partial sum of exponentials passes
+// a limit (2^60; 2^12 with f16 probabilities), which is exact: any reference point works for a
+// softmax as long as nothing overflows.  The two threads of a row agree on that through a barrier
+// with an OR-reduction per block.
 #include "kernels.h"
 #include "fast_items.cuh"
 #include "umma.cuh"
@@ -33,10 +29,9 @@
 namespace mgn {
 namespace {
 
-constexpr int kThreads = 384;
+constexpr int kThreads = 512;
 constexpr int BM = 128;      // rows per query tile
 constexpr int BN = 128;      // keys per block
-constexpr int kStages = 2;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 // A thread's partial row sum (64 columns) above this limit moves the reference points.  Every p stays
@@ -53,52 +48,55 @@ struct Cfg {
     static constexpr int NCH = D / 64;                 // 128-byte chunks per row
     static constexpr int TILE_BYTES = 128 * D * 2;     // a 128-row tile of Q, K or V
     static constexpr int CHUNK_BYTES = 128 * 128;      // one 64-column chunk of a 128-row tile
-    static constexpr int OFF_Q = 0;
-    static constexpr int OFF_K = OFF_Q + 2 * TILE_BYTES;
-    static constexpr int OFF_V = OFF_K + kStages * TILE_BYTES;
-    static constexpr int OFF_OST = OFF_V + kStages * TILE_BYTES;    // output staging, one tile
-    static constexpr int OFF_XCHG = OFF_OST + TILE_BYTES;           // [2 halves][128 rows] f32 exchange
-    static constexpr int OFF_BAR = OFF_XCHG + 2 * 128 * 4;
+    static constexpr int OFF_Q = 0;                                 // two stages (item parity)
+    static constexpr int OFF_K = OFF_Q + 2 * TILE_BYTES;            // two stages (block parity)
+    static constexpr int OFF_V = OFF_K + 2 * TILE_BYTES;
+    static constexpr int OFF_OST = OFF_V + 2 * TILE_BYTES;          // output staging, one tile
+    static constexpr int OFF_XCHG = OFF_OST + TILE_BYTES;           // [2 halves][128 rows] f32 exchange; at item end: l of each half
+    static constexpr int OFF_MREF = OFF_XCHG + 2 * 128 * 4;         // [128 rows] f32: reference point of each row at item end
+    static constexpr int OFF_BAR = OFF_MREF + 128 * 4;
     static constexpr int SMEM = OFF_BAR + 256 + 1024;
     static_assert(SMEM <= 232448, "shared memory budget");
-    static constexpr uint32_t TM_S = 0, TM_O = 256, TM_COLS = 512;
+    static constexpr uint32_t TM_S = 0, TM_P = 256, TM_O = 384, TM_COLS = 512;
 };
 
-// barrier slots (8 bytes each)
-enum { B_Q = 0, B_KFULL = 1, B_KEMPTY = 3, B_VFULL = 5, B_VEMPTY = 7, B_SFULL = 9, B_PFULL = 11, B_OFULL = 13,
-       B_QEMPTY = 15, B_OEMPTY = 16, B_COUNT = 18 };
+// barrier slots (8 bytes each); pairs are indexed by the parity of the item (Q) or of the block
+//   S_GO[b]   (2 arrivals + bytes)   K(g) has landed AND the product P(g-2) V(g-2) has completed: S(g) may be
+//                                    issued -- P(g-2) stored implies S(g-2) read, so the score buffer is free, and
+//                                    by the time S(g) is visible its P buffer is free too
+//   PV_GO[b]  (257 arrivals + bytes) V(g) has landed AND all 256 softmax threads have stored P(g)
+// Every mbarrier operation of an issuing lane costs it 250-350 clocks while the tensor core streams
+// operands from shared memory, hence one wait per product.
+enum { B_QFULL = 0, B_QEMPTY = 2, B_KEMPTY = 4, B_VEMPTY = 6, B_SFULL = 8, B_SGO = 10, B_PVGO = 12, B_PVDONE = 14,
+       B_OFULL = 16, B_OEMPTY = 17, B_STFULL = 18, B_STEMPTY = 19, B_COUNT = 20 };
 
-// Work item `it`: query-tile pair and head.  Order 0 (block-major): heaviest tiles of every head
+// Work item `it`: query tile and head.  Order 0 (block-major): heaviest tiles of every head
 // first, dealt in snake order -- balanced for any item count, but the CTAs running at one time touch
-// every head.  Order 1 (head-major): the tile pairs of a head are consecutive, heaviest and lightest
+// every head.  Order 1 (head-major): the tiles of a head are consecutive, heaviest and lightest
 // remaining in turn, and CTA c takes the item pairs c, c+G, ... -- the CTAs running at one time
 // share the K, V of a few heads, which then stay in L2.  The launcher chooses (pick_schedule).
 struct Item {
-    int pair, bh, bhk, row0[2], nblk[2], n_max;
+    int bh, bhk, row0, nblk;
 };
 // GEN = false is the square multi-head case (Sk == Sq, G == 1): offsets and the head mapping fold away.
 template <bool GEN>
-__device__ __forceinline__ Item make_item(int it, const Dims& dm, int n_pairs, int tpi, int causal, int order) {
+__device__ __forceinline__ Item make_item(int it, const Dims& dm, int n_tiles, int causal, int order) {
     const int BH = dm.BH;
     const int Sk = GEN ? dm.Sk : dm.Sq, off = GEN ? dm.off : 0;
     Item w;
+    int tile;
     if (order == 0) {                          // block-major, heaviest (last) query tiles first
-        w.pair = n_pairs - 1 - it / BH;
+        tile = n_tiles - 1 - it / BH;
         w.bh = it % BH;
-    } else {                                   // head-major, heaviest / lightest remaining tile pair in turn
-        w.bh = it / n_pairs;
-        const int j = it % n_pairs;
-        w.pair = (j & 1) ? (j >> 1) : n_pairs - 1 - (j >> 1);
+    } else {                                   // head-major, heaviest / lightest remaining tile in turn
+        w.bh = it / n_tiles;
+        const int j = it % n_tiles;
+        tile = (j & 1) ? (j >> 1) : n_tiles - 1 - (j >> 1);
     }
     w.bhk = GEN ? (w.bh / dm.H) * (dm.H / dm.G) + (w.bh % dm.H) / dm.G : w.bh;
     const int n_kb = (Sk + BN - 1) / BN;
-#pragma unroll
-    for (int t = 0; t < 2; ++t) {
-        w.row0[t] = (w.pair * tpi + t) * BM;          // tpi = tiles per item: 2, or 1 when items would be too few
-        if (t >= tpi || w.row0[t] >= dm.Sq) w.nblk[t] = 0;
-        else w.nblk[t] = causal ? min(n_kb, (min(w.row0[t] + BM, dm.Sq) - 1 + off) / BN + 1) : n_kb;
-    }
-    w.n_max = max(w.nblk[0], w.nblk[1]);
+    w.row0 = tile * BM;
+    w.nblk = causal ? min(n_kb, (min(w.row0 + BM, dm.Sq) - 1 + off) / BN + 1) : n_kb;
     return w;
 }
 
@@ -109,7 +107,7 @@ template <int D, bool GEN, bool F16>
 __global__ void __launch_bounds__(kThreads, 1)
 fast_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                 const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO,
-                float* __restrict__ LSE, float* __restrict__ O32, const Dims dm, int n_pairs, int tpi, int causal, int order,
+                float* __restrict__ LSE, float* __restrict__ O32, const Dims dm, int n_tiles, int causal, int order,
                 float c2, unsigned* status)
 {
     using C = Cfg<D>;
@@ -123,7 +121,7 @@ fast_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (*reinterpret_cast<volatile unsigned*>(status) != 0) return;   // an earlier wait on this device gave up
 
-    const int n_items = n_pairs * dm.BH;
+    const int n_items = n_tiles * dm.BH;
     const int Sq = dm.Sq, Sk = GEN ? dm.Sk : dm.Sq, coff = GEN ? dm.off : 0;
     const int G = static_cast<int>(gridDim.x), cta = static_cast<int>(blockIdx.x);
     const int n_tiers = 2 * ((n_items + 2 * G - 1) / (2 * G));   // upper bound on items per CTA in either order
@@ -131,8 +129,10 @@ fast_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     if (tid == 0) {
         for (int i = 0; i < B_COUNT; ++i) {
             uint32_t cnt = 1;
-            if (i == B_PFULL || i == B_PFULL + 1 || i == B_OEMPTY || i == B_OEMPTY + 1) cnt = 256;
-            if ((i >= B_KEMPTY && i < B_KEMPTY + 2) || (i >= B_VEMPTY && i < B_VEMPTY + 2) || i == B_QEMPTY) cnt = 2;
+            if (i == B_STFULL) cnt = 256;
+            if (i == B_PVGO || i == B_PVGO + 1) cnt = 257;
+            if (i == B_SGO || i == B_SGO + 1) cnt = 2;
+            if (i == B_OEMPTY || i == B_STEMPTY) cnt = 128;
             mbar_init(bar(i), cnt);
         }
         fence_mbar_init();
@@ -145,7 +145,7 @@ fast_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     const uint32_t tmem = lds32u(tmem_slot);
 
     if (warp < 4) {
-        reg_dealloc<96>();
+        reg_dealloc<72>();
         if (warp == 0 && lane == 0) {
         // ------------------------------------------------------------------ TMA producer
         {
@@ -153,112 +153,192 @@ fast_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             for (int k = 0; k < n_tiers; ++k) {
                 const int it = item_index(cta, k, G, n_items, order);
                 if (it < 0) break;
-                const Item w = make_item<GEN>(it, dm, n_pairs, tpi, causal, order);
-                mbar_wait(bar(B_QEMPTY), (k & 1) ^ 1, status);   // both issuers are done with the previous Q tiles
-                const int nq = (w.nblk[1] > 0) ? 2 : 1;
-                mbar_arrive_expect_tx(bar(B_Q), nq * C::TILE_BYTES);
-                for (int t = 0; t < nq; ++t)
+                const Item w = make_item<GEN>(it, dm, n_tiles, causal, order);
+                const int qs = k & 1;
+                mbar_wait(bar(B_QEMPTY + qs), ((k >> 1) & 1) ^ 1, status);   // the last S product of item k - 2 is done
+                mbar_arrive_expect_tx(bar(B_QFULL + qs), C::TILE_BYTES);
 #pragma unroll
-                    for (int ch = 0; ch < C::NCH; ++ch)
-                        tma_load_3d(sQ + t * C::TILE_BYTES + ch * C::CHUNK_BYTES, &tmQ, bar(B_Q), ch * 64, w.row0[t], w.bh);
-                for (int n = 0; n < w.n_max; ++n, ++g) {
+                for (int ch = 0; ch < C::NCH; ++ch)
+                    tma_load_3d(sQ + qs * C::TILE_BYTES + ch * C::CHUNK_BYTES, &tmQ, bar(B_QFULL + qs), ch * 64, w.row0, w.bh);
+                for (int n = 0; n < w.nblk; ++n, ++g) {
                     const int st = g & 1;
                     const uint32_t ph = (g >> 1) & 1;
                     mbar_wait(bar(B_KEMPTY + st), ph ^ 1, status);
-                    mbar_arrive_expect_tx(bar(B_KFULL + st), C::TILE_BYTES);
+                    mbar_arrive_expect_tx(bar(B_SGO + st), C::TILE_BYTES);
 #pragma unroll
                     for (int ch = 0; ch < C::NCH; ++ch)
-                        tma_load_3d(sK + st * C::TILE_BYTES + ch * C::CHUNK_BYTES, &tmK, bar(B_KFULL + st), ch * 64, n * BN, w.bhk);
-                    mbar_wait(bar(B_VEMPTY + st), ph ^ 1, status);
-                    mbar_arrive_expect_tx(bar(B_VFULL + st), C::TILE_BYTES);
-#pragma unroll
-                    for (int ch = 0; ch < C::NCH; ++ch)
-                        tma_load_3d(sV + st * C::TILE_BYTES + ch * C::CHUNK_BYTES, &tmV, bar(B_VFULL + st), ch * 64, n * BN, w.bhk);
+                        tma_load_3d(sK + st * C::TILE_BYTES + ch * C::CHUNK_BYTES, &tmK, bar(B_SGO + st), ch * 64, n * BN, w.bhk);
                 }
             }
         }
-        } else if ((warp == 1 || warp == 2) && lane == 0) {
-        // ------------------------------------------------------------------ MMA issuer of tile t
+        } else if (warp == 2 && lane == 0) {
+        // ------------------------------------------------------------------ TMA producer of V
+        // A thread of its own: K(g+2) is wanted half a block before P(g) exists, V(g+2) only once the
+        // product with V(g) has completed; one thread loading both in turn would hold K back.
         {
-            const int t = warp - 1;
+            int g = 0;
+            for (int k = 0; k < n_tiers; ++k) {
+                const int it = item_index(cta, k, G, n_items, order);
+                if (it < 0) break;
+                const Item w = make_item<GEN>(it, dm, n_tiles, causal, order);
+                for (int n = 0; n < w.nblk; ++n, ++g) {
+                    const int st = g & 1;
+                    mbar_wait(bar(B_VEMPTY + st), ((g >> 1) & 1) ^ 1, status);
+                    mbar_arrive_expect_tx(bar(B_PVGO + st), C::TILE_BYTES);
+#pragma unroll
+                    for (int ch = 0; ch < C::NCH; ++ch)
+                        tma_load_3d(sV + st * C::TILE_BYTES + ch * C::CHUNK_BYTES, &tmV, bar(B_PVGO + st), ch * 64, n * BN, w.bhk);
+                }
+            }
+        }
+        } else if ((warp == 1 || warp == 3) && lane == 0) {
+        // ------------------------------------------------------------------ MMA issuers
+        // Two lanes, each walking over this CTA's blocks (all items in sequence): warp 1 issues the score
+        // products, which run up to two blocks ahead of the softmax warps, warp 3 the P V products.
+        // Block g uses score buffer, P buffer and K/V stage g & 1.  While one lane sits in a wait the
+        // other keeps the tensor core fed.
+        {
             constexpr uint32_t idesc_s = F16 ? umma_idesc_f16(BM, BN, false, false) : umma_idesc_bf16(BM, BN, false, false);
             constexpr uint32_t idesc_o = F16 ? umma_idesc_f16(BM, D, false, true) : umma_idesc_bf16(BM, D, false, true);
             // Descriptors are built once; inside the loops only the start-address field moves (the
             // field holds address >> 4 and cannot carry out of its 14 bits within shared memory).
-            const uint64_t qd = umma_smem_desc(sQ + t * C::TILE_BYTES, 16, 1024);
-            const uint64_t dK0 = umma_smem_desc(sK, 16, 1024);
-            const uint64_t dV0 = umma_smem_desc(sV, C::CHUNK_BYTES, 1024);
-            const uint32_t tSd = tmem + C::TM_S + t * 128, tOd = tmem + C::TM_O + t * D;
-            auto issue_s = [&](int st) {   // S_t = Q_t K(stage st)^T
-                const uint64_t kd = dK0 + static_cast<uint64_t>((st * C::TILE_BYTES) >> 4);
-#pragma unroll
-                for (int kk = 0; kk < D / 16; ++kk) {
-                    const uint64_t off = static_cast<uint64_t>(((kk >> 2) * C::CHUNK_BYTES + (kk & 3) * 32) >> 4);
-                    umma_ss(tSd, qd + off, kd + off, idesc_s, kk > 0);
-                }
-                umma_commit(bar(B_SFULL + t));
-            };
-            auto issue_o = [&](int st, uint32_t acc0) {   // O_t (+)= P_t V(stage st)
-                const uint64_t vd = dV0 + static_cast<uint64_t>((st * C::TILE_BYTES) >> 4);
-#pragma unroll
-                for (int kk = 0; kk < BN / 16; ++kk)
-                    umma_ts(tOd, tSd + (kk >> 2) * 64 + (kk & 3) * 8, vd + static_cast<uint64_t>((kk * 2048) >> 4), idesc_o,
-                            kk > 0 ? 1u : acc0);
-            };
-            int g = 0;       // key blocks seen so far (all items): stage and phase of the K/V ring
-            int cp = 0;      // P_t blocks consumed so far: phase of P_FULL[t]
-            int co = 0;      // items in which this tile was active: phase of O_EMPTY[t]
-            for (int k = 0; k < n_tiers; ++k) {
-                const int it = item_index(cta, k, G, n_items, order);
-                if (it < 0) break;
-                const Item w = make_item<GEN>(it, dm, n_pairs, tpi, causal, order);
-                const int nb = w.nblk[t];
-                mbar_wait(bar(B_Q), k & 1, status);
-                mbar_wait(bar(B_KFULL + (g & 1)), (g >> 1) & 1, status);
-                tc_fence_after();
-                if (nb > 0) issue_s(g & 1);
-                umma_commit(bar(B_KEMPTY + (g & 1)));
-                if (nb <= 1) umma_commit(bar(B_QEMPTY));          // no further S products of this item from this issuer
-                if (nb > 0) mbar_wait(bar(B_OEMPTY + t), (co & 1) ^ 1, status);   // the last item's O_t has been read out
-                for (int n = 0; n < w.n_max; ++n, ++g) {
-                    const int st = g & 1;
-                    // Every issuer waits for every block, also the ones its tile does not use: an
-                    // issuer that ran ahead could release a ring slot twice in one phase.
-                    mbar_wait(bar(B_VFULL + st), (g >> 1) & 1, status);
-                    if (n < nb) {
-                        mbar_wait(bar(B_PFULL + t), cp & 1, status);
-                        ++cp;
+            int g = 0;
+            if (warp == 1) {
+                const uint64_t dQ0 = umma_smem_desc(sQ, 16, 1024);
+                const uint64_t dK0 = umma_smem_desc(sK, 16, 1024);
+                mbar_arrive(bar(B_SGO));         // blocks 0 and 1 have no product before them to wait for
+                mbar_arrive(bar(B_SGO + 1));
+                for (int k = 0; k < n_tiers; ++k) {
+                    const int it = item_index(cta, k, G, n_items, order);
+                    if (it < 0) break;
+                    const int nblk = make_item<GEN>(it, dm, n_tiles, causal, order).nblk;
+                    const int qs = k & 1;
+                    const uint64_t qd = dQ0 + static_cast<uint64_t>((qs * C::TILE_BYTES) >> 4);
+                    mbar_wait(bar(B_QFULL + qs), (k >> 1) & 1, status);
+                    for (int n = 0; n < nblk; ++n, ++g) {
+                        const int b = g & 1;
+                        mbar_wait(bar(B_SGO + b), (g >> 1) & 1, status);
                         tc_fence_after();
-                        issue_o(st, n > 0);
-                        if (n == nb - 1) umma_commit(bar(B_OFULL + t));
-                    }
-                    umma_commit(bar(B_VEMPTY + st));          // this issuer is done with V(n)
-                    if (n + 1 < w.n_max) {
-                        mbar_wait(bar(B_KFULL + (st ^ 1)), ((g + 1) >> 1) & 1, status);
-                        if (n + 1 < nb) {
-                            tc_fence_after();
-                            issue_s(st ^ 1);
-                            if (n + 2 == nb) umma_commit(bar(B_QEMPTY));   // that was this item's last S product
+                        const uint64_t kd = dK0 + static_cast<uint64_t>((b * C::TILE_BYTES) >> 4);
+                        const uint32_t tS = tmem + C::TM_S + b * 128;
+#pragma unroll
+                        for (int kk = 0; kk < D / 16; ++kk) {
+                            const uint64_t off = static_cast<uint64_t>(((kk >> 2) * C::CHUNK_BYTES + (kk & 3) * 32) >> 4);
+                            umma_ss(tS, qd + off, kd + off, idesc_s, kk > 0);
                         }
-                        umma_commit(bar(B_KEMPTY + (st ^ 1)));   // ... and with K(n+1)
+                        umma_commit(bar(B_SFULL + b));
+                        umma_commit(bar(B_KEMPTY + b));
                     }
+                    umma_commit(bar(B_QEMPTY + qs));      // that was this item's last S product
                 }
-                if (nb > 0) ++co;
+            } else {
+                const uint64_t dV0 = umma_smem_desc(sV, C::CHUNK_BYTES, 1024);
+                const uint32_t tO = tmem + C::TM_O;
+                for (int k = 0; k < n_tiers; ++k) {
+                    const int it = item_index(cta, k, G, n_items, order);
+                    if (it < 0) break;
+                    const int nblk = make_item<GEN>(it, dm, n_tiles, causal, order).nblk;
+                    mbar_wait(bar(B_OEMPTY), (k & 1) ^ 1, status);   // the last item's O has been read out
+                    for (int n = 0; n < nblk; ++n, ++g) {
+                        const int b = g & 1;
+                        mbar_wait(bar(B_PVGO + b), (g >> 1) & 1, status);
+                        tc_fence_after();
+                        const uint64_t vd = dV0 + static_cast<uint64_t>((b * C::TILE_BYTES) >> 4);
+                        const uint32_t tP = tmem + C::TM_P + b * 64;
+#pragma unroll
+                        for (int kk = 0; kk < BN / 16; ++kk)
+                            umma_ts(tO, tP + kk * 8, vd + static_cast<uint64_t>((kk * 2048) >> 4), idesc_o, (kk > 0 || n > 0) ? 1u : 0u);
+                        umma_commit(bar(B_SGO + b));          // with K(g+2): S(g+2) may go
+                        umma_commit(bar(B_VEMPTY + b));
+                        umma_commit(bar(B_PVDONE + b));
+                    }
+                    umma_commit(bar(B_OFULL));
+                }
             }
         }
         }
         __syncwarp();
+    } else if (warp >= 12) {
+        // ------------------------------------------------------------------ epilogue warpgroup
+        // Per item: O / l -> bf16 -> shared (swizzled like the TMA box) -> TMA store; LSE.  The row sums
+        // and reference points come from the softmax warps through shared memory.
+        reg_dealloc<88>();
+        const int r = tid - 384;                           // row within the tile = tensor-memory lane
+        const uint32_t tOr = tmem + (static_cast<uint32_t>(r & ~31) << 16) + C::TM_O;
+        const uint32_t xchg = base + C::OFF_XCHG, mref = base + C::OFF_MREF;
+        const uint32_t ost = base + C::OFF_OST;
+        for (int k = 0; k < n_tiers; ++k) {
+            const int it = item_index(cta, k, G, n_items, order);
+            if (it < 0) break;
+            const Item w = make_item<GEN>(it, dm, n_tiles, causal, order);
+            const int i = w.row0 + r;
+            mbar_wait(bar(B_STFULL), k & 1, status);
+            const float lt = lds32f(xchg + r * 4) + lds32f(xchg + (128 + r) * 4);
+            const float mr = lds32f(mref + r * 4);
+            mbar_arrive(bar(B_STEMPTY));                      // the softmax warps may use the exchange buffer again
+            const float inv = 1.0f / lt;
+            if (i < Sq) LSE[static_cast<size_t>(w.bh) * Sq + i] = (mr + log2f(lt)) * kLn2;
+            if (!F16) {
+                if (r == 0) bulk_wait_group_read0();          // the previous store has finished reading the staging tile
+                named_bar_sync(5, 128);
+            }
+            mbar_wait(bar(B_OFULL), k & 1, status);
+            tc_fence_after();
+#pragma unroll
+            for (int c = 0; c < D / 32; ++c) {
+                uint32_t v[32];
+                tmem_ld32(tOr + 32 * c, v);
+                tmem_ld_wait();
+                if (c == D / 32 - 1) {
+                    tc_fence_before();
+                    mbar_arrive(bar(B_OEMPTY));                // the next item may overwrite O
+                }
+                if constexpr (F16) {
+                    // f32 output: 32 contiguous columns of row i, 16-byte stores
+                    if (i < Sq) {
+                        float* orow = O32 + (static_cast<size_t>(w.bh) * Sq + i) * D + 32 * c;
+#pragma unroll
+                        for (int e = 0; e < 8; ++e)
+                            *reinterpret_cast<float4*>(orow + 4 * e) =
+                                make_float4(__uint_as_float(v[4 * e]) * inv, __uint_as_float(v[4 * e + 1]) * inv,
+                                            __uint_as_float(v[4 * e + 2]) * inv, __uint_as_float(v[4 * e + 3]) * inv);
+                    }
+                } else {
+                    uint32_t u[16];
+#pragma unroll
+                    for (int e = 0; e < 16; ++e)
+                        u[e] = pack_bf16(__uint_as_float(v[2 * e]) * inv, __uint_as_float(v[2 * e + 1]) * inv);
+                    const int col = 32 * c;                        // first output column of this chunk
+                    const uint32_t rowaddr = ost + (col >> 6) * C::CHUNK_BYTES + r * 128;
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const int piece = ((col & 63) >> 3) + q;
+                        sts128(rowaddr + ((piece ^ (r & 7)) << 4), u[4 * q], u[4 * q + 1], u[4 * q + 2], u[4 * q + 3]);
+                    }
+                }
+            }
+            if (!F16) {
+                fence_proxy_async_smem();
+                named_bar_sync(5, 128);
+                if (r == 0) {
+#pragma unroll
+                    for (int ch = 0; ch < C::NCH; ++ch)
+                        tma_store_3d(&tmO, ost + ch * C::CHUNK_BYTES, ch * 64, w.row0, w.bh);
+                    bulk_commit_group();
+                }
+            }
+        }
+        if (!F16 && r == 0) bulk_wait_group_read0();
     } else {
-        // ------------------------------------------------------------------ softmax + epilogue
-        reg_alloc<200>();
+        // ------------------------------------------------------------------ softmax warps
+        reg_alloc<176>();
         const int h = (warp - 4) >> 2;                     // which 64 key columns of every block
         const int r = (tid - 128) & 127;                   // row within the tile = tensor-memory lane
         const uint32_t lane_base = static_cast<uint32_t>(r & ~31) << 16;
         const uint32_t xchg = base + C::OFF_XCHG;
         const uint32_t my_x = xchg + (h * 128 + r) * 4, peer_x = xchg + ((h ^ 1) * 128 + r) * 4;
-        const uint32_t ost = base + C::OFF_OST;
-        int cs[2] = {0, 0};      // S_t blocks consumed so far (all items): phase of S_FULL[t]
-        int co[2] = {0, 0};      // items in which tile t was active: phase of O_FULL[t]
+        const uint32_t tO = tmem + lane_base + C::TM_O + (D / 2) * h;
+        int g = 0;               // blocks seen so far (all items): buffer and phase of S, P
 
         // barrier over the 256 softmax threads with an OR reduction of `pred`
         auto bar_or = [](bool pred) -> bool {
@@ -273,116 +353,119 @@ fast_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         for (int k = 0; k < n_tiers; ++k) {
         const int it = item_index(cta, k, G, n_items, order);
         if (it < 0) break;
-        const Item w = make_item<GEN>(it, dm, n_pairs, tpi, causal, order);
-        const int bh = w.bh, n_max = w.n_max;
-        const int row0[2] = {w.row0[0], w.row0[1]}, nblk[2] = {w.nblk[0], w.nblk[1]};
-        float m_ref[2] = {-INFINITY, -INFINITY}, l[2] = {0.f, 0.f};
+        const Item w = make_item<GEN>(it, dm, n_tiles, causal, order);
+        const int i = w.row0 + r;
+        float m_ref = -INFINITY, l = 0.f;
+        // the exchange buffer carried the row sums of the last item to the epilogue warps
+        if (k > 0) mbar_wait(bar(B_STEMPTY), (k - 1) & 1, status);
 
-        for (int n = 0; n < n_max; ++n) {
-#pragma unroll
-            for (int t = 0; t < 2; ++t) {
-                if (n >= nblk[t]) continue;
-                const uint32_t tS = tmem + lane_base + C::TM_S + t * 128 + 64 * h;   // this thread's 64 score columns
-                const uint32_t tO = tmem + lane_base + C::TM_O + t * D + (D / 2) * h;
-                const int i = row0[t] + r;
-                mbar_wait(bar(B_SFULL + t), (cs[t] + n) & 1, status);
-                tc_fence_after();
-                const int j0 = n * BN + 64 * h;
-                const bool masked = (causal && (j0 + 63 > row0[t] + coff)) || (j0 + 64 > Sk);
-                const int jmax = min(Sk - 1, causal ? i + coff : Sk - 1) - j0;   // columns c <= jmax of this half are visible
+        for (int n = 0; n < w.nblk; ++n, ++g) {
+            const int b = g & 1;
+            const uint32_t ph = (g >> 1) & 1;
+            const uint32_t tS = tmem + lane_base + C::TM_S + b * 128 + 64 * h;   // this thread's 64 score columns
+            const uint32_t tP = tmem + lane_base + C::TM_P + b * 64 + 32 * h;    // ... and where their probabilities go
+            mbar_wait(bar(B_SFULL + b), ph, status);
+            tc_fence_after();
+            const int j0 = n * BN + 64 * h;
+            const bool masked = (causal && (j0 + 63 > w.row0 + coff)) || (j0 + 64 > Sk);
+            const int jmax = min(Sk - 1, causal ? i + coff : Sk - 1) - j0;   // columns c <= jmax of this half are visible
 
-                if (n == 0) {
-                    // first block: the reference point is the row maximum of the scaled scores
-                    float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+            if (n == 0) {
+                // first block: the reference point is the row maximum of the scaled scores
+                float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
 #pragma unroll
-                    for (int c = 0; c < 2; ++c) {
-                        uint32_t v[32];
-                        tmem_ld32(tS + 32 * c, v);
-                        tmem_ld_wait();
-                        float x[32];
+                for (int c = 0; c < 2; ++c) {
+                    uint32_t v[32];
+                    tmem_ld32(tS + 32 * c, v);
+                    tmem_ld_wait();
+                    float x[32];
 #pragma unroll
-                        for (int e = 0; e < 32; ++e) x[e] = __uint_as_float(v[e]) * c2;
-                        if (masked) {
-#pragma unroll
-                            for (int e = 0; e < 32; ++e)
-                                if (32 * c + e > jmax) x[e] = -INFINITY;
-                        }
-#pragma unroll
-                        for (int e = 0; e < 32; e += 4) {
-                            mx0 = fmaxf(mx0, x[e]);
-                            mx1 = fmaxf(mx1, x[e + 1]);
-                            mx2 = fmaxf(mx2, x[e + 2]);
-                            mx3 = fmaxf(mx3, x[e + 3]);
-                        }
-                    }
-                    const float mine = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
-                    sts32(my_x, mine);
-                    bar_or(false);
-                    m_ref[t] = fmaxf(mine, lds32f(peer_x));      // finite: key 0 is visible to every row
-                    bar_or(false);                                // exchange buffer may be reused
-                }
-
-                // One pass: y = s*c2 - m_ref, p = exp2(y), partial row sum, bf16 pack (kept in
-                // registers); two columns per fma / add instruction.  A row that outgrew its reference
-                // point shows in its partial sum (every p <= the sum): if any partial sum passes the
-                // limit, the rows find their current maxima in a second look at S (still intact: P is
-                // written over it only afterwards), move their reference points, rescale O and l, and
-                // the pass is redone.  The common case pays no per-element maximum.
-                uint32_t pk[32];
-                float lsum = 0.f;
-                for (int attempt = 0; attempt < 2; ++attempt) {
-                    uint64_t la = f2_pack(0.f, 0.f), lb = la;
-                    const float neg_m = -m_ref[t];
-                    const uint64_t c2x2 = f2_pack(c2, c2), nm2 = f2_pack(neg_m, neg_m);
-#pragma unroll
-                    for (int c = 0; c < 2; ++c) {
-                        uint32_t v[32];
-                        tmem_ld32(tS + 32 * c, v);
-                        tmem_ld_wait();
-                        float y[32];
-#pragma unroll
-                        for (int e = 0; e < 32; e += 2)
-                            f2_unpack(f2_fma(f2_pack(__uint_as_float(v[e]), __uint_as_float(v[e + 1])), c2x2, nm2), y[e], y[e + 1]);
-                        if (masked) {
-#pragma unroll
-                            for (int e = 0; e < 32; ++e)
-                                if (32 * c + e > jmax) y[e] = -INFINITY;
-                        }
-#pragma unroll
-                        for (int e = 0; e < 32; e += 4) {
-                            const float p0 = ex2(y[e]), p1 = ex2(y[e + 1]), p2 = ex2(y[e + 2]), p3 = ex2(y[e + 3]);
-                            la = f2_add(la, f2_pack(p0, p1));
-                            lb = f2_add(lb, f2_pack(p2, p3));
-                            pk[16 * c + e / 2] = F16 ? pack_f16(p0, p1) : pack_bf16(p0, p1);
-                            pk[16 * c + e / 2 + 1] = F16 ? pack_f16(p2, p3) : pack_bf16(p2, p3);
-                        }
-                    }
-                    {
-                        float a0, a1, a2, a3;
-                        f2_unpack(la, a0, a1);
-                        f2_unpack(lb, a2, a3);
-                        lsum = (a0 + a1) + (a2 + a3);
-                    }
-                    if (attempt == 1) break;
-                    if (!bar_or(!(lsum <= (F16 ? kGrowthLimitF16 : kGrowthLimitBf16)))) break;      // also true for an overflowed (inf / nan) sum
-                    // some row grew: every row moves its reference point to its current maximum
-                    float ymax = -INFINITY;
-#pragma unroll
-                    for (int c = 0; c < 2; ++c) {
-                        uint32_t v[32];
-                        tmem_ld32(tS + 32 * c, v);
-                        tmem_ld_wait();
+                    for (int e = 0; e < 32; ++e) x[e] = __uint_as_float(v[e]) * c2;
+                    if (masked) {
 #pragma unroll
                         for (int e = 0; e < 32; ++e)
-                            if (!masked || 32 * c + e <= jmax) ymax = fmaxf(ymax, fmaf(__uint_as_float(v[e]), c2, neg_m));
+                            if (32 * c + e > jmax) x[e] = -INFINITY;
                     }
-                    sts32(my_x, ymax);
-                    bar_or(false);
-                    const float ym = fmaxf(ymax, lds32f(peer_x));
-                    const float m_new = fmaxf(m_ref[t], m_ref[t] + ym);
-                    const float alpha = ex2(m_ref[t] - m_new);
-                    m_ref[t] = m_new;
-                    l[t] *= alpha;
+#pragma unroll
+                    for (int e = 0; e < 32; e += 4) {
+                        mx0 = fmaxf(mx0, x[e]);
+                        mx1 = fmaxf(mx1, x[e + 1]);
+                        mx2 = fmaxf(mx2, x[e + 2]);
+                        mx3 = fmaxf(mx3, x[e + 3]);
+                    }
+                }
+                const float mine = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
+                sts32(my_x, mine);
+                bar_or(false);
+                m_ref = fmaxf(mine, lds32f(peer_x));      // finite: key 0 is visible to every row
+                bar_or(false);                                // exchange buffer may be reused
+            }
+
+            // One pass: y = s*c2 - m_ref, p = exp2(y), partial row sum, bf16 pack (kept in
+            // registers); two columns per fma / add instruction.  A row that outgrew its reference
+            // point shows in its partial sum (every p <= the sum): if any partial sum passes the
+            // limit, the rows find their current maxima in a second look at S (still intact), move their
+            // reference points, rescale O and l, and the pass is redone.  The common case pays no
+            // per-element maximum.
+            uint32_t pk[32];
+            float lsum = 0.f;
+            for (int attempt = 0; attempt < 2; ++attempt) {
+                uint64_t la = f2_pack(0.f, 0.f), lb = la;
+                const float neg_m = -m_ref;
+                const uint64_t c2x2 = f2_pack(c2, c2), nm2 = f2_pack(neg_m, neg_m);
+#pragma unroll
+                for (int c = 0; c < 2; ++c) {
+                    uint32_t v[32];
+                    tmem_ld32(tS + 32 * c, v);
+                    tmem_ld_wait();
+                    float y[32];
+#pragma unroll
+                    for (int e = 0; e < 32; e += 2)
+                        f2_unpack(f2_fma(f2_pack(__uint_as_float(v[e]), __uint_as_float(v[e + 1])), c2x2, nm2), y[e], y[e + 1]);
+                    if (masked) {
+#pragma unroll
+                        for (int e = 0; e < 32; ++e)
+                            if (32 * c + e > jmax) y[e] = -INFINITY;
+                    }
+#pragma unroll
+                    for (int e = 0; e < 32; e += 4) {
+                        const float p0 = ex2(y[e]), p1 = ex2(y[e + 1]), p2 = ex2(y[e + 2]), p3 = ex2(y[e + 3]);
+                        la = f2_add(la, f2_pack(p0, p1));
+                        lb = f2_add(lb, f2_pack(p2, p3));
+                        pk[16 * c + e / 2] = F16 ? pack_f16(p0, p1) : pack_bf16(p0, p1);
+                        pk[16 * c + e / 2 + 1] = F16 ? pack_f16(p2, p3) : pack_bf16(p2, p3);
+                    }
+                }
+                {
+                    float a0, a1, a2, a3;
+                    f2_unpack(la, a0, a1);
+                    f2_unpack(lb, a2, a3);
+                    lsum = (a0 + a1) + (a2 + a3);
+                }
+                if (attempt == 1) break;
+                if (!bar_or(!(lsum <= (F16 ? kGrowthLimitF16 : kGrowthLimitBf16)))) break;      // also true for an overflowed (inf / nan) sum
+                // some row grew: every row moves its reference point to its current maximum
+                float ymax = -INFINITY;
+#pragma unroll
+                for (int c = 0; c < 2; ++c) {
+                    uint32_t v[32];
+                    tmem_ld32(tS + 32 * c, v);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int e = 0; e < 32; ++e)
+                        if (!masked || 32 * c + e <= jmax) ymax = fmaxf(ymax, fmaf(__uint_as_float(v[e]), c2, neg_m));
+                }
+                sts32(my_x, ymax);
+                bar_or(false);
+                const float ym = fmaxf(ymax, lds32f(peer_x));
+                const float m_new = fmaxf(m_ref, m_ref + ym);
+                const float alpha = ex2(m_ref - m_new);
+                m_ref = m_new;
+                l *= alpha;
+                if (n > 0) {
+                    // O holds the blocks up to n - 1 once the product P(g-1) V(g-1) has completed
+                    mbar_wait(bar(B_PVDONE + (b ^ 1)), ((g - 1) >> 1) & 1, status);
+                    tc_fence_after();
 #pragma unroll 1
                     for (int c = 0; c < D / 64; ++c) {
                         uint32_t v[32];
@@ -392,85 +475,28 @@ fast_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                         for (int e = 0; e < 32; ++e) v[e] = __float_as_uint(__uint_as_float(v[e]) * alpha);
                         tmem_st32(tO + 32 * c, v);
                     }
-                    bar_or(false);                                // everyone has read the exchange buffer
                 }
-                l[t] += lsum;
-#pragma unroll
-                for (int c = 0; c < 2; ++c) {
-                    uint32_t u[16];
-#pragma unroll
-                    for (int e = 0; e < 16; ++e) u[e] = pk[16 * c + e];
-                    tmem_st16(tS + 16 * c, u);
-                }
-                tmem_st_wait();
-                tc_fence_before();
-                mbar_arrive(bar(B_PFULL + t));
+                bar_or(false);                                // everyone has read the exchange buffer
             }
+            l += lsum;
+            // P buffer g & 1 is free: S(g) was issued after the product P(g-2) V(g-2) had completed
+#pragma unroll
+            for (int c = 0; c < 2; ++c) {
+                uint32_t u[16];
+#pragma unroll
+                for (int e = 0; e < 16; ++e) u[e] = pk[16 * c + e];
+                tmem_st16(tP + 16 * c, u);
+            }
+            tmem_st_wait();
+            tc_fence_before();
+            mbar_arrive(bar(B_PVGO + b));
         }
 
-        // ---- epilogue per tile: O / l -> bf16 -> shared (swizzled like the TMA box) -> TMA store; LSE
-#pragma unroll
-        for (int t = 0; t < 2; ++t) {
-            if (nblk[t] == 0) continue;
-            const uint32_t tO = tmem + lane_base + C::TM_O + t * D + (D / 2) * h;
-            const int i = row0[t] + r;
-            sts32(my_x, l[t]);
-            if (!F16 && r == 0 && h == 0) bulk_wait_group_read0();   // the previous store has finished reading the staging tile
-            bar_or(false);
-            const float lt = l[t] + lds32f(peer_x);
-            mbar_wait(bar(B_OFULL + t), co[t] & 1, status);
-            tc_fence_after();
-            const float inv = 1.0f / lt;
-            uint32_t v[D / 64][32];
-#pragma unroll
-            for (int c = 0; c < D / 64; ++c) tmem_ld32(tO + 32 * c, v[c]);
-            tmem_ld_wait();
-            tc_fence_before();
-            mbar_arrive(bar(B_OEMPTY + t));                    // the next item may overwrite O_t
-            if (h == 0 && i < Sq) LSE[static_cast<size_t>(bh) * Sq + i] = (m_ref[t] + log2f(lt)) * kLn2;
-            if constexpr (F16) {
-                // f32 output: this thread's D/2 contiguous columns of row i, 16-byte stores
-                if (i < Sq) {
-                    float* orow = O32 + (static_cast<size_t>(bh) * Sq + i) * D + (D / 2) * h;
-#pragma unroll
-                    for (int c = 0; c < D / 64; ++c)
-#pragma unroll
-                        for (int e = 0; e < 8; ++e)
-                            *reinterpret_cast<float4*>(orow + 32 * c + 4 * e) =
-                                make_float4(__uint_as_float(v[c][4 * e]) * inv, __uint_as_float(v[c][4 * e + 1]) * inv,
-                                            __uint_as_float(v[c][4 * e + 2]) * inv, __uint_as_float(v[c][4 * e + 3]) * inv);
-                }
-                bar_or(false);                                 // exchange buffer may be reused
-            } else {
-#pragma unroll
-                for (int c = 0; c < D / 64; ++c) {
-                    uint32_t u[16];
-#pragma unroll
-                    for (int e = 0; e < 16; ++e)
-                        u[e] = pack_bf16(__uint_as_float(v[c][2 * e]) * inv, __uint_as_float(v[c][2 * e + 1]) * inv);
-                    const int col = (D / 2) * h + 32 * c;          // first output column of this chunk
-                    const uint32_t rowaddr = ost + (col >> 6) * C::CHUNK_BYTES + r * 128;
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        const int piece = ((col & 63) >> 3) + q;
-                        sts128(rowaddr + ((piece ^ (r & 7)) << 4), u[4 * q], u[4 * q + 1], u[4 * q + 2], u[4 * q + 3]);
-                    }
-                }
-                fence_proxy_async_smem();
-                bar_or(false);
-                if (r == 0 && h == 0) {
-#pragma unroll
-                    for (int ch = 0; ch < C::NCH; ++ch)
-                        tma_store_3d(&tmO, ost + ch * C::CHUNK_BYTES, ch * 64, row0[t], bh);
-                    bulk_commit_group();
-                }
-            }
-            ++co[t];
-        }
-        cs[0] += nblk[0];
-        cs[1] += nblk[1];
+        // row sums (one per half) and reference points for the epilogue warps
+        sts32(my_x, l);
+        if (h == 0) sts32(base + C::OFF_MREF + r * 4, m_ref);
+        mbar_arrive(bar(B_STFULL));
         }   // items
-        if (!F16 && r == 0 && h == 0) bulk_wait_group_read0();
     }
 
     tc_fence_before();
@@ -496,19 +522,15 @@ cudaError_t launch_gen(const Problem& p, const void* q, const void* k, const voi
     if (cudaGetDevice(&dev) != cudaSuccess ||
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
         return cudaErrorInvalidValue;
-    // An item is two query tiles of a head (their softmax and products interleave); with fewer such
-    // items than SMs an item is one tile instead, so that twice as many SMs have work.
     const int n_tiles = (p.Sq + BM - 1) / BM;
-    const int tpi = (static_cast<long long>((n_tiles + 1) / 2) * p.BH() < sms && n_tiles > 1) ? 1 : 2;
-    const int n_pairs = (n_tiles + tpi - 1) / tpi;
-    const long long items = static_cast<long long>(n_pairs) * p.BH();
+    const long long items = static_cast<long long>(n_tiles) * p.BH();
     if (items > 0x7fffffffLL) return cudaErrorInvalidValue;
     const long long blocks = items < sms ? items : sms;       // persistent: one CTA per SM
     const Dims dm{p.Sq, p.Sk, p.BH(), p.H, p.group(), p.off()};
     // streamed per block and shared between the query tiles of a head: K, V
     const int order = pick_schedule(items, sms, static_cast<double>(p.BHkv()) * p.Sk * D * (2 + 2), dev);
     kern<<<static_cast<unsigned>(blocks), kThreads, C::SMEM, st>>>(tq, tk, tv, to, lse, F16 ? static_cast<float*>(o) : nullptr, dm,
-                                                                   n_pairs, tpi, p.causal, order,
+                                                                   n_tiles, p.causal, order,
                                                                    p.scale * kLog2e, status);
     return MGN_FAIL(cudaGetLastError(), "forward launch");
 }
