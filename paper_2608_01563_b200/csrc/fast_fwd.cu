@@ -19,7 +19,7 @@
 // Tensor memory (512 columns): S(even blocks) [0,128), S(odd) [128,256), P(even) [256,320),
 // P(odd) [320,384), O [384,384+D).  The softmax reference point of a row only moves (and O is rescaled
 // in tensor memory) when a row outgrows it so far that a thread's partial sum of exponentials passes
-// a limit (2^60; 2^12 with f16 probabilities), which is exact: any reference point works for a
+// a limit (2^60; 2^15 with f16 probabilities), which is exact: any reference point works for a
 // softmax as long as nothing overflows.  The two threads of a row agree on that through a barrier
 // with an OR-reduction per block.
 #include "kernels.h"
@@ -36,11 +36,16 @@ constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 // A thread's partial row sum (64 columns) above this limit moves the reference points.  Every p stays
 // below the limit and the sums of a row below 2^13 times it, so nothing overflows.  With f16
-// probabilities the limit is 2^12 (f16 ends at 65504).  With bf16 it is 2^60: bf16 and f32 share the
+// probabilities the limit is 2^15 (f16 ends at 65504).  With bf16 it is 2^60: bf16 and f32 share the
 // exponent range, a softmax is exact for any reference point, and a low limit is expensive -- one row
 // in 128 passing it makes the whole tile repeat the pass, which heavy-tailed scores (1 % of the
 // inputs scaled by 8 in the decoder sweep) did in most key blocks: forward +50-60 % there.
-constexpr float kGrowthLimitF16 = 4096.0f;
+constexpr float kGrowthLimitF16 = 32768.0f;
+// With f16 probabilities the reference point is set this far (log2 units) above the row maximum, so that a
+// row has to outgrow its first maximum by a factor of 2^21 before its pass is repeated; the probabilities
+// then start at 2^-6 and keep full f16 precision down to 2^-8 of the row maximum (subnormal below: an
+// absolute step of 2^-18 of the maximum).
+constexpr float kMarginF16 = 6.0f;
 constexpr float kGrowthLimitBf16 = 1152921504606846976.0f;   // 2^60
 
 // 2^x for two values on the FMA pipe instead of the special-function unit (16 results per clock
@@ -366,13 +371,16 @@ fast_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         const uint32_t tO = tmem + lane_base + C::TM_O + (D / 2) * h;
         int g = 0;               // blocks seen so far (all items): buffer and phase of S, P
 
-        // barrier over the 256 softmax threads with an OR reduction of `pred`
-        auto bar_or = [](bool pred) -> bool {
+        // Barrier with an OR reduction of `pred` over the two warps that share 32 rows (one per half of the
+        // key columns).  Everything the two threads of a row have to agree on is local to these 64
+        // threads, so a row that outgrows its reference point makes 32 rows repeat their pass, not 128.
+        const uint32_t pair_id = 1 + ((warp - 4) & 3);
+        auto bar_or = [pair_id](bool pred) -> bool {
             uint32_t out;
             asm volatile(
                 "{\n\t.reg .pred P, Q;\n\tsetp.ne.b32 P, %1, 0;\n\t"
-                "barrier.cta.red.or.pred Q, 1, 256, P;\n\tselp.u32 %0, 1, 0, Q;\n\t}"
-                : "=r"(out) : "r"(static_cast<uint32_t>(pred)) : "memory");
+                "barrier.cta.red.or.pred Q, %2, 64, P;\n\tselp.u32 %0, 1, 0, Q;\n\t}"
+                : "=r"(out) : "r"(static_cast<uint32_t>(pred)), "r"(pair_id) : "memory");
             return out != 0;
         };
 
@@ -423,7 +431,7 @@ fast_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                 const float mine = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
                 sts32(my_x, mine);
                 bar_or(false);
-                m_ref = fmaxf(mine, lds32f(peer_x));      // finite: key 0 is visible to every row
+                m_ref = fmaxf(mine, lds32f(peer_x)) + (F16 ? kMarginF16 : 0.f);      // finite: key 0 is visible to every row
                 bar_or(false);                                // exchange buffer may be reused
             }
 
@@ -488,7 +496,7 @@ fast_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                 sts32(my_x, ymax);
                 bar_or(false);
                 const float ym = fmaxf(ymax, lds32f(peer_x));
-                const float m_new = fmaxf(m_ref, m_ref + ym);
+                const float m_new = fmaxf(m_ref, m_ref + ym + (F16 ? kMarginF16 : 0.f));
                 const float alpha = ex2(m_ref - m_new);
                 m_ref = m_new;
                 l *= alpha;
