@@ -63,6 +63,8 @@ def _load():
         lib.ref_out_proj_bwd_weight.restype = None
         lib.ref_qkv_rope.argtypes = [_dp] * 7 + [i] * 6
         lib.ref_qkv_rope.restype = None
+        lib.ref_qkv_rope_bwd.argtypes = [_dp] * 10 + [i] * 6
+        lib.ref_qkv_rope_bwd.restype = None
         lib.ref_max_threads.argtypes = []
         lib.ref_max_threads.restype = i
         _lib = lib
@@ -197,3 +199,20 @@ def qkv_rope(x, w, cos_t, sin_t, H: int, Hkv: int, D: int):
     q = np.empty((B, H, S, D)); k = np.empty((B, Hkv, S, D)); v = np.empty((B, Hkv, S, D))
     _load().ref_qkv_rope(_p(x), _p(w), _p(cos_t), _p(sin_t), _p(q), _p(k), _p(v), B, S, E, H, Hkv, D)
     return q, k, v
+
+
+def qkv_rope_bwd(g_q, g_k, g_v, x, w, cos_t, sin_t):
+    """Backward of qkv_rope: gradients with respect to the rotated Q [B,H,S,D], K, V [B,Hkv,S,D] ->
+    (dX [B,S,E], dW [(H+2Hkv)*D, E], gY [B,S,(H+2Hkv)*D] = the gradient with respect to the unrotated
+    projection, heads concatenated query | key | value), float64."""
+    g_q, g_k, g_v, x, w, cos_t, sin_t = _c(g_q), _c(g_k), _c(g_v), _c(x), _c(w), _c(cos_t), _c(sin_t)
+    B, H, S, D = g_q.shape
+    Hkv = g_k.shape[1]
+    E = x.shape[2]
+    F = (H + 2 * Hkv) * D
+    assert g_k.shape == (B, Hkv, S, D) and g_v.shape == (B, Hkv, S, D) and x.shape == (B, S, E) and w.shape == (F, E)
+    assert cos_t.shape == (S, D // 2) and sin_t.shape == (S, D // 2)
+    gy = np.empty((B, S, F)); dx = np.empty((B, S, E)); dw = np.empty((F, E))
+    _load().ref_qkv_rope_bwd(_p(g_q), _p(g_k), _p(g_v), _p(x), _p(w), _p(cos_t), _p(sin_t), _p(gy), _p(dx), _p(dw),
+                             B, S, E, H, Hkv, D)
+    return dx, dw, gy

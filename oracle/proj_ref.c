@@ -128,3 +128,56 @@ void ref_qkv_rope(const double *X, const double *W, const double *cos_t, const d
         }
     }
 }
+
+/*
+ * Backward of ref_qkv_rope (textbook reverse mode of the two steps it states, written out):
+ *   the rotation of a (d, d + D/2) pair by the angle (c, sn) is linear with an orthogonal matrix, so the
+ *   gradient with respect to the unrotated pair is the rotation by the opposite angle:
+ *       gy[d]       =  g[d] * c + g[d + D/2] * sn
+ *       gy[d + D/2] =  g[d + D/2] * c - g[d] * sn          (query and key heads; value heads: gy = g)
+ *   then, with y[r, hh*D + d] = sum_e X[r, e] W[hh*D + d, e]:
+ *       dX[r, e]        = sum_{hh,d} gy[r, hh, d] W[hh*D + d, e]
+ *       dW[hh*D + d, e] = sum_r      gy[r, hh, d] X[r, e]
+ * gQ [B,H,S,D], gK, gV [B,Hkv,S,D] are the gradients with respect to the ROTATED outputs.
+ * GY (scratch and output) [B*S, (H+2Hkv)*D]: the gradient with respect to the unrotated projection.
+ */
+void ref_qkv_rope_bwd(const double *gQ, const double *gK, const double *gV, const double *X, const double *W,
+                      const double *cos_t, const double *sin_t, double *GY, double *dX, double *dW,
+                      int B, int S, int E, int H, int Hkv, int D)
+{
+    const int heads = H + 2 * Hkv, half = D / 2;
+    const long rows = (long)B * S;
+    const long F = (long)heads * D;
+#pragma omp parallel for schedule(static)
+    for (long r = 0; r < rows; ++r) {
+        const int b = (int)(r / S), s = (int)(r % S);
+        for (int hh = 0; hh < heads; ++hh) {
+            const double *g;
+            int rope = 1;
+            if (hh < H) g = gQ + (((size_t)b * H + hh) * S + s) * D;
+            else if (hh < H + Hkv) g = gK + (((size_t)b * Hkv + (hh - H)) * S + s) * D;
+            else { g = gV + (((size_t)b * Hkv + (hh - H - Hkv)) * S + s) * D; rope = 0; }
+            double *gy = GY + (size_t)r * F + (size_t)hh * D;
+            if (!rope) { for (int d = 0; d < D; ++d) gy[d] = g[d]; continue; }
+            for (int d = 0; d < half; ++d) {
+                const double c = cos_t[(size_t)s * half + d], sn = sin_t[(size_t)s * half + d];
+                gy[d] = g[d] * c + g[d + half] * sn;
+                gy[d + half] = g[d + half] * c - g[d] * sn;
+            }
+        }
+    }
+#pragma omp parallel for schedule(static)
+    for (long r = 0; r < rows; ++r)
+        for (int e = 0; e < E; ++e) {
+            double acc = 0.0;
+            for (long f = 0; f < F; ++f) acc += GY[(size_t)r * F + f] * W[(size_t)f * E + e];
+            dX[(size_t)r * E + e] = acc;
+        }
+#pragma omp parallel for schedule(static)
+    for (long f = 0; f < F; ++f)
+        for (int e = 0; e < E; ++e) {
+            double acc = 0.0;
+            for (long r = 0; r < rows; ++r) acc += GY[(size_t)r * F + f] * X[(size_t)r * E + e];
+            dW[(size_t)f * E + e] = acc;
+        }
+}

@@ -142,3 +142,91 @@ def test_qkv_rope_invariants():
     xs = np.zeros((1, 6, E)); xs[0, 1] = xs[0, 2] = x[0, 0]; xs[0, 3] = xs[0, 4] = x[0, 5]
     q, k, _ = orc.qkv_rope(xs, w, cos_t, sin_t, H, Hkv, D)
     np.testing.assert_allclose(q[0, 0, 3] @ k[0, 0, 1], q[0, 0, 4] @ k[0, 0, 2], rtol=1e-12, atol=1e-12)
+
+
+# ---- backward of the query/key/value projection with rotation --------------------------------------
+
+def _angles_seeded(S, D, seed):
+    th = np.random.default_rng(seed).uniform(-3.0, 3.0, (S, D // 2))
+    return np.cos(th), np.sin(th)
+
+
+def test_qkv_bwd_hand_worked_example():
+    # B=1, S=1, E=1, H=1, Hkv=1, D=2, x = 2, w = [1, 3 | -1, 2 | 4, 5] (query | key | value rows),
+    # angle with cos = 0, sin = 1: out[0] = -y[1], out[1] = y[0].
+    x = np.array([[[2.0]]]); w = np.array([[1.0], [3.0], [-1.0], [2.0], [4.0], [5.0]])
+    c, s = np.array([[0.0]]), np.array([[1.0]])
+    q, k, v = orc.qkv_rope(x, w, c, s, 1, 1, 2)
+    np.testing.assert_allclose(q.ravel(), [-6.0, 2.0]); np.testing.assert_allclose(k.ravel(), [-4.0, -2.0])
+    g_q = np.array([1.0, 10.0]).reshape(1, 1, 1, 2); g_k = np.array([100.0, 1000.0]).reshape(1, 1, 1, 2)
+    g_v = np.array([0.5, 0.25]).reshape(1, 1, 1, 2)
+    dx, dw, gy = orc.qkv_rope_bwd(g_q, g_k, g_v, x, w, c, s)
+    # q0 = -y1, q1 = y0  =>  gy0 = g_q1, gy1 = -g_q0
+    np.testing.assert_allclose(gy.ravel(), [10.0, -1.0, 1000.0, -100.0, 0.5, 0.25], rtol=0, atol=0)
+    np.testing.assert_allclose(dw.ravel(), 2.0 * gy.ravel(), rtol=0, atol=0)
+    np.testing.assert_allclose(dx.ravel(), [10 - 3 - 1000 - 200 + 2 + 1.25], rtol=0, atol=1e-12)
+
+
+@pytest.mark.parametrize("B,S,E,H,Hkv,D", [(2, 5, 7, 3, 1, 4), (1, 6, 5, 2, 2, 8)])
+def test_qkv_bwd_matches_torch_float64_autograd(B, S, E, H, Hkv, D):
+    g = torch.Generator().manual_seed(B + S + E + D)
+    x = torch.randn(B, S, E, generator=g, dtype=torch.float64, requires_grad=True)
+    w = torch.randn((H + 2 * Hkv) * D, E, generator=g, dtype=torch.float64, requires_grad=True)
+    c, s = _angles_seeded(S, D, 5)
+    ct, st = torch.from_numpy(c), torch.from_numpy(s)
+    y = torch.einsum("bse,fe->bsf", x, w).view(B, S, H + 2 * Hkv, D).permute(0, 2, 1, 3)     # [B, heads, S, D]
+    lo, hi = y[..., : D // 2], y[..., D // 2:]
+    rot = torch.cat([lo * ct - hi * st, hi * ct + lo * st], dim=-1)
+    q, k, v = rot[:, :H], rot[:, H:H + Hkv], y[:, H + Hkv:]
+    g_q = torch.randn(q.shape, generator=g, dtype=torch.float64)
+    g_k = torch.randn(k.shape, generator=g, dtype=torch.float64)
+    g_v = torch.randn(v.shape, generator=g, dtype=torch.float64)
+    ((q * g_q).sum() + (k * g_k).sum() + (v * g_v).sum()).backward()
+    dx, dw, _ = orc.qkv_rope_bwd(g_q.numpy(), g_k.numpy(), g_v.numpy(), x.detach().numpy(), w.detach().numpy(), c, s)
+    np.testing.assert_allclose(dx, x.grad.numpy(), rtol=1e-12, atol=1e-12)
+    np.testing.assert_allclose(dw, w.grad.numpy(), rtol=1e-12, atol=1e-12)
+
+
+def test_qkv_bwd_central_finite_differences_of_the_forward_oracle():
+    B, S, E, H, Hkv, D = 1, 3, 3, 2, 1, 4
+    x, w = rnd(11, B, S, E), rnd(12, (H + 2 * Hkv) * D, E)
+    c, s = _angles_seeded(S, D, 13)
+    g_q, g_k, g_v = rnd(14, B, H, S, D), rnd(15, B, Hkv, S, D), rnd(16, B, Hkv, S, D)
+
+    def loss(x_, w_):
+        q, k, v = orc.qkv_rope(x_, w_, c, s, H, Hkv, D)
+        return float((q * g_q).sum() + (k * g_k).sum() + (v * g_v).sum())
+
+    dx, dw, _ = orc.qkv_rope_bwd(g_q, g_k, g_v, x, w, c, s)
+    h = 1e-6
+    for idx in np.ndindex(x.shape):
+        p, m = x.copy(), x.copy()
+        p[idx] += h; m[idx] -= h
+        assert abs((loss(p, w) - loss(m, w)) / (2 * h) - dx[idx]) <= 1e-6
+    for idx in np.ndindex(w.shape):
+        p, m = w.copy(), w.copy()
+        p[idx] += h; m[idx] -= h
+        assert abs((loss(x, p) - loss(x, m)) / (2 * h) - dw[idx]) <= 1e-6
+
+
+def test_qkv_bwd_inverse_rotation_properties():
+    """The gradient with respect to the unrotated projection is the rotation by the opposite angle: it keeps
+    pair norms, undoes the forward rotation, and with zero angles it is the concatenation of the inputs."""
+    B, S, E, H, Hkv, D = 2, 4, 3, 2, 1, 6
+    x, w = rnd(21, B, S, E), rnd(22, (H + 2 * Hkv) * D, E)
+    c, s = _angles_seeded(S, D, 23)
+    q, k, v = orc.qkv_rope(x, w, c, s, H, Hkv, D)
+    _, _, gy = orc.qkv_rope_bwd(q, k, v, x, w, c, s)              # feed the rotated outputs back
+    y = np.einsum("bse,fe->bsf", x, w)                             # the unrotated projection
+    np.testing.assert_allclose(gy, y, rtol=1e-12, atol=1e-12)      # R^T R = I
+    g_q, g_k, g_v = rnd(24, B, H, S, D), rnd(25, B, Hkv, S, D), rnd(26, B, Hkv, S, D)
+    _, _, gy2 = orc.qkv_rope_bwd(g_q, g_k, g_v, x, w, c, s)
+    gq_un = gy2[..., : H * D].reshape(B, S, H, D).transpose(0, 2, 1, 3)
+    half = D // 2
+    np.testing.assert_allclose(gq_un[..., :half] ** 2 + gq_un[..., half:] ** 2,
+                               g_q[..., :half] ** 2 + g_q[..., half:] ** 2, rtol=1e-12)
+    one, zero = np.ones((S, half)), np.zeros((S, half))
+    dx0, _, gy0 = orc.qkv_rope_bwd(g_q, g_k, g_v, x, w, one, zero)
+    cat = np.concatenate([t.transpose(0, 2, 1, 3).reshape(B, S, -1) for t in (g_q, g_k, g_v)], axis=-1)
+    np.testing.assert_allclose(gy0, cat, rtol=0, atol=0)
+    np.testing.assert_allclose(dx0, cat @ w, rtol=1e-12, atol=1e-12)
