@@ -297,7 +297,28 @@ def measure_proj_fusion(mgn, steps, warmup):
         qk = qk * c + rot * s_
         q2.copy_(qk[:, :H]); k2.copy_(qk[:, H:]); v2.copy_(yq[:, 2 * H:])
 
+    # backward of the QKV projection: opposite rotation of dq, dk, then the data and weight gradients
+    gq, gk, gv = (torch.randn(B, H, S, D, device="cuda", generator=g).to(dt) for _ in range(3))
+    d_x = torch.empty(B, S, E, device="cuda", dtype=dt)
+    d_wqkv = torch.empty_like(w_qkv)
+
+    def fused_qkv_bwd():
+        mgn.mgn_rope_bwd_inplace(gq, gk, cos_t, sin_t, mode)
+        mgn.mgn_qkv_bwd_data(gq, gk, gv, w_qkv, d_x, mode)
+        mgn.mgn_qkv_bwd_weight(gq, gk, gv, x, d_wqkv, mode)
+
+    def unfused_qkv_bwd():
+        c = torch.cat([cos_t, cos_t], dim=1).to(dt)
+        s_ = torch.cat([sin_t, sin_t], dim=1).to(dt)
+        qk = torch.cat([gq, gk], dim=1)
+        rot = torch.cat([qk[..., D // 2:], -qk[..., :D // 2]], dim=-1)
+        gy = torch.cat([qk * c + rot * s_, gv], dim=1).transpose(1, 2).reshape(B * S, 3 * H * D)
+        torch.matmul(gy, w_qkv, out=d_x.view(B * S, E))
+        torch.matmul(gy.t(), x.view(B * S, E), out=d_wqkv)
+
     gemm_flops = 2.0 * B * S * H * D * E
+    qb_fused = timed(fused_qkv_bwd)
+    qb_unf = timed(unfused_qkv_bwd)
     w_fused = timed(lambda: mgn.mgn_out_proj_bwd_weight(o, d_y, d_w, mode))
     w_unf = timed(unfused_dw)
     qkv_fused = timed(lambda: mgn.mgn_qkv_rope_fwd(x, w_qkv, cos_t, sin_t, q2, k2, v2, mode))
@@ -314,6 +335,8 @@ def measure_proj_fusion(mgn, steps, warmup):
             "weight_grad_ms": {"fused": round(w_fused, 4), "library_gemm_plus_layout_copy": round(w_unf, 4)},
             "qkv_rope_ms": {"fused": round(qkv_fused, 4), "library_gemm_plus_eager_rotation_and_copies": round(qkv_unf, 4)},
             "qkv_rope_tflops": round(3 * gemm_flops / (qkv_fused * 1e-3) / 1e12, 1),
+            "qkv_bwd_ms": {"fused": round(qb_fused, 4), "library_gemms_plus_eager_rotation_and_copies": round(qb_unf, 4)},
+            "qkv_bwd_tflops": round(6 * gemm_flops / (qb_fused * 1e-3) / 1e12, 1),
             "do_producer_ms": round(p_fused, 4), "do_producer_tflops": round(gemm_flops / (p_fused * 1e-3) / 1e12, 1),
             "proj_bwd_plus_attn_bwd_ms": {"fused": round(b_fused, 4), "library_gemm_plus_layout_copy_plus_attn_bwd": round(b_unf, 4)}}
 

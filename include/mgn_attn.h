@@ -184,6 +184,16 @@ int mgn_attn_bwd_deterministic(const void* q, const void* k, const void* v, cons
  *     cos_t, sin_t [S, D/2] (f32, device): out[d] = y[d] c - y[d+D/2] s, out[d+D/2] = y[d+D/2] c + y[d] s;
  *     value heads are copied.  q [B,H,S,D], k, v [B,H_kv,S,D] (bf16) out, in the layout the attention
  *     entry points read.  The rotation is done in f32 on the accumulators, before the one rounding to bf16.
+ * The backward of that step, in three calls (fast mode, same limits):
+ * mgn_rope_bwd_inplace:  rotates the pairs of dq [B,H,S,D] and dk [B,H_kv,S,D] (bf16, as the attention
+ *     backward wrote them) IN PLACE by the opposite angles: g[d] = dq[d] c + dq[d+D/2] s,
+ *     g[d+D/2] = dq[d+D/2] c - dq[d] s -- the gradient with respect to the unrotated projection.  A
+ *     streaming pass: the rotation depends on the position, i.e. on the row of the operand, so it cannot be
+ *     folded into the two products below.  The result is rounded to bf16 once more.
+ * mgn_qkv_bwd_data:      dx[b,s,e] = sum_n g[b,s,n] * w[n,e], g the concatenation (query | key | value heads)
+ *     of gq [B,H,S,D], gk, gv [B,H_kv,S,D] -- dq and dk after mgn_rope_bwd_inplace, and dv -- read where they
+ *     are (no concatenated copy); w [(H + 2 H_kv) D, E]; dx [B,S,E] (bf16) out.
+ * mgn_qkv_bwd_weight:    dw[n,e] = sum_{b,s} g[b,s,n] * x[b,s,e]; x [B,S,E] in; dw [(H + 2 H_kv) D, E] (bf16) out.
  * mgn_attn_bwd_given_delta: mgn_attn_bwd_ext without `o`, with a ready `delta` [B,H,S_q] (f32, read
  *     only): the pass over o and d_o is skipped.  Either mode.  Workspace as for mgn_attn_bwd_ext.
  * Errors as elsewhere: INVALID_ARG (null pointer, size <= 0, unknown mode), UNSUPPORTED, MISALIGNED,
@@ -196,6 +206,12 @@ int mgn_out_proj_bwd_weight(const void* o, const void* d_y, void* d_w, int B, in
                             void* stream);
 int mgn_qkv_rope_fwd(const void* x, const void* w, const float* cos_t, const float* sin_t, void* q, void* k, void* v,
                      int B, int S, int E, int H, int H_kv, int D, int mode, void* stream);
+int mgn_rope_bwd_inplace(void* dq, void* dk, const float* cos_t, const float* sin_t, int B, int H, int H_kv, int S,
+                         int D, int mode, void* stream);
+int mgn_qkv_bwd_data(const void* gq, const void* gk, const void* gv, const void* w, void* dx, int B, int S, int E, int H,
+                     int H_kv, int D, int mode, void* stream);
+int mgn_qkv_bwd_weight(const void* gq, const void* gk, const void* gv, const void* x, void* dw, int B, int S, int E,
+                       int H, int H_kv, int D, int mode, void* stream);
 int mgn_attn_bwd_given_delta(const void* q, const void* k, const void* v, const void* d_o, const float* lse,
                              const float* delta, void* dq, void* dk, void* dv,
                              void* workspace, size_t workspace_bytes,

@@ -79,6 +79,12 @@ def lib() -> ctypes.CDLL:
         L.mgn_out_proj_bwd_weight.restype = i
         L.mgn_qkv_rope_fwd.argtypes = [vp] * 7 + [i] * 7 + [vp]
         L.mgn_qkv_rope_fwd.restype = i
+        L.mgn_rope_bwd_inplace.argtypes = [vp] * 4 + [i] * 6 + [vp]
+        L.mgn_rope_bwd_inplace.restype = i
+        L.mgn_qkv_bwd_data.argtypes = [vp] * 5 + [i] * 7 + [vp]
+        L.mgn_qkv_bwd_data.restype = i
+        L.mgn_qkv_bwd_weight.argtypes = [vp] * 5 + [i] * 7 + [vp]
+        L.mgn_qkv_bwd_weight.restype = i
         L.mgn_attn_bwd_given_delta.argtypes = [vp] * 9 + [vp, sz, i, i, i, i, i, i, i, f, i, vp]
         L.mgn_attn_bwd_given_delta.restype = i
         L.mgn_selftest_wait_timeout.argtypes = [vp, vp]
@@ -258,6 +264,33 @@ def mgn_qkv_rope_fwd(x, w, cos_t, sin_t, q, k, v, mode: int, stream: Optional[in
                                 int(x.shape[2]), H, int(k.shape[1]), D, int(mode), _stream(stream))
     if st != MGN_OK:
         raise MgnError(st, "mgn_qkv_rope_fwd")
+
+
+def mgn_rope_bwd_inplace(dq, dk, cos_t, sin_t, mode: int, stream: Optional[int] = None) -> None:
+    """dq [B,H,S,D], dk [B,Hkv,S,D] rotated in place by the opposite angles (gradient of the rotary embedding)."""
+    B, H, S, D = _dims(dq)
+    st = lib().mgn_rope_bwd_inplace(_ptr(dq), _ptr(dk), _ptr(cos_t), _ptr(sin_t), B, H, int(dk.shape[1]), S, D,
+                                    int(mode), _stream(stream))
+    if st != MGN_OK:
+        raise MgnError(st, "mgn_rope_bwd_inplace")
+
+
+def mgn_qkv_bwd_data(gq, gk, gv, w, dx, mode: int, stream: Optional[int] = None) -> None:
+    """dx [B,S,E] = (gq | gk | gv heads concatenated) w; gq [B,H,S,D], gk, gv [B,Hkv,S,D], w [(H+2Hkv)D, E]."""
+    B, H, S, D = _dims(gq)
+    st = lib().mgn_qkv_bwd_data(_ptr(gq), _ptr(gk), _ptr(gv), _ptr(w), _ptr(dx), B, S, int(dx.shape[2]), H,
+                                int(gk.shape[1]), D, int(mode), _stream(stream))
+    if st != MGN_OK:
+        raise MgnError(st, "mgn_qkv_bwd_data")
+
+
+def mgn_qkv_bwd_weight(gq, gk, gv, x, dw, mode: int, stream: Optional[int] = None) -> None:
+    """dw [(H+2Hkv)D, E] = (gq | gk | gv heads concatenated)^T x; x [B,S,E]."""
+    B, H, S, D = _dims(gq)
+    st = lib().mgn_qkv_bwd_weight(_ptr(gq), _ptr(gk), _ptr(gv), _ptr(x), _ptr(dw), B, S, int(x.shape[2]), H,
+                                  int(gk.shape[1]), D, int(mode), _stream(stream))
+    if st != MGN_OK:
+        raise MgnError(st, "mgn_qkv_bwd_weight")
 
 
 def mgn_attn_bwd_given_delta(q, k, v, d_o, lse, delta, dq, dk, dv, workspace, causal: bool, scale: float, mode: int,

@@ -353,6 +353,45 @@ int mgn_qkv_rope_fwd(const void* x, const void* w, const float* cos_t, const flo
                ? MGN_OK : MGN_ERR_CUDA;
 }
 
+int mgn_rope_bwd_inplace(void* dq, void* dk, const float* cos_t, const float* sin_t, int B, int H, int H_kv, int S,
+                         int D, int mode, void* stream)
+{
+    if (!cos_t || !sin_t || H_kv <= 0) return MGN_ERR_INVALID_ARG;
+    if (int r = check_proj(dq, dk, cos_t, sin_t, B, H, S, D, 8, mode)) return r;
+    unsigned* status = nullptr;
+    if (int r = device_setup(&status)) return r;
+    return mgn::launch_rope_bwd(dq, dk, cos_t, sin_t, B, H, H_kv, S, D, static_cast<cudaStream_t>(stream)) == cudaSuccess
+               ? MGN_OK : MGN_ERR_CUDA;
+}
+
+int mgn_qkv_bwd_data(const void* gq, const void* gk, const void* gv, const void* w, void* dx, int B, int S, int E, int H,
+                     int H_kv, int D, int mode, void* stream)
+{
+    if (!gv || H_kv <= 0) return MGN_ERR_INVALID_ARG;
+    if (int r = check_proj(gq, gk, w, dx, B, H, S, D, E, mode)) return r;
+    if (static_cast<long long>(H + 2LL * H_kv) * D > 0x7fffffffLL) return MGN_ERR_UNSUPPORTED;
+    if (!aligned16(gv)) return MGN_ERR_MISALIGNED;
+    unsigned* status = nullptr;
+    if (int r = device_setup(&status)) return r;
+    return mgn::launch_qkv_bwd_data(gq, gk, gv, w, dx, B, S, E, H, H_kv, D, status, static_cast<cudaStream_t>(stream)) ==
+                   cudaSuccess
+               ? MGN_OK : MGN_ERR_CUDA;
+}
+
+int mgn_qkv_bwd_weight(const void* gq, const void* gk, const void* gv, const void* x, void* dw, int B, int S, int E,
+                       int H, int H_kv, int D, int mode, void* stream)
+{
+    if (!gv || H_kv <= 0) return MGN_ERR_INVALID_ARG;
+    if (int r = check_proj(gq, gk, x, dw, B, H, S, D, E, mode)) return r;
+    if (static_cast<long long>(H + 2LL * H_kv) * D > 0x7fffffffLL) return MGN_ERR_UNSUPPORTED;
+    if (!aligned16(gv)) return MGN_ERR_MISALIGNED;
+    unsigned* status = nullptr;
+    if (int r = device_setup(&status)) return r;
+    return mgn::launch_qkv_bwd_weight(gq, gk, gv, x, dw, B, S, E, H, H_kv, D, status,
+                                      static_cast<cudaStream_t>(stream)) == cudaSuccess
+               ? MGN_OK : MGN_ERR_CUDA;
+}
+
 int mgn_attn_bwd(const void* q, const void* k, const void* v, const void* o, const void* d_o,
                  const float* lse, void* dq, void* dk, void* dv,
                  void* workspace, size_t workspace_bytes,
@@ -418,6 +457,6 @@ const char* mgn_status_string(int status)
     }
 }
 
-int mgn_version(void) { return 310; }   // 0.2.1: tile-shape query, low-padding strict tiles, leaner fast forward (0.2.0: extended shapes, deterministic backward, accelerated forward)
+int mgn_version(void) { return 320; }   // 0.3.2: projections either side of attention, forward and backward, rebuilt fast forward; 0.2.1: tile-shape query, low-padding strict tiles, leaner fast forward (0.2.0: extended shapes, deterministic backward, accelerated forward)
 
 }  // extern "C"

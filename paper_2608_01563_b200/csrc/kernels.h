@@ -122,6 +122,15 @@ cudaError_t launch_out_proj_bwd_weight(const void* o, const void* d_y, void* d_w
 // (rotate-half pairing, angle tables cos_t, sin_t [S, D/2] f32) applied to q and k; q [B,H,S,D], k, v [B,Hkv,S,D].
 cudaError_t launch_qkv_rope(const void* x, const void* w, const float* cos_t, const float* sin_t, void* q, void* k,
                             void* v, int B, int S, int E, int H, int Hkv, int D, unsigned* status, cudaStream_t st);
+// Its backward.  launch_rope_bwd rotates dq [B,H,S,D] and dk [B,Hkv,S,D] in place by the opposite angles (the
+// gradient with respect to the unrotated projection); then dx [B,S,E] = (gq | gk | gv)_concat w and
+// dw [(H+2Hkv)*D, E] = (gq | gk | gv)_concat^T x, reading the three head-major tensors where they are.
+cudaError_t launch_rope_bwd(void* dq, void* dk, const float* cos_t, const float* sin_t, int B, int H, int Hkv, int S,
+                            int D, cudaStream_t st);
+cudaError_t launch_qkv_bwd_data(const void* gq, const void* gk, const void* gv, const void* w, void* dx, int B, int S,
+                                int E, int H, int Hkv, int D, unsigned* status, cudaStream_t st);
+cudaError_t launch_qkv_bwd_weight(const void* gq, const void* gk, const void* gv, const void* x, void* dw, int B, int S,
+                                  int E, int H, int Hkv, int D, unsigned* status, cudaStream_t st);
 
 // Work-item order of the persistent fast kernels (see the kernels for the two orders).  Head-major
 // order (1) is chosen when the data that the items of one head share (`shared_bytes`, over all

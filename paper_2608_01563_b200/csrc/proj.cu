@@ -12,7 +12,13 @@
 //        epilogue also emits delta = rowsum(dO o O) -- the attention backward's preprocess pass -- while
 //        the dO tile is still in registers;
 //   DW   dW_o = O_concat^T dY contracts over the positions, again reading O head-major (both operands
-//        are fed to the tensor core with the non-contracted index contiguous).
+//        are fed to the tensor core with the non-contracted index contiguous);
+//   DX   dX = (gQ | gK | gV)_concat W_qkv, the data gradient of the QKV projection: like FWD, but the
+//        heads of the concatenated operand live in three tensors ([B,H,S,D] and two [B,Hkv,S,D]);
+//   DWX  dW_qkv = (gQ | gK | gV)_concat^T X, its weight gradient: like DW with the same three tensors.
+// The last two take the gradients with respect to the UNROTATED projection: the rotation depends on the
+// position, i.e. on the row of the operand, and cannot be folded into either product; rope_bwd_kernel
+// applies the opposite rotation to dQ and dK in place first (a streaming pass over those two tensors).
 // One CTA computes a 128 x 256 output tile.  Warp 0 streams 64-wide contraction slices of both
 // operands through a four-stage TMA ring, one lane of warp 1 issues the products into a 256-column
 // tensor-memory accumulator, warps 2-5 (one thread per accumulator row) read it out.
@@ -32,10 +38,10 @@ constexpr int OFF_A = 0, OFF_B = kStages * A_BYTES, OFF_BAR = OFF_B + kStages * 
 constexpr int PAYLOAD = OFF_BAR + 128;
 constexpr int SMEM = PAYLOAD + 1024;
 enum { B_FULL = 0, B_EMPTY = kStages, B_ACC = 2 * kStages, B_COUNT = 2 * kStages + 1 };
-enum { V_FWD = 0, V_DO = 1, V_DW = 2, V_QKV = 3 };
+enum { V_FWD = 0, V_DO = 1, V_DW = 2, V_QKV = 3, V_DX = 4, V_DWX = 5 };
 
 struct ProjArgs {
-    __nv_bfloat16* out;          // FWD: y   DO: d_o   DW: d_w   QKV: q
+    __nv_bfloat16* out;          // FWD: y   DO: d_o   DW, DWX: d_w   QKV: q   DX: d_x
     __nv_bfloat16* out_k;        // QKV: k
     __nv_bfloat16* out_v;        // QKV: v
     const __nv_bfloat16* o;      // DO: attention output, for delta
@@ -80,8 +86,8 @@ __device__ __forceinline__ void epilogue_plain(const ProjArgs& a, const uint32_t
             dl = 0.f;
         }
     } else {
-        // FWD: y[b, row, n..]   DW: d_w[row, n..]   (E is a multiple of 8: whole 16-byte pieces)
-        const size_t r = V == V_FWD ? static_cast<size_t>(b) * a.S + row : static_cast<size_t>(row);
+        // FWD, DX: y[b, row, n..]   DW, DWX: d_w[row, n..]   (E is a multiple of 8: whole 16-byte pieces)
+        const size_t r = (V == V_FWD || V == V_DX) ? static_cast<size_t>(b) * a.S + row : static_cast<size_t>(row);
         store_row32(a.out + r * a.E + n, u, (a.E - n) / 8);
     }
 }
@@ -130,7 +136,8 @@ __device__ __forceinline__ void epilogue_qkv_head(const ProjArgs& a, uint32_t ta
 
 template <int V>
 __global__ void __launch_bounds__(kThreads, 1)
-proj_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const ProjArgs a,
+proj_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmA2,
+            const __grid_constant__ CUtensorMap tmA3, const __grid_constant__ CUtensorMap tmB, const ProjArgs a,
             unsigned* status)
 {
     extern __shared__ uint8_t smem_raw[];
@@ -142,11 +149,21 @@ proj_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     // tile: TN output columns from n0; TM rows from r0 (positions s of batch element b, or for DW rows (h,d) of d_w)
     const int n0 = static_cast<int>(blockIdx.x) * TN, r0 = static_cast<int>(blockIdx.y) * TM, b = static_cast<int>(blockIdx.z);
-    const int HD = a.H * a.D;
-    const int n_sc = (a.S + TK - 1) / TK;                              // DW: 64-position slices per batch element
-    const int N = V == V_DO ? HD : V == V_QKV ? (a.H + 2 * a.Hkv) * a.D : a.E;
-    const int n_kt = V == V_FWD ? HD / TK : V == V_DW ? a.B * n_sc : (a.E + TK - 1) / TK;
-    const int rows = V == V_DW ? HD : a.S;
+    const int HD = a.H * a.D, F = (a.H + 2 * a.Hkv) * a.D;             // features: of the heads of O; of query | key | value
+    const int n_sc = (a.S + TK - 1) / TK;                              // DW, DWX: 64-position slices per batch element
+    const int N = V == V_DO ? HD : V == V_QKV ? F : a.E;
+    const int n_kt = V == V_FWD ? HD / TK : V == V_DX ? F / TK : (V == V_DW || V == V_DWX) ? a.B * n_sc : (a.E + TK - 1) / TK;
+    const int rows = V == V_DW ? HD : V == V_DWX ? F : a.S;
+    // DX, DWX: 64 consecutive features of the concatenation (query | key | value heads) starting at f lie in one
+    // head of one of three tensors; `idx` is that head's index in its tensor for batch element bb.  Past the
+    // last head the index runs off the value tensor, and the load returns zeros.
+    auto head_of = [&](int f, int bb, int& idx) -> const CUtensorMap* {
+        const int hh = f / a.D;
+        if (hh < a.H) { idx = bb * a.H + hh; return &tmA; }
+        if (hh < a.H + a.Hkv) { idx = bb * a.Hkv + hh - a.H; return &tmA2; }
+        idx = hh < a.H + 2 * a.Hkv ? bb * a.Hkv + hh - a.H - a.Hkv : a.B * a.Hkv;
+        return &tmA3;
+    };
 
     if (tid == 0) {
         for (int i = 0; i < B_COUNT; ++i) mbar_init(bar(i), 1);
@@ -169,8 +186,14 @@ proj_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             if constexpr (V == V_DO || V == V_QKV) {
                 tma_load_3d(dA, &tmA, full, k0, r0, b);                                  // 128 positions x 64 e
                 tma_load_3d(dB, &tmB, full, k0, n0, 0);                                  // 256 rows n x 64 e
-            } else if constexpr (V == V_FWD) {
-                tma_load_3d(dA, &tmA, full, k0 % a.D, r0, b * a.H + k0 / a.D);           // 128 positions x 64 d of one head
+            } else if constexpr (V == V_FWD || V == V_DX) {
+                if constexpr (V == V_FWD) {
+                    tma_load_3d(dA, &tmA, full, k0 % a.D, r0, b * a.H + k0 / a.D);       // 128 positions x 64 d of one head
+                } else {
+                    int idx;
+                    const CUtensorMap* m = head_of(k0, b, idx);
+                    tma_load_3d(dA, m, full, k0 % a.D, r0, idx);
+                }
 #pragma unroll
                 for (int c = 0; c < TN / 64; ++c)                                         // four blocks of 64 k rows x 64 n
                     tma_load_3d(dB + c * (TK * 128), &tmB, full, n0 + 64 * c, k0, 0);
@@ -179,7 +202,13 @@ proj_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 #pragma unroll
                 for (int c = 0; c < TM / 64; ++c) {                                       // two blocks of 64 positions x 64 rows m
                     const int m = r0 + 64 * c;
-                    tma_load_3d(dA + c * (TK * 128), &tmA, full, m % a.D, s0, bb * a.H + m / a.D);
+                    if constexpr (V == V_DW) {
+                        tma_load_3d(dA + c * (TK * 128), &tmA, full, m % a.D, s0, bb * a.H + m / a.D);
+                    } else {
+                        int idx;
+                        const CUtensorMap* mp = head_of(m, bb, idx);
+                        tma_load_3d(dA + c * (TK * 128), mp, full, m % a.D, s0, idx);
+                    }
                 }
 #pragma unroll
                 for (int c = 0; c < TN / 64; ++c)                                         // four blocks of 64 positions x 64 e
@@ -188,7 +217,7 @@ proj_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         }
     } else if (warp == 1 && lane == 0) {
         // ---------------------------------------------------------------- MMA issuer
-        constexpr bool A_MN = V == V_DW, B_MN = V == V_FWD || V == V_DW;
+        constexpr bool A_MN = V == V_DW || V == V_DWX, B_MN = V == V_FWD || V == V_DW || V == V_DX || V == V_DWX;
         constexpr uint32_t idesc = umma_idesc_bf16(TM, TN, A_MN, B_MN);
         const uint64_t dA = A_MN ? umma_smem_desc(sA, TK * 128, 1024) : umma_smem_desc(sA, 16, 1024);
         const uint64_t dB = B_MN ? umma_smem_desc(sB, TK * 128, 1024) : umma_smem_desc(sB, 16, 1024);
@@ -237,16 +266,58 @@ proj_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 }
 
 template <int V>
-cudaError_t launch(const CUtensorMap& ta, const CUtensorMap& tb, const ProjArgs& a, unsigned* status, cudaStream_t st)
+cudaError_t launch3(const CUtensorMap& ta, const CUtensorMap& ta2, const CUtensorMap& ta3, const CUtensorMap& tb,
+                    const ProjArgs& a, unsigned* status, cudaStream_t st)
 {
     auto kern = proj_kernel<V>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
     if (e != cudaSuccess) return e;
-    const int N = V == V_DO ? a.H * a.D : V == V_QKV ? (a.H + 2 * a.Hkv) * a.D : a.E;
-    const int rows = V == V_DW ? a.H * a.D : a.S;
-    const dim3 grid((N + TN - 1) / TN, (rows + TM - 1) / TM, V == V_DW ? 1 : a.B);
-    kern<<<grid, kThreads, SMEM, st>>>(ta, tb, a, status);
+    const int F = (a.H + 2 * a.Hkv) * a.D;
+    const int N = V == V_DO ? a.H * a.D : V == V_QKV ? F : a.E;
+    const int rows = V == V_DW ? a.H * a.D : V == V_DWX ? F : a.S;
+    const dim3 grid((N + TN - 1) / TN, (rows + TM - 1) / TM, (V == V_DW || V == V_DWX) ? 1 : a.B);
+    kern<<<grid, kThreads, SMEM, st>>>(ta, ta2, ta3, tb, a, status);
     return cudaGetLastError();
+}
+template <int V>
+cudaError_t launch(const CUtensorMap& ta, const CUtensorMap& tb, const ProjArgs& a, unsigned* status, cudaStream_t st)
+{
+    return launch3<V>(ta, ta, ta, tb, a, status, st);
+}
+
+// Rotation of the (d, d + D/2) pairs of every row of t [rows_bh * S, D] by the OPPOSITE of the angles in
+// cos_t, sin_t [S, D/2], in place: the gradient of the rotary embedding.  Eight pairs per thread and step.
+__global__ void __launch_bounds__(256)
+rope_bwd_kernel(__nv_bfloat16* __restrict__ t, const float* __restrict__ cos_t, const float* __restrict__ sin_t,
+                size_t n_rows, int S, int D)
+{
+    const int half = D / 2, per_row = half / 8;
+    const size_t total = n_rows * per_row;
+    for (size_t i = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x; i < total;
+         i += static_cast<size_t>(gridDim.x) * blockDim.x) {
+        const size_t row = i / per_row;
+        const int d0 = static_cast<int>(i % per_row) * 8, s = static_cast<int>(row % S);
+        uint4* plo = reinterpret_cast<uint4*>(t + row * D + d0);
+        uint4* phi = reinterpret_cast<uint4*>(t + row * D + half + d0);
+        const uint4 lo4 = *plo, hi4 = *phi;
+        const float4 ca = *reinterpret_cast<const float4*>(cos_t + static_cast<size_t>(s) * half + d0);
+        const float4 cb = *reinterpret_cast<const float4*>(cos_t + static_cast<size_t>(s) * half + d0 + 4);
+        const float4 sa = *reinterpret_cast<const float4*>(sin_t + static_cast<size_t>(s) * half + d0);
+        const float4 sb = *reinterpret_cast<const float4*>(sin_t + static_cast<size_t>(s) * half + d0 + 4);
+        const float cc[8] = {ca.x, ca.y, ca.z, ca.w, cb.x, cb.y, cb.z, cb.w};
+        const float ss[8] = {sa.x, sa.y, sa.z, sa.w, sb.x, sb.y, sb.z, sb.w};
+        const uint32_t lw[4] = {lo4.x, lo4.y, lo4.z, lo4.w}, hw[4] = {hi4.x, hi4.y, hi4.z, hi4.w};
+        uint32_t lo_out[4], hi_out[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const float l0 = __uint_as_float(lw[j] << 16), l1 = __uint_as_float(lw[j] & 0xffff0000u);
+            const float h0 = __uint_as_float(hw[j] << 16), h1 = __uint_as_float(hw[j] & 0xffff0000u);
+            lo_out[j] = pack_bf16(l0 * cc[2 * j] + h0 * ss[2 * j], l1 * cc[2 * j + 1] + h1 * ss[2 * j + 1]);
+            hi_out[j] = pack_bf16(h0 * cc[2 * j] - l0 * ss[2 * j], h1 * cc[2 * j + 1] - l1 * ss[2 * j + 1]);
+        }
+        *plo = make_uint4(lo_out[0], lo_out[1], lo_out[2], lo_out[3]);
+        *phi = make_uint4(hi_out[0], hi_out[1], hi_out[2], hi_out[3]);
+    }
 }
 
 }  // namespace
@@ -291,6 +362,45 @@ cudaError_t launch_qkv_rope(const void* x, const void* w, const float* cos_t, co
     ProjArgs a{static_cast<__nv_bfloat16*>(q), static_cast<__nv_bfloat16*>(k), static_cast<__nv_bfloat16*>(v), nullptr,
                nullptr, cos_t, sin_t, B, H, Hkv, S, D, E};
     return launch<V_QKV>(ta, tb, a, status, st);
+}
+
+cudaError_t launch_rope_bwd(void* dq, void* dk, const float* cos_t, const float* sin_t, int B, int H, int Hkv, int S,
+                            int D, cudaStream_t st)
+{
+    void* ts[2] = {dq, dk};
+    const int hs[2] = {H, Hkv};
+    for (int i = 0; i < 2; ++i) {
+        const size_t n_rows = static_cast<size_t>(B) * hs[i] * S, total = n_rows * (D / 16);
+        const unsigned blocks = static_cast<unsigned>(total / 256 + 1 < 148u * 16u ? total / 256 + 1 : 148u * 16u);
+        rope_bwd_kernel<<<blocks, 256, 0, st>>>(static_cast<__nv_bfloat16*>(ts[i]), cos_t, sin_t, n_rows, S, D);
+        const cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+    }
+    return cudaSuccess;
+}
+
+cudaError_t launch_qkv_bwd_data(const void* gq, const void* gk, const void* gv, const void* w, void* dx, int B, int S,
+                                int E, int H, int Hkv, int D, unsigned* status, cudaStream_t st)
+{
+    CUtensorMap ta, ta2, ta3, tb;
+    if (make_tmap_3d(&ta, gq, 2, 1, B * H, S, D, 64, TM)) return cudaErrorInvalidValue;
+    if (make_tmap_3d(&ta2, gk, 2, 1, B * Hkv, S, D, 64, TM)) return cudaErrorInvalidValue;
+    if (make_tmap_3d(&ta3, gv, 2, 1, B * Hkv, S, D, 64, TM)) return cudaErrorInvalidValue;
+    if (make_tmap_3d(&tb, w, 2, 1, 1, (H + 2 * Hkv) * D, E, 64, TK)) return cudaErrorInvalidValue;
+    ProjArgs a{static_cast<__nv_bfloat16*>(dx), nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, B, H, Hkv, S, D, E};
+    return launch3<V_DX>(ta, ta2, ta3, tb, a, status, st);
+}
+
+cudaError_t launch_qkv_bwd_weight(const void* gq, const void* gk, const void* gv, const void* x, void* dw, int B, int S,
+                                  int E, int H, int Hkv, int D, unsigned* status, cudaStream_t st)
+{
+    CUtensorMap ta, ta2, ta3, tb;
+    if (make_tmap_3d(&ta, gq, 2, 1, B * H, S, D, 64, TK)) return cudaErrorInvalidValue;
+    if (make_tmap_3d(&ta2, gk, 2, 1, B * Hkv, S, D, 64, TK)) return cudaErrorInvalidValue;
+    if (make_tmap_3d(&ta3, gv, 2, 1, B * Hkv, S, D, 64, TK)) return cudaErrorInvalidValue;
+    if (make_tmap_3d(&tb, x, 2, 1, B, S, E, 64, TK)) return cudaErrorInvalidValue;
+    ProjArgs a{static_cast<__nv_bfloat16*>(dw), nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, B, H, Hkv, S, D, E};
+    return launch3<V_DWX>(ta, ta2, ta3, tb, a, status, st);
 }
 
 }  // namespace mgn

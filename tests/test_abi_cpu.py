@@ -36,7 +36,8 @@ def test_every_declared_symbol_is_exported(lib):
             "mgn_attn_fast_item_order", "mgn_attn_fwd_ext", "mgn_attn_bwd_ext",
             "mgn_attn_bwd_deterministic", "mgn_attn_fwd_accel", "mgn_attn_fwd_accel_workspace_bytes",
             "mgn_attn_strict_tiles", "mgn_selftest_wait_timeout", "mgn_out_proj_fwd", "mgn_out_proj_bwd_data",
-            "mgn_attn_bwd_given_delta", "mgn_out_proj_bwd_weight", "mgn_qkv_rope_fwd"} <= set(syms)
+            "mgn_attn_bwd_given_delta", "mgn_out_proj_bwd_weight", "mgn_qkv_rope_fwd", "mgn_rope_bwd_inplace",
+            "mgn_qkv_bwd_data", "mgn_qkv_bwd_weight"} <= set(syms)
     for s in syms:
         assert getattr(lib, s) is not None
 
@@ -264,6 +265,39 @@ def test_projection_entry_points_validate_before_any_launch(lib):
     p = [A] * 7
     p[3] = A + 8                                            # the sine table
     assert qk(ptrs=p) == MISALIGNED
+
+    # the backward of the QKV projection: opposite rotation in place, data gradient, weight gradient
+    lib.mgn_rope_bwd_inplace.argtypes = [vp] * 4 + [i] * 6 + [vp]
+    lib.mgn_qkv_bwd_data.argtypes = [vp] * 5 + [i] * 7 + [vp]
+    lib.mgn_qkv_bwd_weight.argtypes = [vp] * 5 + [i] * 7 + [vp]
+
+    def rb(ptrs=None, Hkv=1, D=128, mode=1):
+        p = [A] * 4 if ptrs is None else ptrs
+        return lib.mgn_rope_bwd_inplace(*p, 1, 2, Hkv, 8, D, mode, None)
+
+    for idx in range(4):
+        p = [A] * 4
+        p[idx] = None
+        assert rb(ptrs=p) == INVALID
+    assert rb(Hkv=0) == INVALID and rb(D=32) == UNSUPPORTED and rb(mode=0) == UNSUPPORTED and rb(mode=7) == INVALID
+    p = [A] * 4
+    p[2] = A + 4                                            # the cosine table
+    assert rb(ptrs=p) == MISALIGNED
+
+    for fn in (lib.mgn_qkv_bwd_data, lib.mgn_qkv_bwd_weight):
+        def qb(ptrs=None, Hkv=1, D=64, E=64, mode=1, S=8):
+            p = [A] * 5 if ptrs is None else ptrs
+            return fn(*p, 1, S, E, 2, Hkv, D, mode, None)
+
+        for idx in range(5):
+            p = [A] * 5
+            p[idx] = None
+            assert qb(ptrs=p) == INVALID
+        assert qb(Hkv=0) == INVALID and qb(S=0) == INVALID and qb(mode=0) == UNSUPPORTED
+        assert qb(D=32) == UNSUPPORTED and qb(E=60) == UNSUPPORTED
+        p = [A] * 5
+        p[2] = A + 2                                        # the value gradient
+        assert qb(ptrs=p) == MISALIGNED
 
     def gd(ptrs=None, ws=A, ws_bytes=1 << 30, Sq=8, Sk=16, D=64, causal=0, mode=0, H=4, Hkv=2):
         p = [A] * 9 if ptrs is None else ptrs

@@ -153,3 +153,97 @@ def test_qkv_projection_with_rotary_embedding(B, S, E, H, Hkv, D):
     for name, got, ref in (("Q", q, rq), ("K", k, rk), ("V", v, rv)):
         err = hp.rel_l2(got.check(name).double().numpy(), ref)
         assert err <= hp.FAST_REL_L2, f"{name}: {err:.3e}"
+
+
+QKV_SHAPES = [
+    # B, S, E, H, Hkv, D
+    (1, 128, 64, 2, 2, 128),       # one tile
+    (2, 197, 200, 3, 1, 64),       # ragged rows, E not a slice multiple, (H + 2 Hkv) D = 320: a row tile past the last head
+    (1, 300, 512, 5, 5, 128),      # odd head count
+    (3, 1, 8, 4, 2, 64),           # a single position
+    (2, 520, 1024, 8, 2, 128),     # grouped key/value heads, several row tiles and contraction slices
+]
+
+
+def _qkv_case(seed, B, S, E, H, Hkv, D):
+    g = torch.Generator().manual_seed(seed)
+    x = torch.randn(B, S, E, generator=g).to(BF)
+    w = (torch.randn((H + 2 * Hkv) * D, E, generator=g) / math.sqrt(E)).to(BF)
+    inv = 10000.0 ** (-torch.arange(D // 2, dtype=torch.float64) * 2.0 / D)
+    ang = torch.arange(S, dtype=torch.float64)[:, None] * inv[None, :]
+    cos_t, sin_t = torch.cos(ang).float().contiguous(), torch.sin(ang).float().contiguous()
+    g_q = torch.randn(B, H, S, D, generator=g).to(BF)
+    g_k = torch.randn(B, Hkv, S, D, generator=g).to(BF)
+    g_v = torch.randn(B, Hkv, S, D, generator=g).to(BF)
+    return x, w, cos_t, sin_t, g_q, g_k, g_v
+
+
+@pytest.mark.parametrize("B,S,E,H,Hkv,D", QKV_SHAPES)
+def test_gradient_of_the_rotary_embedding_in_place(B, S, E, H, Hkv, D):
+    x, w, cos_t, sin_t, g_q, g_k, g_v = _qkv_case(60 + S, B, S, E, H, Hkv, D)
+    dq, dk = hp.Guarded((B, H, S, D), BF), hp.Guarded((B, Hkv, S, D), BF)
+    dq.view.copy_(g_q); dk.view.copy_(g_k)
+    mgn.mgn_rope_bwd_inplace(dq.view, dk.view, cos_t.cuda(), sin_t.cuda(), MODE)
+    mgn.mgn_attn_check()
+    _, _, gy = orc.qkv_rope_bwd(g_q.double().numpy(), g_k.double().numpy(), g_v.double().numpy(), x.double().numpy(),
+                                w.double().numpy(), cos_t.double().numpy(), sin_t.double().numpy())
+    ref_q = gy[..., : H * D].reshape(B, S, H, D).transpose(0, 2, 1, 3)
+    ref_k = gy[..., H * D:(H + Hkv) * D].reshape(B, S, Hkv, D).transpose(0, 2, 1, 3)
+    # one rounding to bf16 of an f32 result: relative 2^-9 per element
+    assert hp.rel_l2(dq.check("dq").double().numpy(), ref_q) <= 3e-3
+    assert hp.rel_l2(dk.check("dk").double().numpy(), ref_k) <= 3e-3
+
+
+@pytest.mark.parametrize("B,S,E,H,Hkv,D", QKV_SHAPES)
+def test_qkv_projection_backward_against_the_oracle(B, S, E, H, Hkv, D):
+    """The three calls in sequence -- opposite rotation in place, data gradient, weight gradient -- against the
+    oracle's backward of the rotated projection."""
+    x, w, cos_t, sin_t, g_q, g_k, g_v = _qkv_case(70 + S, B, S, E, H, Hkv, D)
+    dq, dk, dv = g_q.cuda(), g_k.cuda(), g_v.cuda()
+    mgn.mgn_rope_bwd_inplace(dq, dk, cos_t.cuda(), sin_t.cuda(), MODE)
+    dx = hp.Guarded((B, S, E), BF)
+    dw = hp.Guarded(((H + 2 * Hkv) * D, E), BF)
+    mgn.mgn_qkv_bwd_data(dq, dk, dv, w.cuda(), dx.view, MODE)
+    mgn.mgn_qkv_bwd_weight(dq, dk, dv, x.cuda(), dw.view, MODE)
+    mgn.mgn_attn_check()
+    assert torch.equal(dv.cpu(), g_v)                       # the value gradient is only read
+    rdx, rdw, _ = orc.qkv_rope_bwd(g_q.double().numpy(), g_k.double().numpy(), g_v.double().numpy(), x.double().numpy(),
+                                   w.double().numpy(), cos_t.double().numpy(), sin_t.double().numpy())
+    e_dx, e_dw = hp.rel_l2(dx.check("dX").double().numpy(), rdx), hp.rel_l2(dw.check("dW").double().numpy(), rdw)
+    assert e_dx <= hp.FAST_REL_L2, f"dX: {e_dx:.3e}"
+    assert e_dw <= hp.FAST_REL_L2, f"dW: {e_dw:.3e}"
+
+
+def test_whole_layer_backward_chain():
+    """dY -> output-projection backward (dO, delta) -> attention backward with that delta -> opposite rotation ->
+    QKV data gradient, on tensors produced by this library's own forward chain; against the same chain in the
+    oracle (f64 on the bf16-rounded inputs)."""
+    B, S, E, H, Hkv, D = 1, 384, 256, 4, 2, 64
+    x, w, cos_t, sin_t, _, _, _ = _qkv_case(91, B, S, E, H, Hkv, D)
+    g = torch.Generator().manual_seed(92)
+    w_o = (torch.randn(H * D, E, generator=g) / math.sqrt(H * D)).to(BF)
+    d_y = torch.randn(B, S, E, generator=g).to(BF)
+    scale = 1.0 / math.sqrt(D)
+    xd, wd, wod, cd, sd = x.cuda(), w.cuda(), w_o.cuda(), cos_t.cuda(), sin_t.cuda()
+    q = torch.empty(B, H, S, D, dtype=BF, device="cuda")
+    k, v = (torch.empty(B, Hkv, S, D, dtype=BF, device="cuda") for _ in range(2))
+    mgn.mgn_qkv_rope_fwd(xd, wd, cd, sd, q, k, v, MODE)
+    o = torch.empty_like(q); lse = torch.empty(B, H, S, device="cuda")
+    mgn.mgn_attn_fwd_ext(q, k, v, o, lse, True, scale, MODE)
+    d_o = torch.empty_like(q); delta = torch.empty(B, H, S, device="cuda")
+    mgn.mgn_out_proj_bwd_data(d_y.cuda(), wod, o, d_o, delta, MODE)
+    dq = torch.empty_like(q); dk, dv = torch.empty_like(k), torch.empty_like(v)
+    ws = mgn.alloc_workspace(B, H, S, D, MODE)
+    mgn.mgn_attn_bwd_given_delta(q, k, v, d_o, lse, delta, dq, dk, dv, ws, True, scale, MODE)
+    mgn.mgn_rope_bwd_inplace(dq, dk, cd, sd, MODE)
+    dx = hp.Guarded((B, S, E), BF)
+    mgn.mgn_qkv_bwd_data(dq, dk, dv, wd, dx.view, MODE)
+    mgn.mgn_attn_check()
+    # oracle chain
+    c64, s64 = cos_t.double().numpy(), sin_t.double().numpy()
+    rq, rk, rv = orc.qkv_rope(x.double().numpy(), w.double().numpy(), c64, s64, H, Hkv, D)
+    r_do, _, _ = orc.out_proj_bwd(d_y.double().numpy(), w_o.double().numpy(), np.zeros((B, H, S, D)))
+    ref = hp.run_oracle_ext(torch.from_numpy(rq), torch.from_numpy(rk), torch.from_numpy(rv), torch.from_numpy(r_do), True, scale)
+    rdx, _, _ = orc.qkv_rope_bwd(ref["dQ"], ref["dK"], ref["dV"], x.double().numpy(), w.double().numpy(), c64, s64)
+    err = hp.rel_l2(dx.check("dX").double().numpy(), rdx)
+    assert err <= hp.FAST_REL_L2, f"dX through the whole layer: {err:.3e}"
