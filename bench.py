@@ -553,6 +553,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-fast", action="store_true", help="skip the extra measurements (other mode, other shapes, other workloads)")
+    ap.add_argument("--only-proj", action="store_true",
+                    help="time only the projections either side of attention (the proj_fusion object of the line) and print "
+                         "that object; a small command to capture their kernels under a profiler")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -565,6 +568,13 @@ def main():
         return
 
     from paper_2608_01563_b200 import binding as mgn
+
+    if args.only_proj:
+        if not torch.cuda.is_available():
+            raise SystemExit("bench.py needs a CUDA device: the projections have no CPU fallback")
+        if int(os.environ.get("RANK", "0")) == 0:
+            print(json.dumps({"proj_fusion": measure_proj_fusion(mgn, args.steps, args.warmup)}))
+        return
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
