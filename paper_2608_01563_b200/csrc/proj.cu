@@ -19,9 +19,12 @@
 // The last two take the gradients with respect to the UNROTATED projection: the rotation depends on the
 // position, i.e. on the row of the operand, and cannot be folded into either product; rope_bwd_kernel
 // applies the opposite rotation to dQ and dK in place first (a streaming pass over those two tensors).
-// One CTA computes a 128 x 256 output tile.  Warp 0 streams 64-wide contraction slices of both
-// operands through a four-stage TMA ring, one lane of warp 1 issues the products into a 256-column
-// tensor-memory accumulator, warps 2-5 (one thread per accumulator row) read it out.
+// Persistent: one CTA per SM walks over 128 x 256 output tiles (tile t, t + grid, ...; neighbouring tiles
+// share their row block, so the CTAs running at one time share operand tiles in L2).  Warp 0 streams
+// 64-wide contraction slices of both operands through a four-stage TMA ring that keeps running across
+// tiles (a lane of warp 6 does the same for the other operand), one lane of warp 1 issues the products
+// into one of two 256-column tensor-memory accumulators, warps 2-5 (one thread per accumulator row) read
+// the other one out meanwhile.
 #include <cuda_bf16.h>
 
 #include "kernels.h"
@@ -30,14 +33,14 @@
 namespace mgn {
 namespace {
 
-constexpr int kThreads = 192;
+constexpr int kThreads = 224;
 constexpr int TM = 128, TN = 256, TK = 64, kStages = 4;
 constexpr int A_BYTES = TM * TK * 2;          // 16 KB
 constexpr int B_BYTES = TN * TK * 2;          // 32 KB
 constexpr int OFF_A = 0, OFF_B = kStages * A_BYTES, OFF_BAR = OFF_B + kStages * B_BYTES;
 constexpr int PAYLOAD = OFF_BAR + 128;
 constexpr int SMEM = PAYLOAD + 1024;
-enum { B_FULL = 0, B_EMPTY = kStages, B_ACC = 2 * kStages, B_COUNT = 2 * kStages + 1 };
+enum { B_FULL = 0, B_EMPTY = kStages, B_ACCFULL = 2 * kStages, B_ACCEMPTY = 2 * kStages + 2, B_COUNT = 2 * kStages + 4 };
 enum { V_FWD = 0, V_DO = 1, V_DW = 2, V_QKV = 3, V_DX = 4, V_DWX = 5 };
 
 struct ProjArgs {
@@ -98,39 +101,45 @@ template <int D>
 __device__ __forceinline__ void epilogue_qkv_head(const ProjArgs& a, uint32_t tacc_head, int b, int s, int hh, bool row_ok)
 {
     constexpr int NC = D / 32, HALF = D / 2;
-    uint32_t v[NC][32];
-#pragma unroll
-    for (int c = 0; c < NC; ++c) tmem_ld32(tacc_head + 32 * c, v[c]);      // whole warp, whatever the row
-    tmem_ld_wait();
-    if (!row_ok || hh >= a.H + 2 * a.Hkv) return;
-    __nv_bfloat16* dst;
-    if (hh < a.H) dst = a.out + ((static_cast<size_t>(b) * a.H + hh) * a.S + s) * D;
-    else if (hh < a.H + a.Hkv) dst = a.out_k + ((static_cast<size_t>(b) * a.Hkv + (hh - a.H)) * a.S + s) * D;
-    else dst = a.out_v + ((static_cast<size_t>(b) * a.Hkv + (hh - a.H - a.Hkv)) * a.S + s) * D;
-    if (hh < a.H + a.Hkv) {
-        const float* ct = a.cos_t + static_cast<size_t>(s) * HALF;
-        const float* st = a.sin_t + static_cast<size_t>(s) * HALF;
-#pragma unroll
-        for (int c = 0; c < NC / 2; ++c)
+    const bool live = row_ok && hh < a.H + 2 * a.Hkv;
+    __nv_bfloat16* dst = nullptr;
+    if (live) {
+        if (hh < a.H) dst = a.out + ((static_cast<size_t>(b) * a.H + hh) * a.S + s) * D;
+        else if (hh < a.H + a.Hkv) dst = a.out_k + ((static_cast<size_t>(b) * a.Hkv + (hh - a.H)) * a.S + s) * D;
+        else dst = a.out_v + ((static_cast<size_t>(b) * a.Hkv + (hh - a.H - a.Hkv)) * a.S + s) * D;
+    }
+    const bool rotate = hh < a.H + a.Hkv;
+    // 32 columns of the lower half and the 32 columns D/2 further on at a time: the pairs of the rotation
+#pragma unroll 1
+    for (int c = 0; c < NC / 2; ++c) {
+        uint32_t lo[32], hi[32];
+        tmem_ld32(tacc_head + 32 * c, lo);                 // whole warp, whatever the row
+        tmem_ld32(tacc_head + 32 * (c + NC / 2), hi);
+        tmem_ld_wait();
+        if (!live) continue;
+        if (rotate) {
+            const float* ct = a.cos_t + static_cast<size_t>(s) * HALF + 32 * c;
+            const float* st = a.sin_t + static_cast<size_t>(s) * HALF + 32 * c;
 #pragma unroll
             for (int e4 = 0; e4 < 8; ++e4) {
-                const float4 c4 = *reinterpret_cast<const float4*>(ct + 32 * c + 4 * e4);
-                const float4 s4 = *reinterpret_cast<const float4*>(st + 32 * c + 4 * e4);
+                const float4 c4 = *reinterpret_cast<const float4*>(ct + 4 * e4);
+                const float4 s4 = *reinterpret_cast<const float4*>(st + 4 * e4);
                 const float cc[4] = {c4.x, c4.y, c4.z, c4.w}, ss[4] = {s4.x, s4.y, s4.z, s4.w};
 #pragma unroll
                 for (int t = 0; t < 4; ++t) {
-                    const float lo = __uint_as_float(v[c][4 * e4 + t]), hi = __uint_as_float(v[c + NC / 2][4 * e4 + t]);
-                    v[c][4 * e4 + t] = __float_as_uint(lo * cc[t] - hi * ss[t]);
-                    v[c + NC / 2][4 * e4 + t] = __float_as_uint(hi * cc[t] + lo * ss[t]);
+                    const float l = __uint_as_float(lo[4 * e4 + t]), h = __uint_as_float(hi[4 * e4 + t]);
+                    lo[4 * e4 + t] = __float_as_uint(l * cc[t] - h * ss[t]);
+                    hi[4 * e4 + t] = __float_as_uint(h * cc[t] + l * ss[t]);
                 }
             }
-    }
-#pragma unroll
-    for (int c = 0; c < NC; ++c) {
+        }
         uint32_t u[16];
 #pragma unroll
-        for (int e = 0; e < 16; ++e) u[e] = pack_bf16(__uint_as_float(v[c][2 * e]), __uint_as_float(v[c][2 * e + 1]));
+        for (int e = 0; e < 16; ++e) u[e] = pack_bf16(__uint_as_float(lo[2 * e]), __uint_as_float(lo[2 * e + 1]));
         store_row32(dst + 32 * c, u, 4);
+#pragma unroll
+        for (int e = 0; e < 16; ++e) u[e] = pack_bf16(__uint_as_float(hi[2 * e]), __uint_as_float(hi[2 * e + 1]));
+        store_row32(dst + 32 * (c + NC / 2), u, 4);
     }
 }
 
@@ -147,8 +156,7 @@ proj_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     const uint32_t tmem_slot = bars + B_COUNT * 8;
     auto bar = [&](int i) { return bars + 8u * i; };
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    // tile: TN output columns from n0; TM rows from r0 (positions s of batch element b, or for DW rows (h,d) of d_w)
-    const int n0 = static_cast<int>(blockIdx.x) * TN, r0 = static_cast<int>(blockIdx.y) * TM, b = static_cast<int>(blockIdx.z);
+    // tile t: TN output columns from n0; TM rows from r0 (positions s of batch element b, or for DW, DWX rows of d_w)
     const int HD = a.H * a.D, F = (a.H + 2 * a.Hkv) * a.D;             // features: of the heads of O; of query | key | value
     const int n_sc = (a.S + TK - 1) / TK;                              // DW, DWX: 64-position slices per batch element
     const int N = V == V_DO ? HD : V == V_QKV ? F : a.E;
@@ -165,55 +173,83 @@ proj_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         return &tmA3;
     };
 
+    const int tiles_n = (N + TN - 1) / TN, tiles_m = (rows + TM - 1) / TM;
+    const int n_tiles = tiles_n * tiles_m * ((V == V_DW || V == V_DWX) ? 1 : a.B);
+    const int t0 = static_cast<int>(blockIdx.x), dt = static_cast<int>(gridDim.x);
+    auto tile_at = [&](int t, int& n0, int& r0, int& b) {
+        n0 = (t % tiles_n) * TN;
+        r0 = ((t / tiles_n) % tiles_m) * TM;
+        b = t / (tiles_n * tiles_m);
+    };
+
     if (tid == 0) {
-        for (int i = 0; i < B_COUNT; ++i) mbar_init(bar(i), 1);
+        for (int i = 0; i < B_COUNT; ++i)
+            mbar_init(bar(i), (i == B_ACCEMPTY || i == B_ACCEMPTY + 1) ? 128 : (i >= B_FULL && i < B_FULL + kStages) ? 2 : 1);
         fence_mbar_init();
     }
     __syncwarp();
-    if (warp == 0) tmem_alloc(tmem_slot, TN);
+    if (warp == 0) tmem_alloc(tmem_slot, 2 * TN);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = lds32u(tmem_slot);
 
-    if (warp == 0 && lane == 0) {
-        // ---------------------------------------------------------------- TMA producer
-        for (int kt = 0; kt < n_kt; ++kt) {
-            const int st = kt % kStages, k0 = kt * TK;
-            if (kt >= kStages) mbar_wait(bar(B_EMPTY + st), ((kt / kStages) - 1) & 1, status);
-            mbar_arrive_expect_tx(bar(B_FULL + st), A_BYTES + B_BYTES);
+    if ((warp == 0 || warp == 6) && lane == 0) {
+        // ---------------------------------------------------------------- TMA producers
+        // Two lanes, one per operand (warp 0: A, warp 6: B).  A lane's turn per slice is a barrier wait (250-350
+        // clocks while the tensor core streams operands from shared memory) plus up to six copy instructions,
+        // and the products of a slice take 512 clocks: one lane for both operands was the limit of the
+        // variants that fetch their operands in 64-wide blocks.
+        const bool opA = warp == 0;
+        int g = 0;                                     // slices loaded so far (all tiles): stage and phase of the ring
+        for (int t = t0; t < n_tiles; t += dt) {
+        int n0, r0, b;
+        tile_at(t, n0, r0, b);
+        int bb = 0, s0 = 0;                            // DW, DWX: batch element and first position of the slice
+        for (int kt = 0; kt < n_kt; ++kt, ++g) {
+            const int st = g % kStages, k0 = kt * TK;
+            if (g >= kStages) mbar_wait(bar(B_EMPTY + st), ((g / kStages) - 1) & 1, status);
+            mbar_arrive_expect_tx(bar(B_FULL + st), opA ? A_BYTES : B_BYTES);
             const uint32_t dA = sA + st * A_BYTES, dB = sB + st * B_BYTES, full = bar(B_FULL + st);
             if constexpr (V == V_DO || V == V_QKV) {
-                tma_load_3d(dA, &tmA, full, k0, r0, b);                                  // 128 positions x 64 e
-                tma_load_3d(dB, &tmB, full, k0, n0, 0);                                  // 256 rows n x 64 e
+                if (opA) tma_load_3d(dA, &tmA, full, k0, r0, b);                         // 128 positions x 64 e
+                else tma_load_3d(dB, &tmB, full, k0, n0, 0);                             // 256 rows n x 64 e
             } else if constexpr (V == V_FWD || V == V_DX) {
-                if constexpr (V == V_FWD) {
-                    tma_load_3d(dA, &tmA, full, k0 % a.D, r0, b * a.H + k0 / a.D);       // 128 positions x 64 d of one head
-                } else {
-                    int idx;
-                    const CUtensorMap* m = head_of(k0, b, idx);
-                    tma_load_3d(dA, m, full, k0 % a.D, r0, idx);
-                }
-#pragma unroll
-                for (int c = 0; c < TN / 64; ++c)                                         // four blocks of 64 k rows x 64 n
-                    tma_load_3d(dB + c * (TK * 128), &tmB, full, n0 + 64 * c, k0, 0);
-            } else {
-                const int bb = kt / n_sc, s0 = (kt % n_sc) * TK;
-#pragma unroll
-                for (int c = 0; c < TM / 64; ++c) {                                       // two blocks of 64 positions x 64 rows m
-                    const int m = r0 + 64 * c;
-                    if constexpr (V == V_DW) {
-                        tma_load_3d(dA + c * (TK * 128), &tmA, full, m % a.D, s0, bb * a.H + m / a.D);
+                if (opA) {
+                    if constexpr (V == V_FWD) {
+                        tma_load_3d(dA, &tmA, full, k0 % a.D, r0, b * a.H + k0 / a.D);   // 128 positions x 64 d of one head
                     } else {
                         int idx;
-                        const CUtensorMap* mp = head_of(m, bb, idx);
-                        tma_load_3d(dA + c * (TK * 128), mp, full, m % a.D, s0, idx);
+                        const CUtensorMap* m = head_of(k0, b, idx);
+                        tma_load_3d(dA, m, full, k0 % a.D, r0, idx);
                     }
-                }
+                } else {
 #pragma unroll
-                for (int c = 0; c < TN / 64; ++c)                                         // four blocks of 64 positions x 64 e
-                    tma_load_3d(dB + c * (TK * 128), &tmB, full, n0 + 64 * c, s0, bb);
+                    for (int c = 0; c < TN / 64; ++c)                                     // four blocks of 64 k rows x 64 n
+                        tma_load_3d(dB + c * (TK * 128), &tmB, full, n0 + 64 * c, k0, 0);
+                }
+            } else {
+                if (opA) {
+#pragma unroll
+                    for (int c = 0; c < TM / 64; ++c) {                                   // two blocks of 64 positions x 64 rows m
+                        const int m = r0 + 64 * c;
+                        if constexpr (V == V_DW) {
+                            tma_load_3d(dA + c * (TK * 128), &tmA, full, m % a.D, s0, bb * a.H + m / a.D);
+                        } else {
+                            int idx;
+                            const CUtensorMap* mp = head_of(m, bb, idx);
+                            tma_load_3d(dA + c * (TK * 128), mp, full, m % a.D, s0, idx);
+                        }
+                    }
+                } else {
+#pragma unroll
+                    for (int c = 0; c < TN / 64; ++c)                                     // four blocks of 64 positions x 64 e
+                        tma_load_3d(dB + c * (TK * 128), &tmB, full, n0 + 64 * c, s0, bb);
+                }
+                s0 += TK;                              // slices run over the positions of batch element 0, then 1, ...
+                if (s0 >= n_sc * TK) { s0 = 0; ++bb; }
             }
+        }
         }
     } else if (warp == 1 && lane == 0) {
         // ---------------------------------------------------------------- MMA issuer
@@ -221,24 +257,35 @@ proj_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         constexpr uint32_t idesc = umma_idesc_bf16(TM, TN, A_MN, B_MN);
         const uint64_t dA = A_MN ? umma_smem_desc(sA, TK * 128, 1024) : umma_smem_desc(sA, 16, 1024);
         const uint64_t dB = B_MN ? umma_smem_desc(sB, TK * 128, 1024) : umma_smem_desc(sB, 16, 1024);
-        for (int kt = 0; kt < n_kt; ++kt) {
-            const int st = kt % kStages;
-            mbar_wait(bar(B_FULL + st), (kt / kStages) & 1, status);
+        int g = 0, ti = 0;                             // slices and tiles so far
+        for (int t = t0; t < n_tiles; t += dt, ++ti) {
+            const int acc = ti & 1;
+            mbar_wait(bar(B_ACCEMPTY + acc), ((ti >> 1) & 1) ^ 1, status);   // the tile two back has been read out
             tc_fence_after();
+            for (int kt = 0; kt < n_kt; ++kt, ++g) {
+                const int st = g % kStages;
+                mbar_wait(bar(B_FULL + st), (g / kStages) & 1, status);
+                tc_fence_after();
 #pragma unroll
-            for (int kk = 0; kk < TK / 16; ++kk) {
-                const uint64_t da = dA + static_cast<uint64_t>((st * A_BYTES + (A_MN ? kk * 2048 : kk * 32)) >> 4);
-                const uint64_t db = dB + static_cast<uint64_t>((st * B_BYTES + (B_MN ? kk * 2048 : kk * 32)) >> 4);
-                umma_ss(tmem, da, db, idesc, (kt > 0 || kk > 0) ? 1u : 0u);
+                for (int kk = 0; kk < TK / 16; ++kk) {
+                    const uint64_t da = dA + static_cast<uint64_t>((st * A_BYTES + (A_MN ? kk * 2048 : kk * 32)) >> 4);
+                    const uint64_t db = dB + static_cast<uint64_t>((st * B_BYTES + (B_MN ? kk * 2048 : kk * 32)) >> 4);
+                    umma_ss(tmem + acc * TN, da, db, idesc, (kt > 0 || kk > 0) ? 1u : 0u);
+                }
+                umma_commit(bar(B_EMPTY + st));
             }
-            umma_commit(bar(B_EMPTY + st));
+            umma_commit(bar(B_ACCFULL + acc));
         }
-        umma_commit(bar(B_ACC));
-    } else if (warp >= 2) {
+    } else if (warp >= 2 && warp < 6) {
         // ---------------------------------------------------------------- epilogue: one thread per row
-        const int q4 = warp & 3, r = 32 * q4 + lane, row = r0 + r;
-        const uint32_t tacc = tmem + (static_cast<uint32_t>(32 * q4) << 16);
-        mbar_wait(bar(B_ACC), 0, status);
+        const int q4 = warp & 3, r = 32 * q4 + lane;
+        int ti = 0;
+        for (int t = t0; t < n_tiles; t += dt, ++ti) {
+        int n0, r0, b;
+        tile_at(t, n0, r0, b);
+        const int row = r0 + r, acc = ti & 1;
+        const uint32_t tacc = tmem + (static_cast<uint32_t>(32 * q4) << 16) + acc * TN;
+        mbar_wait(bar(B_ACCFULL + acc), (ti >> 1) & 1, status);
         tc_fence_after();
         if constexpr (V == V_QKV) {
             if (a.D == 128) {
@@ -259,10 +306,13 @@ proj_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                 if (row < rows && n < N) epilogue_plain<V>(a, v, b, row, n, dl);
             }
         }
+        tc_fence_before();
+        mbar_arrive(bar(B_ACCEMPTY + acc));             // this accumulator may be overwritten
+        }
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 0) tmem_dealloc(tmem, TN);
+    if (warp == 0) tmem_dealloc(tmem, 2 * TN);
 }
 
 template <int V>
@@ -275,7 +325,13 @@ cudaError_t launch3(const CUtensorMap& ta, const CUtensorMap& ta2, const CUtenso
     const int F = (a.H + 2 * a.Hkv) * a.D;
     const int N = V == V_DO ? a.H * a.D : V == V_QKV ? F : a.E;
     const int rows = V == V_DW ? a.H * a.D : V == V_DWX ? F : a.S;
-    const dim3 grid((N + TN - 1) / TN, (rows + TM - 1) / TM, (V == V_DW || V == V_DWX) ? 1 : a.B);
+    const long long tiles = static_cast<long long>((N + TN - 1) / TN) * ((rows + TM - 1) / TM) *
+                            ((V == V_DW || V == V_DWX) ? 1 : a.B);
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+        sms <= 0 || tiles > 0x7fffffffLL)
+        return cudaErrorInvalidValue;
+    const unsigned grid = static_cast<unsigned>(tiles < sms ? tiles : sms);     // persistent: one CTA per SM
     kern<<<grid, kThreads, SMEM, st>>>(ta, ta2, ta3, tb, a, status);
     return cudaGetLastError();
 }
