@@ -316,6 +316,43 @@ def measure_proj_fusion(mgn, steps, warmup):
         torch.matmul(gy, w_qkv, out=d_x.view(B * S, E))
         torch.matmul(gy.t(), x.view(B * S, E), out=d_wqkv)
 
+    # a whole attention layer, forward and backward, through this library's entry points only ...
+    y2 = torch.empty(B, S, E, device="cuda", dtype=dt)
+    d_wo = torch.empty_like(w)
+
+    def layer_fused():
+        mgn.mgn_qkv_rope_fwd(x, w_qkv, cos_t, sin_t, q2, k2, v2, mode)
+        mgn.mgn_attn_fwd(q2, k2, v2, o, lse, wl.causal, wl.scale, mode)
+        mgn.mgn_out_proj_fwd(o, w, y2, mode)
+        mgn.mgn_out_proj_bwd_weight(o, d_y, d_wo, mode)
+        mgn.mgn_out_proj_bwd_data(d_y, w, o, d_o, delta, mode)
+        mgn.mgn_attn_bwd_given_delta(q2, k2, v2, d_o, lse, delta, dq, dk, dv, ws, wl.causal, wl.scale, mode)
+        mgn.mgn_rope_bwd_inplace(dq, dk, cos_t, sin_t, mode)
+        mgn.mgn_qkv_bwd_data(dq, dk, dv, w_qkv, d_x, mode)
+        mgn.mgn_qkv_bwd_weight(dq, dk, dv, x, d_wqkv, mode)
+
+    # ... and the same layer with library GEMMs, eager rotations and layout copies around this library's
+    # attention kernels (what a caller without the fused projections would run)
+    def layer_unfused():
+        unfused_qkv()
+        mgn.mgn_attn_fwd(q2, k2, v2, o, lse, wl.causal, wl.scale, mode)
+        unfused_fwd()
+        unfused_dw()
+        d_o.copy_(torch.matmul(d_y, w.t()).view(B, S, H, D).transpose(1, 2))
+        mgn.mgn_attn_bwd(q2, k2, v2, o, d_o, lse, dq, dk, dv, ws, wl.causal, wl.scale, mode)
+        c = torch.cat([cos_t, cos_t], dim=1).to(dt)
+        s_ = torch.cat([sin_t, sin_t], dim=1).to(dt)
+        qk = torch.cat([dq, dk], dim=1)
+        rot = torch.cat([qk[..., D // 2:], -qk[..., :D // 2]], dim=-1)
+        gy = torch.cat([qk * c + rot * s_, dv], dim=1).transpose(1, 2).reshape(B * S, 3 * H * D)
+        torch.matmul(gy, w_qkv, out=d_x.view(B * S, E))
+        torch.matmul(gy.t(), x.view(B * S, E), out=d_wqkv)
+
+    layer_f = timed(layer_fused)
+    layer_u = timed(layer_unfused)
+    attn_flops = 14.0 * B * H * (S * S / 2.0) * D if wl.causal else 14.0 * B * H * S * S * D
+    layer_flops = attn_flops + 2.0 * B * S * E * (3 * H * D) * 3 + 2.0 * B * S * (H * D) * E * 3
+
     gemm_flops = 2.0 * B * S * H * D * E
     qb_fused = timed(fused_qkv_bwd)
     qb_unf = timed(unfused_qkv_bwd)
@@ -337,6 +374,8 @@ def measure_proj_fusion(mgn, steps, warmup):
             "qkv_rope_tflops": round(3 * gemm_flops / (qkv_fused * 1e-3) / 1e12, 1),
             "qkv_bwd_ms": {"fused": round(qb_fused, 4), "library_gemms_plus_eager_rotation_and_copies": round(qb_unf, 4)},
             "qkv_bwd_tflops": round(6 * gemm_flops / (qb_fused * 1e-3) / 1e12, 1),
+            "layer_fwd_bwd_ms": {"fused": round(layer_f, 4), "library_gemms_eager_rotation_copies_plus_attn": round(layer_u, 4)},
+            "layer_fwd_bwd_tflops": round(layer_flops / (layer_f * 1e-3) / 1e12, 1),
             "do_producer_ms": round(p_fused, 4), "do_producer_tflops": round(gemm_flops / (p_fused * 1e-3) / 1e12, 1),
             "proj_bwd_plus_attn_bwd_ms": {"fused": round(b_fused, 4), "library_gemm_plus_layout_copy_plus_attn_bwd": round(b_unf, 4)}}
 
